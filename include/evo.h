@@ -1,0 +1,173 @@
+/*
+ * evo.h -- C-ABI of the B200 (sm_100a) library for one evolution-strategy generation:
+ *
+ *     evo_ask      sample the whole population   theta[2j], theta[2j+1] = center +- sigma*eps_j
+ *     evo_rollout  evaluate every member         fitness[m] = mean episode return of policy(theta[m])
+ *     evo_tell     update the search distribution  centred ranks -> ES gradient -> Adam ascent
+ *
+ * The split follows the component interfaces of the EvoJAX paper, Section 4 ("Extending
+ * EvoJAX"): the algorithm's ask/tell ("Devising New Algorithms"), the policy's get_actions
+ * over the whole population ("Exploring Novel Policy Architectures") and the stateless
+ * vectorised task's reset/step ("Experimenting with More Tasks"); the roll-out loop and the
+ * central generation of roll-out seeds are the simulation manager's job (Section 2).  The
+ * paper prints no formulas; the ones quoted below are the textbook PGPE (symmetric sampling)
+ * and Adam definitions the paper names (Sections 2 and 5).
+ *
+ * Conventions for every call
+ *   - All pointers named d_* are DEVICE pointers owned by the caller; everything else is host
+ *     memory.  The library never allocates or frees device memory, and launches all work on the
+ *     CUDA stream given to evo_create (a cudaStream_t passed as void*).
+ *   - No call synchronises the device except evo_sync_status.  Device-side conditions (a NaN
+ *     fitness) are recorded in a status word inside the workspace and reported there.
+ *   - Every call returns an evo_status; nothing prints, aborts or throws.
+ *   - One solver = one stream = one host thread at a time.
+ *   - Notation: P = pop_size (even), H = P/2 antithetic pairs, D = param_dim,
+ *     ldD = D rounded up to a multiple of 32 floats (row pitch), E = episodes, T = horizon.
+ */
+#ifndef EVO_H
+#define EVO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct evo_solver evo_solver;   /* opaque, host memory, freed by evo_destroy */
+
+typedef enum {
+    EVO_OK = 0,
+    EVO_ERR_INVALID_ARG = 1,   /* NULL / misaligned pointer, bad size, bad enum            */
+    EVO_ERR_BAD_ORDER   = 2,   /* e.g. evo_tell before evo_ask                              */
+    EVO_ERR_WORKSPACE   = 3,   /* workspace too small                                       */
+    EVO_ERR_CUDA        = 4,   /* a CUDA runtime call or launch failed                      */
+    EVO_ERR_NONFINITE   = 5,   /* a NaN fitness reached evo_tell; that update was skipped   */
+    EVO_ERR_TIMEOUT     = 6,   /* a bounded device-side wait gave up                        */
+    EVO_ERR_UNSUPPORTED = 7    /* valid request this build has no kernel for                */
+} evo_status;
+
+enum { EVO_NOISE_STORED = 0, EVO_NOISE_REGENERATED = 1 };
+enum { EVO_POLICY_NONE = 0, EVO_POLICY_MLP = 1, EVO_POLICY_CNN_28 = 2 };
+enum { EVO_TASK_NONE = 0, EVO_TASK_CARTPOLE = 1, EVO_TASK_TANH_LINEAR = 2, EVO_TASK_SUPERVISED = 3 };
+enum { EVO_ROLLOUT_AUTO = 0, EVO_ROLLOUT_GENERIC = 1, EVO_ROLLOUT_TILED = 2 };
+
+/* indices into evo_config.task_param for EVO_TASK_CARTPOLE */
+enum { EVO_CP_CART_MASS = 0, EVO_CP_POLE_MASS = 1, EVO_CP_POLE_HALF_LENGTH = 2, EVO_CP_GRAVITY = 3,
+       EVO_CP_DT = 4, EVO_CP_INIT_RANGE = 5 };
+
+#define EVO_MAX_LAYERS 8
+
+typedef struct evo_config {
+    uint32_t struct_size;          /* sizeof(evo_config), checked                               */
+    uint32_t pop_size;             /* P, even, >= 2                                             */
+    uint64_t seed;                 /* Philox key of every random stream of this solver          */
+    uint32_t param_dim;            /* D >= 1                                                    */
+    uint32_t noise_mode;           /* EVO_NOISE_*: keep eps[H][ldD] from ask, or recompute it   */
+    float    sigma;                /* > 0, constant                                             */
+    float    lr;                   /* Adam step size                                            */
+    float    beta1, beta2, adam_eps;   /* 0 selects 0.9 / 0.999 / 1e-8                          */
+    uint32_t policy_kind;          /* EVO_POLICY_*                                              */
+    uint32_t n_layers;             /* MLP: number of weight matrices, 1..EVO_MAX_LAYERS         */
+    uint32_t layer_sizes[EVO_MAX_LAYERS + 1];  /* MLP widths, input first                       */
+    float    action_scale;         /* MLP output = scale * tanh(.)                              */
+    uint32_t task_kind;            /* EVO_TASK_*; NONE = caller computes fitness itself         */
+    uint32_t episodes;             /* E >= 1 (control tasks)                                    */
+    uint32_t horizon;              /* T >= 1 (control tasks)                                    */
+    uint32_t batch;                /* images per member (supervised task)                       */
+    uint32_t trace_steps;          /* leading steps recorded when evo_rollout gets d_trace      */
+    uint32_t rollout_kernel;       /* EVO_ROLLOUT_*: AUTO picks the tiled kernel when one fits  */
+    float    task_param[16];       /* cart-pole: EVO_CP_* ; others unused                       */
+} evo_config;
+
+/* Bytes of device workspace a solver with this configuration needs.  Pure host function. */
+evo_status evo_workspace_bytes(const evo_config* cfg, size_t* bytes);
+
+/*
+ * Create a solver.  d_workspace: device memory, 256-byte aligned, at least
+ * evo_workspace_bytes() long, owned by the caller and kept alive until evo_destroy.
+ * cuda_stream: a cudaStream_t (NULL = default stream).  Enqueues the initialisation (centre,
+ * Adam moments = 0, task constants) on the stream; generation and Adam step start at 0.
+ * Errors: INVALID_ARG (bad config / pointer / alignment), WORKSPACE, UNSUPPORTED, CUDA.
+ */
+evo_status evo_create(const evo_config* cfg, void* d_workspace, size_t workspace_bytes,
+                      void* cuda_stream, evo_solver** out);
+
+/*
+ * ask (paper Section 4, NEAlgorithm.ask; PGPE symmetric sampling, Section 5).  For pair j and
+ * dimension d, eps[j][d] ~ N(0,1) from the counter-based generator at (seed, generation);
+ * theta[2j][d] = fma(+sigma, eps, center[d]), theta[2j+1][d] = fma(-sigma, eps, center[d]).
+ * Returns the device pointer of theta[P][ldD] (fp32, row-major, padding columns zero), which
+ * lives in the workspace and is valid until the next evo_ask, and its row pitch in floats.
+ */
+evo_status evo_ask(evo_solver* s, const float** d_theta, size_t* ld_theta);
+
+/*
+ * rollout (paper Sections 2 and 4: the simulation manager's loop of PolicyNetwork.get_actions
+ * and VectorizedTask.step over the population; supervised learning is a single-step task,
+ * Section 3).  Evaluates all P members of d_theta (NULL = the matrix of the last evo_ask; a
+ * caller matrix must be [P][ldD] with the same pitch, 16-byte aligned) and writes
+ * d_fitness[P] (fp32).  Control tasks: E episodes of T steps per member from seeded initial
+ * states shared by all members; fitness = mean episode return.  Supervised task: fitness =
+ * -mean cross-entropy on the batch bound with evo_set_batch.
+ * d_trace: NULL, or [P][E][trace_steps][state_dim] floats receiving the post-step task state
+ * (state_dim = 4 cart-pole: x, x', theta, theta'; 28 tanh-linear).
+ * Errors: BAD_ORDER (d_theta NULL before any ask; supervised without a batch), INVALID_ARG,
+ * UNSUPPORTED (task NONE), CUDA.
+ */
+evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, float* d_trace);
+
+/*
+ * tell (paper Section 4, NEAlgorithm.tell; Section 2 "Modern ML Optimizers").  With
+ * rank_m = #{k: f_k < f_m or (f_k == f_m and k < m)} and u_m = rank_m/(P-1) - 1/2:
+ *   g[d] = (sigma/P) * sum_j (u[2j] - u[2j+1]) * eps[j][d]
+ *   t += 1;  m = b1 m + (1-b1) g;  v = b2 v + (1-b2) g^2
+ *   center += lr * (m/(1-b1^t)) / (sqrt(v/(1-b2^t)) + adam_eps)          (ascent)
+ * eps is the noise of the matching evo_ask (read back in STORED mode, recomputed from the
+ * counters in REGENERATED mode).  Advances the generation.  A NaN in d_fitness[P] skips the
+ * update (centre, moments, t unchanged) and raises EVO_ERR_NONFINITE at the next
+ * evo_sync_status.  Errors: BAD_ORDER (no ask since the last tell), INVALID_ARG, CUDA.
+ */
+evo_status evo_tell(evo_solver* s, const float* d_fitness);
+
+/* Frees the host handle.  Does not touch the workspace; does not synchronise. */
+evo_status evo_destroy(evo_solver* s);
+
+/* ---- helpers -------------------------------------------------------------------------- */
+
+/* Supervised task: bind the batch scored by every member (paper Section 3, supervised tasks
+ * provide data and labels).  d_images [batch][28][28] fp32, d_labels [batch] int32 in 0..9;
+ * both stay owned by the caller and must outlive the rollouts that use them. */
+evo_status evo_set_batch(evo_solver* s, const float* d_images, const int32_t* d_labels);
+
+/* Device pointers into the workspace (valid for the solver's lifetime): centre, Adam moments,
+ * last gradient (each [ldD] floats, padding zero); ranks [P] int32 and centred-rank weights
+ * [P] fp32 of the last tell; eps[H][ldD] of the last ask (NULL in REGENERATED mode). */
+evo_status evo_get_center (evo_solver* s, const float** d_center);
+evo_status evo_get_moments(evo_solver* s, const float** d_m, const float** d_v);
+evo_status evo_get_gradient(evo_solver* s, const float** d_g);
+evo_status evo_get_ranks  (evo_solver* s, const int32_t** d_rank, const float** d_u);
+evo_status evo_get_eps    (evo_solver* s, const float** d_eps);
+
+/* Checkpoint / resume: counters are (generation, Adam step).  evo_set_state copies D floats
+ * from each non-NULL device pointer into the solver (asynchronously, on the solver's stream)
+ * and sets the counters; the Adam step is read back from the device by evo_get_counters,
+ * which therefore synchronises the stream. */
+evo_status evo_get_counters(evo_solver* s, uint32_t* generation, uint32_t* adam_step);
+evo_status evo_set_state(evo_solver* s, const float* d_center, const float* d_m, const float* d_v,
+                         uint32_t generation, uint32_t adam_step);
+
+/* Waits for the solver's stream, returns and clears the device status (EVO_OK,
+ * EVO_ERR_NONFINITE, EVO_ERR_TIMEOUT) or EVO_ERR_CUDA if the stream reports a fault. */
+evo_status evo_sync_status(evo_solver* s);
+
+/* Number of kernels the library has launched for this solver so far. */
+evo_status evo_launch_count(evo_solver* s, uint64_t* launches);
+
+const char* evo_status_string(evo_status st);
+uint32_t    evo_version(void);            /* major*10000 + minor*100 + patch */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EVO_H */

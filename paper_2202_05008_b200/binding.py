@@ -1,0 +1,236 @@
+"""ctypes binding of ``libevo.so`` (declared in ``include/evo.h``).
+
+Argument marshalling only: every step of ask / rollout / tell runs in the library's CUDA
+kernels.  PyTorch supplies device memory (the workspace, fitness and trace buffers) and the
+stream.  There is no fallback: if the shared library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+from . import workloads as W
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libevo.so")
+
+EVO_MAX_LAYERS = 8
+STATUS = {0: "EVO_OK", 1: "EVO_ERR_INVALID_ARG", 2: "EVO_ERR_BAD_ORDER", 3: "EVO_ERR_WORKSPACE",
+          4: "EVO_ERR_CUDA", 5: "EVO_ERR_NONFINITE", 6: "EVO_ERR_TIMEOUT", 7: "EVO_ERR_UNSUPPORTED"}
+ROLLOUT_AUTO, ROLLOUT_GENERIC, ROLLOUT_TILED = 0, 1, 2
+
+
+class EvoConfig(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("pop_size", C.c_uint32), ("seed", C.c_uint64),
+        ("param_dim", C.c_uint32), ("noise_mode", C.c_uint32),
+        ("sigma", C.c_float), ("lr", C.c_float),
+        ("beta1", C.c_float), ("beta2", C.c_float), ("adam_eps", C.c_float),
+        ("policy_kind", C.c_uint32), ("n_layers", C.c_uint32),
+        ("layer_sizes", C.c_uint32 * (EVO_MAX_LAYERS + 1)), ("action_scale", C.c_float),
+        ("task_kind", C.c_uint32), ("episodes", C.c_uint32), ("horizon", C.c_uint32),
+        ("batch", C.c_uint32), ("trace_steps", C.c_uint32), ("rollout_kernel", C.c_uint32),
+        ("task_param", C.c_float * 16),
+    ]
+
+
+class EvoError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {STATUS.get(code, code)}")
+
+
+_lib = None
+
+
+def load_library():
+    """Loads libevo.so; raises if it has not been built (no CPU fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2202_05008_b200.build`")
+    L = C.CDLL(LIB_PATH)
+    vp, u32p, szp = C.c_void_p, C.POINTER(C.c_uint32), C.POINTER(C.c_size_t)
+    cfgp = C.POINTER(EvoConfig)
+    L.evo_workspace_bytes.argtypes = [cfgp, szp]
+    L.evo_create.argtypes = [cfgp, vp, C.c_size_t, vp, C.POINTER(vp)]
+    L.evo_ask.argtypes = [vp, C.POINTER(vp), szp]
+    L.evo_rollout.argtypes = [vp, vp, vp, vp]
+    L.evo_tell.argtypes = [vp, vp]
+    L.evo_destroy.argtypes = [vp]
+    L.evo_set_batch.argtypes = [vp, vp, vp]
+    L.evo_get_center.argtypes = [vp, C.POINTER(vp)]
+    L.evo_get_moments.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
+    L.evo_get_gradient.argtypes = [vp, C.POINTER(vp)]
+    L.evo_get_ranks.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
+    L.evo_get_eps.argtypes = [vp, C.POINTER(vp)]
+    L.evo_get_counters.argtypes = [vp, u32p, u32p]
+    L.evo_set_state.argtypes = [vp, vp, vp, vp, C.c_uint32, C.c_uint32]
+    L.evo_sync_status.argtypes = [vp]
+    L.evo_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+    L.evo_status_string.argtypes = [C.c_int]
+    L.evo_status_string.restype = C.c_char_p
+    L.evo_version.restype = C.c_uint32
+    for name in ("evo_workspace_bytes", "evo_create", "evo_ask", "evo_rollout", "evo_tell",
+                 "evo_destroy", "evo_set_batch", "evo_get_center", "evo_get_moments",
+                 "evo_get_gradient", "evo_get_ranks", "evo_get_eps", "evo_get_counters",
+                 "evo_set_state", "evo_sync_status", "evo_launch_count"):
+        getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def make_config(w: W.Workload, *, trace_steps: int = 0, rollout_kernel: int = ROLLOUT_AUTO,
+                noise_mode: Optional[int] = None) -> EvoConfig:
+    c = EvoConfig()
+    c.struct_size = C.sizeof(EvoConfig)
+    c.pop_size, c.param_dim, c.seed = w.pop_size, w.param_dim, w.seed
+    c.noise_mode = w.noise_mode if noise_mode is None else noise_mode
+    c.sigma, c.lr = w.sigma, w.lr
+    c.policy_kind = w.policy_kind
+    c.n_layers = max(len(w.layer_sizes) - 1, 0)
+    for i, s in enumerate(w.layer_sizes):
+        c.layer_sizes[i] = s
+    c.action_scale = w.action_scale
+    c.task_kind, c.episodes, c.horizon, c.batch = w.task_kind, w.episodes, w.horizon, w.batch
+    c.trace_steps, c.rollout_kernel = trace_steps, rollout_kernel
+    for i, v in enumerate(w.task_param):
+        c.task_param[i] = v
+    return c
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise EvoError(code, where)
+
+
+class Solver:
+    """One ES solver bound to a CUDA device, a stream and a caller-owned workspace tensor."""
+
+    def __init__(self, workload: W.Workload, device="cuda:0", stream: Optional[torch.cuda.Stream] = None,
+                 **cfg_kw):
+        self.lib = load_library()
+        self.workload = workload
+        self.cfg = make_config(workload, **cfg_kw)
+        self.device = torch.device(device)
+        nbytes = C.c_size_t(0)
+        _check(self.lib.evo_workspace_bytes(C.byref(self.cfg), C.byref(nbytes)), "evo_workspace_bytes")
+        self.workspace_bytes = nbytes.value
+        with torch.cuda.device(self.device):
+            self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.device)
+            base = self.workspace.data_ptr()
+            self._ws_ptr = (base + 255) // 256 * 256
+            h = C.c_void_p()
+            _check(self.lib.evo_create(C.byref(self.cfg), self._ws_ptr, self.workspace_bytes,
+                                       self.stream.cuda_stream, C.byref(h)), "evo_create")
+        self._h = h
+        self.P, self.D = workload.pop_size, workload.param_dim
+        self.ldD = (self.D + 31) // 32 * 32
+        self._batch = None
+
+    # -- the five calls ------------------------------------------------------------------
+    def ask(self) -> torch.Tensor:
+        """theta[P][D] as a strided view (row pitch ldD) of the workspace."""
+        p, ld = C.c_void_p(), C.c_size_t()
+        _check(self.lib.evo_ask(self._h, C.byref(p), C.byref(ld)), "evo_ask")
+        return self._view_f32(p.value, self.P, ld.value)[:, :self.D]
+
+    def rollout(self, theta: Optional[torch.Tensor] = None, fitness: Optional[torch.Tensor] = None,
+                trace: Optional[torch.Tensor] = None) -> torch.Tensor:
+        if fitness is None:
+            fitness = torch.empty(self.P, dtype=torch.float32, device=self.device)
+        tp = None
+        if theta is not None:
+            assert theta.dtype == torch.float32 and theta.is_cuda and theta.stride(1) == 1
+            assert theta.shape[0] == self.P and theta.stride(0) == self.ldD
+            tp = theta.data_ptr()
+        _check(self.lib.evo_rollout(self._h, tp, fitness.data_ptr(),
+                                    None if trace is None else trace.data_ptr()), "evo_rollout")
+        return fitness
+
+    def tell(self, fitness: torch.Tensor) -> None:
+        assert fitness.dtype == torch.float32 and fitness.is_cuda and fitness.numel() == self.P
+        _check(self.lib.evo_tell(self._h, fitness.data_ptr()), "evo_tell")
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None:
+            self.lib.evo_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    # -- helpers -------------------------------------------------------------------------
+    def set_batch(self, images: torch.Tensor, labels: torch.Tensor) -> None:
+        assert images.dtype == torch.float32 and images.is_cuda and images.is_contiguous()
+        assert labels.dtype == torch.int32 and labels.is_cuda and labels.is_contiguous()
+        self._batch = (images, labels)           # keep alive
+        _check(self.lib.evo_set_batch(self._h, images.data_ptr(), labels.data_ptr()), "evo_set_batch")
+
+    def padded_rows(self, rows: int) -> torch.Tensor:
+        """A zeroed [rows][ldD] device matrix with the pitch evo_rollout expects."""
+        return torch.zeros(rows, self.ldD, dtype=torch.float32, device=self.device)
+
+    def _view_f32(self, ptr: int, rows: int, cols: int) -> torch.Tensor:
+        off = ptr - self.workspace.data_ptr()
+        flat = self.workspace[off:off + rows * cols * 4].view(torch.float32)
+        return flat.view(rows, cols)
+
+    def _view_i32(self, ptr: int, n: int) -> torch.Tensor:
+        off = ptr - self.workspace.data_ptr()
+        return self.workspace[off:off + n * 4].view(torch.int32)
+
+    def center(self) -> torch.Tensor:
+        p = C.c_void_p()
+        _check(self.lib.evo_get_center(self._h, C.byref(p)), "evo_get_center")
+        return self._view_f32(p.value, 1, self.ldD)[0, :self.D]
+
+    def moments(self):
+        m, v = C.c_void_p(), C.c_void_p()
+        _check(self.lib.evo_get_moments(self._h, C.byref(m), C.byref(v)), "evo_get_moments")
+        return (self._view_f32(m.value, 1, self.ldD)[0, :self.D],
+                self._view_f32(v.value, 1, self.ldD)[0, :self.D])
+
+    def gradient(self) -> torch.Tensor:
+        p = C.c_void_p()
+        _check(self.lib.evo_get_gradient(self._h, C.byref(p)), "evo_get_gradient")
+        return self._view_f32(p.value, 1, self.ldD)[0, :self.D]
+
+    def ranks(self):
+        r, u = C.c_void_p(), C.c_void_p()
+        _check(self.lib.evo_get_ranks(self._h, C.byref(r), C.byref(u)), "evo_get_ranks")
+        return self._view_i32(r.value, self.P), self._view_f32(u.value, 1, self.P)[0]
+
+    def eps(self) -> Optional[torch.Tensor]:
+        p = C.c_void_p()
+        _check(self.lib.evo_get_eps(self._h, C.byref(p)), "evo_get_eps")
+        if not p.value:
+            return None
+        return self._view_f32(p.value, self.P // 2, self.ldD)[:, :self.D]
+
+    def counters(self):
+        g, t = C.c_uint32(), C.c_uint32()
+        _check(self.lib.evo_get_counters(self._h, C.byref(g), C.byref(t)), "evo_get_counters")
+        return g.value, t.value
+
+    def set_state(self, center=None, m=None, v=None, generation=0, adam_step=0) -> None:
+        def ptr(x):
+            if x is None:
+                return None
+            assert x.dtype == torch.float32 and x.is_cuda and x.is_contiguous() and x.numel() == self.D
+            return x.data_ptr()
+        _check(self.lib.evo_set_state(self._h, ptr(center), ptr(m), ptr(v), generation, adam_step),
+               "evo_set_state")
+
+    def sync_status(self) -> int:
+        return self.lib.evo_sync_status(self._h)
+
+    def launch_count(self) -> int:
+        n = C.c_uint64()
+        _check(self.lib.evo_launch_count(self._h, C.byref(n)), "evo_launch_count")
+        return n.value

@@ -1,0 +1,369 @@
+// Host side of the C-ABI declared in include/evo.h: argument checks, workspace layout and
+// kernel launches.  No device memory is allocated here; nothing synchronises except
+// evo_sync_status / evo_get_counters.
+#include "internal.h"
+
+#include <cmath>
+#include <cstring>
+#include <new>
+
+using namespace evo;
+
+struct evo_solver {
+    evo_config   cfg;
+    Layout       lay;
+    char*        ws;
+    cudaStream_t stream;
+    uint32_t     generation;
+    bool         asked;            // an ask without a matching tell is outstanding
+    bool         ever_asked;
+    const float*   d_images;
+    const int32_t* d_labels;
+    uint64_t     launches;
+    uint32_t     k0, k1;
+};
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static evo_status check_config(const evo_config* c)
+{
+    if (!c || c->struct_size != sizeof(evo_config)) return EVO_ERR_INVALID_ARG;
+    if (c->pop_size < 2 || (c->pop_size & 1u) || c->param_dim < 1) return EVO_ERR_INVALID_ARG;
+    if (!(c->sigma > 0.f) || !std::isfinite(c->sigma) || !std::isfinite(c->lr)) return EVO_ERR_INVALID_ARG;
+    if (c->noise_mode > EVO_NOISE_REGENERATED) return EVO_ERR_INVALID_ARG;
+    if (c->beta1 < 0.f || c->beta1 >= 1.f || c->beta2 < 0.f || c->beta2 >= 1.f || c->adam_eps < 0.f)
+        return EVO_ERR_INVALID_ARG;
+    if (c->rollout_kernel > EVO_ROLLOUT_TILED) return EVO_ERR_INVALID_ARG;
+    switch (c->task_kind) {
+        case EVO_TASK_NONE: break;
+        case EVO_TASK_CARTPOLE:
+        case EVO_TASK_TANH_LINEAR:
+            if (c->policy_kind != EVO_POLICY_MLP) return EVO_ERR_INVALID_ARG;
+            if (c->episodes < 1 || c->horizon < 1) return EVO_ERR_INVALID_ARG;
+            if (!rollout_mlp_supported(*c)) return EVO_ERR_INVALID_ARG;
+            if (c->task_kind == EVO_TASK_CARTPOLE) {
+                const float* tp = c->task_param;
+                if (!(tp[EVO_CP_CART_MASS] > 0.f) || !(tp[EVO_CP_POLE_MASS] > 0.f) ||
+                    !(tp[EVO_CP_POLE_HALF_LENGTH] > 0.f) || !(tp[EVO_CP_DT] > 0.f) ||
+                    !(tp[EVO_CP_INIT_RANGE] >= 0.f))
+                    return EVO_ERR_INVALID_ARG;
+            }
+            break;
+        case EVO_TASK_SUPERVISED:
+            if (c->policy_kind != EVO_POLICY_CNN_28 || c->param_dim != kCnnParams || c->batch < 1)
+                return EVO_ERR_INVALID_ARG;
+            break;
+        default: return EVO_ERR_INVALID_ARG;
+    }
+    return EVO_OK;
+}
+
+static evo_status make_layout(const evo_config& c, Layout* L)
+{
+    const size_t P = c.pop_size, H = P / 2;
+    const uint32_t ldD = static_cast<uint32_t>(align_up(c.param_dim, 32));
+    L->ldD = ldD;
+    L->grad_splits = gradient_splits(static_cast<uint32_t>(H), ldD);
+    L->EB = 1; L->n_eb = 1;
+    if (c.task_kind == EVO_TASK_CARTPOLE || c.task_kind == EVO_TASK_TANH_LINEAR)
+        rollout_mlp_plan(c, &L->EB, &L->n_eb);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t row = static_cast<size_t>(ldD) * sizeof(float);
+    L->status = take(sizeof(DeviceStatus));
+    L->center = take(row);
+    L->m = take(row);
+    L->v = take(row);
+    L->g = take(row);
+    L->u = take(P * sizeof(float));
+    L->rank = take(P * sizeof(int32_t));
+    L->grad_partial = take(row * L->grad_splits);
+    L->fit_partial = take(P * L->n_eb * sizeof(float));
+    L->task_const = take(kTlNx * (kTlNx + kTlNa) * sizeof(float));
+    L->cnn_scratch = take(c.task_kind == EVO_TASK_SUPERVISED ? cnn_scratch_bytes(c.pop_size, c.batch) : 0);
+    L->theta = take(row * P);
+    L->eps = take(c.noise_mode == EVO_NOISE_STORED ? row * H : 0);
+    L->total = off;
+    return EVO_OK;
+}
+
+extern "C" {
+
+evo_status evo_workspace_bytes(const evo_config* cfg, size_t* bytes)
+{
+    if (!bytes) return EVO_ERR_INVALID_ARG;
+    evo_status st = check_config(cfg);
+    if (st != EVO_OK) return st;
+    Layout L;
+    make_layout(*cfg, &L);
+    *bytes = L.total;
+    return EVO_OK;
+}
+
+evo_status evo_create(const evo_config* cfg_in, void* d_workspace, size_t workspace_bytes,
+                      void* cuda_stream, evo_solver** out)
+{
+    if (!out) return EVO_ERR_INVALID_ARG;
+    *out = nullptr;
+    evo_status st = check_config(cfg_in);
+    if (st != EVO_OK) return st;
+    if (!d_workspace || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return EVO_ERR_INVALID_ARG;
+    evo_solver* s = new (std::nothrow) evo_solver();
+    if (!s) return EVO_ERR_INVALID_ARG;
+    s->cfg = *cfg_in;
+    if (s->cfg.beta1 == 0.f) s->cfg.beta1 = 0.9f;
+    if (s->cfg.beta2 == 0.f) s->cfg.beta2 = 0.999f;
+    if (s->cfg.adam_eps == 0.f) s->cfg.adam_eps = 1e-8f;
+    make_layout(s->cfg, &s->lay);
+    if (workspace_bytes < s->lay.total) { delete s; return EVO_ERR_WORKSPACE; }
+    s->ws = static_cast<char*>(d_workspace);
+    s->stream = static_cast<cudaStream_t>(cuda_stream);
+    s->generation = 0;
+    s->asked = false;
+    s->ever_asked = false;
+    s->d_images = nullptr;
+    s->d_labels = nullptr;
+    s->launches = 0;
+    s->k0 = static_cast<uint32_t>(s->cfg.seed & 0xFFFFFFFFull);
+    s->k1 = static_cast<uint32_t>(s->cfg.seed >> 32);
+    const Layout& L = s->lay;
+    int n = launch_init(s->stream, reinterpret_cast<float*>(s->ws + L.center),
+                        reinterpret_cast<float*>(s->ws + L.m), reinterpret_cast<float*>(s->ws + L.v),
+                        reinterpret_cast<float*>(s->ws + L.g), L.ldD,
+                        reinterpret_cast<DeviceStatus*>(s->ws + L.status));
+    if (n < 0) { delete s; return EVO_ERR_CUDA; }
+    s->launches += n;
+    n = launch_task_constants(s->stream, s->cfg.task_kind, s->k0, s->k1,
+                              reinterpret_cast<float*>(s->ws + L.task_const));
+    if (n < 0) { delete s; return EVO_ERR_CUDA; }
+    s->launches += n;
+    *out = s;
+    return EVO_OK;
+}
+
+evo_status evo_ask(evo_solver* s, const float** d_theta, size_t* ld_theta)
+{
+    if (!s) return EVO_ERR_INVALID_ARG;
+    const Layout& L = s->lay;
+    float* theta = reinterpret_cast<float*>(s->ws + L.theta);
+    float* eps = s->cfg.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<float*>(s->ws + L.eps) : nullptr;
+    const int n = launch_ask(s->stream, reinterpret_cast<const float*>(s->ws + L.center), s->cfg.sigma,
+                             s->k0, s->k1, s->generation, s->cfg.pop_size / 2, s->cfg.param_dim, L.ldD,
+                             theta, eps);
+    if (n < 0) return EVO_ERR_CUDA;
+    s->launches += n;
+    s->asked = true;
+    s->ever_asked = true;
+    if (d_theta) *d_theta = theta;
+    if (ld_theta) *ld_theta = L.ldD;
+    return EVO_OK;
+}
+
+evo_status evo_set_batch(evo_solver* s, const float* d_images, const int32_t* d_labels)
+{
+    if (!s || !d_images || !d_labels) return EVO_ERR_INVALID_ARG;
+    if (s->cfg.task_kind != EVO_TASK_SUPERVISED) return EVO_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(d_images) & 15u) return EVO_ERR_INVALID_ARG;
+    s->d_images = d_images;
+    s->d_labels = d_labels;
+    return EVO_OK;
+}
+
+evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, float* d_trace)
+{
+    if (!s || !d_fitness) return EVO_ERR_INVALID_ARG;
+    const evo_config& c = s->cfg;
+    const Layout& L = s->lay;
+    if (c.task_kind == EVO_TASK_NONE) return EVO_ERR_UNSUPPORTED;
+    if (!d_theta) {
+        if (!s->ever_asked) return EVO_ERR_BAD_ORDER;
+        d_theta = reinterpret_cast<const float*>(s->ws + L.theta);
+    } else if (reinterpret_cast<uintptr_t>(d_theta) & 15u) {
+        return EVO_ERR_INVALID_ARG;
+    }
+    if (c.task_kind == EVO_TASK_SUPERVISED) {
+        if (!s->d_images) return EVO_ERR_BAD_ORDER;
+        if (d_trace) return EVO_ERR_UNSUPPORTED;
+        const int n = launch_rollout_cnn(s->stream, d_theta, L.ldD, c.pop_size, s->d_images, s->d_labels,
+                                         c.batch, s->ws + L.cnn_scratch, d_fitness);
+        if (n < 0) return n == -2 ? EVO_ERR_UNSUPPORTED : EVO_ERR_CUDA;
+        s->launches += n;
+        return EVO_OK;
+    }
+    if (d_trace && c.trace_steps == 0) return EVO_ERR_INVALID_ARG;
+    RolloutMlpArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.theta = d_theta;
+    a.fit_partial = reinterpret_cast<float*>(s->ws + L.fit_partial);
+    a.trace = d_trace;
+    a.task_const = reinterpret_cast<const float*>(s->ws + L.task_const);
+    a.P = c.pop_size;
+    a.ldD = L.ldD;
+    a.n_layers = c.n_layers;
+    a.max_width = 0;
+    for (uint32_t l = 0; l <= c.n_layers; ++l) {
+        a.sizes[l] = c.layer_sizes[l];
+        if (c.layer_sizes[l] > a.max_width) a.max_width = c.layer_sizes[l];
+    }
+    a.action_scale = c.action_scale;
+    a.task = c.task_kind;
+    a.E = c.episodes; a.T = c.horizon; a.EB = L.EB; a.n_eb = L.n_eb;
+    a.trace_T = c.trace_steps < c.horizon ? c.trace_steps : c.horizon;
+    a.k0 = s->k0; a.k1 = s->k1; a.generation = s->generation;
+    std::memcpy(a.tp, c.task_param, sizeof(a.tp));
+    const int n = launch_rollout_mlp(s->stream, a, c.rollout_kernel, d_fitness);
+    if (n < 0) return n == -2 ? EVO_ERR_UNSUPPORTED : EVO_ERR_CUDA;
+    s->launches += n;
+    return EVO_OK;
+}
+
+evo_status evo_tell(evo_solver* s, const float* d_fitness)
+{
+    if (!s || !d_fitness) return EVO_ERR_INVALID_ARG;
+    if (!s->asked) return EVO_ERR_BAD_ORDER;
+    const evo_config& c = s->cfg;
+    const Layout& L = s->lay;
+    DeviceStatus* status = reinterpret_cast<DeviceStatus*>(s->ws + L.status);
+    float* u = reinterpret_cast<float*>(s->ws + L.u);
+    int n = launch_rank(s->stream, d_fitness, c.pop_size, reinterpret_cast<int32_t*>(s->ws + L.rank), u,
+                        status);
+    if (n < 0) return EVO_ERR_CUDA;
+    s->launches += n;
+    const float* eps = c.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<const float*>(s->ws + L.eps)
+                                                        : nullptr;
+    n = launch_gradient_adam(s->stream, u, eps, s->k0, s->k1, s->generation, c.pop_size / 2, c.param_dim,
+                             L.ldD, L.grad_splits, reinterpret_cast<float*>(s->ws + L.grad_partial),
+                             c.sigma, c.lr, c.beta1, c.beta2, c.adam_eps,
+                             reinterpret_cast<float*>(s->ws + L.center),
+                             reinterpret_cast<float*>(s->ws + L.m), reinterpret_cast<float*>(s->ws + L.v),
+                             reinterpret_cast<float*>(s->ws + L.g), status);
+    if (n < 0) return EVO_ERR_CUDA;
+    s->launches += n;
+    s->asked = false;
+    s->generation += 1;
+    return EVO_OK;
+}
+
+evo_status evo_destroy(evo_solver* s)
+{
+    if (!s) return EVO_ERR_INVALID_ARG;
+    delete s;
+    return EVO_OK;
+}
+
+evo_status evo_get_center(evo_solver* s, const float** d_center)
+{
+    if (!s || !d_center) return EVO_ERR_INVALID_ARG;
+    *d_center = reinterpret_cast<const float*>(s->ws + s->lay.center);
+    return EVO_OK;
+}
+
+evo_status evo_get_moments(evo_solver* s, const float** d_m, const float** d_v)
+{
+    if (!s || !d_m || !d_v) return EVO_ERR_INVALID_ARG;
+    *d_m = reinterpret_cast<const float*>(s->ws + s->lay.m);
+    *d_v = reinterpret_cast<const float*>(s->ws + s->lay.v);
+    return EVO_OK;
+}
+
+evo_status evo_get_gradient(evo_solver* s, const float** d_g)
+{
+    if (!s || !d_g) return EVO_ERR_INVALID_ARG;
+    *d_g = reinterpret_cast<const float*>(s->ws + s->lay.g);
+    return EVO_OK;
+}
+
+evo_status evo_get_ranks(evo_solver* s, const int32_t** d_rank, const float** d_u)
+{
+    if (!s || !d_rank || !d_u) return EVO_ERR_INVALID_ARG;
+    *d_rank = reinterpret_cast<const int32_t*>(s->ws + s->lay.rank);
+    *d_u = reinterpret_cast<const float*>(s->ws + s->lay.u);
+    return EVO_OK;
+}
+
+evo_status evo_get_eps(evo_solver* s, const float** d_eps)
+{
+    if (!s || !d_eps) return EVO_ERR_INVALID_ARG;
+    *d_eps = s->cfg.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<const float*>(s->ws + s->lay.eps)
+                                                   : nullptr;
+    return EVO_OK;
+}
+
+evo_status evo_get_counters(evo_solver* s, uint32_t* generation, uint32_t* adam_step)
+{
+    if (!s || !generation || !adam_step) return EVO_ERR_INVALID_ARG;
+    DeviceStatus h;
+    if (cudaMemcpyAsync(&h, s->ws + s->lay.status, sizeof(h), cudaMemcpyDeviceToHost, s->stream) != cudaSuccess)
+        return EVO_ERR_CUDA;
+    if (cudaStreamSynchronize(s->stream) != cudaSuccess) return EVO_ERR_CUDA;
+    *generation = s->generation;
+    *adam_step = h.adam_step;
+    return EVO_OK;
+}
+
+evo_status evo_set_state(evo_solver* s, const float* d_center, const float* d_m, const float* d_v,
+                         uint32_t generation, uint32_t adam_step)
+{
+    if (!s) return EVO_ERR_INVALID_ARG;
+    const size_t bytes = static_cast<size_t>(s->cfg.param_dim) * sizeof(float);
+    const Layout& L = s->lay;
+    if (d_center && cudaMemcpyAsync(s->ws + L.center, d_center, bytes, cudaMemcpyDeviceToDevice, s->stream) != cudaSuccess)
+        return EVO_ERR_CUDA;
+    if (d_m && cudaMemcpyAsync(s->ws + L.m, d_m, bytes, cudaMemcpyDeviceToDevice, s->stream) != cudaSuccess)
+        return EVO_ERR_CUDA;
+    if (d_v && cudaMemcpyAsync(s->ws + L.v, d_v, bytes, cudaMemcpyDeviceToDevice, s->stream) != cudaSuccess)
+        return EVO_ERR_CUDA;
+    if (cudaMemcpyAsync(s->ws + L.status + offsetof(DeviceStatus, adam_step), &adam_step, sizeof(uint32_t),
+                        cudaMemcpyHostToDevice, s->stream) != cudaSuccess)
+        return EVO_ERR_CUDA;
+    if (cudaStreamSynchronize(s->stream) != cudaSuccess) return EVO_ERR_CUDA;   // adam_step is a stack value
+    s->generation = generation;
+    s->asked = false;
+    return EVO_OK;
+}
+
+evo_status evo_sync_status(evo_solver* s)
+{
+    if (!s) return EVO_ERR_INVALID_ARG;
+    DeviceStatus h;
+    if (cudaMemcpyAsync(&h, s->ws + s->lay.status, sizeof(h), cudaMemcpyDeviceToHost, s->stream) != cudaSuccess)
+        return EVO_ERR_CUDA;
+    if (cudaStreamSynchronize(s->stream) != cudaSuccess) return EVO_ERR_CUDA;
+    if (h.sticky) {
+        const uint32_t zero = 0;
+        if (cudaMemcpyAsync(s->ws + s->lay.status + offsetof(DeviceStatus, sticky), &zero, sizeof(zero),
+                            cudaMemcpyHostToDevice, s->stream) != cudaSuccess)
+            return EVO_ERR_CUDA;
+        if (cudaStreamSynchronize(s->stream) != cudaSuccess) return EVO_ERR_CUDA;
+        if (h.sticky & (1u << EVO_ERR_TIMEOUT)) return EVO_ERR_TIMEOUT;
+        if (h.sticky & (1u << EVO_ERR_NONFINITE)) return EVO_ERR_NONFINITE;
+        return EVO_ERR_CUDA;
+    }
+    return EVO_OK;
+}
+
+evo_status evo_launch_count(evo_solver* s, uint64_t* launches)
+{
+    if (!s || !launches) return EVO_ERR_INVALID_ARG;
+    *launches = s->launches;
+    return EVO_OK;
+}
+
+const char* evo_status_string(evo_status st)
+{
+    switch (st) {
+        case EVO_OK: return "ok";
+        case EVO_ERR_INVALID_ARG: return "invalid argument";
+        case EVO_ERR_BAD_ORDER: return "call out of order";
+        case EVO_ERR_WORKSPACE: return "workspace too small";
+        case EVO_ERR_CUDA: return "CUDA error";
+        case EVO_ERR_NONFINITE: return "non-finite fitness, update skipped";
+        case EVO_ERR_TIMEOUT: return "device-side wait timed out";
+        case EVO_ERR_UNSUPPORTED: return "unsupported configuration";
+    }
+    return "unknown status";
+}
+
+uint32_t evo_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,72 @@
+// Internal declarations shared by the host API (evo.cu) and the kernel files.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/evo.h"
+
+namespace evo {
+
+// Device-resident control block at the start of the workspace.
+struct DeviceStatus {
+    uint32_t sticky;        // OR of (1u << evo_status) for conditions raised on the device
+    uint32_t nonfinite;     // set by the rank kernel of the current tell, cleared by its finish
+    uint32_t adam_step;     // t
+    uint32_t pad;
+};
+
+constexpr uint32_t kTlNx = 28;   // tanh-linear task: state width
+constexpr uint32_t kTlNa = 8;    // tanh-linear task: action width
+constexpr uint32_t kCnnParams = 5994;
+
+struct RolloutMlpArgs {
+    const float* theta;          // [P][ldD]
+    float*       fit_partial;    // [P][n_episode_blocks] sums of episode returns
+    float*       trace;          // nullable
+    const float* task_const;     // tanh-linear: A[28][28] then B[28][8]
+    uint32_t P, ldD;
+    uint32_t n_layers;
+    uint32_t sizes[EVO_MAX_LAYERS + 1];
+    uint32_t max_width;
+    float    action_scale;
+    uint32_t task;
+    uint32_t E, T, EB, n_eb;     // episodes, horizon, episodes per block, blocks per member
+    uint32_t trace_T;
+    uint32_t k0, k1, generation;
+    float    tp[16];
+    uint32_t weights_in_smem;
+};
+
+struct Layout {                  // byte offsets into the workspace
+    size_t status, center, m, v, g, theta, eps, u, rank, grad_partial, fit_partial, task_const,
+           cnn_scratch, total;
+    uint32_t ldD, grad_splits, n_eb, EB;
+};
+
+// ---- launchers (each returns the number of kernels it launched, or -1 on a launch error) ----
+int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, uint32_t ldD,
+                DeviceStatus* status);
+int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t k1, float* task_const);
+int launch_ask(cudaStream_t st, const float* center, float sigma, uint32_t k0, uint32_t k1,
+               uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, float* theta, float* eps);
+int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank, float* u,
+                DeviceStatus* status);
+int launch_gradient_adam(cudaStream_t st, const float* u, const float* eps /*NULL = regenerate*/,
+                         uint32_t k0, uint32_t k1, uint32_t generation, uint32_t H, uint32_t D,
+                         uint32_t ldD, uint32_t splits, float* partial, float sigma, float lr,
+                         float beta1, float beta2, float adam_eps, float* center, float* m, float* v,
+                         float* g, DeviceStatus* status);
+uint32_t gradient_splits(uint32_t H, uint32_t ldD);
+
+int  launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a, uint32_t kernel_choice,
+                        float* fitness);
+bool rollout_mlp_supported(const evo_config& cfg);
+void rollout_mlp_plan(const evo_config& cfg, uint32_t* EB, uint32_t* n_eb);
+
+size_t cnn_scratch_bytes(uint32_t P, uint32_t batch);
+int launch_rollout_cnn(cudaStream_t st, const float* theta, uint32_t ldD, uint32_t P,
+                       const float* images, const int32_t* labels, uint32_t batch, void* scratch,
+                       float* fitness);
+
+}  // namespace evo

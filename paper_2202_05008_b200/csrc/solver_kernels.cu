@@ -1,0 +1,292 @@
+// Solver kernels: ask (antithetic sampling), centred rank, ES gradient (stored or regenerated
+// noise) and the Adam ascent step.  Paper Section 4 (NEAlgorithm ask / tell), Section 2
+// ("Modern ML Optimizers"); the algorithm is PGPE with symmetric sampling (Section 5).
+#include "internal.h"
+#include "noise.cuh"
+
+namespace evo {
+
+// ------------------------------------------------------------------------------------------
+// init / task constants
+// ------------------------------------------------------------------------------------------
+__global__ void k_init(float* center, float* m, float* v, float* g, uint32_t ldD, DeviceStatus* status)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < ldD) { center[i] = 0.f; m[i] = 0.f; v[i] = 0.f; g[i] = 0.f; }
+    if (i == 0) { status->sticky = 0; status->nonfinite = 0; status->adam_step = 0; status->pad = 0; }
+}
+
+int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, uint32_t ldD,
+                DeviceStatus* status)
+{
+    k_init<<<(ldD + 255) / 256, 256, 0, st>>>(center, m, v, g, ldD, status);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+// Tanh-linear task constants: A[28][28] = z * fp32(0.9/sqrt(28)), B[28][8] = z * fp32(1/sqrt(8)),
+// z from stream 4 (row 0 = A, row 1 = B), generation 0.
+__global__ void k_tanh_linear_constants(PhiloxKey key, float* out)
+{
+    const uint32_t quad = threadIdx.x;
+    constexpr uint32_t qa = kTlNx * kTlNx / 4, qb = kTlNx * kTlNa / 4;
+    if (quad < qa) {
+        const float4 z = stream_normal4(key, 4u, 0u, 0u, quad);
+        const float sc = __uint_as_float(0x3E2E2A81u);
+        float4 r = make_float4(__fmul_rn(z.x, sc), __fmul_rn(z.y, sc), __fmul_rn(z.z, sc), __fmul_rn(z.w, sc));
+        reinterpret_cast<float4*>(out)[quad] = r;
+    } else if (quad < qa + qb) {
+        const float4 z = stream_normal4(key, 4u, 0u, 1u, quad - qa);
+        const float sc = __uint_as_float(0x3EB504F3u);
+        float4 r = make_float4(__fmul_rn(z.x, sc), __fmul_rn(z.y, sc), __fmul_rn(z.z, sc), __fmul_rn(z.w, sc));
+        reinterpret_cast<float4*>(out)[quad] = r;
+    }
+}
+
+int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t k1, float* task_const)
+{
+    if (task != EVO_TASK_TANH_LINEAR) return 0;
+    k_tanh_linear_constants<<<1, 256, 0, st>>>(PhiloxKey{k0, k1}, task_const);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+// ------------------------------------------------------------------------------------------
+// ask: one thread per (column quad, chunk of pairs).  Writes are 128-bit and coalesced along
+// the row; the centre quad is loaded once per thread and reused for all pairs of the chunk.
+// ------------------------------------------------------------------------------------------
+constexpr uint32_t kAskPairsPerThread = 8;
+
+__global__ void __launch_bounds__(256)
+k_ask(const float* __restrict__ center, float sigma, PhiloxKey key, uint32_t generation,
+      uint32_t H, uint32_t D, uint32_t ldD, float* __restrict__ theta, float* __restrict__ eps)
+{
+    const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
+    if (quad * 4u >= ldD) return;
+    const uint32_t d0 = quad * 4u;
+    const float4 c = reinterpret_cast<const float4*>(center)[quad];
+    const float nsigma = -sigma;
+    const bool full = d0 + 4u <= D;
+    for (uint32_t j = blockIdx.y * kAskPairsPerThread; j < H; j += gridDim.y * kAskPairsPerThread) {
+        const uint32_t jend = min(j + kAskPairsPerThread, H);
+        for (uint32_t jj = j; jj < jend; ++jj) {
+            float4 z = stream_normal4(key, 0u, generation, jj, quad);
+            if (!full) {                       // ragged tail and padding columns carry zeros
+                if (d0 + 0u >= D) z.x = 0.f;
+                if (d0 + 1u >= D) z.y = 0.f;
+                if (d0 + 2u >= D) z.z = 0.f;
+                if (d0 + 3u >= D) z.w = 0.f;
+            }
+            const float4 tp = make_float4(__fmaf_rn(sigma, z.x, c.x), __fmaf_rn(sigma, z.y, c.y),
+                                          __fmaf_rn(sigma, z.z, c.z), __fmaf_rn(sigma, z.w, c.w));
+            const float4 tm = make_float4(__fmaf_rn(nsigma, z.x, c.x), __fmaf_rn(nsigma, z.y, c.y),
+                                          __fmaf_rn(nsigma, z.z, c.z), __fmaf_rn(nsigma, z.w, c.w));
+            float* row = theta + static_cast<size_t>(2u * jj) * ldD + d0;
+            __stcs(reinterpret_cast<float4*>(row), tp);
+            __stcs(reinterpret_cast<float4*>(row + ldD), tm);
+            if (eps) __stcs(reinterpret_cast<float4*>(eps + static_cast<size_t>(jj) * ldD + d0), z);
+        }
+    }
+}
+
+int launch_ask(cudaStream_t st, const float* center, float sigma, uint32_t k0, uint32_t k1,
+               uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, float* theta, float* eps)
+{
+    const uint32_t quads = ldD / 4u;
+    dim3 grid((quads + 255u) / 256u, (H + kAskPairsPerThread - 1u) / kAskPairsPerThread);
+    if (grid.y > 65535u) grid.y = 65535u;
+    k_ask<<<grid, 256, 0, st>>>(center, sigma, PhiloxKey{k0, k1}, generation, H, D, ldD, theta, eps);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+// ------------------------------------------------------------------------------------------
+// centred rank by counting: rank_m = #{k : f_k < f_m or (f_k == f_m and k < m)}
+// ------------------------------------------------------------------------------------------
+constexpr uint32_t kRankTile = 2048;
+
+__global__ void __launch_bounds__(256)
+k_rank(const float* __restrict__ fitness, uint32_t P, int32_t* __restrict__ rank,
+       float* __restrict__ u, DeviceStatus* status)
+{
+    __shared__ float tile[kRankTile];
+    const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
+    const float fm = (m < P) ? fitness[m] : 0.f;
+    if (m < P && fm != fm) atomicOr(&status->nonfinite, 1u);
+    uint32_t below = 0;
+    for (uint32_t base = 0; base < P; base += kRankTile) {
+        const uint32_t n = min(kRankTile, P - base);
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) tile[i] = fitness[base + i];
+        __syncthreads();
+        if (m < P) {
+            for (uint32_t i = 0; i < n; ++i) {
+                const float fk = tile[i];
+                below += (fk < fm || (fk == fm && base + i < m)) ? 1u : 0u;
+            }
+        }
+    }
+    if (m < P) {
+        rank[m] = static_cast<int32_t>(below);
+        u[m] = __fadd_rn(__fdiv_rn(__uint2float_rn(below), __uint2float_rn(P - 1u)), -0.5f);
+    }
+}
+
+int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank, float* u,
+                DeviceStatus* status)
+{
+    k_rank<<<(P + 255u) / 256u, 256, 0, st>>>(fitness, P, rank, u, status);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+// ------------------------------------------------------------------------------------------
+// ES gradient.  partial[s][d] = sum over the pairs of split s of (u[2j]-u[2j+1]) * eps[j][d],
+// one thread per column quad, fixed summation order (four interleaved accumulators combined
+// as (a0+a1)+(a2+a3)); no floating-point atomics anywhere, so results are run-to-run identical.
+// REGEN recomputes eps from the Philox counters instead of reading it.
+// ------------------------------------------------------------------------------------------
+template <bool REGEN>
+__global__ void __launch_bounds__(128)
+k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, PhiloxKey key,
+               uint32_t generation, uint32_t H, uint32_t ldD, uint32_t pairs_per_split,
+               float* __restrict__ partial, const DeviceStatus* status)
+{
+    if (status->nonfinite) return;
+    const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
+    if (quad * 4u >= ldD) return;
+    const uint32_t j0 = blockIdx.y * pairs_per_split;
+    const uint32_t j1 = min(H, j0 + pairs_per_split);
+    float4 acc[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float2* up = reinterpret_cast<const float2*>(u);
+    uint32_t j = j0;
+    for (; j + 4u <= j1; j += 4u) {
+        float4 e[4];
+        float w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (REGEN) e[i] = stream_normal4(key, 0u, generation, j + i, quad);
+            else e[i] = __ldcs(reinterpret_cast<const float4*>(eps + static_cast<size_t>(j + i) * ldD) + quad);
+            const float2 uu = __ldg(up + j + i);
+            w[i] = uu.x - uu.y;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            acc[i].x = fmaf(w[i], e[i].x, acc[i].x);
+            acc[i].y = fmaf(w[i], e[i].y, acc[i].y);
+            acc[i].z = fmaf(w[i], e[i].z, acc[i].z);
+            acc[i].w = fmaf(w[i], e[i].w, acc[i].w);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {                  // tail keeps the accumulator assignment j % 4
+        if (j + i < j1) {
+            float4 e;
+            if (REGEN) e = stream_normal4(key, 0u, generation, j + i, quad);
+            else e = __ldcs(reinterpret_cast<const float4*>(eps + static_cast<size_t>(j + i) * ldD) + quad);
+            const float2 uu = __ldg(up + j + i);
+            const float w = uu.x - uu.y;
+            acc[i].x = fmaf(w, e.x, acc[i].x);
+            acc[i].y = fmaf(w, e.y, acc[i].y);
+            acc[i].z = fmaf(w, e.z, acc[i].z);
+            acc[i].w = fmaf(w, e.w, acc[i].w);
+        }
+    }
+    float4 r;
+    r.x = (acc[0].x + acc[1].x) + (acc[2].x + acc[3].x);
+    r.y = (acc[0].y + acc[1].y) + (acc[2].y + acc[3].y);
+    r.z = (acc[0].z + acc[1].z) + (acc[2].z + acc[3].z);
+    r.w = (acc[0].w + acc[1].w) + (acc[2].w + acc[3].w);
+    reinterpret_cast<float4*>(partial + static_cast<size_t>(blockIdx.y) * ldD)[quad] = r;
+}
+
+// Sum the splits in order, scale, and take the Adam ascent step in place.
+__global__ void __launch_bounds__(256)
+k_adam(const float* __restrict__ partial, uint32_t splits, uint32_t ldD, float scale, float lr,
+       float beta1, float beta2, float adam_eps, float* __restrict__ center, float* __restrict__ m,
+       float* __restrict__ v, float* __restrict__ g, const DeviceStatus* status)
+{
+    if (status->nonfinite) return;
+    __shared__ float corr[2];
+    if (threadIdx.x == 0) {
+        const double t = static_cast<double>(status->adam_step + 1u);
+        corr[0] = static_cast<float>(1.0 / (1.0 - pow(static_cast<double>(beta1), t)));
+        corr[1] = static_cast<float>(1.0 / (1.0 - pow(static_cast<double>(beta2), t)));
+    }
+    __syncthreads();
+    const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
+    if (quad * 4u >= ldD) return;
+    float4 s = reinterpret_cast<const float4*>(partial)[quad];
+    for (uint32_t k = 1; k < splits; ++k) {
+        const float4 p = reinterpret_cast<const float4*>(partial + static_cast<size_t>(k) * ldD)[quad];
+        s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+    }
+    float gg[4] = { s.x * scale, s.y * scale, s.z * scale, s.w * scale };
+    float4 c4 = reinterpret_cast<float4*>(center)[quad];
+    float4 m4 = reinterpret_cast<float4*>(m)[quad];
+    float4 v4 = reinterpret_cast<float4*>(v)[quad];
+    float cc[4] = { c4.x, c4.y, c4.z, c4.w }, mm[4] = { m4.x, m4.y, m4.z, m4.w },
+          vv[4] = { v4.x, v4.y, v4.z, v4.w };
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        mm[i] = beta1 * mm[i] + (1.f - beta1) * gg[i];
+        vv[i] = beta2 * vv[i] + (1.f - beta2) * gg[i] * gg[i];
+        const float mhat = mm[i] * corr[0];
+        const float vhat = vv[i] * corr[1];
+        cc[i] += lr * mhat / (sqrtf(vhat) + adam_eps);
+    }
+    reinterpret_cast<float4*>(g)[quad] = make_float4(gg[0], gg[1], gg[2], gg[3]);
+    reinterpret_cast<float4*>(m)[quad] = make_float4(mm[0], mm[1], mm[2], mm[3]);
+    reinterpret_cast<float4*>(v)[quad] = make_float4(vv[0], vv[1], vv[2], vv[3]);
+    reinterpret_cast<float4*>(center)[quad] = make_float4(cc[0], cc[1], cc[2], cc[3]);
+}
+
+// Closes a tell: the Adam step counter advances only if the update was applied.
+__global__ void k_tell_finish(DeviceStatus* status)
+{
+    if (status->nonfinite) {
+        status->sticky |= (1u << EVO_ERR_NONFINITE);
+        status->nonfinite = 0;
+    } else {
+        status->adam_step += 1u;
+    }
+}
+
+uint32_t gradient_splits(uint32_t H, uint32_t ldD)
+{
+    // enough thread blocks to fill 148 SMs several times over, a pure function of the shape
+    const uint32_t blocks_x = (ldD / 4u + 127u) / 128u;
+    uint32_t s = (148u * 8u + blocks_x - 1u) / blocks_x;
+    if (s > 64u) s = 64u;
+    const uint32_t max_s = (H + 15u) / 16u;            // at least 16 pairs per split
+    if (s > max_s) s = max_s;
+    if (s < 1u) s = 1u;
+    return s;
+}
+
+int launch_gradient_adam(cudaStream_t st, const float* u, const float* eps, uint32_t k0, uint32_t k1,
+                         uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, uint32_t splits,
+                         float* partial, float sigma, float lr, float beta1, float beta2,
+                         float adam_eps, float* center, float* m, float* v, float* g,
+                         DeviceStatus* status)
+{
+    (void)D;
+    const uint32_t quads = ldD / 4u;
+    const uint32_t pps = (H + splits - 1u) / splits;
+    const uint32_t used = (H + pps - 1u) / pps;        // splits that own at least one pair
+    dim3 grid((quads + 127u) / 128u, used);
+    if (eps)
+        k_grad_partial<false><<<grid, 128, 0, st>>>(u, eps, PhiloxKey{k0, k1}, generation, H, ldD, pps,
+                                                    partial, status);
+    else
+        k_grad_partial<true><<<grid, 128, 0, st>>>(u, nullptr, PhiloxKey{k0, k1}, generation, H, ldD,
+                                                   pps, partial, status);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    const float scale = sigma / static_cast<float>(2u * H);
+    k_adam<<<(quads + 255u) / 256u, 256, 0, st>>>(partial, used, ldD, scale, lr, beta1, beta2, adam_eps,
+                                                  center, m, v, g, status);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    k_tell_finish<<<1, 1, 0, st>>>(status);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 3;
+}
+
+}  // namespace evo

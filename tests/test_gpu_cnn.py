@@ -1,0 +1,54 @@
+"""Supervised (CNN) rollout on the GPU against the oracle: fitness within 1e-3."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import rel_err
+from paper_2202_05008_b200 import Solver, workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(w, theta_np=None, generation=0, members=None):
+    s = Solver(w)
+    images, labels = W.image_batch(w.seed, generation, w.batch)
+    s.set_batch(torch.tensor(images, device="cuda"), torch.tensor(labels, device="cuda"))
+    if theta_np is None:
+        theta_np = s.ask().cpu().numpy(); arg = None
+    else:
+        arg = s.padded_rows(w.pop_size); arg[:, :w.param_dim] = torch.tensor(theta_np, device="cuda")
+    fit = s.rollout(arg).cpu().numpy()
+    assert s.sync_status() == 0
+    members = range(w.pop_size) if members is None else members
+    want = np.array([oracle.cnn_fitness(theta_np[m], images, labels, True) for m in members])
+    assert rel_err(fit[list(members)], want, floor=1.0) < 1e-3
+    s.close()
+    return fit
+
+
+def test_cnn_zero_parameters_is_minus_ln10():
+    w = W.CFG3.with_(pop_size=2, batch=64)
+    fit = _run(w, theta_np=np.zeros((2, W.CNN_PARAMS), dtype=np.float32))
+    assert np.abs(fit + math.log(10)).max() < 1e-6
+
+
+def test_cnn_cfg3_first_generation_sampled_members():
+    _run(W.CFG3, members=[0, 1, 31, 63])
+
+
+def test_cnn_random_large_parameters_ragged_batch():
+    w = W.CFG3.with_(pop_size=4, batch=77)
+    _run(w, theta_np=W.random_parameters(5, 4, W.CNN_PARAMS, scale=0.2))
+
+
+def test_cnn_rollout_needs_a_batch():
+    from paper_2202_05008_b200 import EvoError
+    s = Solver(W.CFG3.with_(pop_size=2, batch=8))
+    s.ask()
+    with pytest.raises(EvoError) as e:
+        s.rollout()
+    assert e.value.code == 2
+    s.close()

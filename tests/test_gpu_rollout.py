@@ -1,0 +1,125 @@
+"""Control-task rollouts on the GPU against the oracle (teacher-forced: same parameters,
+same seeded initial states): per-step state <= 1e-4, fitness <= 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import rel_err, oracle_fitness, cartpole_features
+from paper_2202_05008_b200 import Solver, workloads as W
+from paper_2202_05008_b200.binding import ROLLOUT_GENERIC, ROLLOUT_TILED, ROLLOUT_AUTO, EvoError
+
+pytestmark = pytest.mark.gpu
+
+STATE_TOL, FIT_TOL = 1e-4, 1e-3
+
+
+def _state_dim(w):
+    return 4 if w.task_kind == W.TASK_CARTPOLE else 28
+
+
+def _rollout_check(w, T, members, kernel, theta_np=None, generation=0, check_trace=True):
+    """Roll `members` rows on the GPU (whole population is rolled; rows are compared)."""
+    w = w.with_(horizon=T)
+    s = Solver(w, trace_steps=T if check_trace else 0, rollout_kernel=kernel)
+    if theta_np is None:
+        theta_dev = s.ask()
+        theta_np = theta_dev.cpu().numpy()
+        arg = None
+    else:
+        arg = s.padded_rows(w.pop_size)
+        arg[:, :w.param_dim] = torch.tensor(theta_np, device="cuda")
+    sd = _state_dim(w)
+    trace = torch.zeros(w.pop_size, w.episodes, T, sd, device="cuda") if check_trace else None
+    fit = s.rollout(arg, trace=trace).cpu().numpy()
+    assert s.sync_status() == 0
+    fit_o, traces_o = oracle_fitness(w, theta_np[members], generation, T, want_trace=check_trace)
+    assert rel_err(fit[members], fit_o, floor=1.0) < FIT_TOL
+    if check_trace:
+        tr = trace.cpu().numpy()
+        for k, m in enumerate(members):
+            got, want = tr[m].astype(np.float64), traces_o[k]
+            if w.task_kind == W.TASK_CARTPOLE:
+                got, want = cartpole_features(got), cartpole_features(want)
+            for i in range(got.shape[-1]):          # per state component, floor = its RMS
+                assert rel_err(got[..., i], want[..., i]) < STATE_TOL, (m, i)
+    s.close()
+    return fit
+
+
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_AUTO])
+def test_cfg1_full(kernel):
+    fit = _rollout_check(W.CFG1, 200, list(range(16)), kernel)
+    assert np.abs(fit).max() <= 200
+
+
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_AUTO])
+def test_cfg1_random_policies_strong_forces(kernel):
+    theta = W.random_parameters(1, 16, 385, scale=0.7)
+    _rollout_check(W.CFG1, 200, list(range(16)), kernel, theta_np=theta)
+
+
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_AUTO])
+def test_cfg2_T200_sampled_members(kernel):
+    _rollout_check(W.CFG2, 200, [0, 1, 77, 128, 255], kernel)
+
+
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_AUTO])
+def test_cfg4_T200_sampled_members(kernel):
+    _rollout_check(W.CFG4, 200, [0, 1, 2047, 4095], kernel)
+
+
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_AUTO])
+def test_cfg4_random_policies(kernel):
+    w = W.CFG4.with_(pop_size=8)
+    theta = W.random_parameters(2, 8, w.param_dim, scale=0.3)
+    _rollout_check(w, 100, list(range(8)), kernel, theta_np=theta)
+
+
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_AUTO])
+def test_zero_policy_is_the_free_pendulum(kernel):
+    theta = np.zeros((16, 385), dtype=np.float32)
+    _rollout_check(W.CFG1, 150, [0, 15], kernel, theta_np=theta)
+
+
+def test_generic_kernel_odd_shapes_and_episode_counts():
+    # 3 layers of odd widths, episodes not a multiple of the episode block
+    sizes = (5, 7, 3, 9, 1)
+    w = W.CFG1.with_(layer_sizes=sizes, param_dim=W.mlp_param_count(sizes), pop_size=6, episodes=37,
+                     task_param=(1.0, 0.1, 0.5, 9.8, 0.01, 0.2))
+    theta = W.random_parameters(3, 6, w.param_dim, scale=0.6)
+    _rollout_check(w, 50, list(range(6)), ROLLOUT_GENERIC, theta_np=theta)
+    sizes = (28, 8)
+    w = W.CFG4.with_(layer_sizes=sizes, param_dim=W.mlp_param_count(sizes), pop_size=4, episodes=3)
+    theta = W.random_parameters(4, 4, w.param_dim, scale=0.3)
+    _rollout_check(w, 30, list(range(4)), ROLLOUT_GENERIC, theta_np=theta)
+
+
+def test_rollout_later_generation_uses_new_initial_states():
+    w = W.CFG1.with_(horizon=50)
+    s = Solver(w)
+    f = []
+    for gen in range(2):
+        theta = s.ask()
+        fit = s.rollout()
+        fit_o, _ = oracle_fitness(w, theta.cpu().numpy(), gen, 50)
+        assert rel_err(fit.cpu().numpy(), fit_o, floor=1.0) < FIT_TOL
+        s.tell(fit)
+        f.append(fit.cpu().numpy())
+    assert s.sync_status() == 0
+    s.close()
+
+
+def test_full_horizon_reward_bounds_and_determinism():
+    for w in (W.CFG2.with_(pop_size=32), W.CFG4.with_(pop_size=64)):
+        s = Solver(w)
+        s.ask()
+        a = s.rollout().clone()
+        b = s.rollout().clone()
+        assert torch.equal(a, b)
+        a = a.cpu().numpy()
+        if w.task_kind == W.TASK_CARTPOLE:
+            assert np.abs(a).max() <= w.horizon
+        else:
+            assert a.max() <= 0 and np.isfinite(a).all()
+        s.close()
