@@ -1,0 +1,441 @@
+#!/usr/bin/env python
+"""Benchmark of one evolution-strategy generation (ask -> rollout -> tell) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl ours|reference]
+
+One "step" is one whole generation of the workload.  Prints ONE JSON line (rank 0).
+For N > 1 (launched by torch.distributed.run) every rank runs an independent solver on its own
+GPU with its own seed (replicas; the generation itself needs no exchange on one GPU), timing is
+the max over ranks and the value is the sum of the work of all ranks.
+
+`--impl reference` times the CPU oracle (single-threaded C, fp64) on a bounded sample of the same
+workload; it is a deliberately slow, plain program and serves as a baseline only.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+FP32_LANES_PER_SM = 128
+L2_FLUSH_BYTES = 256 << 20
+
+
+# ------------------------------------------------------------------------------------------
+# workload arithmetic (algorithmic work per generation)
+# ------------------------------------------------------------------------------------------
+def mlp_macs(sizes):
+    return sum(a * b for a, b in zip(sizes[:-1], sizes[1:]))
+
+
+def rollout_flops_per_env_step(w):
+    from paper_2202_05008_b200 import workloads as W
+    if w.task_kind == W.TASK_SUPERVISED:
+        return 645120.0                       # conv1 230,400 + conv2 409,600 + fc 5,120 (2 x MAC)
+    macs = mlp_macs(w.layer_sizes)
+    if w.task_kind == W.TASK_TANH_LINEAR:
+        macs += 28 * 28 + 28 * 8              # the task's own x' = tanh(Ax + Ba)
+    return 2.0 * macs
+
+
+def stage_work(w, stored):
+    """Algorithmic bytes / flops of each stage of one generation."""
+    P, D = w.pop_size, w.param_dim
+    H = P // 2
+    ask_bytes = 4.0 * P * D + (4.0 * H * D if stored else 0.0) + 4.0 * D
+    tell_bytes = (4.0 * H * D if stored else 0.0) + 28.0 * D + 8.0 * P
+    rollout_flops = rollout_flops_per_env_step(w) * w.env_steps_per_generation
+    return {"ask_bytes": ask_bytes, "tell_bytes": tell_bytes, "rollout_flops": rollout_flops}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Polls NVML for SM clock and throttle reasons while the timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, device_index):
+        self.samples, self.reason_bits, self.max_mhz = [], 0, None
+        self._stop = threading.Event()
+        self._thread = None
+        self.h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.h = None
+
+    def sample(self):
+        if self.h is None:
+            return
+        try:
+            self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+            self.reason_bits |= int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+        except Exception:
+            try:
+                self.reason_bits |= int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            except Exception:
+                pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample()
+            time.sleep(0.02)
+
+    def start(self):
+        if self.h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------
+def oracle_generation_sample(w, n_members, generation=0):
+    """Times the oracle on ask + tell for the whole population (a column sample for very wide
+    problems) and the rollout of n_members members; returns seconds for a full generation
+    extrapolated linearly (members and columns are independent)."""
+    import oracle
+    from paper_2202_05008_b200 import workloads as W
+    P, D = w.pop_size, w.param_dim
+    cols = D if P * D <= 50_000_000 else 4096
+    t0 = time.perf_counter()
+    theta, eps = oracle.ask(w.seed, generation, P, cols, np.zeros(cols, np.float32), w.sigma)
+    t_ask = (time.perf_counter() - t0) * (D / cols)
+    t_roll, n_done = 0.0, 0
+    fitness = W.synthetic_fitness(w.seed, generation, P)
+    if w.task_kind != W.TASK_NONE:
+        full = np.zeros((n_members, D), dtype=np.float32)
+        if cols == D:
+            full[:] = theta[:n_members]
+        t0 = time.perf_counter()
+        if w.task_kind == W.TASK_SUPERVISED:
+            images, labels = W.image_batch(w.seed, generation, w.batch)
+            for m in range(n_members):
+                fitness[m] = oracle.cnn_fitness(full[m], images, labels, True)
+        elif w.task_kind == W.TASK_CARTPOLE:
+            tp = w.task_param
+            p = oracle.cartpole_params(tp[0], tp[1], tp[2], tp[3], tp[4])
+            for m in range(n_members):
+                fitness[m] = oracle.rollout_cartpole(full[m], w.layer_sizes, w.action_scale, p, tp[5],
+                                                     w.seed, generation, w.episodes, w.horizon)[0]
+        else:
+            A, B = oracle.tanh_linear_constants(w.seed)
+            for m in range(n_members):
+                fitness[m] = oracle.rollout_tanh_linear(full[m], w.layer_sizes, w.action_scale, A, B,
+                                                        w.seed, generation, w.episodes, w.horizon)[0]
+        t_roll = (time.perf_counter() - t0) * (P / n_members)
+        n_done = n_members
+    t0 = time.perf_counter()
+    _, u, _ = oracle.centered_rank(fitness)
+    g = oracle.gradient(u, eps, w.sigma)
+    oracle.adam(np.zeros(cols), np.zeros(cols), np.zeros(cols), g, 1, w.lr)
+    t_tell = (time.perf_counter() - t0) * (D / cols)
+    sample = (f"ask+tell on all {P} members x {cols} of {D} columns; rollout of {n_done} of {P} members "
+              f"x {w.episodes} episodes x {w.horizon} steps; scaled linearly to one generation")
+    return t_ask + t_roll + t_tell, sample
+
+
+def unit_of(w):
+    from paper_2202_05008_b200 import workloads as W
+    if w.task_kind == W.TASK_NONE:
+        return "generations_per_sec", "generations/s", 1.0
+    return "env_steps_per_sec", "env-steps/s", float(w.env_steps_per_generation)
+
+
+def members_for_budget(w, seconds):
+    """Members whose oracle rollout takes about `seconds` (from a one-member probe)."""
+    from paper_2202_05008_b200 import workloads as W
+    if w.task_kind == W.TASK_NONE:
+        return 0
+    t, _ = oracle_generation_sample(w.with_(pop_size=2, param_dim=w.param_dim), 1)
+    per_member = max(t / 2.0, 1e-4)
+    return int(max(1, min(w.pop_size, seconds / per_member)))
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    metric, unit, units_per_gen = unit_of(w)
+    n = members_for_budget(w, 1.0)
+    times, sample = [], ""
+    for i in range(args.warmup + args.steps):
+        t, sample = oracle_generation_sample(w, max(n, 1), generation=i)
+        if i >= args.warmup:
+            times.append(t)
+    t_step = sum(times) / len(times)
+    value = units_per_gen / t_step
+    line = {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": config_of(w, args, stored=True),
+            "generations_per_sec": 1.0 / t_step,
+            "cpu_baseline": {"value": value, "unit": unit, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def config_of(w, args, stored):
+    from paper_2202_05008_b200 import workloads as W
+    task = {W.TASK_NONE: "none", W.TASK_CARTPOLE: "cartpole_swingup", W.TASK_TANH_LINEAR: "tanh_linear",
+            W.TASK_SUPERVISED: "supervised_28x28"}[w.task_kind]
+    return {"workload": w.name, "pop_size": w.pop_size, "param_dim": w.param_dim, "task": task,
+            "policy": "mlp " + "-".join(map(str, w.layer_sizes)) if w.layer_sizes else
+                      ("cnn_28" if w.policy_kind == W.POLICY_CNN_28 else "none"),
+            "episodes": w.episodes, "horizon": w.horizon, "batch": w.batch,
+            "noise": "stored" if stored else "regenerated", "parallelism": f"replicas x{args.gpus}",
+            "l2": "flushed between timed steps (256 MiB write, untimed)"}
+
+
+# ------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2202_05008_b200 import Solver, workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the GPU arm has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    stored = args.noise == "stored"
+    w_rank = w.with_(seed=w.seed + 1000 * rank)         # independent replicas
+    s = Solver(w_rank, device=dev, noise_mode=W.NOISE_STORED if stored else W.NOISE_REGENERATED)
+    P, D = w.pop_size, w.param_dim
+    supervised = w.task_kind == W.TASK_SUPERVISED
+    no_task = w.task_kind == W.TASK_NONE
+    fitness = torch.empty(P, dtype=torch.float32, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    if supervised:
+        batches = []
+        for g in range(4):
+            im, lb = W.image_batch(w_rank.seed, g, w.batch)
+            batches.append((torch.tensor(im, device=dev), torch.tensor(lb, device=dev)))
+    if no_task:
+        fits = [torch.tensor(W.synthetic_fitness(w_rank.seed, g, P), device=dev) for g in range(4)]
+
+    def generation(i, ev=None):
+        if ev: ev[0].record()
+        s.ask()
+        if ev: ev[1].record()
+        if supervised:
+            s.set_batch(*batches[i % 4])
+        if no_task:
+            f = fits[i % 4]
+        else:
+            f = s.rollout(fitness=fitness)
+        if ev: ev[2].record()
+        s.tell(f)
+        if ev: ev[3].record()
+
+    for i in range(args.warmup):
+        flush.fill_(i & 255)
+        generation(i)
+    torch.cuda.synchronize()
+    if s.sync_status() != 0:
+        raise SystemExit("bench.py: device status not ok after warm-up")
+
+    sampler = ClockSampler(local)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    launches0 = s.launch_count()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    for i in range(args.steps):
+        flush.fill_(i & 255)                            # evict L2 (untimed)
+        generation(args.warmup + i, events[i])
+    sampler.sample()
+    torch.cuda.synchronize()
+    sampler.stop()
+    if world > 1:
+        dist.barrier()
+    launches = s.launch_count() - launches0
+    status = s.sync_status()
+    if status != 0:
+        raise SystemExit(f"bench.py: device status {status} after the timed region")
+
+    t_ask = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
+    t_roll = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
+    t_tell = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
+    t_total_ms = sum(e[0].elapsed_time(e[3]) for e in events)
+    tt = torch.tensor([t_total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    t_step_ms = float(tt.item()) / args.steps
+
+    # ---- end to end: host-resident centre in, fitness and centre out, every step -----------
+    h_center = torch.zeros(D, dtype=torch.float32).pin_memory()
+    h_fit = torch.zeros(P, dtype=torch.float32).pin_memory()
+    d_center = torch.zeros(D, dtype=torch.float32, device=dev)
+    if supervised:
+        h_batches = [(b[0].cpu().pin_memory(), b[1].cpu().pin_memory()) for b in batches]
+        d_im = torch.empty_like(batches[0][0]); d_lb = torch.empty_like(batches[0][1])
+    if no_task:
+        h_fits = [f.cpu().pin_memory() for f in fits]
+    h_center.copy_(s.center().cpu())
+    gen0, t0_adam = s.counters()
+    e2e_steps = max(3, min(args.steps, 50))
+    h2d = 4 * D + (w.batch * (784 * 4 + 4) if supervised else 0) + (4 * P if no_task else 0)
+    d2h = 4 * D + 4 * P
+
+    def e2e_step(i):
+        d_center.copy_(h_center, non_blocking=True)
+        s.set_state(center=d_center, generation=gen0 + i, adam_step=t0_adam + i)
+        s.ask()
+        if supervised:
+            d_im.copy_(h_batches[i % 4][0], non_blocking=True)
+            d_lb.copy_(h_batches[i % 4][1], non_blocking=True)
+            s.set_batch(d_im, d_lb)
+        if no_task:
+            fitness.copy_(h_fits[i % 4], non_blocking=True)
+        else:
+            s.rollout(fitness=fitness)
+        s.tell(fitness)
+        h_fit.copy_(fitness, non_blocking=True)
+        h_center.copy_(s.center(), non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    e2e_step(0)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(1, e2e_steps + 1):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+    te = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_ms = float(te.item())
+
+    if rank == 0:
+        metric, unit, units_per_gen = unit_of(w)
+        value = world * units_per_gen / (t_step_ms * 1e-3)
+        peaks = measured_peaks()
+        clocks = sampler.summary()
+        sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+        max_mhz = clocks["sm_max_mhz"] or 1965
+        work = stage_work(w, stored)
+        alu_peak = sm_count * FP32_LANES_PER_SM * 2 * max_mhz * 1e6 / 1e12      # TFLOP/s fp32 FMA
+        stages = {
+            "ask": {"ms": t_ask, "GB/s": work["ask_bytes"] / (t_ask * 1e-3) / 1e9},
+            "rollout": {"ms": t_roll, "TFLOP/s": work["rollout_flops"] / (t_roll * 1e-3) / 1e12 if t_roll > 0 else 0.0},
+            "tell": {"ms": t_tell, "GB/s": work["tell_bytes"] / (t_tell * 1e-3) / 1e9},
+        }
+        if no_task:
+            dom = "ask" if t_ask >= t_tell else "tell"
+            achieved = stages[dom]["GB/s"]
+            roofline = {"kernel": "k_ask" if dom == "ask" else "k_grad_partial", "bound": "hbm",
+                        "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                        "traffic": None}
+        elif supervised:
+            achieved = stages["rollout"]["TFLOP/s"]
+            roofline = {"kernel": "k_cnn", "bound": "tensor", "achieved": achieved,
+                        "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                        "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"],
+                        "traffic": None}
+        else:
+            achieved = stages["rollout"]["TFLOP/s"]
+            roofline = {"kernel": "k_rollout_mlp", "bound": "alu", "achieved": achieved, "peak": alu_peak,
+                        "unit": "TFLOP/s", "frac": achieved / alu_peak,
+                        "peak_source": f"{sm_count} SMs x 128 fp32 lanes x 2 x {max_mhz} MHz",
+                        "traffic": None}
+        cpu = None
+        if world == 1 or rank == 0:
+            n = members_for_budget(w, 12.0)
+            t_cpu, sample = oracle_generation_sample(w, max(n, 1))
+            cpu = {"value": units_per_gen / t_cpu, "unit": unit, "cores": 1, "kind": "oracle",
+                   "sample": sample}
+        line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": t_step_ms, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": config_of(w, args, stored),
+                "generations_per_sec": world / (t_step_ms * 1e-3),
+                "e2e": {"value": world * units_per_gen / (e2e_ms * 1e-3), "unit": unit,
+                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+                "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
+                "stages": stages, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    s.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--noise", default="stored", choices=["stored", "regenerated"])
+    ap.add_argument("--pop", type=int, default=0, help="override the population size (experiments)")
+    ap.add_argument("--dim", type=int, default=0, help="override the parameter count (cfg5 only)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from paper_2202_05008_b200 import workloads as W
+    w = W.CONFIGS[args.workload]
+    if args.pop:
+        w = w.with_(pop_size=args.pop)
+    if args.dim and args.workload == "cfg5":
+        w = w.with_(param_dim=args.dim)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -77,7 +77,7 @@ static evo_status make_layout(const evo_config& c, Layout* L)
     L->g = take(row);
     L->u = take(P * sizeof(float));
     L->rank = take(P * sizeof(int32_t));
-    L->grad_partial = take(row * L->grad_splits);
+    L->grad_partial = take(2 * row * L->grad_splits);          // fp64 partial sums
     L->fit_partial = take(P * L->n_eb * sizeof(float));
     L->task_const = take(kTlNx * (kTlNx + kTlNa) * sizeof(float));
     L->cnn_scratch = take(c.task_kind == EVO_TASK_SUPERVISED ? cnn_scratch_bytes(c.pop_size, c.batch) : 0);
@@ -232,7 +232,7 @@ evo_status evo_tell(evo_solver* s, const float* d_fitness)
     const float* eps = c.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<const float*>(s->ws + L.eps)
                                                         : nullptr;
     n = launch_gradient_adam(s->stream, u, eps, s->k0, s->k1, s->generation, c.pop_size / 2, c.param_dim,
-                             L.ldD, L.grad_splits, reinterpret_cast<float*>(s->ws + L.grad_partial),
+                             L.ldD, L.grad_splits, reinterpret_cast<double*>(s->ws + L.grad_partial),
                              c.sigma, c.lr, c.beta1, c.beta2, c.adam_eps,
                              reinterpret_cast<float*>(s->ws + L.center),
                              reinterpret_cast<float*>(s->ws + L.m), reinterpret_cast<float*>(s->ws + L.v),

@@ -54,7 +54,7 @@ int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank
                 DeviceStatus* status);
 int launch_gradient_adam(cudaStream_t st, const float* u, const float* eps /*NULL = regenerate*/,
                          uint32_t k0, uint32_t k1, uint32_t generation, uint32_t H, uint32_t D,
-                         uint32_t ldD, uint32_t splits, float* partial, float sigma, float lr,
+                         uint32_t ldD, uint32_t splits, double* partial, float sigma, float lr,
                          float beta1, float beta2, float adam_eps, float* center, float* m, float* v,
                          float* g, DeviceStatus* status);
 uint32_t gradient_splits(uint32_t H, uint32_t ldD);

@@ -138,69 +138,75 @@ int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank
 
 // ------------------------------------------------------------------------------------------
 // ES gradient.  partial[s][d] = sum over the pairs of split s of (u[2j]-u[2j+1]) * eps[j][d],
-// one thread per column quad, fixed summation order (four interleaved accumulators combined
-// as (a0+a1)+(a2+a3)); no floating-point atomics anywhere, so results are run-to-run identical.
+// one thread per column quad.  Products and sums are fp64: the Adam step lr*g/(|g|+eps) is
+// ill-conditioned where |g| is near adam_eps, so the cancellation error of an fp32 sum
+// (~1e-7 of RMS(g)) would move those coordinates by far more than the 1e-5 parity bound.  The
+// stored-noise kernel is HBM-bound (4 bytes per term), so the fp64 arithmetic is hidden.
+// Summation order is fixed (two interleaved accumulators per column, splits added in order);
+// no floating-point atomics anywhere, so results are run-to-run identical.
 // REGEN recomputes eps from the Philox counters instead of reading it.
 // ------------------------------------------------------------------------------------------
+struct Acc4 { double x, y, z, w; };
+
+__device__ __forceinline__ void acc_fma(Acc4& a, double wd, const float4& e)
+{
+    a.x = fma(wd, static_cast<double>(e.x), a.x);
+    a.y = fma(wd, static_cast<double>(e.y), a.y);
+    a.z = fma(wd, static_cast<double>(e.z), a.z);
+    a.w = fma(wd, static_cast<double>(e.w), a.w);
+}
+
 template <bool REGEN>
 __global__ void __launch_bounds__(128)
 k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, PhiloxKey key,
-               uint32_t generation, uint32_t H, uint32_t ldD, uint32_t pairs_per_split,
-               float* __restrict__ partial, const DeviceStatus* status)
+               uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, uint32_t pairs_per_split,
+               double* __restrict__ partial, const DeviceStatus* status)
 {
     if (status->nonfinite) return;
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
     const uint32_t j0 = blockIdx.y * pairs_per_split;
     const uint32_t j1 = min(H, j0 + pairs_per_split);
-    float4 acc[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    Acc4 acc[2] = { {0., 0., 0., 0.}, {0., 0., 0., 0.} };
     const float2* up = reinterpret_cast<const float2*>(u);
     uint32_t j = j0;
     for (; j + 4u <= j1; j += 4u) {
         float4 e[4];
-        float w[4];
+        double w[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if (REGEN) e[i] = stream_normal4(key, 0u, generation, j + i, quad);
             else e[i] = __ldcs(reinterpret_cast<const float4*>(eps + static_cast<size_t>(j + i) * ldD) + quad);
             const float2 uu = __ldg(up + j + i);
-            w[i] = uu.x - uu.y;
+            w[i] = static_cast<double>(uu.x) - static_cast<double>(uu.y);   // exact
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            acc[i].x = fmaf(w[i], e[i].x, acc[i].x);
-            acc[i].y = fmaf(w[i], e[i].y, acc[i].y);
-            acc[i].z = fmaf(w[i], e[i].z, acc[i].z);
-            acc[i].w = fmaf(w[i], e[i].w, acc[i].w);
-        }
+        for (int i = 0; i < 4; ++i) acc_fma(acc[i & 1], w[i], e[i]);
     }
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {                  // tail keeps the accumulator assignment j % 4
+    for (int i = 0; i < 3; ++i) {                  // tail keeps the accumulator assignment j % 2
         if (j + i < j1) {
             float4 e;
             if (REGEN) e = stream_normal4(key, 0u, generation, j + i, quad);
             else e = __ldcs(reinterpret_cast<const float4*>(eps + static_cast<size_t>(j + i) * ldD) + quad);
             const float2 uu = __ldg(up + j + i);
-            const float w = uu.x - uu.y;
-            acc[i].x = fmaf(w, e.x, acc[i].x);
-            acc[i].y = fmaf(w, e.y, acc[i].y);
-            acc[i].z = fmaf(w, e.z, acc[i].z);
-            acc[i].w = fmaf(w, e.w, acc[i].w);
+            acc_fma(acc[i & 1], static_cast<double>(uu.x) - static_cast<double>(uu.y), e);
         }
     }
-    float4 r;
-    r.x = (acc[0].x + acc[1].x) + (acc[2].x + acc[3].x);
-    r.y = (acc[0].y + acc[1].y) + (acc[2].y + acc[3].y);
-    r.z = (acc[0].z + acc[1].z) + (acc[2].z + acc[3].z);
-    r.w = (acc[0].w + acc[1].w) + (acc[2].w + acc[3].w);
-    reinterpret_cast<float4*>(partial + static_cast<size_t>(blockIdx.y) * ldD)[quad] = r;
+    double r[4] = { acc[0].x + acc[1].x, acc[0].y + acc[1].y, acc[0].z + acc[1].z, acc[0].w + acc[1].w };
+    if (REGEN && quad * 4u + 4u > D) {             // recomputed noise exists only for real columns
+#pragma unroll
+        for (uint32_t i = 0; i < 4u; ++i)
+            if (quad * 4u + i >= D) r[i] = 0.;
+    }
+    double2* out = reinterpret_cast<double2*>(partial + static_cast<size_t>(blockIdx.y) * ldD) + 2u * quad;
+    out[0] = make_double2(r[0], r[1]);
+    out[1] = make_double2(r[2], r[3]);
 }
 
-// Sum the splits in order, scale, and take the Adam ascent step in place.
+// Sum the splits in order, scale, round the gradient to fp32 and take the Adam ascent step.
 __global__ void __launch_bounds__(256)
-k_adam(const float* __restrict__ partial, uint32_t splits, uint32_t ldD, float scale, float lr,
+k_adam(const double* __restrict__ partial, uint32_t splits, uint32_t ldD, double scale, float lr,
        float beta1, float beta2, float adam_eps, float* __restrict__ center, float* __restrict__ m,
        float* __restrict__ v, float* __restrict__ g, const DeviceStatus* status)
 {
@@ -214,12 +220,15 @@ k_adam(const float* __restrict__ partial, uint32_t splits, uint32_t ldD, float s
     __syncthreads();
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
-    float4 s = reinterpret_cast<const float4*>(partial)[quad];
-    for (uint32_t k = 1; k < splits; ++k) {
-        const float4 p = reinterpret_cast<const float4*>(partial + static_cast<size_t>(k) * ldD)[quad];
-        s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+    double sum[4] = { 0., 0., 0., 0. };
+    for (uint32_t k = 0; k < splits; ++k) {
+        const double2* p = reinterpret_cast<const double2*>(partial + static_cast<size_t>(k) * ldD) + 2u * quad;
+        const double2 a = p[0], b = p[1];
+        sum[0] += a.x; sum[1] += a.y; sum[2] += b.x; sum[3] += b.y;
     }
-    float gg[4] = { s.x * scale, s.y * scale, s.z * scale, s.w * scale };
+    float gg[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) gg[i] = static_cast<float>(sum[i] * scale);
     float4 c4 = reinterpret_cast<float4*>(center)[quad];
     float4 m4 = reinterpret_cast<float4*>(m)[quad];
     float4 v4 = reinterpret_cast<float4*>(v)[quad];
@@ -264,23 +273,22 @@ uint32_t gradient_splits(uint32_t H, uint32_t ldD)
 
 int launch_gradient_adam(cudaStream_t st, const float* u, const float* eps, uint32_t k0, uint32_t k1,
                          uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, uint32_t splits,
-                         float* partial, float sigma, float lr, float beta1, float beta2,
+                         double* partial, float sigma, float lr, float beta1, float beta2,
                          float adam_eps, float* center, float* m, float* v, float* g,
                          DeviceStatus* status)
 {
-    (void)D;
     const uint32_t quads = ldD / 4u;
     const uint32_t pps = (H + splits - 1u) / splits;
     const uint32_t used = (H + pps - 1u) / pps;        // splits that own at least one pair
     dim3 grid((quads + 127u) / 128u, used);
     if (eps)
-        k_grad_partial<false><<<grid, 128, 0, st>>>(u, eps, PhiloxKey{k0, k1}, generation, H, ldD, pps,
+        k_grad_partial<false><<<grid, 128, 0, st>>>(u, eps, PhiloxKey{k0, k1}, generation, H, D, ldD, pps,
                                                     partial, status);
     else
-        k_grad_partial<true><<<grid, 128, 0, st>>>(u, nullptr, PhiloxKey{k0, k1}, generation, H, ldD,
+        k_grad_partial<true><<<grid, 128, 0, st>>>(u, nullptr, PhiloxKey{k0, k1}, generation, H, D, ldD,
                                                    pps, partial, status);
     if (cudaGetLastError() != cudaSuccess) return -1;
-    const float scale = sigma / static_cast<float>(2u * H);
+    const double scale = static_cast<double>(sigma) / static_cast<double>(2u * H);
     k_adam<<<(quads + 255u) / 256u, 256, 0, st>>>(partial, used, ldD, scale, lr, beta1, beta2, adam_eps,
                                                   center, m, v, g, status);
     if (cudaGetLastError() != cudaSuccess) return -1;

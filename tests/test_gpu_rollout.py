@@ -72,7 +72,7 @@ def test_cfg4_T200_sampled_members(kernel):
 @pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_AUTO])
 def test_cfg4_random_policies(kernel):
     w = W.CFG4.with_(pop_size=8)
-    theta = W.random_parameters(2, 8, w.param_dim, scale=0.3)
+    theta = W.random_parameters(2, 8, w.param_dim, scale=0.05)   # contracting closed loop
     _rollout_check(w, 100, list(range(8)), kernel, theta_np=theta)
 
 

@@ -52,7 +52,11 @@ def test_tell_cfg1_first_step_is_plus_minus_lr():
     s.ask()
     s.tell(torch.tensor(W.synthetic_fitness(0, 0, 16), device="cuda"))
     c = s.center().cpu().numpy()
-    assert np.abs(np.abs(c) - 0.01).max() < 1e-5
+    g = s.gradient().cpu().numpy()
+    big = np.abs(g) > 1e-4                    # |step| = lr/(1 + eps/|g|)
+    assert big.sum() > 300
+    assert np.abs(np.abs(c[big]) - 0.01).max() < 2e-6
+    assert (np.sign(c) == np.sign(g)).all()   # ascent
     s.close()
 
 
