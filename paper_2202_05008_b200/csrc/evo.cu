@@ -211,7 +211,8 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
     a.trace_T = c.trace_steps < c.horizon ? c.trace_steps : c.horizon;
     a.k0 = s->k0; a.k1 = s->k1; a.generation = s->generation;
     std::memcpy(a.tp, c.task_param, sizeof(a.tp));
-    const int n = launch_rollout_mlp(s->stream, a, c.rollout_kernel, d_fitness);
+    const int n = launch_rollout_mlp(s->stream, a, c.rollout_kernel, d_fitness,
+                                     reinterpret_cast<DeviceStatus*>(s->ws + L.status));
     if (n < 0) return n == -2 ? EVO_ERR_UNSUPPORTED : EVO_ERR_CUDA;
     s->launches += n;
     return EVO_OK;

@@ -60,7 +60,7 @@ int launch_gradient_adam(cudaStream_t st, const float* u, const float* eps /*NUL
 uint32_t gradient_splits(uint32_t H, uint32_t ldD);
 
 int  launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a, uint32_t kernel_choice,
-                        float* fitness);
+                        float* fitness, DeviceStatus* status);
 bool rollout_mlp_supported(const evo_config& cfg);
 void rollout_mlp_plan(const evo_config& cfg, uint32_t* EB, uint32_t* n_eb);
 

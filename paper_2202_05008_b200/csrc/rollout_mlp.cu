@@ -10,79 +10,9 @@
 //   k_rollout_mlp_tiled<..> compile-time shapes with register-tiled layers (the fast path)
 #include "internal.h"
 #include "noise.cuh"
+#include "tasks.cuh"
 
 namespace evo {
-
-// ------------------------------------------------------------------------------------------
-// task arithmetic (fp32)
-// ------------------------------------------------------------------------------------------
-struct CartpoleConst {
-    float total_mass, pole_mass_length, gravity, length, dt, inv_total;
-    float pole_mass;
-};
-
-__device__ __forceinline__ CartpoleConst cartpole_const(const float* tp)
-{
-    CartpoleConst c;
-    c.total_mass = tp[EVO_CP_CART_MASS] + tp[EVO_CP_POLE_MASS];
-    c.inv_total = 1.0f / c.total_mass;
-    c.pole_mass = tp[EVO_CP_POLE_MASS];
-    c.length = tp[EVO_CP_POLE_HALF_LENGTH];
-    c.pole_mass_length = tp[EVO_CP_POLE_MASS] * tp[EVO_CP_POLE_HALF_LENGTH];
-    c.gravity = tp[EVO_CP_GRAVITY];
-    c.dt = tp[EVO_CP_DT];
-    return c;
-}
-
-struct CpState { float x, xd, th, thd; };
-
-// time derivative of (x, x', theta, theta') for the uniform-rod cart-pole, theta = 0 upright
-__device__ __forceinline__ CpState cartpole_deriv(const CartpoleConst& c, const CpState& s, float force)
-{
-    float sn, cs;
-    sincosf(s.th, &sn, &cs);
-    const float tmp = (force + c.pole_mass_length * s.thd * s.thd * sn) * c.inv_total;
-    const float th_acc = (c.gravity * sn - cs * tmp) /
-                         (c.length * (4.0f / 3.0f - c.pole_mass * cs * cs * c.inv_total));
-    const float x_acc = tmp - c.pole_mass_length * th_acc * cs * c.inv_total;
-    return CpState{ s.xd, x_acc, s.thd, th_acc };
-}
-
-__device__ __forceinline__ CpState cp_axpy(const CpState& s, float h, const CpState& k)
-{
-    return CpState{ fmaf(h, k.x, s.x), fmaf(h, k.xd, s.xd), fmaf(h, k.th, s.th), fmaf(h, k.thd, s.thd) };
-}
-
-// classical RK4, force held over the step
-__device__ __forceinline__ CpState cartpole_step(const CartpoleConst& c, const CpState& s, float force)
-{
-    const float h = c.dt;
-    const CpState k1 = cartpole_deriv(c, s, force);
-    const CpState k2 = cartpole_deriv(c, cp_axpy(s, 0.5f * h, k1), force);
-    const CpState k3 = cartpole_deriv(c, cp_axpy(s, 0.5f * h, k2), force);
-    const CpState k4 = cartpole_deriv(c, cp_axpy(s, h, k3), force);
-    const float w = h * (1.0f / 6.0f);
-    CpState n;
-    n.x   = s.x   + w * (k1.x   + 2.0f * k2.x   + 2.0f * k3.x   + k4.x);
-    n.xd  = s.xd  + w * (k1.xd  + 2.0f * k2.xd  + 2.0f * k3.xd  + k4.xd);
-    n.th  = s.th  + w * (k1.th  + 2.0f * k2.th  + 2.0f * k3.th  + k4.th);
-    n.thd = s.thd + w * (k1.thd + 2.0f * k2.thd + 2.0f * k3.thd + k4.thd);
-    return n;
-}
-
-// seeded start shared by all members: (0, 0, pi, 0) + Uniform(-a, a)^4, stream 1, row = episode
-__device__ __forceinline__ CpState cartpole_reset(PhiloxKey key, uint32_t generation, uint32_t episode,
-                                                  float a)
-{
-    const uint4 r = philox4x32_10(0u, episode, generation, 1u, key);
-    const float two_a = __fmul_rn(2.0f, a);
-    CpState s;
-    s.x   = __fmaf_rn(two_a, uniform_half(r.x), -a);
-    s.xd  = __fmaf_rn(two_a, uniform_half(r.y), -a);
-    s.th  = __fadd_rn(__uint_as_float(0x40490FDBu), __fmaf_rn(two_a, uniform_half(r.z), -a));
-    s.thd = __fmaf_rn(two_a, uniform_half(r.w), -a);
-    return s;
-}
 
 // ------------------------------------------------------------------------------------------
 // generic kernel: block = (member, episode block); 128 threads; activations in shared memory
@@ -258,8 +188,22 @@ bool rollout_mlp_supported(const evo_config& cfg)
     return false;
 }
 
+int rollout_mlp_tiled_shape(uint32_t task, uint32_t n_layers, const uint32_t* sizes);
+uint32_t rollout_mlp_tiled_eb(int shape);
+int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus* status);
+
+static bool use_tiled(uint32_t task, uint32_t n_layers, const uint32_t* sizes, uint32_t choice)
+{
+    return choice != EVO_ROLLOUT_GENERIC && rollout_mlp_tiled_shape(task, n_layers, sizes) >= 0;
+}
+
 void rollout_mlp_plan(const evo_config& cfg, uint32_t* EB, uint32_t* n_eb)
 {
+    if (use_tiled(cfg.task_kind, cfg.n_layers, cfg.layer_sizes, cfg.rollout_kernel)) {
+        *EB = rollout_mlp_tiled_eb(rollout_mlp_tiled_shape(cfg.task_kind, cfg.n_layers, cfg.layer_sizes));
+        *n_eb = (cfg.episodes + *EB - 1u) / *EB;
+        return;
+    }
     uint32_t eb = cfg.episodes < 32u ? cfg.episodes : 32u;
     // few members: split the episodes of a member over more blocks to fill the SMs
     while (eb > 4u && static_cast<uint64_t>(cfg.pop_size) * ((cfg.episodes + eb - 1u) / eb) < 4u * 148u)
@@ -278,17 +222,15 @@ static size_t generic_smem_bytes(const RolloutMlpArgs& a, bool with_weights)
     return f * sizeof(float);
 }
 
-int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a);   // defined below
-bool rollout_mlp_tiled_available(const RolloutMlpArgs& a);
-
-int launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a_in, uint32_t kernel_choice, float* fitness)
+int launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a_in, uint32_t kernel_choice, float* fitness,
+                       DeviceStatus* status)
 {
     RolloutMlpArgs a = a_in;
     int launches = 0;
-    const bool tiled_ok = rollout_mlp_tiled_available(a);
+    const bool tiled_ok = rollout_mlp_tiled_shape(a.task, a.n_layers, a.sizes) >= 0;
     if (kernel_choice == EVO_ROLLOUT_TILED && !tiled_ok) return -2;
     if (tiled_ok && kernel_choice != EVO_ROLLOUT_GENERIC) {
-        const int r = launch_rollout_mlp_tiled(st, a);
+        const int r = launch_rollout_mlp_tiled(st, a, status);
         if (r < 0) return r;
         launches += r;
     } else {
@@ -307,11 +249,5 @@ int launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a_in, uint32_t ker
     if (cudaGetLastError() != cudaSuccess) return -1;
     return launches + 1;
 }
-
-// ------------------------------------------------------------------------------------------
-// tiled kernel (compile-time shapes) -- not built yet for any shape
-// ------------------------------------------------------------------------------------------
-bool rollout_mlp_tiled_available(const RolloutMlpArgs&) { return false; }
-int launch_rollout_mlp_tiled(cudaStream_t, const RolloutMlpArgs&) { return -2; }
 
 }  // namespace evo

@@ -1,0 +1,389 @@
+// Fast control-task rollout for compile-time network shapes.
+//
+// Block = (member, block of EB episodes).  The member's parameter row is fetched from HBM once
+// with a single bulk asynchronous copy (cp.async.bulk, completion on an mbarrier), then every
+// thread moves its slice of each weight matrix into REGISTERS, where it stays for all T steps:
+// the FP32 pipe needs one operand per FMA from somewhere, and shared memory (128 B/clk/SM) can
+// feed only a quarter of the 128 FMA lanes, so weights live in registers and only the small
+// activation vectors ([unit][episode], a few hundred bytes) travel through shared memory as
+// broadcast 128-bit loads.  A thread owns TI output rows x KS inputs of a layer; the S threads
+// that share a row group are adjacent lanes and combine their partial sums with shuffles.
+// Task state stays in registers / shared memory; nothing but the optional debug trace and one
+// partial return per block goes back to HBM.
+//
+// Paper: Section 2 (roll-out loop, central seeds), Section 4 (get_actions over the population
+// with parameters as data; stateless task step; identical initial observations).
+#include "internal.h"
+#include "noise.cuh"
+#include "tasks.cuh"
+
+namespace evo {
+
+// tanh(x) = 1 - 2/(exp(2x)+1) on the special-function unit; absolute error ~2e-7
+__device__ __forceinline__ float tanh_fast(float x)
+{
+    const float e = __expf(2.0f * x);
+    return 1.0f - __fdividef(2.0f, e + 1.0f);
+}
+
+template <int EB> struct EpVec;
+template <> struct EpVec<1> { static __device__ __forceinline__ void load(const float* p, float* a) { a[0] = p[0]; } };
+template <> struct EpVec<2> { static __device__ __forceinline__ void load(const float* p, float* a) {
+    const float2 v = *reinterpret_cast<const float2*>(p); a[0] = v.x; a[1] = v.y; } };
+template <> struct EpVec<4> { static __device__ __forceinline__ void load(const float* p, float* a) {
+    const float4 v = *reinterpret_cast<const float4*>(p); a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w; } };
+template <> struct EpVec<8> { static __device__ __forceinline__ void load(const float* p, float* a) {
+    const float4 v = reinterpret_cast<const float4*>(p)[0], u = reinterpret_cast<const float4*>(p)[1];
+    a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w; a[4] = u.x; a[5] = u.y; a[6] = u.z; a[7] = u.w; } };
+template <> struct EpVec<16> { static __device__ __forceinline__ void load(const float* p, float* a) {
+    EpVec<8>::load(p, a); EpVec<8>::load(p + 8, a + 8); } };
+
+__host__ __device__ constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x / 2); }
+
+// Sum v[0..N) over the S adjacent lanes that share a row group.  While more than one value is
+// left each stage halves the set a lane keeps (lanes exchange the halves they give up); after
+// that the remaining stages are plain butterflies.  On return the lane holds CNT = max(N/S, 1)
+// finished sums, v[0..CNT), belonging to indices [offset, offset + CNT).
+template <int N, int S>
+__device__ __forceinline__ int reduce_lanes(float (&v)[N], int s)
+{
+    int offset = 0;
+    int cur = N;
+#pragma unroll
+    for (int b = 0; b < ilog2(S); ++b) {
+        const bool upper = (s >> b) & 1;
+        if (cur > 1) {
+            const int half = cur / 2;
+#pragma unroll
+            for (int i = 0; i < N / 2; ++i) {
+                if (i < half) {
+                    const float keep = upper ? v[half + i] : v[i];
+                    const float give = upper ? v[i] : v[half + i];
+                    v[i] = keep + __shfl_xor_sync(0xffffffffu, give, 1 << b);
+                }
+            }
+            if (upper) offset += half;
+            cur = half;
+        } else {
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1 << b);
+        }
+    }
+    return offset;
+}
+
+// One dense layer y = f(W x + b) for EB episodes at once.
+//   NI inputs, NO outputs, thread tile TI rows x KS = NI/S inputs, S lanes per row group.
+template <int NI, int NO, int TI, int S, int EB, int THREADS>
+struct Dense {
+    static_assert(NI % S == 0, "S must divide the input width");
+    static_assert((S & (S - 1)) == 0 && S <= 32, "S is a power of two within a warp");
+    static constexpr int KS = NI / S;
+    static constexpr int GROUPS = (NO + TI - 1) / TI;
+    static constexpr int ACTIVE = GROUPS * S;
+    static_assert(ACTIVE <= THREADS, "layer needs more threads than the block has");
+    static constexpr int N = TI * EB;
+    static constexpr int CNT = (N >= S) ? N / S : 1;
+
+    float w[TI][KS];
+    float bias[TI];
+    int   row0, s;
+    bool  active;
+
+    // weights from a row-major [NO][NI] matrix followed by bias[NO] (shared or global memory)
+    __device__ __forceinline__ void load(const float* W, const float* b, int tid)
+    {
+        active = tid < ACTIVE;
+        s = tid % S;
+        row0 = (tid / S) * TI;
+#pragma unroll
+        for (int r = 0; r < TI; ++r) {
+            const bool ok = active && (row0 + r < NO);
+#pragma unroll
+            for (int k = 0; k < KS; ++k) w[r][k] = ok ? W[(row0 + r) * NI + s * KS + k] : 0.f;
+            bias[r] = (ok && s == 0 && b) ? b[row0 + r] : 0.f;
+        }
+    }
+
+    // in: [NI][EB], out: [NO][EB]; out = scale * tanh(.) if ACT else the plain sum
+    template <bool ACT, class Hook>
+    __device__ __forceinline__ void run(const float* __restrict__ in, float* __restrict__ out,
+                                        float scale, Hook&& hook) const
+    {
+        float acc[N];
+#pragma unroll
+        for (int r = 0; r < TI; ++r)
+#pragma unroll
+            for (int e = 0; e < EB; ++e) acc[r * EB + e] = bias[r];
+#pragma unroll
+        for (int k = 0; k < KS; ++k) {
+            float a[EB];
+            EpVec<EB>::load(in + (s * KS + k) * EB, a);
+            hook(k, a);
+#pragma unroll
+            for (int r = 0; r < TI; ++r)
+#pragma unroll
+                for (int e = 0; e < EB; ++e) acc[r * EB + e] = fmaf(w[r][k], a[e], acc[r * EB + e]);
+        }
+        const int offset = reduce_lanes<N, S>(acc, s);
+        // with N < S several lanes end with the same sum: the one whose spare bits are 0 writes
+        const bool writer = active && ((N >= S) || ((s >> ilog2(N)) == 0));
+        if (writer) {
+#pragma unroll
+            for (int i = 0; i < CNT; ++i) {
+                const int n = offset + i;
+                const int row = row0 + n / EB, e = n % EB;
+                if (row < NO) out[row * EB + e] = ACT ? scale * tanh_fast(acc[i]) : acc[i];
+            }
+        }
+    }
+};
+
+struct NoHook { __device__ __forceinline__ void operator()(int, const float*) const {} };
+
+// bounded wait on an mbarrier phase; returns false if it gave up
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t max_iter)
+{
+    for (uint32_t it = 0; it < max_iter; ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+        if (it > 64) __nanosleep(64);
+    }
+    return false;
+}
+
+template <int NIN, int H1, int H2, int NOUT, int EB, int THREADS, int TASK,
+          int TI1, int S1, int TI2, int S2, int TI3, int S3>
+__global__ void __launch_bounds__(THREADS)
+k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
+{
+    constexpr bool CART = (TASK == EVO_TASK_CARTPOLE);
+    constexpr int NOBS = CART ? 5 : (kTlNx + kTlNa);        // tanh-linear: [x ; a] feeds the dynamics
+    static_assert(CART ? (NIN == 5 && NOUT == 1) : (NIN == kTlNx && NOUT == kTlNa), "task/policy shape");
+
+    extern __shared__ __align__(128) float smem[];
+    __shared__ __align__(8) uint64_t mbar;
+    float* stage = smem;                                      // parameter row, ldD floats
+    float* obs0 = stage + a.ldD;                              // [NOBS][EB]
+    float* obs1 = obs0 + NOBS * EB;                           // second x buffer (tanh-linear)
+    float* h1 = obs1 + NOBS * EB;                             // [H1][EB]
+    float* h2 = h1 + H1 * EB;                                 // [H2][EB]
+    float* actb = h2 + H2 * EB;                               // [NOUT][EB] (cart-pole)
+
+    const int tid = threadIdx.x;
+    const uint32_t member = blockIdx.x, eb = blockIdx.y;
+    const uint32_t e0 = eb * EB;
+    const int nE = min(static_cast<uint32_t>(EB), a.E - e0);
+    const PhiloxKey key{ a.k0, a.k1 };
+
+    // ---- parameter row: one bulk copy HBM -> shared memory ---------------------------------
+    const uint32_t bar = static_cast<uint32_t>(__cvta_generic_to_shared(&mbar));
+    const uint32_t bytes = a.ldD * 4u;
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const float* src = a.theta + static_cast<size_t>(member) * a.ldD;
+        const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+    }
+
+    // ---- reset (overlaps the copy) -----------------------------------------------------------
+    CartpoleConst cpc{};
+    CpState cps{};
+    float ret = 0.f;                        // cart-pole: lane e of warp 0; tanh-linear: see below
+    if (CART) {
+        cpc = cartpole_const(a.tp);
+        if (tid < EB) {
+            cps = cartpole_reset(key, a.generation, e0 + min(tid, nE - 1), a.tp[EVO_CP_INIT_RANGE]);
+            float sn, cs;
+            sincosf(cps.th, &sn, &cs);
+            obs0[0 * EB + tid] = cps.x;  obs0[1 * EB + tid] = cps.xd;
+            obs0[2 * EB + tid] = cs;     obs0[3 * EB + tid] = sn;
+            obs0[4 * EB + tid] = cps.thd;
+        }
+    } else {
+        for (int item = tid; item < (kTlNx / 4) * EB; item += THREADS) {
+            const int q = item / EB, e = item % EB;
+            const float4 z = stream_normal4(key, 1u, a.generation, e0 + min(e, nE - 1), q);
+            obs0[(4 * q + 0) * EB + e] = z.x; obs0[(4 * q + 1) * EB + e] = z.y;
+            obs0[(4 * q + 2) * EB + e] = z.z; obs0[(4 * q + 3) * EB + e] = z.w;
+        }
+    }
+
+    // one thread waits (bounded) and publishes the outcome, so the whole block takes one branch
+    __shared__ int copy_ok;
+    if (tid == 0) {
+        copy_ok = mbar_wait(bar, 0u, 1u << 22) ? 1 : 0;
+        if (!copy_ok) {
+            // the copy did not land in time: flag it, give it one more bounded chance, leave
+            atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
+            mbar_wait(bar, 0u, 1u << 22);
+        }
+    }
+    __syncthreads();
+    if (!copy_ok) return;
+
+    // ---- weights into registers ----------------------------------------------------------------
+    Dense<NIN, H1, TI1, S1, EB, THREADS> L1;
+    Dense<H1, H2, TI2, S2, EB, THREADS> L2;
+    Dense<H2, NOUT, TI3, S3, EB, THREADS> L3;
+    {
+        const float* p = stage;
+        L1.load(p, p + H1 * NIN, tid); p += H1 * NIN + H1;
+        L2.load(p, p + H2 * H1, tid);  p += H2 * H1 + H2;
+        L3.load(p, p + NOUT * H2, tid);
+    }
+    // tanh-linear dynamics x' = tanh([A B][x ; a]) as a fourth layer with shared weights
+    constexpr int SD = CART ? 1 : 4;
+    constexpr int NID = CART ? 1 : NOBS, NOD = CART ? 1 : kTlNx;
+    Dense<NID, NOD, 1, SD, EB, THREADS> LD;
+    if (!CART) {
+        LD.active = tid < LD.ACTIVE; LD.s = tid % SD; LD.row0 = tid / SD; LD.bias[0] = 0.f;
+        const bool ok = LD.active && LD.row0 < NOD;
+#pragma unroll
+        for (int k = 0; k < LD.KS; ++k) {
+            const int col = LD.s * LD.KS + k;
+            const float* A = a.task_const;
+            const float* B = a.task_const + kTlNx * kTlNx;
+            LD.w[0][k] = !ok ? 0.f : (col < static_cast<int>(kTlNx) ? A[LD.row0 * kTlNx + col]
+                                                                    : B[LD.row0 * kTlNa + (col - kTlNx)]);
+        }
+    }
+    __syncthreads();
+
+    float* obs = obs0;
+    float* obs_next = obs1;
+    const bool tracing = a.trace != nullptr;
+
+    // ---- time loop -------------------------------------------------------------------------------
+    for (uint32_t t = 0; t < a.T; ++t) {
+        L1.template run<true>(obs, h1, 1.0f, NoHook{});
+        __syncthreads();
+        L2.template run<true>(h1, h2, 1.0f, NoHook{});
+        __syncthreads();
+        if (CART) {
+            L3.template run<true>(h2, actb, a.action_scale, NoHook{});
+            __syncthreads();
+            if (tid < EB) {
+                cps = cartpole_step(cpc, cps, actb[tid]);
+                float sn, cs;
+                sincosf(cps.th, &sn, &cs);
+                ret += cs * __expf(-cps.x * cps.x);           // reward on the post-step state
+                obs[0 * EB + tid] = cps.x;  obs[1 * EB + tid] = cps.xd;
+                obs[2 * EB + tid] = cs;     obs[3 * EB + tid] = sn;
+                obs[4 * EB + tid] = cps.thd;
+                if (tracing && t < a.trace_T && tid < nE) {
+                    float4* tr = reinterpret_cast<float4*>(
+                        a.trace + ((static_cast<size_t>(member) * a.E + e0 + tid) * a.trace_T + t) * 4);
+                    *tr = make_float4(cps.x, cps.xd, cps.th, cps.thd);
+                }
+            }
+            __syncthreads();
+        } else {
+            // actions go straight behind x so that [x ; a] is one input vector of the dynamics
+            L3.template run<true>(h2, obs + kTlNx * EB, a.action_scale, NoHook{});
+            __syncthreads();
+            // reward -|x|^2 - 0.01|a|^2 on (x_t, a_t): the S lanes of row group 0 see every input
+            float sq[EB];
+#pragma unroll
+            for (int e = 0; e < EB; ++e) sq[e] = 0.f;
+            const int sD = LD.s, KSD = LD.KS;
+            const bool group0 = tid < SD;
+            LD.template run<true>(obs, obs_next, 1.0f, [&](int k, const float* v) {
+                if (group0) {
+                    const float c = (sD * KSD + k < static_cast<int>(kTlNx)) ? -1.0f : -0.01f;
+#pragma unroll
+                    for (int e = 0; e < EB; ++e) sq[e] = fmaf(c * v[e], v[e], sq[e]);
+                }
+            });
+            if (tid < SD) {                                    // row group 0, whole warp-converged
+#pragma unroll
+                for (int e = 0; e < EB; ++e) if (e < nE) ret += sq[e];
+            }
+            if (tracing && t < a.trace_T) {
+                __syncthreads();
+                for (int item = tid; item < static_cast<int>(kTlNx) * nE; item += THREADS) {
+                    const int i = item / nE, e = item % nE;
+                    a.trace[((static_cast<size_t>(member) * a.E + e0 + e) * a.trace_T + t) * kTlNx + i] =
+                        obs_next[i * EB + e];
+                }
+            }
+            __syncthreads();
+            float* tmp = obs; obs = obs_next; obs_next = tmp;
+        }
+    }
+
+    // ---- block return: fixed-order sum over the block's episodes ---------------------------------
+    if (tid < 32) {
+        float v;
+        if (CART) v = (tid < nE) ? ret : 0.f;
+        else      v = (tid < SD) ? ret : 0.f;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        if (tid == 0) a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// shapes with a compiled kernel
+// ------------------------------------------------------------------------------------------
+struct TiledShape { uint32_t task, nin, h1, h2, nout, EB; };
+static const TiledShape kShapes[] = {
+    { EVO_TASK_CARTPOLE, 5, 16, 16, 1, 1 },
+    { EVO_TASK_CARTPOLE, 5, 64, 64, 1, 8 },
+    { EVO_TASK_TANH_LINEAR, 28, 128, 128, 8, 4 },
+};
+
+int rollout_mlp_tiled_shape(uint32_t task, uint32_t n_layers, const uint32_t* sizes)
+{
+    if (n_layers != 3) return -1;
+    for (int i = 0; i < static_cast<int>(sizeof(kShapes) / sizeof(kShapes[0])); ++i) {
+        const TiledShape& s = kShapes[i];
+        if (s.task == task && s.nin == sizes[0] && s.h1 == sizes[1] && s.h2 == sizes[2] && s.nout == sizes[3])
+            return i;
+    }
+    return -1;
+}
+
+uint32_t rollout_mlp_tiled_eb(int shape) { return kShapes[shape].EB; }
+
+template <class K>
+static int launch_one(K kernel, int threads, size_t act_floats, cudaStream_t st, const RolloutMlpArgs& a,
+                      DeviceStatus* status)
+{
+    const size_t bytes = (static_cast<size_t>(a.ldD) + act_floats) * sizeof(float);
+    if (bytes > 220u * 1024u) return -2;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) != cudaSuccess)
+        return -1;
+    dim3 grid(a.P, a.n_eb);
+    kernel<<<grid, threads, bytes, st>>>(a, status);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus* status)
+{
+    const int shape = rollout_mlp_tiled_shape(a.task, a.n_layers, a.sizes);
+    if (shape < 0 || a.EB != kShapes[shape].EB) return -2;
+    switch (shape) {
+        case 0:
+            return launch_one(k_rollout_mlp_tiled<5, 16, 16, 1, 1, 32, EVO_TASK_CARTPOLE, 1, 1, 1, 2, 1, 16>,
+                              32, (2 * 5 + 16 + 16 + 1) * 1, st, a, status);
+        case 1:
+            return launch_one(k_rollout_mlp_tiled<5, 64, 64, 1, 8, 64, EVO_TASK_CARTPOLE, 1, 1, 4, 4, 1, 32>,
+                              64, (2 * 5 + 64 + 64 + 1) * 8, st, a, status);
+        case 2:
+            return launch_one(k_rollout_mlp_tiled<28, 128, 128, 8, 4, 128, EVO_TASK_TANH_LINEAR, 4, 4, 4, 4, 1, 16>,
+                              128, (2 * 36 + 128 + 128 + 8) * 4, st, a, status);
+    }
+    return -2;
+}
+
+}  // namespace evo
