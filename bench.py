@@ -393,7 +393,7 @@ def run_ours(args, w):
                         "peak_source": f"{sm_count} SMs x 128 fp32 lanes x 2 x {max_mhz} MHz",
                         "traffic": None}
         cpu = None
-        if world == 1 or rank == 0:
+        if not args.skip_cpu_baseline:
             n = members_for_budget(w, 12.0)
             t_cpu, sample = oracle_generation_sample(w, max(n, 1))
             cpu = {"value": units_per_gen / t_cpu, "unit": unit, "cores": 1, "kind": "oracle",
@@ -421,6 +421,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--noise", default="stored", choices=["stored", "regenerated"])
+    ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing leg")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (experiments)")
     ap.add_argument("--dim", type=int, default=0, help="override the parameter count (cfg5 only)")
     args = ap.parse_args()

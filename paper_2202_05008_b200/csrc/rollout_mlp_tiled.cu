@@ -6,7 +6,8 @@
 // the FP32 pipe needs one operand per FMA from somewhere, and shared memory (128 B/clk/SM) can
 // feed only a quarter of the 128 FMA lanes, so weights live in registers and only the small
 // activation vectors ([unit][episode], a few hundred bytes) travel through shared memory as
-// broadcast 128-bit loads.  A thread owns TI output rows x KS inputs of a layer; the S threads
+// broadcast 128-bit loads.  A thread owns TI output rows x KS inputs of a layer (inputs s, s+S,
+// s+2S, ... so that the S lanes read adjacent shared-memory words); the S threads
 // that share a row group are adjacent lanes and combine their partial sums with shuffles.
 // Task state stays in registers / shared memory; nothing but the optional debug trace and one
 // partial return per block goes back to HBM.
@@ -99,7 +100,7 @@ struct Dense {
         for (int r = 0; r < TI; ++r) {
             const bool ok = active && (row0 + r < NO);
 #pragma unroll
-            for (int k = 0; k < KS; ++k) w[r][k] = ok ? W[(row0 + r) * NI + s * KS + k] : 0.f;
+            for (int k = 0; k < KS; ++k) w[r][k] = ok ? W[(row0 + r) * NI + k * S + s] : 0.f;
             bias[r] = (ok && s == 0 && b) ? b[row0 + r] : 0.f;
         }
     }
@@ -117,8 +118,8 @@ struct Dense {
 #pragma unroll
         for (int k = 0; k < KS; ++k) {
             float a[EB];
-            EpVec<EB>::load(in + (s * KS + k) * EB, a);
-            hook(k, a);
+            EpVec<EB>::load(in + (k * S + s) * EB, a);     // lane s takes inputs s, s+S, ... (no bank conflicts)
+            hook(k * S + s, a);
 #pragma unroll
             for (int r = 0; r < TI; ++r)
 #pragma unroll
@@ -128,11 +129,25 @@ struct Dense {
         // with N < S several lanes end with the same sum: the one whose spare bits are 0 writes
         const bool writer = active && ((N >= S) || ((s >> ilog2(N)) == 0));
         if (writer) {
+            if constexpr (CNT >= EB && EB >= 4) {              // whole rows: 128-bit stores
 #pragma unroll
-            for (int i = 0; i < CNT; ++i) {
-                const int n = offset + i;
-                const int row = row0 + n / EB, e = n % EB;
-                if (row < NO) out[row * EB + e] = ACT ? scale * tanh_fast(acc[i]) : acc[i];
+                for (int i = 0; i < CNT; i += 4) {
+                    const int n = offset + i;
+                    const int row = row0 + n / EB, e = n % EB;
+                    float4 y;
+                    y.x = ACT ? scale * tanh_fast(acc[i + 0]) : acc[i + 0];
+                    y.y = ACT ? scale * tanh_fast(acc[i + 1]) : acc[i + 1];
+                    y.z = ACT ? scale * tanh_fast(acc[i + 2]) : acc[i + 2];
+                    y.w = ACT ? scale * tanh_fast(acc[i + 3]) : acc[i + 3];
+                    if (row < NO) *reinterpret_cast<float4*>(out + row * EB + e) = y;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < CNT; ++i) {
+                    const int n = offset + i;
+                    const int row = row0 + n / EB, e = n % EB;
+                    if (row < NO) out[row * EB + e] = ACT ? scale * tanh_fast(acc[i]) : acc[i];
+                }
             }
         }
     }
@@ -162,6 +177,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
 {
     constexpr bool CART = (TASK == EVO_TASK_CARTPOLE);
     constexpr int NOBS = CART ? 5 : (kTlNx + kTlNa);        // tanh-linear: [x ; a] feeds the dynamics
+    static_assert(!CART || S3 * ((NOUT + TI3 - 1) / TI3) <= 32, "cart-pole action layer runs in warp 0");
     static_assert(CART ? (NIN == 5 && NOUT == 1) : (NIN == kTlNx && NOUT == kTlNa), "task/policy shape");
 
     extern __shared__ __align__(128) float smem[];
@@ -204,7 +220,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
         if (tid < EB) {
             cps = cartpole_reset(key, a.generation, e0 + min(tid, nE - 1), a.tp[EVO_CP_INIT_RANGE]);
             float sn, cs;
-            sincosf(cps.th, &sn, &cs);
+            sincos_fast(cps.th, sn, cs);
             obs0[0 * EB + tid] = cps.x;  obs0[1 * EB + tid] = cps.xd;
             obs0[2 * EB + tid] = cs;     obs0[3 * EB + tid] = sn;
             obs0[4 * EB + tid] = cps.thd;
@@ -250,7 +266,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
         const bool ok = LD.active && LD.row0 < NOD;
 #pragma unroll
         for (int k = 0; k < LD.KS; ++k) {
-            const int col = LD.s * LD.KS + k;
+            const int col = k * SD + LD.s;
             const float* A = a.task_const;
             const float* B = a.task_const + kTlNx * kTlNx;
             LD.w[0][k] = !ok ? 0.f : (col < static_cast<int>(kTlNx) ? A[LD.row0 * kTlNx + col]
@@ -270,20 +286,23 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
         L2.template run<true>(h1, h2, 1.0f, NoHook{});
         __syncthreads();
         if (CART) {
-            L3.template run<true>(h2, actb, a.action_scale, NoHook{});
-            __syncthreads();
-            if (tid < EB) {
-                cps = cartpole_step(cpc, cps, actb[tid]);
-                float sn, cs;
-                sincosf(cps.th, &sn, &cs);
-                ret += cs * __expf(-cps.x * cps.x);           // reward on the post-step state
-                obs[0 * EB + tid] = cps.x;  obs[1 * EB + tid] = cps.xd;
-                obs[2 * EB + tid] = cs;     obs[3 * EB + tid] = sn;
-                obs[4 * EB + tid] = cps.thd;
-                if (tracing && t < a.trace_T && tid < nE) {
-                    float4* tr = reinterpret_cast<float4*>(
-                        a.trace + ((static_cast<size_t>(member) * a.E + e0 + tid) * a.trace_T + t) * 4);
-                    *tr = make_float4(cps.x, cps.xd, cps.th, cps.thd);
+            // the action and the task step are one warp's work: no block-wide barrier in between
+            if (tid < 32) {
+                L3.template run<true>(h2, actb, a.action_scale, NoHook{});
+                __syncwarp();
+                if (tid < EB) {
+                    cps = cartpole_step_fast(cpc, cps, actb[tid]);
+                    float sn, cs;
+                    sincos_fast(cps.th, sn, cs);
+                    ret += cs * __expf(-cps.x * cps.x);       // reward on the post-step state
+                    obs[0 * EB + tid] = cps.x;  obs[1 * EB + tid] = cps.xd;
+                    obs[2 * EB + tid] = cs;     obs[3 * EB + tid] = sn;
+                    obs[4 * EB + tid] = cps.thd;
+                    if (tracing && t < a.trace_T && tid < nE) {
+                        float4* tr = reinterpret_cast<float4*>(
+                            a.trace + ((static_cast<size_t>(member) * a.E + e0 + tid) * a.trace_T + t) * 4);
+                        *tr = make_float4(cps.x, cps.xd, cps.th, cps.thd);
+                    }
                 }
             }
             __syncthreads();
@@ -295,11 +314,10 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
             float sq[EB];
 #pragma unroll
             for (int e = 0; e < EB; ++e) sq[e] = 0.f;
-            const int sD = LD.s, KSD = LD.KS;
             const bool group0 = tid < SD;
-            LD.template run<true>(obs, obs_next, 1.0f, [&](int k, const float* v) {
+            LD.template run<true>(obs, obs_next, 1.0f, [&](int col, const float* v) {
                 if (group0) {
-                    const float c = (sD * KSD + k < static_cast<int>(kTlNx)) ? -1.0f : -0.01f;
+                    const float c = (col < static_cast<int>(kTlNx)) ? -1.0f : -0.01f;
 #pragma unroll
                     for (int e = 0; e < EB; ++e) sq[e] = fmaf(c * v[e], v[e], sq[e]);
                 }

@@ -76,4 +76,58 @@ __device__ __forceinline__ CpState cartpole_reset(PhiloxKey key, uint32_t genera
 }
 
 
+// ---- latency-trimmed variants for the tiled kernel ---------------------------------------------
+// The roll-out is a serial chain per episode, so the task step's dependent-instruction latency
+// sets the step time.  sin/cos by quarter-turn reduction (two-term pi/2) and short Taylor
+// polynomials evaluated side by side (abs. error < 1e-7 for |theta| < 1e3), divisions by
+// reciprocal approximation (2 ulp).
+
+__device__ __forceinline__ void sincos_fast(float th, float& sn, float& cs)
+{
+    const float kf = rintf(th * 0.636619772f);
+    float r = fmaf(kf, -1.57079637f, th);
+    r = fmaf(kf, 4.37113883e-8f, r);
+    const float z = r * r;
+    float sp = fmaf(z, 2.75573192e-6f, -1.98412698e-4f);
+    float cp = fmaf(z, 2.48015873e-5f, -1.38888889e-3f);
+    sp = fmaf(sp, z, 8.33333333e-3f);
+    cp = fmaf(cp, z, 4.16666667e-2f);
+    sp = fmaf(sp, z, -1.66666667e-1f);
+    cp = fmaf(cp, z, -0.5f);
+    const float s0 = fmaf(sp * z, r, r);
+    const float c0 = fmaf(cp, z, 1.0f);
+    const int q = __float2int_rn(kf) & 3;
+    const float a = (q & 1) ? s0 : c0;
+    const float b = (q & 1) ? c0 : s0;
+    cs = (q == 1 || q == 2) ? -a : a;
+    sn = (q >= 2) ? -b : b;
+}
+
+__device__ __forceinline__ CpState cartpole_deriv_fast(const CartpoleConst& c, const CpState& s, float force)
+{
+    float sn, cs;
+    sincos_fast(s.th, sn, cs);
+    const float tmp = fmaf(c.pole_mass_length * s.thd * s.thd, sn, force) * c.inv_total;
+    const float den = c.length * fmaf(-c.pole_mass * c.inv_total * cs, cs, 4.0f / 3.0f);
+    const float th_acc = __fdividef(fmaf(c.gravity, sn, -cs * tmp), den);
+    const float x_acc = fmaf(-c.pole_mass_length * c.inv_total * th_acc, cs, tmp);
+    return CpState{ s.xd, x_acc, s.thd, th_acc };
+}
+
+__device__ __forceinline__ CpState cartpole_step_fast(const CartpoleConst& c, const CpState& s, float force)
+{
+    const float h = c.dt;
+    const CpState k1 = cartpole_deriv_fast(c, s, force);
+    const CpState k2 = cartpole_deriv_fast(c, cp_axpy(s, 0.5f * h, k1), force);
+    const CpState k3 = cartpole_deriv_fast(c, cp_axpy(s, 0.5f * h, k2), force);
+    const CpState k4 = cartpole_deriv_fast(c, cp_axpy(s, h, k3), force);
+    const float w = h * (1.0f / 6.0f);
+    CpState n;
+    n.x   = fmaf(w, (k1.x   + k4.x)   + 2.0f * (k2.x   + k3.x),   s.x);
+    n.xd  = fmaf(w, (k1.xd  + k4.xd)  + 2.0f * (k2.xd  + k3.xd),  s.xd);
+    n.th  = fmaf(w, (k1.th  + k4.th)  + 2.0f * (k2.th  + k3.th),  s.th);
+    n.thd = fmaf(w, (k1.thd + k4.thd) + 2.0f * (k2.thd + k3.thd), s.thd);
+    return n;
+}
+
 }  // namespace evo
