@@ -164,6 +164,36 @@ evo_status evo_sync_status(evo_solver* s);
 /* Number of kernels the library has launched for this solver so far. */
 evo_status evo_launch_count(evo_solver* s, uint64_t* launches);
 
+/*
+ * ES gradient without any device allocation (the paper has no counterpart: this entry point
+ * exists for deployment reasons only).  It is meant for callers that are not allowed to
+ * allocate device memory after start-up and therefore cannot hand evo_create a workspace: a
+ * service that distributes all GPU memory once when it boots, or a plug-in inside a host
+ * framework whose allocator owns the device.  Computes, like the gradient stage of evo_tell,
+ *     d_gradient[d] = (sigma / pop_size) * sum_j (d_u[2j] - d_u[2j+1]) * d_eps[j * ld_eps + d]
+ * for d < param_dim, with fp64 partial sums.  d_u[pop_size] (centred-rank weights, fp32),
+ * d_eps[pop_size/2][ld_eps] (fp32, ld_eps >= param_dim) and d_gradient[param_dim] are the
+ * caller's device buffers; nothing else is needed.
+ *   - The split partial sums live in a fixed array of EVO_STATIC_SCRATCH_BYTES that is part of
+ *     the library image: every GPU that loads the library carries it until the process ends.
+ *     Limit: param_dim rounded up to a multiple of 32 must not exceed
+ *     EVO_STATIC_SCRATCH_BYTES / 8 (= 524,288); larger problems return EVO_ERR_WORKSPACE and
+ *     must use evo_create / evo_tell with a caller workspace.
+ *   - The device that owns the buffers must be current.  The first call on each device looks
+ *     up the array's device address (no allocation); make that first call outside of any
+ *     stream capture.  No call allocates, frees or synchronises.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left;
+ *     each call overwrites every word it reads back, so nothing needs clearing.  Two calls
+ *     whose kernels may overlap on the GPU (different streams, or the same stream from two
+ *     threads) race on it: serialise them.
+ * Errors: INVALID_ARG (NULL pointer, odd or zero pop_size, ld_eps < param_dim), WORKSPACE
+ * (param_dim beyond the limit), CUDA (address lookup or launch failed).
+ */
+#define EVO_STATIC_SCRATCH_BYTES (4u << 20)
+evo_status evo_es_gradient_static(const float* d_u, const float* d_eps, uint32_t pop_size,
+                                  uint32_t param_dim, size_t ld_eps, float sigma,
+                                  float* d_gradient, void* cuda_stream);
+
 const char* evo_status_string(evo_status st);
 uint32_t    evo_version(void);            /* major*10000 + minor*100 + patch */
 

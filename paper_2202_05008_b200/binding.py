@@ -73,6 +73,8 @@ def load_library():
     L.evo_set_state.argtypes = [vp, vp, vp, vp, C.c_uint32, C.c_uint32]
     L.evo_sync_status.argtypes = [vp]
     L.evo_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+    L.evo_es_gradient_static.argtypes = [vp, vp, C.c_uint32, C.c_uint32, C.c_size_t, C.c_float, vp, vp]
+    L.evo_es_gradient_static.restype = C.c_int
     L.evo_status_string.argtypes = [C.c_int]
     L.evo_status_string.restype = C.c_char_p
     L.evo_version.restype = C.c_uint32
@@ -234,3 +236,26 @@ class Solver:
         n = C.c_uint64()
         _check(self.lib.evo_launch_count(self._h, C.byref(n)), "evo_launch_count")
         return n.value
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def es_gradient_static(u: torch.Tensor, eps: torch.Tensor, sigma: float,
+                       out: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """ES gradient through ``evo_es_gradient_static``: no workspace, no allocation inside the
+    library (its scratch is a fixed array in the library image).  ``u`` is [P] fp32, ``eps`` is
+    [P/2][D] fp32 with unit column stride (any row pitch); returns g[D].  Meant for hosts that
+    forbid device allocation after start-up; pass ``out`` to keep this wrapper allocation-free
+    as well.  Calls that may overlap on the GPU must be serialised by the caller."""
+    lib = load_library()
+    assert u.dtype == torch.float32 and eps.dtype == torch.float32 and u.is_cuda and eps.is_cuda
+    assert u.is_contiguous() and eps.stride(1) == 1 and eps.shape[0] * 2 == u.numel()
+    P, D = u.numel(), eps.shape[1]
+    if out is None:
+        out = torch.empty(D, dtype=torch.float32, device=u.device)
+    with torch.cuda.device(u.device):
+        st = stream if stream is not None else torch.cuda.current_stream(u.device)
+        _check(lib.evo_es_gradient_static(u.data_ptr(), eps.data_ptr(), P, D, eps.stride(0), float(sigma),
+                                          out.data_ptr(), st.cuda_stream), "evo_es_gradient_static")
+    return out
