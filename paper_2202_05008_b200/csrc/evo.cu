@@ -80,7 +80,13 @@ static evo_status make_layout(const evo_config& c, Layout* L)
     L->grad_partial = take(2 * row * L->grad_splits);          // fp64 partial sums
     L->fit_partial = take(P * L->n_eb * sizeof(float));
     L->task_const = take(kTlNx * (kTlNx + kTlNa) * sizeof(float));
-    L->cnn_scratch = take(c.task_kind == EVO_TASK_SUPERVISED ? cnn_scratch_bytes(c.pop_size, c.batch) : 0);
+    size_t cnn = 0;
+    if (c.task_kind == EVO_TASK_SUPERVISED) {
+        cnn = cnn_scratch_bytes(c.pop_size, c.batch);
+        const size_t tc = cnn_tc_scratch_bytes(c.pop_size, c.batch);
+        if (tc > cnn) cnn = tc;
+    }
+    L->cnn_scratch = take(cnn);
     L->theta = take(row * P);
     L->eps = take(c.noise_mode == EVO_NOISE_STORED ? row * H : 0);
     L->total = off;
@@ -184,8 +190,13 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
     if (c.task_kind == EVO_TASK_SUPERVISED) {
         if (!s->d_images) return EVO_ERR_BAD_ORDER;
         if (d_trace) return EVO_ERR_UNSUPPORTED;
-        const int n = launch_rollout_cnn(s->stream, d_theta, L.ldD, c.pop_size, s->d_images, s->d_labels,
-                                         c.batch, s->ws + L.cnn_scratch, d_fitness);
+        // GENERIC selects the CUDA-core kernel, anything else the tensor-core path
+        const int n = c.rollout_kernel == EVO_ROLLOUT_GENERIC
+            ? launch_rollout_cnn(s->stream, d_theta, L.ldD, c.pop_size, s->d_images, s->d_labels, c.batch,
+                                 s->ws + L.cnn_scratch, d_fitness)
+            : launch_rollout_cnn_tc(s->stream, d_theta, L.ldD, c.pop_size, s->d_images, s->d_labels, c.batch,
+                                    s->ws + L.cnn_scratch, d_fitness,
+                                    reinterpret_cast<DeviceStatus*>(s->ws + L.status));
         if (n < 0) return n == -2 ? EVO_ERR_UNSUPPORTED : EVO_ERR_CUDA;
         s->launches += n;
         return EVO_OK;

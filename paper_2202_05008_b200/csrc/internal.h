@@ -65,6 +65,10 @@ bool rollout_mlp_supported(const evo_config& cfg);
 void rollout_mlp_plan(const evo_config& cfg, uint32_t* EB, uint32_t* n_eb);
 
 size_t cnn_scratch_bytes(uint32_t P, uint32_t batch);
+size_t cnn_tc_scratch_bytes(uint32_t P, uint32_t batch);
+int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uint32_t P, const float* images,
+                          const int32_t* labels, uint32_t batch, void* scratch, float* fitness,
+                          DeviceStatus* status);
 int launch_rollout_cnn(cudaStream_t st, const float* theta, uint32_t ldD, uint32_t P,
                        const float* images, const int32_t* labels, uint32_t batch, void* scratch,
                        float* fitness);

@@ -1,0 +1,532 @@
+// Supervised rollout on the 5th-generation tensor cores (tcgen05, accumulators in TMEM).
+//
+// The convolutional policy (conv 1->8 5x5, ReLU, pool; conv 8->16 5x5, ReLU, pool; linear
+// 256->10) evaluated for every member on the same batch is two dense contractions:
+//
+//   k_cnn_conv1_tc   conv1 for ALL members at once.  The batch is shared, so the im2col rows
+//                    (one per output pixel, K = 25 taps padded to 32) are the A operand for every
+//                    member, and the 8P filters of the population sit side by side on N:
+//                    D[128 pixels][256 filters] per tcgen05.mma, 512 TMEM columns per tile.  The
+//                    epilogue takes bias/ReLU/2x2-max-pool out of TMEM and writes the pooled
+//                    activation as bf16, 8 channels = 16 bytes per pixel.
+//   k_cnn_conv2_tc   per member: conv2 as an implicit GEMM with NO im2col copy.  With channels
+//                    innermost, the 8 channels of a pixel are one 16-byte row of a UMMA core
+//                    matrix, 8 consecutive output columns are 8 consecutive pixels = one 128-byte
+//                    core matrix, and the (kh,kw) tap is just an address offset, so the shared
+//                    memory descriptors of the A operand point straight into the pooled image
+//                    pair that a single bulk copy brought in.  D[128 = 2 images x 8x8][16 filters]
+//                    in TMEM; pool, linear layer and cross-entropy on CUDA cores.
+//
+// Operands are bf16 (round to nearest even), accumulation fp32 in TMEM.  Every wait is bounded:
+// on expiry the block records EVO_ERR_TIMEOUT, frees its TMEM and leaves.
+// Paper: Section 3 (supervised tasks are single-step tasks; ConvNet on 28x28 images).
+#include "internal.h"
+#include <cuda_bf16.h>
+
+namespace evo {
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// K-major operand without swizzle: 8-row x 16-byte core matrices; lbo = bytes between the core
+// matrices adjacent in K, sbo = bytes between 8-row groups adjacent in M (or N).
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32;
+    d |= static_cast<uint64_t>(1) << 46;                 // descriptor version of sm_100
+    return d;                                            // layout type 0: no swizzle
+}
+
+// kind::f16 instruction descriptor: bf16 x bf16 -> fp32, both operands K-major
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(uint32_t M, uint32_t N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 :: "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(slot_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// 32 lanes x 16 consecutive 32-bit columns: thread = lane, r[i] = column i
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* r)
+{
+    uint32_t u[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+                   "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(u[i]);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t max_iter)
+{
+    for (uint32_t it = 0; it < max_iter; ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+        if (it > 32) __nanosleep(32);
+    }
+    return false;
+}
+constexpr uint32_t kWaitIters = 1u << 22;
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// ------------------------------------------------------------------------------------------
+// conv1 for a group of up to 64 members
+// ------------------------------------------------------------------------------------------
+constexpr int kC1Threads = 128;
+constexpr int kC1SmemB = 512 * 32 * 2;        // all filters of the group, bf16, K = 32
+constexpr int kC1SmemA = 128 * 32 * 2;        // one im2col tile
+constexpr int kC1Dyn = kC1SmemB + kC1SmemA + 512 * 4;
+// the block owns all 512 TMEM columns, so it must be alone on its SM: ask for more than half
+// of the SM's shared memory
+constexpr int kC1DynRequest = 120 * 1024;
+
+// pooled-1 layout: [member][image pair][y 12][image in pair 2][x 12][channel 8] bf16
+__device__ __forceinline__ size_t pooled1_offset(uint32_t member, uint32_t n_pairs, uint32_t image,
+                                                 uint32_t py, uint32_t px)
+{
+    return (((static_cast<size_t>(member) * n_pairs + (image >> 1)) * 12 + py) * 2 + (image & 1u)) * 12 + px;
+}
+
+__global__ void __launch_bounds__(kC1Threads, 1)
+k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const float* __restrict__ images,
+               uint32_t batch, uint4* __restrict__ pooled1, uint32_t* work_counter, DeviceStatus* status)
+{
+    extern __shared__ __align__(1024) unsigned char dyn[];
+    __shared__ __align__(8) uint64_t mma_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int wait_ok;
+
+    unsigned char* Bsm = dyn;
+    unsigned char* Asm = dyn + kC1SmemB;
+    float* bias = reinterpret_cast<float*>(dyn + kC1SmemB + kC1SmemA);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t group0 = blockIdx.y * 64u;                         // first member of this group
+    const uint32_t n_members = min(64u, P - group0);
+    const uint32_t n_half = (n_members > 32u) ? 2u : 1u;
+    const uint32_t n_pairs = (batch + 1u) / 2u;
+    const uint32_t n_pooled = batch * 144u;
+    const uint32_t n_tiles = (n_pooled + 31u) / 32u;
+
+    if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *work_counter = 0;   // for the conv2 kernel
+
+    // ---- B operand: W1 of every member of the group, [filter][k] -> core matrices (k-group, n-group)
+    for (uint32_t idx = tid; idx < 512u * 4u; idx += kC1Threads) {
+        const uint32_t f = idx >> 2, kg = idx & 3u;                   // filter, 8-tap group
+        const uint32_t m = f >> 3, ch = f & 7u;
+        uint32_t w[4] = { 0, 0, 0, 0 };
+        if (m < n_members) {
+            const float* src = theta + static_cast<size_t>(group0 + m) * ldD + ch * 25u + kg * 8u;
+            float v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v[k] = (kg * 8u + k < 25u) ? src[k] : 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) w[k] = pack_bf16(v[2 * k], v[2 * k + 1]);
+        }
+        *reinterpret_cast<uint4*>(Bsm + (kg * 64u + (f >> 3)) * 128u + (f & 7u) * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    for (uint32_t f = tid; f < 512u; f += kC1Threads)
+        bias[f] = ((f >> 3) < n_members) ? theta[static_cast<size_t>(group0 + (f >> 3)) * ldD + 200u + (f & 7u)] : 0.f;
+
+    const uint32_t bar = smem_u32(&mma_bar);
+    if (tid == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512);
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+    constexpr uint32_t idesc = umma_idesc_bf16(128, 256);
+    uint32_t phase = 0;
+    bool failed = false;
+
+    for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        // ---- A operand: im2col rows, row m = (pooled pixel m/4, window element m%4) ----------
+        {
+            const uint32_t gp = tile * 32u + (tid >> 2), wnd = tid & 3u;
+            uint32_t packed[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) packed[k] = 0;
+            if (gp < n_pooled) {
+                const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
+                const float* src = images + static_cast<size_t>(img) * 784u + (2u * py + (wnd >> 1)) * 28u + 2u * px + (wnd & 1u);
+                float v[26];
+#pragma unroll
+                for (int kh = 0; kh < 5; ++kh)
+#pragma unroll
+                    for (int kw = 0; kw < 5; ++kw) v[kh * 5 + kw] = __ldg(src + kh * 28 + kw);
+                v[25] = 0.f;
+#pragma unroll
+                for (int k = 0; k < 13; ++k) packed[k] = pack_bf16(v[2 * k], v[2 * k + 1]);
+            }
+#pragma unroll
+            for (int kg = 0; kg < 4; ++kg)
+                *reinterpret_cast<uint4*>(Asm + (kg * 16 + (tid >> 3)) * 128 + (tid & 7) * 16) =
+                    make_uint4(packed[4 * kg], packed[4 * kg + 1], packed[4 * kg + 2], packed[4 * kg + 3]);
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t a0 = smem_u32(Asm), b0 = smem_u32(Bsm);
+            for (uint32_t h = 0; h < n_half; ++h)
+                for (uint32_t ks = 0; ks < 2u; ++ks) {
+                    const uint64_t ad = umma_smem_desc(a0 + ks * 2u * 2048u, 2048u, 128u);
+                    const uint64_t bd = umma_smem_desc(b0 + ks * 2u * 8192u + h * 4096u, 8192u, 128u);
+                    umma_bf16(tmem + h * 256u, ad, bd, idesc, ks);
+                }
+            umma_commit(bar);
+            wait_ok = mbar_wait_bounded(bar, phase, kWaitIters) ? 1 : 0;
+        }
+        __syncthreads();
+        if (!wait_ok) { failed = true; break; }
+        phase ^= 1u;
+        tc_fence_after();
+
+        // ---- epilogue: 32 filters (4 members) at a time; 2x2 max over the 4 lanes of a pixel ----
+        const uint32_t gp = tile * 32u + warp * 8u + (lane >> 2);
+        const bool pix_ok = gp < n_pooled;
+        const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
+        const bool b0 = lane & 1, b1 = lane & 2;
+        for (uint32_t grp = 0; grp < n_half * 8u; ++grp) {
+            float r[32];
+            const uint32_t taddr = tmem + (static_cast<uint32_t>(warp * 32) << 16) + grp * 32u;
+            tmem_ld16(taddr, r);
+            tmem_ld16(taddr + 16u, r + 16);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float keep = b0 ? r[16 + i] : r[i];
+                const float give = b0 ? r[i] : r[16 + i];
+                r[i] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 1));
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float keep = b1 ? r[8 + i] : r[i];
+                const float give = b1 ? r[i] : r[8 + i];
+                r[i] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 2));
+            }
+            const uint32_t m = grp * 4u + (b0 ? 2u : 0u) + (b1 ? 1u : 0u);   // member whose 8 channels I hold
+            if (pix_ok && m < n_members) {
+                const float* bb = bias + m * 8u;
+                uint32_t o[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    o[c] = pack_bf16(fmaxf(r[2 * c] + bb[2 * c], 0.f), fmaxf(r[2 * c + 1] + bb[2 * c + 1], 0.f));
+                pooled1[pooled1_offset(group0 + m, n_pairs, img, py, px)] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+            __syncwarp();
+        }
+        tc_fence_before();
+        __syncthreads();
+    }
+
+    if (failed && tid == 0) atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+// ------------------------------------------------------------------------------------------
+// conv2 + pool + linear + cross-entropy, one work item = (member, 16 image pairs)
+// ------------------------------------------------------------------------------------------
+constexpr int kC2Threads = 128;
+constexpr int kPairsPerItem = 16;
+constexpr uint32_t kPairBytes = 12 * 2 * 12 * 16;        // 4608
+
+struct __align__(128) C2Smem {
+    unsigned char a[2][kPairBytes];                      // pooled image pairs (double buffer)
+    unsigned char b[26 * 2 * 128];                       // W2 as core matrices (k-group, n-group)
+    float wf[10 * 256];                                  // linear layer, bf16-rounded values
+    float p2[2][256];                                    // pooled-2 activations of the pair
+    float logits[2][10];
+    float b2[16];
+    float bfc[10];
+    uint64_t full[2];
+    uint64_t mma_bar;
+    uint32_t tmem_slot;
+    int      wait_ok;
+    uint32_t item;
+    float    loss;
+};
+
+__global__ void __launch_bounds__(kC2Threads)
+k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const unsigned char* __restrict__ pooled1,
+               const int32_t* __restrict__ labels, uint32_t batch, uint32_t items_per_member,
+               float* __restrict__ partial, uint32_t* work_counter, DeviceStatus* status)
+{
+    extern __shared__ __align__(1024) unsigned char dyn[];
+    C2Smem& S = *reinterpret_cast<C2Smem*>(dyn);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t n_pairs = (batch + 1u) / 2u;
+    const uint32_t n_items = P * items_per_member;
+
+    const uint32_t bar_full0 = smem_u32(&S.full[0]), bar_full1 = smem_u32(&S.full[1]), bar_mma = smem_u32(&S.mma_bar);
+    if (tid == 0) {
+        mbar_init(bar_full0, 1); mbar_init(bar_full1, 1); mbar_init(bar_mma, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (warp == 0) tmem_alloc(smem_u32(&S.tmem_slot), 32);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = S.tmem_slot;
+    constexpr uint32_t idesc = umma_idesc_bf16(128, 16);
+    uint32_t full_phase[2] = { 0, 0 }, mma_phase = 0;
+    bool failed = false;
+
+    while (!failed) {
+        if (tid == 0) S.item = atomicAdd(work_counter, 1u);
+        __syncthreads();
+        const uint32_t item = S.item;
+        if (item >= n_items) break;
+        const uint32_t member = item / items_per_member;
+        const uint32_t pair0 = (item % items_per_member) * kPairsPerItem;
+        const uint32_t pair1 = min(n_pairs, pair0 + kPairsPerItem);
+        const float* prm = theta + static_cast<size_t>(member) * ldD;
+        const unsigned char* src = pooled1 + (static_cast<size_t>(member) * n_pairs) * kPairBytes;
+
+        // ---- first pair on its way while the weights are converted -----------------------------
+        if (tid == 0) {
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar_full0), "r"(kPairBytes) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         :: "r"(smem_u32(S.a[0])), "l"(src + static_cast<size_t>(pair0) * kPairBytes), "r"(kPairBytes), "r"(bar_full0) : "memory");
+            S.loss = 0.f;
+        }
+        // W2[oc][ic][kh][kw] -> k = (kh*5+kw)*8 + ic, core matrix (tap g, oc/8), row oc%8, 16 bytes = 8 ic
+        for (uint32_t idx = tid; idx < 26u * 16u; idx += kC2Threads) {
+            const uint32_t g = idx >> 4, oc = idx & 15u;
+            uint32_t w[4] = { 0, 0, 0, 0 };
+            if (g < 25u) {
+                float v[8];
+#pragma unroll
+                for (int ic = 0; ic < 8; ++ic) v[ic] = prm[208u + (oc * 8u + ic) * 25u + g];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) w[k] = pack_bf16(v[2 * k], v[2 * k + 1]);
+            }
+            *reinterpret_cast<uint4*>(S.b + (g * 2u + (oc >> 3)) * 128u + (oc & 7u) * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        for (uint32_t i = tid; i < 2560u; i += kC2Threads)
+            S.wf[i] = __bfloat162float(__float2bfloat16_rn(prm[3424u + i]));
+        if (tid < 16) S.b2[tid] = prm[3408u + tid];
+        if (tid < 10) S.bfc[tid] = prm[5984u + tid];
+        fence_async_smem();
+        __syncthreads();
+
+        for (uint32_t pair = pair0; pair < pair1; ++pair) {
+            const uint32_t buf = (pair - pair0) & 1u;
+            if (tid == 0) {
+                // next pair into the other buffer (its last reader, the previous MMA, has completed)
+                if (pair + 1u < pair1) {
+                    const uint32_t nb = buf ^ 1u, nbar = nb ? bar_full1 : bar_full0;
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(nbar), "r"(kPairBytes) : "memory");
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 :: "r"(smem_u32(S.a[nb])), "l"(src + static_cast<size_t>(pair + 1u) * kPairBytes), "r"(kPairBytes), "r"(nbar) : "memory");
+                }
+                int ok = mbar_wait_bounded(buf ? bar_full1 : bar_full0, full_phase[buf], kWaitIters) ? 1 : 0;
+                if (ok) {
+                    tc_fence_after();
+                    const uint32_t a0 = smem_u32(S.a[buf]), b0 = smem_u32(S.b);
+#pragma unroll 1
+                    for (uint32_t j = 0; j < 13u; ++j) {
+                        const uint32_t g0 = 2u * j, g1 = 2u * j + 1u;
+                        const uint32_t off0 = (g0 / 5u) * 384u + (g0 % 5u) * 16u;
+                        const uint32_t off1 = (g1 < 25u) ? (g1 / 5u) * 384u + (g1 % 5u) * 16u : off0;
+                        const uint64_t ad = umma_smem_desc(a0 + off0, off1 - off0, 192u);
+                        const uint64_t bd = umma_smem_desc(b0 + j * 512u, 256u, 128u);
+                        umma_bf16(tmem, ad, bd, idesc, j);
+                    }
+                    umma_commit(bar_mma);
+                    ok = mbar_wait_bounded(bar_mma, mma_phase, kWaitIters) ? 1 : 0;
+                }
+                S.wait_ok = ok;
+            }
+            __syncthreads();
+            if (!S.wait_ok) { failed = true; break; }
+            full_phase[buf] ^= 1u;
+            mma_phase ^= 1u;
+            tc_fence_after();
+
+            // ---- epilogue: lane = (y%2, image, x); 2x2 max = lanes ^1 and ^16; + bias, ReLU, bf16 ----
+            {
+                float r[16];
+                tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16), r);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    float v = fmaxf(r[c], __shfl_xor_sync(0xffffffffu, r[c], 1));
+                    v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 16));
+                    r[c] = v;
+                }
+                if ((lane & 17) == 0) {
+                    const int im = (lane >> 3) & 1, px = (lane & 7) >> 1, py = warp;
+#pragma unroll
+                    for (int c = 0; c < 16; ++c)
+                        S.p2[im][c * 16 + py * 4 + px] =
+                            __bfloat162float(__float2bfloat16_rn(fmaxf(r[c] + S.b2[c], 0.f)));
+                }
+            }
+            tc_fence_before();
+            __syncthreads();
+            // ---- linear 256 -> 10 for both images: 4 lanes per logit -------------------------------
+            if (warp < 3) {                                   // 20 logits x 4 lanes = threads 0..79 of 96
+                const int out = tid >> 2, part = tid & 3;
+                const bool valid = out < 20;
+                const int im = valid ? out / 10 : 0, cls = valid ? out % 10 : 0;
+                float acc = 0.f;
+                if (valid) {
+#pragma unroll 8
+                    for (int i = 0; i < 64; ++i) acc = fmaf(S.wf[cls * 256 + i * 4 + part], S.p2[im][i * 4 + part], acc);
+                }
+                __syncwarp();
+                acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+                acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+                if (valid && part == 0) S.logits[im][cls] = acc + S.bfc[cls];
+            }
+            __syncthreads();
+            if (tid < 2) {
+                const uint32_t image = pair * 2u + tid;
+                if (image < batch) {
+                    const float* lg = S.logits[tid];
+                    float mx = lg[0];
+#pragma unroll
+                    for (int k = 1; k < 10; ++k) mx = fmaxf(mx, lg[k]);
+                    float se = 0.f;
+#pragma unroll
+                    for (int k = 0; k < 10; ++k) se += expf(lg[k] - mx);
+                    const int lab = min(max(labels[image], 0), 9);
+                    const float l = (mx + logf(se)) - lg[lab];
+                    // image 0 then image 1 of the pair, in a fixed order
+                    if (tid == 1) S.logits[1][0] = l; else S.logits[0][0] = l;
+                } else {
+                    S.logits[tid][0] = 0.f;
+                }
+            }
+            __syncthreads();
+            if (tid == 0) S.loss += S.logits[0][0] + S.logits[1][0];
+        }
+        __syncthreads();
+        if (!failed && tid == 0) partial[item] = S.loss;
+    }
+
+    if (failed && tid == 0) atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 32);
+}
+
+__global__ void k_cnn_tc_finalize(const float* __restrict__ partial, uint32_t P, uint32_t items_per_member,
+                                  uint32_t batch, float* __restrict__ fitness)
+{
+    const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= P) return;
+    float s = 0.f;
+    for (uint32_t t = 0; t < items_per_member; ++t) s += partial[static_cast<size_t>(m) * items_per_member + t];
+    fitness[m] = -s / static_cast<float>(batch);
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+static uint32_t items_per_member_of(uint32_t batch)
+{
+    const uint32_t n_pairs = (batch + 1u) / 2u;
+    return (n_pairs + kPairsPerItem - 1u) / kPairsPerItem;
+}
+
+size_t cnn_tc_scratch_bytes(uint32_t P, uint32_t batch)
+{
+    const size_t n_pairs = (batch + 1u) / 2u;
+    size_t b = 256;                                                        // work counter
+    b += (static_cast<size_t>(P) * items_per_member_of(batch) * sizeof(float) + 255) / 256 * 256;
+    b += static_cast<size_t>(P) * n_pairs * kPairBytes;
+    return b;
+}
+
+int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uint32_t P, const float* images,
+                          const int32_t* labels, uint32_t batch, void* scratch, float* fitness,
+                          DeviceStatus* status)
+{
+    static int sm_count = 0;
+    if (sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+    }
+    unsigned char* base = static_cast<unsigned char*>(scratch);
+    uint32_t* counter = reinterpret_cast<uint32_t*>(base);
+    float* partial = reinterpret_cast<float*>(base + 256);
+    const uint32_t ipm = items_per_member_of(batch);
+    unsigned char* pooled1 = base + 256 + (static_cast<size_t>(P) * ipm * sizeof(float) + 255) / 256 * 256;
+
+    if (cudaFuncSetAttribute(k_cnn_conv1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kC1DynRequest) != cudaSuccess) return -1;
+    const uint32_t n_tiles = (batch * 144u + 31u) / 32u;
+    dim3 g1(min(static_cast<uint32_t>(sm_count), n_tiles), (P + 63u) / 64u);
+    k_cnn_conv1_tc<<<g1, kC1Threads, kC1DynRequest, st>>>(theta, ldD, P, images, batch,
+                                                          reinterpret_cast<uint4*>(pooled1), counter, status);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+
+    const int c2_bytes = static_cast<int>(sizeof(C2Smem));
+    if (cudaFuncSetAttribute(k_cnn_conv2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, c2_bytes) != cudaSuccess) return -1;
+    const uint32_t n_items = P * ipm;
+    const uint32_t g2 = min(n_items, static_cast<uint32_t>(sm_count) * 4u);
+    k_cnn_conv2_tc<<<g2, kC2Threads, c2_bytes, st>>>(theta, ldD, P, pooled1, labels, batch, ipm, partial, counter, status);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    k_cnn_tc_finalize<<<(P + 255u) / 256u, 256, 0, st>>>(partial, P, ipm, batch, fitness);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 3;
+}
+
+}  // namespace evo

@@ -8,12 +8,15 @@ import torch
 import oracle
 from helpers import rel_err
 from paper_2202_05008_b200 import Solver, workloads as W
+from paper_2202_05008_b200.binding import ROLLOUT_GENERIC, ROLLOUT_AUTO
+
+KERNELS = [ROLLOUT_GENERIC, ROLLOUT_AUTO]      # CUDA-core kernel, tensor-core (tcgen05) path
 
 pytestmark = pytest.mark.gpu
 
 
-def _run(w, theta_np=None, generation=0, members=None):
-    s = Solver(w)
+def _run(w, theta_np=None, generation=0, members=None, kernel=ROLLOUT_AUTO):
+    s = Solver(w, rollout_kernel=kernel)
     images, labels = W.image_batch(w.seed, generation, w.batch)
     s.set_batch(torch.tensor(images, device="cuda"), torch.tensor(labels, device="cuda"))
     if theta_np is None:
@@ -29,19 +32,39 @@ def _run(w, theta_np=None, generation=0, members=None):
     return fit
 
 
-def test_cnn_zero_parameters_is_minus_ln10():
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_cnn_zero_parameters_is_minus_ln10(kernel):
     w = W.CFG3.with_(pop_size=2, batch=64)
-    fit = _run(w, theta_np=np.zeros((2, W.CNN_PARAMS), dtype=np.float32))
+    fit = _run(w, theta_np=np.zeros((2, W.CNN_PARAMS), dtype=np.float32), kernel=kernel)
     assert np.abs(fit + math.log(10)).max() < 1e-6
 
 
-def test_cnn_cfg3_first_generation_sampled_members():
-    _run(W.CFG3, members=[0, 1, 31, 63])
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_cnn_cfg3_first_generation_sampled_members(kernel):
+    _run(W.CFG3, members=[0, 1, 31, 32, 63], kernel=kernel)
 
 
-def test_cnn_random_large_parameters_ragged_batch():
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_cnn_random_large_parameters_ragged_batch(kernel):
     w = W.CFG3.with_(pop_size=4, batch=77)
-    _run(w, theta_np=W.random_parameters(5, 4, W.CNN_PARAMS, scale=0.2))
+    _run(w, theta_np=W.random_parameters(5, 4, W.CNN_PARAMS, scale=0.2), kernel=kernel)
+
+
+def test_cnn_more_than_one_member_group_and_tiny_batch():
+    # 70 members = two conv1 groups (64 + 6); batch 3 = one full pair and one half pair
+    w = W.CFG3.with_(pop_size=70, batch=3)
+    _run(w, theta_np=W.random_parameters(6, 70, W.CNN_PARAMS, scale=0.1), members=[0, 5, 63, 64, 69])
+
+
+def test_cnn_tensor_core_path_is_deterministic():
+    w = W.CFG3.with_(pop_size=8, batch=256)
+    s = Solver(w)
+    images, labels = W.image_batch(w.seed, 0, w.batch)
+    s.set_batch(torch.tensor(images, device="cuda"), torch.tensor(labels, device="cuda"))
+    s.ask()
+    a = s.rollout().clone(); b = s.rollout().clone()
+    assert torch.equal(a, b) and s.sync_status() == 0
+    s.close()
 
 
 def test_cnn_rollout_needs_a_batch():
