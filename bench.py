@@ -230,6 +230,29 @@ def config_of(w, args, stored):
 
 
 # ------------------------------------------------------------------------------------------
+# cross-rank plumbing (works with gloo on CPU tensors and nccl on CUDA tensors)
+# ------------------------------------------------------------------------------------------
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Replicas are independent problems: every rank gets its own random streams."""
+    return base_seed + 1000 * rank
+
+
+def max_over_ranks(value_ms: float, device, world: int) -> float:
+    """Timing of a multi-rank run is the slowest rank's."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank_step: float, world: int, ms_per_step: float) -> float:
+    """Aggregate throughput of all ranks (weak scaling: every rank does one full generation)."""
+    return world * units_per_rank_step / (ms_per_step * 1e-3)
+
+
+# ------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------
 def run_ours(args, w):
@@ -248,7 +271,7 @@ def run_ours(args, w):
         dist.init_process_group("nccl", device_id=dev)
 
     stored = args.noise == "stored"
-    w_rank = w.with_(seed=w.seed + 1000 * rank)         # independent replicas
+    w_rank = w.with_(seed=rank_seed(w.seed, rank))      # independent replicas
     s = Solver(w_rank, device=dev, noise_mode=W.NOISE_STORED if stored else W.NOISE_REGENERATED)
     P, D = w.pop_size, w.param_dim
     supervised = w.task_kind == W.TASK_SUPERVISED
@@ -308,10 +331,7 @@ def run_ours(args, w):
     t_roll = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
     t_tell = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
     t_total_ms = sum(e[0].elapsed_time(e[3]) for e in events)
-    tt = torch.tensor([t_total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-    t_step_ms = float(tt.item()) / args.steps
+    t_step_ms = max_over_ranks(t_total_ms, dev, world) / args.steps
 
     # ---- end to end: host-resident centre in, fitness and centre out, every step -----------
     h_center = torch.zeros(D, dtype=torch.float32).pin_memory()
@@ -354,14 +374,11 @@ def run_ours(args, w):
         e2e_step(i)
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
-    te = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_ms = float(te.item())
+    e2e_ms = max_over_ranks(e2e_ms, dev, world)
 
     if rank == 0:
         metric, unit, units_per_gen = unit_of(w)
-        value = world * units_per_gen / (t_step_ms * 1e-3)
+        value = whole_job_value(units_per_gen, world, t_step_ms)
         peaks = measured_peaks()
         clocks = sampler.summary()
         sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
@@ -403,7 +420,7 @@ def run_ours(args, w):
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": config_of(w, args, stored),
                 "generations_per_sec": world / (t_step_ms * 1e-3),
-                "e2e": {"value": world * units_per_gen / (e2e_ms * 1e-3), "unit": unit,
+                "e2e": {"value": whole_job_value(units_per_gen, world, e2e_ms), "unit": unit,
                         "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
                 "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
                 "stages": stages, "cpu_baseline": cpu}

@@ -1,0 +1,52 @@
+"""The N > 1 plumbing of bench.py on CPU: two gloo ranks (no GPU involved)."""
+import json
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    local_ms = 10.0 + 5.0 * rank                       # rank 1 is the slow one
+    slowest = bench.max_over_ranks(local_ms, torch.device("cpu"), world)
+    seeds = [None] * world
+    dist.all_gather_object(seeds, bench.rank_seed(7, rank))
+    dist.barrier()
+    if rank == 0:
+        json.dump({"slowest": slowest, "seeds": seeds,
+                   "value": bench.whole_job_value(1000.0, world, slowest)}, open(out, "w"))
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_max_timing_distinct_seeds_and_aggregate(tmp_path):
+    out = str(tmp_path / "r.json")
+    port = 29500 + os.getpid() % 2000
+    mp.spawn(_worker, args=(2, port, out), nprocs=2, join=True)
+    r = json.load(open(out))
+    assert r["slowest"] == 15.0
+    assert len(set(r["seeds"])) == 2
+    assert abs(r["value"] - 2 * 1000.0 / 0.015) < 1e-6
+
+
+def test_reference_arm_under_torchrun_prints_one_line_from_rank_zero():
+    port = 31500 + os.getpid() % 2000
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.join(ROOT, "bench.py"),
+           "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0", "--workload", "cfg1"]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["cpu_baseline"]["kind"] == "oracle"
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["value"] > 0
