@@ -189,7 +189,7 @@ bool rollout_mlp_supported(const evo_config& cfg)
 }
 
 int rollout_mlp_tiled_shape(uint32_t task, uint32_t n_layers, const uint32_t* sizes);
-uint32_t rollout_mlp_tiled_eb(int shape);
+uint32_t rollout_mlp_tiled_eb(int shape, uint32_t episodes);
 int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus* status);
 
 static bool use_tiled(uint32_t task, uint32_t n_layers, const uint32_t* sizes, uint32_t choice)
@@ -200,7 +200,7 @@ static bool use_tiled(uint32_t task, uint32_t n_layers, const uint32_t* sizes, u
 void rollout_mlp_plan(const evo_config& cfg, uint32_t* EB, uint32_t* n_eb)
 {
     if (use_tiled(cfg.task_kind, cfg.n_layers, cfg.layer_sizes, cfg.rollout_kernel)) {
-        *EB = rollout_mlp_tiled_eb(rollout_mlp_tiled_shape(cfg.task_kind, cfg.n_layers, cfg.layer_sizes));
+        *EB = rollout_mlp_tiled_eb(rollout_mlp_tiled_shape(cfg.task_kind, cfg.n_layers, cfg.layer_sizes), cfg.episodes);
         *n_eb = (cfg.episodes + *EB - 1u) / *EB;
         return;
     }

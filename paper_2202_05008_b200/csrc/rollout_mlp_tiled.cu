@@ -23,8 +23,10 @@ namespace evo {
 // tanh(x) = 1 - 2/(exp(2x)+1) on the special-function unit; absolute error ~2e-7
 __device__ __forceinline__ float tanh_fast(float x)
 {
-    const float e = __expf(2.0f * x);
-    return 1.0f - __fdividef(2.0f, e + 1.0f);
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * 2.885390082f));      // e^(2x) = 2^(2x log2 e)
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+    return fmaf(-2.0f, r, 1.0f);
 }
 
 template <int EB> struct EpVec;
@@ -72,9 +74,39 @@ __device__ __forceinline__ int reduce_lanes(float (&v)[N], int s)
     return offset;
 }
 
+// Select-free variant for TI >= S: register slot i of lane s holds output row i ^ rowmask(s) with
+// rowmask(s) = sum_b bit_b(s) * (TI >> (b+1)), so at every stage a lane keeps its lower slots and
+// hands over its upper ones.  Returns rowmask(s): the lane ends with rows rowmask(s) .. + TI/S - 1.
+template <int S> __device__ __forceinline__ int row_mask(int s, int TI)
+{
+    int m = 0;
+#pragma unroll
+    for (int b = 0; b < ilog2(S); ++b) m += ((s >> b) & 1) * (TI >> (b + 1));
+    return m;
+}
+
+template <int TI, int EB, int S>
+__device__ __forceinline__ void reduce_lanes_perm(float (&v)[TI * EB])
+{
+#pragma unroll
+    for (int b = 0; b < ilog2(S); ++b) {
+        const int half = TI >> (b + 1);
+#pragma unroll
+        for (int i = 0; i < TI / 2; ++i) {
+            if (i < half) {
+#pragma unroll
+                for (int e = 0; e < EB; ++e)
+                    v[i * EB + e] += __shfl_xor_sync(0xffffffffu, v[(half + i) * EB + e], 1 << b);
+            }
+        }
+    }
+}
+
 // One dense layer y = f(W x + b) for EB episodes at once.
 //   NI inputs, NO outputs, thread tile TI rows x KS = NI/S inputs, S lanes per row group.
-template <int NI, int NO, int TI, int S, int EB, int THREADS>
+//   LD = floats between consecutive units of the activation arrays (>= EB; a team that owns only
+//   some of the episodes of a wider array passes the array's full episode count).
+template <int NI, int NO, int TI, int S, int EB, int THREADS, int LD = EB>
 struct Dense {
     static_assert(NI % S == 0, "S must divide the input width");
     static_assert((S & (S - 1)) == 0 && S <= 32, "S is a power of two within a warp");
@@ -84,6 +116,7 @@ struct Dense {
     static_assert(ACTIVE <= THREADS, "layer needs more threads than the block has");
     static constexpr int N = TI * EB;
     static constexpr int CNT = (N >= S) ? N / S : 1;
+    static constexpr bool PERM = (TI >= S) && (S > 1);        // select-free reduction possible
 
     float w[TI][KS];
     float bias[TI];
@@ -97,11 +130,14 @@ struct Dense {
         s = tid % S;
         row0 = (tid / S) * TI;
 #pragma unroll
-        for (int r = 0; r < TI; ++r) {
-            const bool ok = active && (row0 + r < NO);
+        const int rm = PERM ? row_mask<S>(s, TI) : 0;
 #pragma unroll
-            for (int k = 0; k < KS; ++k) w[r][k] = ok ? W[(row0 + r) * NI + k * S + s] : 0.f;
-            bias[r] = (ok && s == 0 && b) ? b[row0 + r] : 0.f;
+        for (int r = 0; r < TI; ++r) {
+            const int row = row0 + (r ^ rm);                     // slot r holds this output row
+            const bool ok = active && (row < NO);
+#pragma unroll
+            for (int k = 0; k < KS; ++k) w[r][k] = ok ? W[row * NI + k * S + s] : 0.f;
+            bias[r] = (ok && s == 0 && b) ? b[row] : 0.f;
         }
     }
 
@@ -118,14 +154,16 @@ struct Dense {
 #pragma unroll
         for (int k = 0; k < KS; ++k) {
             float a[EB];
-            EpVec<EB>::load(in + (k * S + s) * EB, a);     // lane s takes inputs s, s+S, ... (no bank conflicts)
+            EpVec<EB>::load(in + (k * S + s) * LD, a);     // lane s takes inputs s, s+S, ... (no bank conflicts)
             hook(k * S + s, a);
 #pragma unroll
             for (int r = 0; r < TI; ++r)
 #pragma unroll
                 for (int e = 0; e < EB; ++e) acc[r * EB + e] = fmaf(w[r][k], a[e], acc[r * EB + e]);
         }
-        const int offset = reduce_lanes<N, S>(acc, s);
+        int offset;
+        if constexpr (PERM) { reduce_lanes_perm<TI, EB, S>(acc); offset = row_mask<S>(s, TI) * EB; }
+        else offset = reduce_lanes<N, S>(acc, s);
         // with N < S several lanes end with the same sum: the one whose spare bits are 0 writes
         const bool writer = active && ((N >= S) || ((s >> ilog2(N)) == 0));
         if (writer) {
@@ -139,14 +177,14 @@ struct Dense {
                     y.y = ACT ? scale * tanh_fast(acc[i + 1]) : acc[i + 1];
                     y.z = ACT ? scale * tanh_fast(acc[i + 2]) : acc[i + 2];
                     y.w = ACT ? scale * tanh_fast(acc[i + 3]) : acc[i + 3];
-                    if (row < NO) *reinterpret_cast<float4*>(out + row * EB + e) = y;
+                    if (row < NO) *reinterpret_cast<float4*>(out + row * LD + e) = y;
                 }
             } else {
 #pragma unroll
                 for (int i = 0; i < CNT; ++i) {
                     const int n = offset + i;
                     const int row = row0 + n / EB, e = n % EB;
-                    if (row < NO) out[row * EB + e] = ACT ? scale * tanh_fast(acc[i]) : acc[i];
+                    if (row < NO) out[row * LD + e] = ACT ? scale * tanh_fast(acc[i]) : acc[i];
                 }
             }
         }
@@ -351,6 +389,162 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
 }
 
 // ------------------------------------------------------------------------------------------
+// Cart-pole, warp-specialised: the task step (action layer + RK4, ~1 us of dependent latency on
+// a handful of lanes) and the two wide policy layers take about equally long, so a block carries
+// two groups of EB episodes and runs them half a step apart: while the task warp advances group
+// A, the policy warps compute the hidden layers of group B, and vice versa.  Block = (member,
+// 2*EB episodes); warp 0 = task warp; the policy warps form NT teams of MT threads, each team
+// owning EB/NT episodes of the group (the weights are replicated in each team's registers).
+// ------------------------------------------------------------------------------------------
+template <int H1, int H2, int EB, int MT, int NT, int TI1, int S1, int TI2, int S2, int TI3, int S3>
+__global__ void __launch_bounds__(32 + MT * NT)
+k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
+{
+    constexpr int NIN = 5;
+    extern __shared__ __align__(128) float smem[];
+    __shared__ __align__(8) uint64_t mbar;
+    __shared__ int copy_ok;
+    float* stage = smem;                                   // parameter row
+    float* obs = stage + a.ldD;                            // [2][NIN][EB]
+    float* h1 = obs + 2 * NIN * EB;                        // [H1][EB]   (policy warps only)
+    float* h2 = h1 + H1 * EB;                              // [2][H2][EB]
+    float* actb = h2 + 2 * H2 * EB;                        // [EB]       (task warp only)
+
+    const int tid = threadIdx.x;
+    const uint32_t member = blockIdx.x, eb = blockIdx.y;
+    const uint32_t e0 = eb * (2 * EB);
+    const int nE = min(static_cast<uint32_t>(2 * EB), a.E - e0);      // episodes of this block
+    const int nA = min(nE, EB), nB = nE - nA;                        // group sizes
+    const PhiloxKey key{ a.k0, a.k1 };
+
+    const uint32_t bar = static_cast<uint32_t>(__cvta_generic_to_shared(&mbar));
+    const uint32_t bytes = a.ldD * 4u;
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const float* src = a.theta + static_cast<size_t>(member) * a.ldD;
+        const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+    }
+    // seeded starts of both groups (lanes e < EB of the task warp keep the states in registers)
+    const CartpoleConst cpc = cartpole_const(a.tp);
+    CpState cps[2] = {};
+    float ret[2] = { 0.f, 0.f };
+    if (tid < EB) {
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            const int ng = g ? nB : nA;
+            const uint32_t ep = e0 + g * EB + min(tid, max(ng, 1) - 1);
+            cps[g] = cartpole_reset(key, a.generation, min(ep, a.E - 1u), a.tp[EVO_CP_INIT_RANGE]);
+            float sn, cs;
+            sincos_fast(cps[g].th, sn, cs);
+            float* o = obs + g * NIN * EB;
+            o[0 * EB + tid] = cps[g].x;  o[1 * EB + tid] = cps[g].xd;
+            o[2 * EB + tid] = cs;        o[3 * EB + tid] = sn;
+            o[4 * EB + tid] = cps[g].thd;
+        }
+    }
+    if (tid == 0) {
+        copy_ok = mbar_wait(bar, 0u, 1u << 22) ? 1 : 0;
+        if (!copy_ok) {
+            atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
+            mbar_wait(bar, 0u, 1u << 22);
+        }
+    }
+    __syncthreads();
+    if (!copy_ok) return;
+
+    const bool tracing = a.trace != nullptr;
+    const float* p1 = stage;
+    const float* p2 = p1 + H1 * NIN + H1;
+    const float* p3 = p2 + H2 * H1 + H2;
+
+    if (tid >= 32) {
+        // ---------------- policy warps: hidden layers of one group per half step ----------------
+        constexpr int ET = EB / NT;                        // episodes per team
+        static_assert(EB % NT == 0, "teams split the group's episodes evenly");
+        const int team = (tid - 32) / MT, mt = (tid - 32) % MT;
+        const int eoff = team * ET;
+        Dense<NIN, H1, TI1, S1, ET, MT, EB> L1;
+        Dense<H1, H2, TI2, S2, ET, MT, EB> L2;
+        L1.load(p1, p1 + H1 * NIN, mt);
+        L2.load(p2, p2 + H2 * H1, mt);
+        auto hidden = [&](int g) {
+            L1.template run<true>(obs + g * NIN * EB + eoff, h1 + eoff, 1.0f, NoHook{});
+            asm volatile("bar.sync %0, %1;" :: "r"(1 + team), "n"(MT) : "memory");   // the team's own barrier
+            L2.template run<true>(h1 + eoff, h2 + g * H2 * EB + eoff, 1.0f, NoHook{});
+        };
+        __syncthreads();                                   // weights are in registers everywhere
+        hidden(0);
+        __syncthreads();
+        for (uint32_t t = 0; t < a.T; ++t) {
+            hidden(1);
+            __syncthreads();
+            if (t + 1u < a.T) hidden(0);
+            __syncthreads();
+        }
+    } else {
+        // ---------------- task warp: action layer + RK4 step of the other group ------------------
+        // action layer H2 -> 1: lane = (episode e = lane % EB, input slice q = lane / EB); every lane
+        // ends with its episode's action after log2(32/EB) butterfly stages, no shared-memory trip
+        constexpr int Q = 32 / EB, KQ = H2 / Q;
+        static_assert(32 % EB == 0 && H2 % Q == 0, "action layer mapping");
+        const int le = tid % EB, lq = tid / EB;
+        float w3[KQ];
+#pragma unroll
+        for (int i = 0; i < KQ; ++i) w3[i] = p3[lq + Q * i];
+        const float b3 = p3[H2];
+        auto advance = [&](int g, uint32_t t) {
+            const float* hin = h2 + g * H2 * EB;
+            float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+            for (int i = 0; i < KQ; i += 2) {
+                acc0 = fmaf(w3[i], hin[(lq + Q * i) * EB + le], acc0);
+                acc1 = fmaf(w3[i + 1], hin[(lq + Q * (i + 1)) * EB + le], acc1);
+            }
+            float pre = acc0 + acc1;
+#pragma unroll
+            for (int off = EB; off < 32; off <<= 1) pre += __shfl_xor_sync(0xffffffffu, pre, off);
+            const float force = a.action_scale * tanh_fast(pre + b3);
+            if (tid < EB) {
+                cps[g] = cartpole_step_fast(cpc, cps[g], force);
+                float sn, cs;
+                sincos_fast(cps[g].th, sn, cs);
+                ret[g] += cs * __expf(-cps[g].x * cps[g].x);       // reward on the post-step state
+                float* o = obs + g * NIN * EB;
+                o[0 * EB + tid] = cps[g].x;  o[1 * EB + tid] = cps[g].xd;
+                o[2 * EB + tid] = cs;        o[3 * EB + tid] = sn;
+                o[4 * EB + tid] = cps[g].thd;
+                if (tracing && t < a.trace_T && tid < (g ? nB : nA)) {
+                    float4* tr = reinterpret_cast<float4*>(
+                        a.trace + ((static_cast<size_t>(member) * a.E + e0 + g * EB + tid) * a.trace_T + t) * 4);
+                    *tr = make_float4(cps[g].x, cps[g].xd, cps[g].th, cps[g].thd);
+                }
+            }
+            __syncwarp();
+        };
+        __syncthreads();
+        __syncthreads();
+        for (uint32_t t = 0; t < a.T; ++t) {
+            advance(0, t);
+            __syncthreads();
+            advance(1, t);
+            __syncthreads();
+        }
+        // block return: group A's episodes then group B's, butterfly sum (fixed order)
+        float v = ((tid < nA) ? ret[0] : 0.f) + ((tid < nB) ? ret[1] : 0.f);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        if (tid == 0) a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // shapes with a compiled kernel
 // ------------------------------------------------------------------------------------------
 struct TiledShape { uint32_t task, nin, h1, h2, nout, EB; };
@@ -371,7 +565,13 @@ int rollout_mlp_tiled_shape(uint32_t task, uint32_t n_layers, const uint32_t* si
     return -1;
 }
 
-uint32_t rollout_mlp_tiled_eb(int shape) { return kShapes[shape].EB; }
+// episodes per block; the 5-64-64-1 cart-pole shape switches to the warp-specialised kernel
+// (two groups of 8) once a member has more than 8 episodes
+uint32_t rollout_mlp_tiled_eb(int shape, uint32_t episodes)
+{
+    if (shape == 1 && episodes > kShapes[1].EB) return 2u * kShapes[1].EB;
+    return kShapes[shape].EB;
+}
 
 template <class K>
 static int launch_one(K kernel, int threads, size_t act_floats, cudaStream_t st, const RolloutMlpArgs& a,
@@ -389,7 +589,11 @@ static int launch_one(K kernel, int threads, size_t act_floats, cudaStream_t st,
 int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus* status)
 {
     const int shape = rollout_mlp_tiled_shape(a.task, a.n_layers, a.sizes);
-    if (shape < 0 || a.EB != kShapes[shape].EB) return -2;
+    if (shape < 0) return -2;
+    if (shape == 1 && a.EB == 2u * kShapes[1].EB)
+        return launch_one(k_rollout_cartpole_ws<64, 64, 8, 64, 2, 1, 1, 4, 4, 1, 32>, 32 + 64 * 2,
+                          (2 * 5 + 64 + 2 * 64 + 1) * 8, st, a, status);
+    if (a.EB != kShapes[shape].EB) return -2;
     switch (shape) {
         case 0:
             return launch_one(k_rollout_mlp_tiled<5, 16, 16, 1, 1, 32, EVO_TASK_CARTPOLE, 1, 1, 1, 2, 1, 16>,

@@ -95,6 +95,19 @@ def test_generic_kernel_odd_shapes_and_episode_counts():
     _rollout_check(w, 30, list(range(4)), ROLLOUT_GENERIC, theta_np=theta)
 
 
+@pytest.mark.parametrize("episodes", [5, 8, 9, 37])
+def test_cfg2_shape_tiled_variants_and_ragged_episode_counts(episodes):
+    # <= 8 episodes: one group per block; more: the two-group warp-specialised kernel, incl. ragged tails
+    w = W.CFG2.with_(pop_size=6, episodes=episodes)
+    theta = W.random_parameters(7, 6, w.param_dim, scale=0.3)
+    _rollout_check(w, 60, list(range(6)), ROLLOUT_TILED, theta_np=theta)
+
+
+def test_cfg1_shape_with_several_episodes():
+    w = W.CFG1.with_(episodes=3)
+    _rollout_check(w, 80, list(range(16)), ROLLOUT_TILED)
+
+
 def test_rollout_later_generation_uses_new_initial_states():
     w = W.CFG1.with_(horizon=50)
     s = Solver(w)
