@@ -123,7 +123,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 constexpr int kC1Threads = 128;
 constexpr int kC1SmemB = 512 * 32 * 2;        // all filters of the group, bf16, K = 32
 constexpr int kC1SmemA = 128 * 32 * 2;        // one im2col tile
-constexpr int kC1Dyn = kC1SmemB + kC1SmemA + 512 * 4;
 // the block owns all 512 TMEM columns, so it must be alone on its SM: ask for more than half
 // of the SM's shared memory
 constexpr int kC1DynRequest = 120 * 1024;
@@ -280,27 +279,57 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 }
 
 // ------------------------------------------------------------------------------------------
-// conv2 + pool + linear + cross-entropy, one work item = (member, 16 image pairs)
+// conv2 + pool + linear + cross-entropy, one work item = (member, 16 image pairs).
+// Pipeline per item: pooled pairs arrive through a 4-deep ring of bulk copies; the MMAs of pair
+// i+1 are issued before the epilogue of pair i (two 16-column accumulators in TMEM); the pooled
+// conv2 activations of all 32 images are kept in shared memory and the linear layer and the
+// cross-entropy run once per item on all of them.
 // ------------------------------------------------------------------------------------------
 constexpr int kC2Threads = 128;
 constexpr int kPairsPerItem = 16;
 constexpr uint32_t kPairBytes = 12 * 2 * 12 * 16;        // 4608
+constexpr int kC2Bufs = 4;
+constexpr int kP2Stride = 257;                           // odd pitch: image rows fall in distinct banks
 
 struct __align__(128) C2Smem {
-    unsigned char a[2][kPairBytes];                      // pooled image pairs (double buffer)
-    unsigned char b[26 * 2 * 128];                       // W2 as core matrices (k-group, n-group)
-    float wf[10 * 256];                                  // linear layer, bf16-rounded values
-    float p2[2][256];                                    // pooled-2 activations of the pair
-    float logits[2][10];
+    unsigned char a[kC2Bufs][kPairBytes];                // pooled image pairs (ring)
+    unsigned char b[26 * 2 * 128];                       // W2 as core matrices (tap, filter group)
+    float wfT[256 * 12];                                 // linear layer transposed [k][class], bf16-rounded
+    float p2[2 * kPairsPerItem][kP2Stride];              // pooled-2 activations of the item's images
+    float logit[2 * kPairsPerItem][12];
     float b2[16];
-    float bfc[10];
-    uint64_t full[2];
-    uint64_t mma_bar;
+    float bfc[12];
+    uint64_t full[kC2Bufs];
+    uint64_t mma_bar[2];
     uint32_t tmem_slot;
     int      wait_ok;
     uint32_t item;
-    float    loss;
 };
+
+__device__ __forceinline__ void c2_load_pair(C2Smem& S, int buf, const unsigned char* src)
+{
+    const uint32_t bar = smem_u32(&S.full[buf]);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(kPairBytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(S.a[buf])), "l"(src), "r"(kPairBytes), "r"(bar) : "memory");
+}
+
+// 13 MMAs (K = 16 each = two 5x5 taps x 8 channels) of one image pair into one accumulator
+__device__ __forceinline__ void c2_issue_mma(C2Smem& S, int buf, uint32_t d_tmem, uint32_t bar)
+{
+    constexpr uint32_t idesc = umma_idesc_bf16(128, 16);
+    const uint32_t a0 = smem_u32(S.a[buf]), b0 = smem_u32(S.b);
+#pragma unroll 1
+    for (uint32_t j = 0; j < 13u; ++j) {
+        const uint32_t g0 = 2u * j, g1 = 2u * j + 1u;
+        const uint32_t off0 = (g0 / 5u) * 384u + (g0 % 5u) * 16u;
+        const uint32_t off1 = (g1 < 25u) ? (g1 / 5u) * 384u + (g1 % 5u) * 16u : off0;   // tap 25 = zero weights
+        const uint64_t ad = umma_smem_desc(a0 + off0, off1 - off0, 192u);
+        const uint64_t bd = umma_smem_desc(b0 + j * 512u, 256u, 128u);
+        umma_bf16(d_tmem, ad, bd, idesc, j);
+    }
+    umma_commit(bar);
+}
 
 __global__ void __launch_bounds__(kC2Threads)
 k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const unsigned char* __restrict__ pooled1,
@@ -313,19 +342,21 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     const uint32_t n_pairs = (batch + 1u) / 2u;
     const uint32_t n_items = P * items_per_member;
 
-    const uint32_t bar_full0 = smem_u32(&S.full[0]), bar_full1 = smem_u32(&S.full[1]), bar_mma = smem_u32(&S.mma_bar);
     if (tid == 0) {
-        mbar_init(bar_full0, 1); mbar_init(bar_full1, 1); mbar_init(bar_mma, 1);
+        for (int i = 0; i < kC2Bufs; ++i) mbar_init(smem_u32(&S.full[i]), 1);
+        mbar_init(smem_u32(&S.mma_bar[0]), 1);
+        mbar_init(smem_u32(&S.mma_bar[1]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    for (int k = tid; k < 256; k += kC2Threads) { S.wfT[k * 12 + 10] = 0.f; S.wfT[k * 12 + 11] = 0.f; }
+    if (tid < 2) S.bfc[10 + tid] = 0.f;
     __syncwarp();
     if (warp == 0) tmem_alloc(smem_u32(&S.tmem_slot), 32);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = S.tmem_slot;
-    constexpr uint32_t idesc = umma_idesc_bf16(128, 16);
-    uint32_t full_phase[2] = { 0, 0 }, mma_phase = 0;
+    uint32_t full_par = 0, mma_par = 0;           // parity bit per ring slot / per accumulator
     bool failed = false;
 
     while (!failed) {
@@ -335,75 +366,67 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         if (item >= n_items) break;
         const uint32_t member = item / items_per_member;
         const uint32_t pair0 = (item % items_per_member) * kPairsPerItem;
-        const uint32_t pair1 = min(n_pairs, pair0 + kPairsPerItem);
+        const int n = static_cast<int>(min(n_pairs, pair0 + kPairsPerItem) - pair0);
+        const int n_img = static_cast<int>(min(batch, 2u * (pair0 + n)) - 2u * pair0);
         const float* prm = theta + static_cast<size_t>(member) * ldD;
-        const unsigned char* src = pooled1 + (static_cast<size_t>(member) * n_pairs) * kPairBytes;
+        const unsigned char* src = pooled1 + (static_cast<size_t>(member) * n_pairs + pair0) * kPairBytes;
 
-        // ---- first pair on its way while the weights are converted -----------------------------
-        if (tid == 0) {
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar_full0), "r"(kPairBytes) : "memory");
-            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         :: "r"(smem_u32(S.a[0])), "l"(src + static_cast<size_t>(pair0) * kPairBytes), "r"(kPairBytes), "r"(bar_full0) : "memory");
-            S.loss = 0.f;
-        }
-        // W2[oc][ic][kh][kw] -> k = (kh*5+kw)*8 + ic, core matrix (tap g, oc/8), row oc%8, 16 bytes = 8 ic
+        if (tid == 0)
+            for (int i = 0; i < min(kC2Bufs, n); ++i) c2_load_pair(S, i, src + static_cast<size_t>(i) * kPairBytes);
+
+        // ---- weights: coalesced reads, then the operand layouts are built from shared memory ----
+        float* raw = &S.p2[0][0];                                   // 3,200 floats of scratch
+        for (uint32_t i = tid; i < 3200u; i += kC2Threads) raw[i] = prm[208u + i];
+        for (uint32_t i = tid; i < 2560u; i += kC2Threads)
+            S.wfT[(i & 255u) * 12u + (i >> 8)] = __bfloat162float(__float2bfloat16_rn(prm[3424u + i]));
+        if (tid < 16) S.b2[tid] = prm[3408u + tid];
+        if (tid < 10) S.bfc[tid] = prm[5984u + tid];
+        __syncthreads();
+        // W2[oc][ic][kh][kw] -> k = (kh*5+kw)*8 + ic: core matrix (tap g, oc/8), row oc%8, 16 bytes = 8 ic
         for (uint32_t idx = tid; idx < 26u * 16u; idx += kC2Threads) {
             const uint32_t g = idx >> 4, oc = idx & 15u;
             uint32_t w[4] = { 0, 0, 0, 0 };
             if (g < 25u) {
-                float v[8];
 #pragma unroll
-                for (int ic = 0; ic < 8; ++ic) v[ic] = prm[208u + (oc * 8u + ic) * 25u + g];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) w[k] = pack_bf16(v[2 * k], v[2 * k + 1]);
+                for (int k = 0; k < 4; ++k)
+                    w[k] = pack_bf16(raw[(oc * 8u + 2 * k) * 25u + g], raw[(oc * 8u + 2 * k + 1) * 25u + g]);
             }
             *reinterpret_cast<uint4*>(S.b + (g * 2u + (oc >> 3)) * 128u + (oc & 7u) * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        for (uint32_t i = tid; i < 2560u; i += kC2Threads)
-            S.wf[i] = __bfloat162float(__float2bfloat16_rn(prm[3424u + i]));
-        if (tid < 16) S.b2[tid] = prm[3408u + tid];
-        if (tid < 10) S.bfc[tid] = prm[5984u + tid];
         fence_async_smem();
         __syncthreads();
 
-        for (uint32_t pair = pair0; pair < pair1; ++pair) {
-            const uint32_t buf = (pair - pair0) & 1u;
+        if (tid == 0) {                                             // first pair's MMAs
+            int ok = mbar_wait_bounded(smem_u32(&S.full[0]), full_par & 1u, kWaitIters) ? 1 : 0;
+            if (ok) { tc_fence_after(); c2_issue_mma(S, 0, tmem, smem_u32(&S.mma_bar[0])); }
+            S.wait_ok = ok;
+        }
+        __syncthreads();
+        if (!S.wait_ok) { failed = true; break; }
+        full_par ^= 1u;
+
+        for (int i = 0; i < n; ++i) {
+            const int acc = i & 1, nxt = (i + 1) % kC2Bufs;
             if (tid == 0) {
-                // next pair into the other buffer (its last reader, the previous MMA, has completed)
-                if (pair + 1u < pair1) {
-                    const uint32_t nb = buf ^ 1u, nbar = nb ? bar_full1 : bar_full0;
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(nbar), "r"(kPairBytes) : "memory");
-                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                 :: "r"(smem_u32(S.a[nb])), "l"(src + static_cast<size_t>(pair + 1u) * kPairBytes), "r"(kPairBytes), "r"(nbar) : "memory");
+                int ok = 1;
+                if (i + 1 < n) {                                    // run one pair ahead of the epilogue
+                    ok = mbar_wait_bounded(smem_u32(&S.full[nxt]), (full_par >> nxt) & 1u, kWaitIters) ? 1 : 0;
+                    if (ok) { tc_fence_after(); c2_issue_mma(S, nxt, tmem + 16u * (acc ^ 1), smem_u32(&S.mma_bar[acc ^ 1])); }
                 }
-                int ok = mbar_wait_bounded(buf ? bar_full1 : bar_full0, full_phase[buf], kWaitIters) ? 1 : 0;
-                if (ok) {
-                    tc_fence_after();
-                    const uint32_t a0 = smem_u32(S.a[buf]), b0 = smem_u32(S.b);
-#pragma unroll 1
-                    for (uint32_t j = 0; j < 13u; ++j) {
-                        const uint32_t g0 = 2u * j, g1 = 2u * j + 1u;
-                        const uint32_t off0 = (g0 / 5u) * 384u + (g0 % 5u) * 16u;
-                        const uint32_t off1 = (g1 < 25u) ? (g1 / 5u) * 384u + (g1 % 5u) * 16u : off0;
-                        const uint64_t ad = umma_smem_desc(a0 + off0, off1 - off0, 192u);
-                        const uint64_t bd = umma_smem_desc(b0 + j * 512u, 256u, 128u);
-                        umma_bf16(tmem, ad, bd, idesc, j);
-                    }
-                    umma_commit(bar_mma);
-                    ok = mbar_wait_bounded(bar_mma, mma_phase, kWaitIters) ? 1 : 0;
-                }
+                if (ok) ok = mbar_wait_bounded(smem_u32(&S.mma_bar[acc]), (mma_par >> acc) & 1u, kWaitIters) ? 1 : 0;
+                // pair i has been consumed: its ring slot takes pair i + ring depth
+                if (ok && i + kC2Bufs < n) c2_load_pair(S, i % kC2Bufs, src + static_cast<size_t>(i + kC2Bufs) * kPairBytes);
                 S.wait_ok = ok;
             }
             __syncthreads();
             if (!S.wait_ok) { failed = true; break; }
-            full_phase[buf] ^= 1u;
-            mma_phase ^= 1u;
+            if (i + 1 < n) full_par ^= (1u << nxt);
+            mma_par ^= (1u << acc);
             tc_fence_after();
-
             // ---- epilogue: lane = (y%2, image, x); 2x2 max = lanes ^1 and ^16; + bias, ReLU, bf16 ----
             {
                 float r[16];
-                tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16), r);
+                tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + 16u * acc, r);
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     float v = fmaxf(r[c], __shfl_xor_sync(0xffffffffu, r[c], 1));
@@ -412,53 +435,54 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 }
                 if ((lane & 17) == 0) {
                     const int im = (lane >> 3) & 1, px = (lane & 7) >> 1, py = warp;
+                    float* dst = S.p2[2 * i + im] + py * 4 + px;
 #pragma unroll
                     for (int c = 0; c < 16; ++c)
-                        S.p2[im][c * 16 + py * 4 + px] =
-                            __bfloat162float(__float2bfloat16_rn(fmaxf(r[c] + S.b2[c], 0.f)));
+                        dst[c * 16] = __bfloat162float(__float2bfloat16_rn(fmaxf(r[c] + S.b2[c], 0.f)));
                 }
+                __syncwarp();
             }
             tc_fence_before();
             __syncthreads();
-            // ---- linear 256 -> 10 for both images: 4 lanes per logit -------------------------------
-            if (warp < 3) {                                   // 20 logits x 4 lanes = threads 0..79 of 96
-                const int out = tid >> 2, part = tid & 3;
-                const bool valid = out < 20;
-                const int im = valid ? out / 10 : 0, cls = valid ? out % 10 : 0;
-                float acc = 0.f;
-                if (valid) {
+        }
+        if (failed) break;
+
+        // ---- linear 256 -> 10 for all images of the item: thread = (image, group of 4 classes) ----
+        if (warp < 3) {
+            float acc4[4] = { 0.f, 0.f, 0.f, 0.f };
+            if (lane < 2 * n) {
+                const float* x = S.p2[lane];
+                const float* wr = S.wfT + 4 * warp;
 #pragma unroll 8
-                    for (int i = 0; i < 64; ++i) acc = fmaf(S.wf[cls * 256 + i * 4 + part], S.p2[im][i * 4 + part], acc);
-                }
-                __syncwarp();
-                acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-                acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-                if (valid && part == 0) S.logits[im][cls] = acc + S.bfc[cls];
-            }
-            __syncthreads();
-            if (tid < 2) {
-                const uint32_t image = pair * 2u + tid;
-                if (image < batch) {
-                    const float* lg = S.logits[tid];
-                    float mx = lg[0];
-#pragma unroll
-                    for (int k = 1; k < 10; ++k) mx = fmaxf(mx, lg[k]);
-                    float se = 0.f;
-#pragma unroll
-                    for (int k = 0; k < 10; ++k) se += expf(lg[k] - mx);
-                    const int lab = min(max(labels[image], 0), 9);
-                    const float l = (mx + logf(se)) - lg[lab];
-                    // image 0 then image 1 of the pair, in a fixed order
-                    if (tid == 1) S.logits[1][0] = l; else S.logits[0][0] = l;
-                } else {
-                    S.logits[tid][0] = 0.f;
+                for (int k = 0; k < 256; ++k) {
+                    const float xv = x[k];
+                    const float4 w4 = *reinterpret_cast<const float4*>(wr + k * 12);
+                    acc4[0] = fmaf(w4.x, xv, acc4[0]); acc4[1] = fmaf(w4.y, xv, acc4[1]);
+                    acc4[2] = fmaf(w4.z, xv, acc4[2]); acc4[3] = fmaf(w4.w, xv, acc4[3]);
                 }
             }
-            __syncthreads();
-            if (tid == 0) S.loss += S.logits[0][0] + S.logits[1][0];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) S.logit[lane][4 * warp + j] = acc4[j] + S.bfc[4 * warp + j];
         }
         __syncthreads();
-        if (!failed && tid == 0) partial[item] = S.loss;
+        if (warp == 0) {
+            float l = 0.f;
+            if (lane < n_img) {
+                const float* lg = S.logit[lane];
+                float mx = lg[0];
+#pragma unroll
+                for (int k = 1; k < 10; ++k) mx = fmaxf(mx, lg[k]);
+                float se = 0.f;
+#pragma unroll
+                for (int k = 0; k < 10; ++k) se += expf(lg[k] - mx);
+                const int lab = min(max(labels[2u * pair0 + lane], 0), 9);
+                l = (mx + logf(se)) - lg[lab];
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);   // fixed order
+            if (lane == 0) partial[item] = l;
+        }
+        __syncthreads();
     }
 
     if (failed && tid == 0) atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
@@ -521,7 +545,7 @@ int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uin
     const int c2_bytes = static_cast<int>(sizeof(C2Smem));
     if (cudaFuncSetAttribute(k_cnn_conv2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, c2_bytes) != cudaSuccess) return -1;
     const uint32_t n_items = P * ipm;
-    const uint32_t g2 = min(n_items, static_cast<uint32_t>(sm_count) * 4u);
+    const uint32_t g2 = min(n_items, static_cast<uint32_t>(sm_count) * 3u);      // 3 blocks of ~72 KB per SM
     k_cnn_conv2_tc<<<g2, kC2Threads, c2_bytes, st>>>(theta, ldD, P, pooled1, labels, batch, ipm, partial, counter, status);
     if (cudaGetLastError() != cudaSuccess) return -1;
     k_cnn_tc_finalize<<<(P + 255u) / 256u, 256, 0, st>>>(partial, P, ipm, batch, fitness);

@@ -129,7 +129,6 @@ struct Dense {
         active = tid < ACTIVE;
         s = tid % S;
         row0 = (tid / S) * TI;
-#pragma unroll
         const int rm = PERM ? row_mask<S>(s, TI) : 0;
 #pragma unroll
         for (int r = 0; r < TI; ++r) {
@@ -408,7 +407,6 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
     float* obs = stage + a.ldD;                            // [2][NIN][EB]
     float* h1 = obs + 2 * NIN * EB;                        // [H1][EB]   (policy warps only)
     float* h2 = h1 + H1 * EB;                              // [2][H2][EB]
-    float* actb = h2 + 2 * H2 * EB;                        // [EB]       (task warp only)
 
     const int tid = threadIdx.x;
     const uint32_t member = blockIdx.x, eb = blockIdx.y;
@@ -592,7 +590,7 @@ int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceSta
     if (shape < 0) return -2;
     if (shape == 1 && a.EB == 2u * kShapes[1].EB)
         return launch_one(k_rollout_cartpole_ws<64, 64, 8, 64, 2, 1, 1, 4, 4, 1, 32>, 32 + 64 * 2,
-                          (2 * 5 + 64 + 2 * 64 + 1) * 8, st, a, status);
+                          (2 * 5 + 64 + 2 * 64) * 8, st, a, status);
     if (a.EB != kShapes[shape].EB) return -2;
     switch (shape) {
         case 0:
