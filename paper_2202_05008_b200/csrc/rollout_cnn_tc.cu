@@ -96,20 +96,23 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t max_iter)
+// Bounded wait: try_wait suspends the thread for a hardware-chosen short time by itself, so this
+// loop just re-arms it until the phase completes or ~max_cycles SM clocks have passed.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t max_cycles_log2)
 {
-    for (uint32_t it = 0; it < max_iter; ++it) {
+    const long long t0 = clock64();
+    const long long limit = 1ll << max_cycles_log2;
+    for (;;) {
         uint32_t done;
         asm volatile("{\n\t.reg .pred p;\n\t"
                      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
                      "selp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
         if (done) return true;
-        if (it > 32) __nanosleep(32);
+        if (clock64() - t0 > limit) return false;
     }
-    return false;
 }
-constexpr uint32_t kWaitIters = 1u << 22;
+constexpr uint32_t kWaitIters = 31;        // log2 of the cycle budget of a wait: ~1 s
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
@@ -280,16 +283,20 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 
 // ------------------------------------------------------------------------------------------
 // conv2 + pool + linear + cross-entropy, one work item = (member, 16 image pairs).
-// Pipeline per item: pooled pairs arrive through a 4-deep ring of bulk copies; the MMAs of pair
-// i+1 are issued before the epilogue of pair i (two 16-column accumulators in TMEM); the pooled
-// conv2 activations of all 32 images are kept in shared memory and the linear layer and the
-// cross-entropy run once per item on all of them.
+// Warp-specialised: warp 4 only issues tensor-core work (13 MMAs per image pair, running ahead
+// of the epilogue through two 16-column TMEM accumulators); warps 0-3 take the accumulators out
+// of TMEM (pool, bias, ReLU), keep the pooled activations of the item's 32 images in shared
+// memory and run the linear layer and the cross-entropy once per item.  Pooled image pairs
+// arrive through a 4-deep ring of bulk copies.  The roles meet only on mbarriers; every wait is
+// bounded, and after a time-out all later waits fall through so that no role is left behind.
 // ------------------------------------------------------------------------------------------
-constexpr int kC2Threads = 128;
+constexpr int kC2EpiThreads = 128;
+constexpr int kC2Threads = kC2EpiThreads + 32;
 constexpr int kPairsPerItem = 16;
 constexpr uint32_t kPairBytes = 12 * 2 * 12 * 16;        // 4608
 constexpr int kC2Bufs = 4;
 constexpr int kP2Stride = 257;                           // odd pitch: image rows fall in distinct banks
+constexpr uint32_t kNoItem = 0xFFFFFFFFu;
 
 struct __align__(128) C2Smem {
     unsigned char a[kC2Bufs][kPairBytes];                // pooled image pairs (ring)
@@ -299,12 +306,30 @@ struct __align__(128) C2Smem {
     float logit[2 * kPairsPerItem][12];
     float b2[16];
     float bfc[12];
-    uint64_t full[kC2Bufs];
-    uint64_t mma_bar[2];
+    uint64_t full[kC2Bufs];                              // a ring slot has landed
+    uint64_t mma_done[2];                                // an accumulator is complete
+    uint64_t acc_free[2];                                // an accumulator has been read out
+    uint64_t item_ready;                                 // weights of the next item are staged
     uint32_t tmem_slot;
-    int      wait_ok;
-    uint32_t item;
+    volatile int abort;
+    volatile uint32_t item;
+    volatile int n;
 };
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+
+// Wait that cannot hang: after one time-out anywhere in the block every later wait returns at once.
+__device__ __forceinline__ void c2_wait(C2Smem& S, uint64_t* bar, uint32_t parity, DeviceStatus* status)
+{
+    if (S.abort) return;
+    if (!mbar_wait_bounded(smem_u32(bar), parity, kWaitIters)) {
+        S.abort = 1;
+        atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
+    }
+}
 
 __device__ __forceinline__ void c2_load_pair(C2Smem& S, int buf, const unsigned char* src)
 {
@@ -314,12 +339,13 @@ __device__ __forceinline__ void c2_load_pair(C2Smem& S, int buf, const unsigned 
                  :: "r"(smem_u32(S.a[buf])), "l"(src), "r"(kPairBytes), "r"(bar) : "memory");
 }
 
-// 13 MMAs (K = 16 each = two 5x5 taps x 8 channels) of one image pair into one accumulator
-__device__ __forceinline__ void c2_issue_mma(C2Smem& S, int buf, uint32_t d_tmem, uint32_t bar)
+// 13 MMAs (K = 16 each = two 5x5 taps x 8 channels) of one image pair into one accumulator.
+// Tap g = (kh, kw) of the A operand is the pooled pair shifted by kh rows (384 B) and kw pixels
+// (16 B); the loop is unrolled so that all offsets are immediates.
+__device__ __forceinline__ void c2_issue_mma(uint32_t a0, uint32_t b0, uint32_t d_tmem, uint32_t bar)
 {
     constexpr uint32_t idesc = umma_idesc_bf16(128, 16);
-    const uint32_t a0 = smem_u32(S.a[buf]), b0 = smem_u32(S.b);
-#pragma unroll 1
+#pragma unroll
     for (uint32_t j = 0; j < 13u; ++j) {
         const uint32_t g0 = 2u * j, g1 = 2u * j + 1u;
         const uint32_t off0 = (g0 / 5u) * 384u + (g0 % 5u) * 16u;
@@ -344,8 +370,9 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 
     if (tid == 0) {
         for (int i = 0; i < kC2Bufs; ++i) mbar_init(smem_u32(&S.full[i]), 1);
-        mbar_init(smem_u32(&S.mma_bar[0]), 1);
-        mbar_init(smem_u32(&S.mma_bar[1]), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&S.mma_done[i]), 1); mbar_init(smem_u32(&S.acc_free[i]), 4); }
+        mbar_init(smem_u32(&S.item_ready), 1);
+        S.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int k = tid; k < 256; k += kC2Threads) { S.wfT[k * 12 + 10] = 0.f; S.wfT[k * 12 + 11] = 0.f; }
@@ -356,77 +383,89 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = S.tmem_slot;
-    uint32_t full_par = 0, mma_par = 0;           // parity bit per ring slot / per accumulator
-    bool failed = false;
 
-    while (!failed) {
-        if (tid == 0) S.item = atomicAdd(work_counter, 1u);
-        __syncthreads();
-        const uint32_t item = S.item;
-        if (item >= n_items) break;
-        const uint32_t member = item / items_per_member;
-        const uint32_t pair0 = (item % items_per_member) * kPairsPerItem;
-        const int n = static_cast<int>(min(n_pairs, pair0 + kPairsPerItem) - pair0);
-        const int n_img = static_cast<int>(min(batch, 2u * (pair0 + n)) - 2u * pair0);
-        const float* prm = theta + static_cast<size_t>(member) * ldD;
-        const unsigned char* src = pooled1 + (static_cast<size_t>(member) * n_pairs + pair0) * kPairBytes;
-
-        if (tid == 0)
-            for (int i = 0; i < min(kC2Bufs, n); ++i) c2_load_pair(S, i, src + static_cast<size_t>(i) * kPairBytes);
-
-        // ---- weights: coalesced reads, then the operand layouts are built from shared memory ----
-        float* raw = &S.p2[0][0];                                   // 3,200 floats of scratch
-        for (uint32_t i = tid; i < 3200u; i += kC2Threads) raw[i] = prm[208u + i];
-        for (uint32_t i = tid; i < 2560u; i += kC2Threads)
-            S.wfT[(i & 255u) * 12u + (i >> 8)] = __bfloat162float(__float2bfloat16_rn(prm[3424u + i]));
-        if (tid < 16) S.b2[tid] = prm[3408u + tid];
-        if (tid < 10) S.bfc[tid] = prm[5984u + tid];
-        __syncthreads();
-        // W2[oc][ic][kh][kw] -> k = (kh*5+kw)*8 + ic: core matrix (tap g, oc/8), row oc%8, 16 bytes = 8 ic
-        for (uint32_t idx = tid; idx < 26u * 16u; idx += kC2Threads) {
-            const uint32_t g = idx >> 4, oc = idx & 15u;
-            uint32_t w[4] = { 0, 0, 0, 0 };
-            if (g < 25u) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    w[k] = pack_bf16(raw[(oc * 8u + 2 * k) * 25u + g], raw[(oc * 8u + 2 * k + 1) * 25u + g]);
-            }
-            *reinterpret_cast<uint4*>(S.b + (g * 2u + (oc >> 3)) * 128u + (oc & 7u) * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-        fence_async_smem();
-        __syncthreads();
-
-        if (tid == 0) {                                             // first pair's MMAs
-            int ok = mbar_wait_bounded(smem_u32(&S.full[0]), full_par & 1u, kWaitIters) ? 1 : 0;
-            if (ok) { tc_fence_after(); c2_issue_mma(S, 0, tmem, smem_u32(&S.mma_bar[0])); }
-            S.wait_ok = ok;
-        }
-        __syncthreads();
-        if (!S.wait_ok) { failed = true; break; }
-        full_par ^= 1u;
-
-        for (int i = 0; i < n; ++i) {
-            const int acc = i & 1, nxt = (i + 1) % kC2Bufs;
-            if (tid == 0) {
-                int ok = 1;
-                if (i + 1 < n) {                                    // run one pair ahead of the epilogue
-                    ok = mbar_wait_bounded(smem_u32(&S.full[nxt]), (full_par >> nxt) & 1u, kWaitIters) ? 1 : 0;
-                    if (ok) { tc_fence_after(); c2_issue_mma(S, nxt, tmem + 16u * (acc ^ 1), smem_u32(&S.mma_bar[acc ^ 1])); }
+    if (warp == 4) {
+        // ================= MMA issuer: one thread, runs ahead of the epilogue =================
+        if (lane == 0) {
+            uint32_t gp = 0, item_par = 0, full_par = 0, free_par = 0;
+            const uint32_t b0 = smem_u32(S.b);
+            for (;;) {
+                c2_wait(S, &S.item_ready, item_par, status);
+                item_par ^= 1u;
+                if (S.item == kNoItem || S.abort) break;
+                const int n = S.n;
+                for (int i = 0; i < n; ++i, ++gp) {
+                    const uint32_t slot = gp % kC2Bufs, acc = gp & 1u;
+                    c2_wait(S, &S.full[slot], (full_par >> slot) & 1u, status);
+                    full_par ^= (1u << slot);
+                    c2_wait(S, &S.acc_free[acc], (free_par >> acc) & 1u, status);
+                    free_par ^= (1u << acc);
+                    tc_fence_after();
+                    c2_issue_mma(smem_u32(S.a[slot]), b0, tmem + 16u * acc, smem_u32(&S.mma_done[acc]));
                 }
-                if (ok) ok = mbar_wait_bounded(smem_u32(&S.mma_bar[acc]), (mma_par >> acc) & 1u, kWaitIters) ? 1 : 0;
-                // pair i has been consumed: its ring slot takes pair i + ring depth
-                if (ok && i + kC2Bufs < n) c2_load_pair(S, i % kC2Bufs, src + static_cast<size_t>(i + kC2Bufs) * kPairBytes);
-                S.wait_ok = ok;
             }
-            __syncthreads();
-            if (!S.wait_ok) { failed = true; break; }
-            if (i + 1 < n) full_par ^= (1u << nxt);
-            mma_par ^= (1u << acc);
-            tc_fence_after();
-            // ---- epilogue: lane = (y%2, image, x); 2x2 max = lanes ^1 and ^16; + bias, ReLU, bf16 ----
-            {
+        }
+    } else {
+        // ================= epilogue warps ========================================================
+        // both accumulators start out free
+        if (lane == 0) { mbar_arrive(smem_u32(&S.acc_free[0])); mbar_arrive(smem_u32(&S.acc_free[1])); }
+        uint32_t gp = 0, done_par = 0;
+        for (;;) {
+            if (tid == 0) {                          // one thread decides, so the whole team takes one branch
+                const uint32_t next = atomicAdd(work_counter, 1u);
+                S.item = S.abort ? kNoItem : next;
+            }
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+            const uint32_t item = S.item;
+            if (item >= n_items) break;
+            const uint32_t member = item / items_per_member;
+            const uint32_t pair0 = (item % items_per_member) * kPairsPerItem;
+            const int n = static_cast<int>(min(n_pairs, pair0 + kPairsPerItem) - pair0);
+            const int n_img = static_cast<int>(min(batch, 2u * (pair0 + n)) - 2u * pair0);
+            const float* prm = theta + static_cast<size_t>(member) * ldD;
+            const unsigned char* src = pooled1 + (static_cast<size_t>(member) * n_pairs + pair0) * kPairBytes;
+
+            // every earlier pair has been consumed (its accumulator was waited for), so the ring is free
+            if (tid == 0)
+                for (int i = 0; i < min(kC2Bufs, n); ++i)
+                    c2_load_pair(S, (gp + i) % kC2Bufs, src + static_cast<size_t>(i) * kPairBytes);
+
+            // ---- weights: coalesced reads, then the operand layouts are built from shared memory ----
+            float* raw = &S.p2[0][0];                               // 3,200 floats of scratch
+            for (uint32_t i = tid; i < 3200u; i += kC2EpiThreads) raw[i] = prm[208u + i];
+            for (uint32_t i = tid; i < 2560u; i += kC2EpiThreads)
+                S.wfT[(i & 255u) * 12u + (i >> 8)] = __bfloat162float(__float2bfloat16_rn(prm[3424u + i]));
+            if (tid < 16) S.b2[tid] = prm[3408u + tid];
+            if (tid < 10) S.bfc[tid] = prm[5984u + tid];
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+            // W2[oc][ic][kh][kw] -> k = (kh*5+kw)*8 + ic: core matrix (tap g, oc/8), row oc%8, 16 bytes = 8 ic
+            for (uint32_t idx = tid; idx < 26u * 16u; idx += kC2EpiThreads) {
+                const uint32_t g = idx >> 4, oc = idx & 15u;
+                uint32_t w[4] = { 0, 0, 0, 0 };
+                if (g < 25u) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        w[k] = pack_bf16(raw[(oc * 8u + 2 * k) * 25u + g], raw[(oc * 8u + 2 * k + 1) * 25u + g]);
+                }
+                *reinterpret_cast<uint4*>(S.b + (g * 2u + (oc >> 3)) * 128u + (oc & 7u) * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            fence_async_smem();
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+            if (tid == 0) { S.n = n; __threadfence_block(); mbar_arrive(smem_u32(&S.item_ready)); }
+
+            for (int i = 0; i < n; ++i, ++gp) {
+                const uint32_t slot = gp % kC2Bufs, acc = gp & 1u;
+                c2_wait(S, &S.mma_done[acc], (done_par >> acc) & 1u, status);
+                done_par ^= (1u << acc);
+                tc_fence_after();
+                // pair i has been consumed by the tensor core: its ring slot takes pair i + ring depth
+                if (tid == 0 && i + kC2Bufs < n) c2_load_pair(S, slot, src + static_cast<size_t>(i + kC2Bufs) * kPairBytes);
+                // lane = (y%2, image, x); 2x2 max = lanes ^1 and ^16; + bias, ReLU, bf16
                 float r[16];
                 tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + 16u * acc, r);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&S.acc_free[acc]));   // values are in registers now
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     float v = fmaxf(r[c], __shfl_xor_sync(0xffffffffu, r[c], 1));
@@ -442,50 +481,49 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 }
                 __syncwarp();
             }
-            tc_fence_before();
-            __syncthreads();
-        }
-        if (failed) break;
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
 
-        // ---- linear 256 -> 10 for all images of the item: thread = (image, group of 4 classes) ----
-        if (warp < 3) {
-            float acc4[4] = { 0.f, 0.f, 0.f, 0.f };
-            if (lane < 2 * n) {
-                const float* x = S.p2[lane];
-                const float* wr = S.wfT + 4 * warp;
+            // ---- linear 256 -> 10 for all images of the item: thread = (image, group of 4 classes) ----
+            if (warp < 3) {
+                float acc4[4] = { 0.f, 0.f, 0.f, 0.f };
+                if (lane < 2 * n) {
+                    const float* x = S.p2[lane];
+                    const float* wr = S.wfT + 4 * warp;
 #pragma unroll 8
-                for (int k = 0; k < 256; ++k) {
-                    const float xv = x[k];
-                    const float4 w4 = *reinterpret_cast<const float4*>(wr + k * 12);
-                    acc4[0] = fmaf(w4.x, xv, acc4[0]); acc4[1] = fmaf(w4.y, xv, acc4[1]);
-                    acc4[2] = fmaf(w4.z, xv, acc4[2]); acc4[3] = fmaf(w4.w, xv, acc4[3]);
+                    for (int k = 0; k < 256; ++k) {
+                        const float xv = x[k];
+                        const float4 w4 = *reinterpret_cast<const float4*>(wr + k * 12);
+                        acc4[0] = fmaf(w4.x, xv, acc4[0]); acc4[1] = fmaf(w4.y, xv, acc4[1]);
+                        acc4[2] = fmaf(w4.z, xv, acc4[2]); acc4[3] = fmaf(w4.w, xv, acc4[3]);
+                    }
                 }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) S.logit[lane][4 * warp + j] = acc4[j] + S.bfc[4 * warp + j];
             }
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+            if (warp == 0) {
+                float l = 0.f;
+                if (lane < n_img) {
+                    const float* lg = S.logit[lane];
+                    float mx = lg[0];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) S.logit[lane][4 * warp + j] = acc4[j] + S.bfc[4 * warp + j];
-        }
-        __syncthreads();
-        if (warp == 0) {
-            float l = 0.f;
-            if (lane < n_img) {
-                const float* lg = S.logit[lane];
-                float mx = lg[0];
+                    for (int k = 1; k < 10; ++k) mx = fmaxf(mx, lg[k]);
+                    float se = 0.f;
 #pragma unroll
-                for (int k = 1; k < 10; ++k) mx = fmaxf(mx, lg[k]);
-                float se = 0.f;
+                    for (int k = 0; k < 10; ++k) se += expf(lg[k] - mx);
+                    const int lab = min(max(labels[2u * pair0 + lane], 0), 9);
+                    l = (mx + logf(se)) - lg[lab];
+                }
 #pragma unroll
-                for (int k = 0; k < 10; ++k) se += expf(lg[k] - mx);
-                const int lab = min(max(labels[2u * pair0 + lane], 0), 9);
-                l = (mx + logf(se)) - lg[lab];
+                for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);   // fixed order
+                if (lane == 0 && !S.abort) partial[item] = l;
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);   // fixed order
-            if (lane == 0) partial[item] = l;
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
         }
-        __syncthreads();
+        // release the issuer
+        if (tid == 0) { S.item = kNoItem; __threadfence_block(); mbar_arrive(smem_u32(&S.item_ready)); }
     }
 
-    if (failed && tid == 0) atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 32);
