@@ -96,18 +96,24 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
 }
-// Bounded wait: try_wait suspends the thread for a hardware-chosen short time by itself, so this
-// loop just re-arms it until the phase completes or ~max_cycles SM clocks have passed.
+// Bounded wait.  try_wait is given a suspend-time hint, so a waiting warp sleeps in hardware
+// instead of taking issue slots from the warps that work; the loop re-arms it until the phase
+// completes or ~2^max_cycles_log2 SM clocks have passed.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t max_cycles_log2)
 {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
     const long long t0 = clock64();
     const long long limit = 1ll << max_cycles_log2;
     for (;;) {
-        uint32_t done;
         asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
                      "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+                     : "=r"(done) : "r"(bar), "r"(parity), "r"(20000u) : "memory");     // hint: 20 us
         if (done) return true;
         if (clock64() - t0 > limit) return false;
     }
@@ -432,9 +438,29 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 
             // ---- weights: coalesced reads, then the operand layouts are built from shared memory ----
             float* raw = &S.p2[0][0];                               // 3,200 floats of scratch
-            for (uint32_t i = tid; i < 3200u; i += kC2EpiThreads) raw[i] = prm[208u + i];
-            for (uint32_t i = tid; i < 2560u; i += kC2EpiThreads)
-                S.wfT[(i & 255u) * 12u + (i >> 8)] = __bfloat162float(__float2bfloat16_rn(prm[3424u + i]));
+            {   // conv2 weights (offset 208) and linear weights (offset 3424) start 16-byte aligned
+                const float4* w2v = reinterpret_cast<const float4*>(prm + 208u);
+                const float4* wfv = reinterpret_cast<const float4*>(prm + 3424u);
+                float4 t2[7], tf[5];
+#pragma unroll
+                for (int k = 0; k < 7; ++k) t2[k] = (tid + k * kC2EpiThreads < 800) ? __ldg(w2v + tid + k * kC2EpiThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int k = 0; k < 5; ++k) tf[k] = __ldg(wfv + tid + k * kC2EpiThreads);
+#pragma unroll
+                for (int k = 0; k < 7; ++k)
+                    if (tid + k * kC2EpiThreads < 800) reinterpret_cast<float4*>(raw)[tid + k * kC2EpiThreads] = t2[k];
+#pragma unroll
+                for (int k = 0; k < 5; ++k) {
+                    // flat index cls*256 + (c*16 + pos), 4 consecutive pos; stored at row pos*16 + c
+                    const uint32_t i = 4u * (tid + k * kC2EpiThreads);
+                    const uint32_t cls = i >> 8, c = (i >> 4) & 15u, pos = i & 15u;
+                    float* d = S.wfT + (pos * 16u + c) * 12u + cls;
+                    d[0 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].x));
+                    d[1 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].y));
+                    d[2 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].z));
+                    d[3 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].w));
+                }
+            }
             if (tid < 16) S.b2[tid] = prm[3408u + tid];
             if (tid < 10) S.bfc[tid] = prm[5984u + tid];
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
@@ -453,6 +479,14 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
             if (tid == 0) { S.n = n; __threadfence_block(); mbar_arrive(smem_u32(&S.item_ready)); }
 
+            // After the 2x2 max (lanes ^1 = x parity, ^16 = y parity) done as a reduce-scatter, this
+            // lane owns channels c0..c0+3 of pooled pixel (image im, row py = warp, column px).
+            const int c0 = 8 * (lane & 1) + 4 * ((lane >> 4) & 1);
+            const int im = (lane >> 3) & 1, px = (lane & 7) >> 1, py = warp;
+            float bias4[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) bias4[j] = S.b2[c0 + j];
+
             for (int i = 0; i < n; ++i, ++gp) {
                 const uint32_t slot = gp % kC2Bufs, acc = gp & 1u;
                 c2_wait(S, &S.mma_done[acc], (done_par >> acc) & 1u, status);
@@ -466,40 +500,60 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&S.acc_free[acc]));   // values are in registers now
+                {
+                    const bool up0 = lane & 1, up1 = lane & 16;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    float v = fmaxf(r[c], __shfl_xor_sync(0xffffffffu, r[c], 1));
-                    v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 16));
-                    r[c] = v;
-                }
-                if ((lane & 17) == 0) {
-                    const int im = (lane >> 3) & 1, px = (lane & 7) >> 1, py = warp;
-                    float* dst = S.p2[2 * i + im] + py * 4 + px;
+                    for (int c = 0; c < 8; ++c) {
+                        const float keep = up0 ? r[8 + c] : r[c];
+                        const float give = up0 ? r[c] : r[8 + c];
+                        r[c] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 1));
+                    }
 #pragma unroll
-                    for (int c = 0; c < 16; ++c)
-                        dst[c * 16] = __bfloat162float(__float2bfloat16_rn(fmaxf(r[c] + S.b2[c], 0.f)));
+                    for (int c = 0; c < 4; ++c) {
+                        const float keep = up1 ? r[4 + c] : r[c];
+                        const float give = up1 ? r[c] : r[4 + c];
+                        r[c] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 16));
+                    }
+                    // activation index inside the item: (pixel, channel), channel innermost
+                    float* dst = S.p2[2 * i + im] + (py * 4 + px) * 16 + c0;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        dst[j] = __bfloat162float(__float2bfloat16_rn(fmaxf(r[j] + bias4[j], 0.f)));
                 }
-                __syncwarp();
             }
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
 
-            // ---- linear 256 -> 10 for all images of the item: thread = (image, group of 4 classes) ----
-            if (warp < 3) {
-                float acc4[4] = { 0.f, 0.f, 0.f, 0.f };
+            // ---- linear 256 -> 10 for all images of the item: thread = (image, quarter of the inputs);
+            //      the partial logits meet in the ring buffers, which are idle now ----
+            float* part = reinterpret_cast<float*>(S.a[0]);            // [4][32][12]
+            {
+                float acc[12];
+#pragma unroll
+                for (int j = 0; j < 12; ++j) acc[j] = 0.f;
                 if (lane < 2 * n) {
-                    const float* x = S.p2[lane];
-                    const float* wr = S.wfT + 4 * warp;
-#pragma unroll 8
-                    for (int k = 0; k < 256; ++k) {
+                    const float* x = S.p2[lane] + 64 * warp;
+                    const float* wr = S.wfT + 64 * warp * 12;
+#pragma unroll 4
+                    for (int k = 0; k < 64; ++k) {
                         const float xv = x[k];
-                        const float4 w4 = *reinterpret_cast<const float4*>(wr + k * 12);
-                        acc4[0] = fmaf(w4.x, xv, acc4[0]); acc4[1] = fmaf(w4.y, xv, acc4[1]);
-                        acc4[2] = fmaf(w4.z, xv, acc4[2]); acc4[3] = fmaf(w4.w, xv, acc4[3]);
+                        const float4 w0 = *reinterpret_cast<const float4*>(wr + k * 12);
+                        const float4 w1 = *reinterpret_cast<const float4*>(wr + k * 12 + 4);
+                        const float4 w2 = *reinterpret_cast<const float4*>(wr + k * 12 + 8);
+                        acc[0] = fmaf(w0.x, xv, acc[0]); acc[1] = fmaf(w0.y, xv, acc[1]);
+                        acc[2] = fmaf(w0.z, xv, acc[2]); acc[3] = fmaf(w0.w, xv, acc[3]);
+                        acc[4] = fmaf(w1.x, xv, acc[4]); acc[5] = fmaf(w1.y, xv, acc[5]);
+                        acc[6] = fmaf(w1.z, xv, acc[6]); acc[7] = fmaf(w1.w, xv, acc[7]);
+                        acc[8] = fmaf(w2.x, xv, acc[8]); acc[9] = fmaf(w2.y, xv, acc[9]);
                     }
                 }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) S.logit[lane][4 * warp + j] = acc4[j] + S.bfc[4 * warp + j];
+                float4* pw = reinterpret_cast<float4*>(part + (warp * 32 + lane) * 12);
+                pw[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                pw[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                pw[2] = make_float4(acc[8], acc[9], 0.f, 0.f);
             }
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+            for (int o = tid; o < 32 * 12; o += kC2EpiThreads)          // quarters added in a fixed order
+                S.logit[o / 12][o % 12] = ((part[o] + part[384 + o]) + (part[768 + o] + part[1152 + o])) + S.bfc[o % 12];
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
             if (warp == 0) {
                 float l = 0.f;
@@ -518,6 +572,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);   // fixed order
                 if (lane == 0 && !S.abort) partial[item] = l;
             }
+            fence_async_smem();        // the ring buffers held partial logits; bulk copies write them next
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
         }
         // release the issuer
