@@ -126,15 +126,67 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+
+// Wait that cannot hang: after one time-out anywhere in the block every later wait returns at
+// once (the block then finishes with meaningless numbers and EVO_ERR_TIMEOUT set).
+__device__ __forceinline__ void wait_or_abort(volatile int* abort_flag, uint64_t* bar, uint32_t parity,
+                                              DeviceStatus* status)
+{
+    if (*abort_flag) return;
+    if (!mbar_wait_bounded(smem_u32(bar), parity, kWaitIters)) {
+        *abort_flag = 1;
+        atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
+    }
+}
+
+// asynchronous TMEM load of 16 columns; the registers are valid after tmem_ld16_fence on them
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* u)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+                   "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16_fence(uint32_t* u)
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]),
+                   "+r"(u[8]), "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15])
+                 :: "memory");
+}
+
 // ------------------------------------------------------------------------------------------
-// conv1 for a group of up to 64 members
+// conv1 for a group of up to 64 members.
+//
+// GEMM rows are POOLED pixels (128 per tile); the four conv outputs of a 2x2 pooling window are
+// four separate A operands (the same 6x6 image patch shifted by (dy,dx)) accumulated into four
+// TMEM column blocks, so the max-pool is a max over four registers of one thread, with no
+// shuffles.  Unit of work = (tile, 8 members = 64 filters): 8 MMAs (4 windows x K = 2 x 16)
+// into one of two 256-column accumulators.  Warp 4 issues the MMAs and runs ahead; warps 0-3 read
+// the accumulators (pool, bias, ReLU, bf16) and store 16 bytes per (member, pixel), and stage the
+// next tile's A operands from a register-prefetched image patch.
 // ------------------------------------------------------------------------------------------
-constexpr int kC1Threads = 128;
-constexpr int kC1SmemB = 512 * 32 * 2;        // all filters of the group, bf16, K = 32
-constexpr int kC1SmemA = 128 * 32 * 2;        // one im2col tile
+constexpr int kC1EpiThreads = 128;
+constexpr int kC1Threads = kC1EpiThreads + 32;
+constexpr int kC1SmemB = 512 * 32 * 2;                  // all filters of the group, bf16, K = 32
+constexpr int kC1SmemAWin = 128 * 32 * 2;               // one window's im2col tile
+constexpr int kC1SmemA = 4 * kC1SmemAWin;               // four windows
 // the block owns all 512 TMEM columns, so it must be alone on its SM: ask for more than half
-// of the SM's shared memory
+// of the SM's shared memory (it uses ~100 KB of it)
 constexpr int kC1DynRequest = 120 * 1024;
+
+struct C1Ctl {
+    uint64_t a_full[2];          // the A operands of a tile are staged
+    uint64_t mma_done[2];        // an accumulator is complete
+    uint64_t acc_free[2];        // an accumulator has been read out
+    uint32_t tmem_slot;
+    volatile int abort;
+};
 
 // pooled-1 layout: [member][image pair][y 12][image in pair 2][x 12][channel 8] bf16
 __device__ __forceinline__ size_t pooled1_offset(uint32_t member, uint32_t n_pairs, uint32_t image,
@@ -143,32 +195,74 @@ __device__ __forceinline__ size_t pooled1_offset(uint32_t member, uint32_t n_pai
     return (((static_cast<size_t>(member) * n_pairs + (image >> 1)) * 12 + py) * 2 + (image & 1u)) * 12 + px;
 }
 
+// 6x6 image patch under one pooled pixel (zero for rows past the batch)
+__device__ __forceinline__ void c1_load_patch(const float* __restrict__ images, uint32_t gp, uint32_t n_pooled,
+                                              float (&patch)[36])
+{
+    if (gp < n_pooled) {
+        const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
+        const float* src = images + static_cast<size_t>(img) * 784u + (2u * py) * 28u + 2u * px;
+#pragma unroll
+        for (int r = 0; r < 6; ++r) {
+            const float2* row = reinterpret_cast<const float2*>(src + r * 28);     // 2*px is even: 8-byte aligned
+#pragma unroll
+            for (int c = 0; c < 3; ++c) {
+                const float2 v = __ldg(row + c);
+                patch[r * 6 + 2 * c] = v.x; patch[r * 6 + 2 * c + 1] = v.y;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 36; ++i) patch[i] = 0.f;
+    }
+}
+
+// im2col rows of the four windows of pooled pixel `row` into the A buffers (core matrices: 8 rows
+// x 16 bytes, k-group kg at +kg*2048, row group at +128)
+__device__ __forceinline__ void c1_stage_rows(unsigned char* Abuf, int row, const float (&patch)[36])
+{
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        const int dy = w >> 1, dx = w & 1;
+        uint32_t packed[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const int k0 = 2 * k, k1 = 2 * k + 1;
+            const float v0 = (k0 < 25) ? patch[(dy + k0 / 5) * 6 + dx + k0 % 5] : 0.f;
+            const float v1 = (k1 < 25) ? patch[(dy + k1 / 5) * 6 + dx + k1 % 5] : 0.f;
+            packed[k] = pack_bf16(v0, v1);
+        }
+#pragma unroll
+        for (int kg = 0; kg < 4; ++kg)
+            *reinterpret_cast<uint4*>(Abuf + w * kC1SmemAWin + (kg * 16 + (row >> 3)) * 128 + (row & 7) * 16) =
+                make_uint4(packed[4 * kg], packed[4 * kg + 1], packed[4 * kg + 2], packed[4 * kg + 3]);
+    }
+}
+
 __global__ void __launch_bounds__(kC1Threads, 1)
 k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const float* __restrict__ images,
                uint32_t batch, uint4* __restrict__ pooled1, uint32_t* work_counter, DeviceStatus* status)
 {
     extern __shared__ __align__(1024) unsigned char dyn[];
-    __shared__ __align__(8) uint64_t mma_bar;
-    __shared__ uint32_t tmem_slot;
-    __shared__ int wait_ok;
+    __shared__ __align__(8) C1Ctl ctl;
 
-    unsigned char* Bsm = dyn;
-    unsigned char* Asm = dyn + kC1SmemB;
-    float* bias = reinterpret_cast<float*>(dyn + kC1SmemB + kC1SmemA);
+    unsigned char* Bsm = dyn;                                           // 32 KB
+    unsigned char* Asm = dyn + kC1SmemB;                                // 2 x 32 KB
+    float* bias = reinterpret_cast<float*>(dyn + kC1SmemB + 2 * kC1SmemA);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t group0 = blockIdx.y * 64u;                         // first member of this group
+    const uint32_t group0 = blockIdx.y * 64u;                           // first member of this block's group
     const uint32_t n_members = min(64u, P - group0);
-    const uint32_t n_half = (n_members > 32u) ? 2u : 1u;
+    const uint32_t n_gm = (n_members + 7u) / 8u;                        // units per tile
     const uint32_t n_pairs = (batch + 1u) / 2u;
     const uint32_t n_pooled = batch * 144u;
-    const uint32_t n_tiles = (n_pooled + 31u) / 32u;
+    const uint32_t n_tiles = (n_pooled + 127u) / 128u;
 
     if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *work_counter = 0;   // for the conv2 kernel
 
-    // ---- B operand: W1 of every member of the group, [filter][k] -> core matrices (k-group, n-group)
+    // ---- B operand: W1 of every member of the group, [filter][k] -> core matrices (k-group, member)
     for (uint32_t idx = tid; idx < 512u * 4u; idx += kC1Threads) {
-        const uint32_t f = idx >> 2, kg = idx & 3u;                   // filter, 8-tap group
+        const uint32_t f = idx >> 2, kg = idx & 3u;                     // filter, 8-tap group
         const uint32_t m = f >> 3, ch = f & 7u;
         uint32_t w[4] = { 0, 0, 0, 0 };
         if (m < n_members) {
@@ -184,104 +278,120 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     for (uint32_t f = tid; f < 512u; f += kC1Threads)
         bias[f] = ((f >> 3) < n_members) ? theta[static_cast<size_t>(group0 + (f >> 3)) * ldD + 200u + (f & 7u)] : 0.f;
 
-    const uint32_t bar = smem_u32(&mma_bar);
     if (tid == 0) {
-        mbar_init(bar, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&ctl.a_full[i]), 1);
+            mbar_init(smem_u32(&ctl.mma_done[i]), 1);
+            mbar_init(smem_u32(&ctl.acc_free[i]), 4);
+        }
+        ctl.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512);
+    if (warp == 0) tmem_alloc(smem_u32(&ctl.tmem_slot), 512);
     fence_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = tmem_slot;
-    constexpr uint32_t idesc = umma_idesc_bf16(128, 256);
-    uint32_t phase = 0;
-    bool failed = false;
+    const uint32_t tmem = ctl.tmem_slot;
 
-    for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        // ---- A operand: im2col rows, row m = (pooled pixel m/4, window element m%4) ----------
-        {
-            const uint32_t gp = tile * 32u + (tid >> 2), wnd = tid & 3u;
-            uint32_t packed[16];
+    if (warp == 4) {
+        // ================= MMA issuer =============================================================
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
+            const uint32_t a_base = smem_u32(Asm), b_base = smem_u32(Bsm);
+            uint32_t u = 0, ti = 0;
+            for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++ti) {
+                wait_or_abort(&ctl.abort, &ctl.a_full[ti & 1u], (ti >> 1) & 1u, status);
+                const uint32_t a0 = a_base + (ti & 1u) * kC1SmemA;
+                for (uint32_t gm = 0; gm < n_gm; ++gm, ++u) {
+                    const uint32_t buf = u & 1u;
+                    wait_or_abort(&ctl.abort, &ctl.acc_free[buf], (u >> 1) & 1u, status);
+                    tc_fence_after();
 #pragma unroll
-            for (int k = 0; k < 16; ++k) packed[k] = 0;
-            if (gp < n_pooled) {
-                const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
-                const float* src = images + static_cast<size_t>(img) * 784u + (2u * py + (wnd >> 1)) * 28u + 2u * px + (wnd & 1u);
-                float v[26];
+                    for (uint32_t w = 0; w < 4u; ++w)
 #pragma unroll
-                for (int kh = 0; kh < 5; ++kh)
-#pragma unroll
-                    for (int kw = 0; kw < 5; ++kw) v[kh * 5 + kw] = __ldg(src + kh * 28 + kw);
-                v[25] = 0.f;
-#pragma unroll
-                for (int k = 0; k < 13; ++k) packed[k] = pack_bf16(v[2 * k], v[2 * k + 1]);
-            }
-#pragma unroll
-            for (int kg = 0; kg < 4; ++kg)
-                *reinterpret_cast<uint4*>(Asm + (kg * 16 + (tid >> 3)) * 128 + (tid & 7) * 16) =
-                    make_uint4(packed[4 * kg], packed[4 * kg + 1], packed[4 * kg + 2], packed[4 * kg + 3]);
-        }
-        fence_async_smem();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after();
-            const uint32_t a0 = smem_u32(Asm), b0 = smem_u32(Bsm);
-            for (uint32_t h = 0; h < n_half; ++h)
-                for (uint32_t ks = 0; ks < 2u; ++ks) {
-                    const uint64_t ad = umma_smem_desc(a0 + ks * 2u * 2048u, 2048u, 128u);
-                    const uint64_t bd = umma_smem_desc(b0 + ks * 2u * 8192u + h * 4096u, 8192u, 128u);
-                    umma_bf16(tmem + h * 256u, ad, bd, idesc, ks);
+                        for (uint32_t ks = 0; ks < 2u; ++ks) {
+                            const uint64_t ad = umma_smem_desc(a0 + w * kC1SmemAWin + ks * 2u * 2048u, 2048u, 128u);
+                            const uint64_t bd = umma_smem_desc(b_base + ks * 2u * 8192u + gm * 8u * 128u, 8192u, 128u);
+                            umma_bf16(tmem + buf * 256u + w * 64u, ad, bd, idesc, ks);
+                        }
+                    umma_commit(smem_u32(&ctl.mma_done[buf]));
                 }
-            umma_commit(bar);
-            wait_ok = mbar_wait_bounded(bar, phase, kWaitIters) ? 1 : 0;
+            }
         }
-        __syncthreads();
-        if (!wait_ok) { failed = true; break; }
-        phase ^= 1u;
-        tc_fence_after();
+    } else {
+        // ================= epilogue warps (also stage the A operands) ==============================
+        if (lane == 0) { mbar_arrive(smem_u32(&ctl.acc_free[0])); mbar_arrive(smem_u32(&ctl.acc_free[1])); }
+        float patch[36];
+        // first tile
+        c1_load_patch(images, blockIdx.x * 128u + tid, n_pooled, patch);
+        if (blockIdx.x < n_tiles) {
+            c1_stage_rows(Asm, tid, patch);
+            fence_async_smem();
+            asm volatile("bar.sync 1, %0;" :: "n"(kC1EpiThreads) : "memory");
+            if (tid == 0) mbar_arrive(smem_u32(&ctl.a_full[0]));
+        }
+        uint32_t u = 0, ti = 0;
+        for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++ti) {
+            const uint32_t next = tile + gridDim.x;
+            const bool has_next = next < n_tiles;
+            if (has_next) c1_load_patch(images, next * 128u + tid, n_pooled, patch);     // lands during the epilogues
+            const uint32_t stage_after = min(2u, n_gm - 1u);
 
-        // ---- epilogue: 32 filters (4 members) at a time; 2x2 max over the 4 lanes of a pixel ----
-        const uint32_t gp = tile * 32u + warp * 8u + (lane >> 2);
-        const bool pix_ok = gp < n_pooled;
-        const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
-        const bool b0 = lane & 1, b1 = lane & 2;
-        for (uint32_t grp = 0; grp < n_half * 8u; ++grp) {
-            float r[32];
-            const uint32_t taddr = tmem + (static_cast<uint32_t>(warp * 32) << 16) + grp * 32u;
-            tmem_ld16(taddr, r);
-            tmem_ld16(taddr + 16u, r + 16);
+            const uint32_t gp = tile * 128u + tid;                     // my pooled pixel = my TMEM lane
+            const bool pix_ok = gp < n_pooled;
+            const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
+
+            for (uint32_t gm = 0; gm < n_gm; ++gm, ++u) {
+                const uint32_t buf = u & 1u;
+                wait_or_abort(&ctl.abort, &ctl.mma_done[buf], (u >> 1) & 1u, status);
+                tc_fence_after();
+                const uint32_t t0 = tmem + (static_cast<uint32_t>(warp * 32) << 16) + buf * 256u;
+#pragma unroll 1
+                for (uint32_t chunk = 0; chunk < 4u; ++chunk) {         // 16 filters = 2 members at a time
+                    uint32_t r0[16], r1[16], r2[16], r3[16];
+                    tmem_ld16_issue(t0 + 0u * 64u + chunk * 16u, r0);
+                    tmem_ld16_issue(t0 + 1u * 64u + chunk * 16u, r1);
+                    tmem_ld16_issue(t0 + 2u * 64u + chunk * 16u, r2);
+                    tmem_ld16_issue(t0 + 3u * 64u + chunk * 16u, r3);
+                    tmem_ld16_fence(r0); tmem_ld16_fence(r1); tmem_ld16_fence(r2); tmem_ld16_fence(r3);
+                    if (chunk == 3u) {                                   // accumulator is in registers: hand it back
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctl.acc_free[buf]));
+                    }
+                    const uint32_t m0 = gm * 8u + chunk * 2u;            // first of the two members
+                    const float* bb = bias + m0 * 8u;
+                    uint32_t o[8];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float keep = b0 ? r[16 + i] : r[i];
-                const float give = b0 ? r[i] : r[16 + i];
-                r[i] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 1));
+                    for (int c = 0; c < 8; ++c) {
+                        const float v0 = fmaxf(fmaxf(__uint_as_float(r0[2 * c]), __uint_as_float(r1[2 * c])),
+                                               fmaxf(__uint_as_float(r2[2 * c]), __uint_as_float(r3[2 * c])));
+                        const float v1 = fmaxf(fmaxf(__uint_as_float(r0[2 * c + 1]), __uint_as_float(r1[2 * c + 1])),
+                                               fmaxf(__uint_as_float(r2[2 * c + 1]), __uint_as_float(r3[2 * c + 1])));
+                        o[c] = pack_bf16(fmaxf(v0 + bb[2 * c], 0.f), fmaxf(v1 + bb[2 * c + 1], 0.f));
+                    }
+                    if (pix_ok) {
+                        if (m0 < n_members)
+                            pooled1[pooled1_offset(group0 + m0, n_pairs, img, py, px)] = make_uint4(o[0], o[1], o[2], o[3]);
+                        if (m0 + 1u < n_members)
+                            pooled1[pooled1_offset(group0 + m0 + 1u, n_pairs, img, py, px)] = make_uint4(o[4], o[5], o[6], o[7]);
+                    }
+                    __syncwarp();
+                }
+                if (has_next && gm == stage_after) {
+                    // the other A buffer was last read by the previous tile, whose accumulators have all
+                    // been waited for: refill it for the next tile
+                    c1_stage_rows(Asm + ((ti + 1u) & 1u) * kC1SmemA, tid, patch);
+                    fence_async_smem();
+                    asm volatile("bar.sync 1, %0;" :: "n"(kC1EpiThreads) : "memory");
+                    if (tid == 0) mbar_arrive(smem_u32(&ctl.a_full[(ti + 1u) & 1u]));
+                }
             }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float keep = b1 ? r[8 + i] : r[i];
-                const float give = b1 ? r[i] : r[8 + i];
-                r[i] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 2));
-            }
-            const uint32_t m = grp * 4u + (b0 ? 2u : 0u) + (b1 ? 1u : 0u);   // member whose 8 channels I hold
-            if (pix_ok && m < n_members) {
-                const float* bb = bias + m * 8u;
-                uint32_t o[4];
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    o[c] = pack_bf16(fmaxf(r[2 * c] + bb[2 * c], 0.f), fmaxf(r[2 * c + 1] + bb[2 * c + 1], 0.f));
-                pooled1[pooled1_offset(group0 + m, n_pairs, img, py, px)] = make_uint4(o[0], o[1], o[2], o[3]);
-            }
-            __syncwarp();
         }
-        tc_fence_before();
-        __syncthreads();
     }
 
-    if (failed && tid == 0) atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 512);
@@ -322,19 +432,9 @@ struct __align__(128) C2Smem {
     volatile int n;
 };
 
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
-}
-
-// Wait that cannot hang: after one time-out anywhere in the block every later wait returns at once.
 __device__ __forceinline__ void c2_wait(C2Smem& S, uint64_t* bar, uint32_t parity, DeviceStatus* status)
 {
-    if (S.abort) return;
-    if (!mbar_wait_bounded(smem_u32(bar), parity, kWaitIters)) {
-        S.abort = 1;
-        atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
-    }
+    wait_or_abort(&S.abort, bar, parity, status);
 }
 
 __device__ __forceinline__ void c2_load_pair(C2Smem& S, int buf, const unsigned char* src)
@@ -629,7 +729,7 @@ int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uin
     unsigned char* pooled1 = base + 256 + (static_cast<size_t>(P) * ipm * sizeof(float) + 255) / 256 * 256;
 
     if (cudaFuncSetAttribute(k_cnn_conv1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kC1DynRequest) != cudaSuccess) return -1;
-    const uint32_t n_tiles = (batch * 144u + 31u) / 32u;
+    const uint32_t n_tiles = (batch * 144u + 127u) / 128u;
     dim3 g1(min(static_cast<uint32_t>(sm_count), n_tiles), (P + 63u) / 64u);
     k_cnn_conv1_tc<<<g1, kC1Threads, kC1DynRequest, st>>>(theta, ldD, P, images, batch,
                                                           reinterpret_cast<uint4*>(pooled1), counter, status);
