@@ -171,7 +171,7 @@ __device__ __forceinline__ void tmem_ld16_fence(uint32_t* u)
 // the accumulators (pool, bias, ReLU, bf16) and store 16 bytes per (member, pixel), and stage the
 // next tile's A operands from a register-prefetched image patch.
 // ------------------------------------------------------------------------------------------
-constexpr int kC1EpiThreads = 128;
+constexpr int kC1EpiThreads = 256;                     // two warps per TMEM lane quarter
 constexpr int kC1Threads = kC1EpiThreads + 32;
 constexpr int kC1SmemB = 512 * 32 * 2;                  // all filters of the group, bf16, K = 32
 constexpr int kC1SmemAWin = 128 * 32 * 2;               // one window's im2col tile
@@ -219,11 +219,11 @@ __device__ __forceinline__ void c1_load_patch(const float* __restrict__ images, 
 
 // im2col rows of the four windows of pooled pixel `row` into the A buffers (core matrices: 8 rows
 // x 16 bytes, k-group kg at +kg*2048, row group at +128)
-__device__ __forceinline__ void c1_stage_rows(unsigned char* Abuf, int row, const float (&patch)[36])
+__device__ __forceinline__ void c1_stage_rows(unsigned char* Abuf, int row, int dy, const float (&patch)[36])
 {
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
-        const int dy = w >> 1, dx = w & 1;
+    for (int dx = 0; dx < 2; ++dx) {                     // the two windows of conv row parity dy
+        const int w = 2 * dy + dx;
         uint32_t packed[16];
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
@@ -282,7 +282,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl.a_full[i]), 1);
             mbar_init(smem_u32(&ctl.mma_done[i]), 1);
-            mbar_init(smem_u32(&ctl.acc_free[i]), 4);
+            mbar_init(smem_u32(&ctl.acc_free[i]), kC1EpiThreads / 32);
         }
         ctl.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -295,7 +295,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     tc_fence_after();
     const uint32_t tmem = ctl.tmem_slot;
 
-    if (warp == 4) {
+    if (warp == kC1EpiThreads / 32) {
         // ================= MMA issuer =============================================================
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
@@ -325,9 +325,10 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         if (lane == 0) { mbar_arrive(smem_u32(&ctl.acc_free[0])); mbar_arrive(smem_u32(&ctl.acc_free[1])); }
         float patch[36];
         // first tile
-        c1_load_patch(images, blockIdx.x * 128u + tid, n_pooled, patch);
+        const int row = tid & 127, half = tid >> 7;       // my pooled pixel (= TMEM lane) and my half of the work
+        c1_load_patch(images, blockIdx.x * 128u + row, n_pooled, patch);
         if (blockIdx.x < n_tiles) {
-            c1_stage_rows(Asm, tid, patch);
+            if (half) c1_stage_rows(Asm, row, 1, patch); else c1_stage_rows(Asm, row, 0, patch);
             fence_async_smem();
             asm volatile("bar.sync 1, %0;" :: "n"(kC1EpiThreads) : "memory");
             if (tid == 0) mbar_arrive(smem_u32(&ctl.a_full[0]));
@@ -336,10 +337,10 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++ti) {
             const uint32_t next = tile + gridDim.x;
             const bool has_next = next < n_tiles;
-            if (has_next) c1_load_patch(images, next * 128u + tid, n_pooled, patch);     // lands during the epilogues
+            if (has_next) c1_load_patch(images, next * 128u + row, n_pooled, patch);     // lands during the epilogues
             const uint32_t stage_after = min(2u, n_gm - 1u);
 
-            const uint32_t gp = tile * 128u + tid;                     // my pooled pixel = my TMEM lane
+            const uint32_t gp = tile * 128u + row;                     // my pooled pixel = my TMEM lane
             const bool pix_ok = gp < n_pooled;
             const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
 
@@ -347,16 +348,16 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 const uint32_t buf = u & 1u;
                 wait_or_abort(&ctl.abort, &ctl.mma_done[buf], (u >> 1) & 1u, status);
                 tc_fence_after();
-                const uint32_t t0 = tmem + (static_cast<uint32_t>(warp * 32) << 16) + buf * 256u;
+                const uint32_t t0 = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + buf * 256u;
 #pragma unroll 1
-                for (uint32_t chunk = 0; chunk < 4u; ++chunk) {         // 16 filters = 2 members at a time
+                for (uint32_t chunk = 2u * half; chunk < 2u * half + 2u; ++chunk) {   // 16 filters = 2 members at a time
                     uint32_t r0[16], r1[16], r2[16], r3[16];
                     tmem_ld16_issue(t0 + 0u * 64u + chunk * 16u, r0);
                     tmem_ld16_issue(t0 + 1u * 64u + chunk * 16u, r1);
                     tmem_ld16_issue(t0 + 2u * 64u + chunk * 16u, r2);
                     tmem_ld16_issue(t0 + 3u * 64u + chunk * 16u, r3);
                     tmem_ld16_fence(r0); tmem_ld16_fence(r1); tmem_ld16_fence(r2); tmem_ld16_fence(r3);
-                    if (chunk == 3u) {                                   // accumulator is in registers: hand it back
+                    if (chunk == 2u * half + 1u) {                        // my part of the accumulator is in registers
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&ctl.acc_free[buf]));
@@ -383,7 +384,8 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 if (has_next && gm == stage_after) {
                     // the other A buffer was last read by the previous tile, whose accumulators have all
                     // been waited for: refill it for the next tile
-                    c1_stage_rows(Asm + ((ti + 1u) & 1u) * kC1SmemA, tid, patch);
+                    if (half) c1_stage_rows(Asm + ((ti + 1u) & 1u) * kC1SmemA, row, 1, patch);
+                    else      c1_stage_rows(Asm + ((ti + 1u) & 1u) * kC1SmemA, row, 0, patch);
                     fence_async_smem();
                     asm volatile("bar.sync 1, %0;" :: "n"(kC1EpiThreads) : "memory");
                     if (tid == 0) mbar_arrive(smem_u32(&ctl.a_full[(ti + 1u) & 1u]));
