@@ -129,11 +129,58 @@ k_rank(const float* __restrict__ fitness, uint32_t P, int32_t* __restrict__ rank
     }
 }
 
+// Large populations: the comparisons of a member are split over blockIdx.y (one fitness tile each)
+// and summed with integer atomics (exact, order-independent); a second kernel turns counts into
+// centred ranks.
+__global__ void __launch_bounds__(256)
+k_rank_count(const float* __restrict__ fitness, uint32_t P, int32_t* __restrict__ rank, DeviceStatus* status)
+{
+    __shared__ float tile[kRankTile];
+    const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t base = blockIdx.y * kRankTile;
+    const uint32_t n = min(kRankTile, P - base);
+    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) tile[i] = fitness[base + i];
+    __syncthreads();
+    if (m >= P) return;
+    const float fm = fitness[m];
+    if (blockIdx.y == 0 && fm != fm) atomicOr(&status->nonfinite, 1u);
+    uint32_t below = 0;
+#pragma unroll 8
+    for (uint32_t i = 0; i < n; ++i) {
+        const float fk = tile[i];
+        below += (fk < fm || (fk == fm && base + i < m)) ? 1u : 0u;
+    }
+    atomicAdd(rank + m, static_cast<int32_t>(below));
+}
+
+__global__ void k_rank_zero(int32_t* __restrict__ rank, uint32_t P)
+{
+    const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m < P) rank[m] = 0;
+}
+
+__global__ void k_rank_finish(const int32_t* __restrict__ rank, uint32_t P, float* __restrict__ u)
+{
+    const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m < P)
+        u[m] = __fadd_rn(__fdiv_rn(__uint2float_rn(static_cast<uint32_t>(rank[m])), __uint2float_rn(P - 1u)), -0.5f);
+}
+
 int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank, float* u,
                 DeviceStatus* status)
 {
-    k_rank<<<(P + 255u) / 256u, 256, 0, st>>>(fitness, P, rank, u, status);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    const uint32_t bx = (P + 255u) / 256u;
+    if (P <= 2u * kRankTile) {
+        k_rank<<<bx, 256, 0, st>>>(fitness, P, rank, u, status);
+        return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    }
+    k_rank_zero<<<bx, 256, 0, st>>>(rank, P);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    dim3 grid(bx, (P + kRankTile - 1u) / kRankTile);
+    k_rank_count<<<grid, 256, 0, st>>>(fitness, P, rank, status);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    k_rank_finish<<<bx, 256, 0, st>>>(rank, P, u);
+    return cudaGetLastError() == cudaSuccess ? 3 : -1;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -156,8 +203,11 @@ __device__ __forceinline__ void acc_fma(Acc4& a, double wd, const float4& e)
     a.w = fma(wd, static_cast<double>(e.w), a.w);
 }
 
+constexpr int kGradThreads = 256;      // threads per block of the gradient kernel
+constexpr int kGradRows = 4;           // noise rows in flight per thread (multiple of 2)
+
 template <bool REGEN>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kGradThreads)
 k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, PhiloxKey key,
                uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, uint32_t pairs_per_split,
                double* __restrict__ partial, const DeviceStatus* status)
@@ -170,21 +220,21 @@ k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, Philo
     Acc4 acc[2] = { {0., 0., 0., 0.}, {0., 0., 0., 0.} };
     const float2* up = reinterpret_cast<const float2*>(u);
     uint32_t j = j0;
-    for (; j + 4u <= j1; j += 4u) {
-        float4 e[4];
-        double w[4];
+    for (; j + kGradRows <= j1; j += kGradRows) {
+        float4 e[kGradRows];
+        double w[kGradRows];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kGradRows; ++i) {
             if (REGEN) e[i] = stream_normal4(key, 0u, generation, j + i, quad);
             else e[i] = __ldcs(reinterpret_cast<const float4*>(eps + static_cast<size_t>(j + i) * ldD) + quad);
             const float2 uu = __ldg(up + j + i);
             w[i] = static_cast<double>(uu.x) - static_cast<double>(uu.y);   // exact
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc_fma(acc[i & 1], w[i], e[i]);
+        for (int i = 0; i < kGradRows; ++i) acc_fma(acc[i & 1], w[i], e[i]);
     }
 #pragma unroll
-    for (int i = 0; i < 3; ++i) {                  // tail keeps the accumulator assignment j % 2
+    for (int i = 0; i < kGradRows - 1; ++i) {      // tail keeps the accumulator assignment j % 2
         if (j + i < j1) {
             float4 e;
             if (REGEN) e = stream_normal4(key, 0u, generation, j + i, quad);
@@ -262,8 +312,8 @@ __global__ void k_tell_finish(DeviceStatus* status)
 uint32_t gradient_splits(uint32_t H, uint32_t ldD)
 {
     // enough thread blocks to fill 148 SMs several times over, a pure function of the shape
-    const uint32_t blocks_x = (ldD / 4u + 127u) / 128u;
-    uint32_t s = (148u * 8u + blocks_x - 1u) / blocks_x;
+    const uint32_t blocks_x = (ldD / 4u + kGradThreads - 1u) / kGradThreads;
+    uint32_t s = (148u * 32u + blocks_x - 1u) / blocks_x;
     if (s > 64u) s = 64u;
     const uint32_t max_s = (H + 15u) / 16u;            // at least 16 pairs per split
     if (s > max_s) s = max_s;
@@ -280,12 +330,12 @@ int launch_gradient_adam(cudaStream_t st, const float* u, const float* eps, uint
     const uint32_t quads = ldD / 4u;
     const uint32_t pps = (H + splits - 1u) / splits;
     const uint32_t used = (H + pps - 1u) / pps;        // splits that own at least one pair
-    dim3 grid((quads + 127u) / 128u, used);
+    dim3 grid((quads + kGradThreads - 1u) / kGradThreads, used);
     if (eps)
-        k_grad_partial<false><<<grid, 128, 0, st>>>(u, eps, PhiloxKey{k0, k1}, generation, H, D, ldD, pps,
+        k_grad_partial<false><<<grid, kGradThreads, 0, st>>>(u, eps, PhiloxKey{k0, k1}, generation, H, D, ldD, pps,
                                                     partial, status);
     else
-        k_grad_partial<true><<<grid, 128, 0, st>>>(u, nullptr, PhiloxKey{k0, k1}, generation, H, D, ldD,
+        k_grad_partial<true><<<grid, kGradThreads, 0, st>>>(u, nullptr, PhiloxKey{k0, k1}, generation, H, D, ldD,
                                                    pps, partial, status);
     if (cudaGetLastError() != cudaSuccess) return -1;
     const double scale = static_cast<double>(sigma) / static_cast<double>(2u * H);

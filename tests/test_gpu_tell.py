@@ -88,6 +88,23 @@ def test_rank_ties_and_specials_bitwise():
     _tell_check(W.Workload("ties", 4096 + 2, 8, seed=1, sigma=0.5), 2, True, fit)
 
 
+def test_rank_large_population_split_path():
+    # P > 4096 takes the split counting path (integer atomics); ties and specials included
+    def fit(seed, gen, P):
+        f = np.round(np.random.default_rng(gen + 5).standard_normal(P) * 50).astype(np.float32)
+        f[1] = np.inf; f[2] = -np.inf; f[3] = 0.0; f[4] = -0.0
+        return f
+    _tell_check(W.Workload("bigP", 16384, 40, seed=2, sigma=0.5), 2, True, fit)
+    _tell_check(W.Workload("bigP", 5000, 9, seed=3, sigma=0.5), 1, False)
+    # NaN is still caught on this path
+    w = W.Workload("bigP", 6000, 8, seed=4, sigma=0.5)
+    s = Solver(w); s.ask()
+    f = W.synthetic_fitness(4, 0, 6000); f[5999] = np.nan
+    s.tell(torch.tensor(f, device="cuda"))
+    assert s.sync_status() == 5
+    s.close()
+
+
 def test_nan_fitness_skips_the_update_and_is_reported():
     w = _bare(W.CFG1)
     s = Solver(w)
