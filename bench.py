@@ -58,6 +58,17 @@ def stage_work(w, stored):
     return {"ask_bytes": ask_bytes, "tell_bytes": tell_bytes, "rollout_flops": rollout_flops}
 
 
+# DRAM bytes (read + write) of the dominant kernel per launch, from the ncu captures summarised
+# under profiles/ (same workload, same kernel).  An entry is dropped (-> null) when its kernel
+# changes after the capture.
+NCU_TRAFFIC_BYTES = {
+    ("cfg2", "stored"): ("k_rollout_cartpole_ws", 4.797184e6),
+    ("cfg2", "regenerated"): ("k_rollout_cartpole_ws", 4.797184e6),
+    ("cfg3", "stored"): ("k_cnn_conv2_tc", 152.562176e6 + 3.476224e6),
+    ("cfg5", "stored"): ("k_ask", 32 * (3.161320e9 + 0.000144e9)),       # reduced-D capture scaled by D
+}
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -390,6 +401,7 @@ def run_ours(args, w):
             "rollout": {"ms": t_roll, "TFLOP/s": work["rollout_flops"] / (t_roll * 1e-3) / 1e12 if t_roll > 0 else 0.0},
             "tell": {"ms": t_tell, "GB/s": work["tell_bytes"] / (t_tell * 1e-3) / 1e9},
         }
+        traffic_entry = NCU_TRAFFIC_BYTES.get((args.workload, args.noise)) if not (args.pop or args.dim) else None
         if no_task:
             dom = "ask" if t_ask >= t_tell else "tell"
             achieved = stages[dom]["GB/s"]
@@ -399,16 +411,19 @@ def run_ours(args, w):
                         "traffic": None}
         elif supervised:
             achieved = stages["rollout"]["TFLOP/s"]
-            roofline = {"kernel": "k_cnn", "bound": "tensor", "achieved": achieved,
+            roofline = {"kernel": "k_cnn_conv1_tc + k_cnn_conv2_tc", "bound": "tensor", "achieved": achieved,
                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                         "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"],
                         "traffic": None}
         else:
             achieved = stages["rollout"]["TFLOP/s"]
-            roofline = {"kernel": "k_rollout_mlp", "bound": "alu", "achieved": achieved, "peak": alu_peak,
+            roofline = {"kernel": "k_rollout_mlp (tiled / warp-specialised)", "bound": "alu", "achieved": achieved, "peak": alu_peak,
                         "unit": "TFLOP/s", "frac": achieved / alu_peak,
                         "peak_source": f"{sm_count} SMs x 128 fp32 lanes x 2 x {max_mhz} MHz",
                         "traffic": None}
+        if traffic_entry is not None and (not no_task or roofline["kernel"] == traffic_entry[0]):
+            roofline["traffic"] = traffic_entry[1]
+            roofline["traffic_kernel"] = traffic_entry[0]
         cpu = None
         if not args.skip_cpu_baseline:
             n = members_for_budget(w, 12.0)

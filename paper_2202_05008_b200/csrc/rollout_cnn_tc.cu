@@ -4,10 +4,11 @@
 // 256->10) evaluated for every member on the same batch is two dense contractions:
 //
 //   k_cnn_conv1_tc   conv1 for ALL members at once.  The batch is shared, so the im2col rows
-//                    (one per output pixel, K = 25 taps padded to 32) are the A operand for every
-//                    member, and the 8P filters of the population sit side by side on N:
-//                    D[128 pixels][256 filters] per tcgen05.mma, 512 TMEM columns per tile.  The
-//                    epilogue takes bias/ReLU/2x2-max-pool out of TMEM and writes the pooled
+//                    (K = 25 taps padded to 32) are the A operand for every member and the 8P
+//                    filters of the population sit side by side on N.  GEMM rows are pooled
+//                    pixels; the four conv outputs under a pooling window are four A operands
+//                    accumulated into four TMEM column blocks, so the 2x2 max-pool is a max over
+//                    registers.  The epilogue adds bias, applies ReLU and writes the pooled
 //                    activation as bf16, 8 channels = 16 bytes per pixel.
 //   k_cnn_conv2_tc   per member: conv2 as an implicit GEMM with NO im2col copy.  With channels
 //                    innermost, the 8 channels of a pixel are one 16-byte row of a UMMA core
