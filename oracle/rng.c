@@ -58,34 +58,37 @@ static uint32_t f32_bits(float x) { uint32_t b; memcpy(&b, &x, 4); return b; }
 static float bits_f32(uint32_t b) { float x; memcpy(&x, &b, 4); return x; }
 
 /*
- * ln(u) for a positive normal fp32 u.  Split u = m * 2^e with m in [sqrt(1/2), sqrt(2)),
- * then ln m = 2 atanh(s), s = (m-1)/(m+1), by the odd series up to s^11/11.
+ * ln(u) for a positive normal fp32 u.  Split u = m * 2^e with m in [sqrt(1/2), sqrt(2)) and
+ * f = m - 1 (exact); ln m = f - f^2/2 + f^3 P(f) with a degree-7 polynomial P fitted to
+ * (ln(1+f) - f + f^2/2)/f^3 on that interval (coefficients are part of the definition, given as
+ * fp32 bit patterns).  The form keeps full relative accuracy as u -> 1, and needs no division.
  */
+static const uint32_t LN_POLY_BITS[8] = {
+    0x3EAAAAA9u, 0xBE800064u, 0x3E4CD0A6u, 0xBE2A6AA7u, 0x3E116E25u, 0xBE04D5F2u, 0x3E022C8Du, 0xBDA5EB80u
+};
+
 float oracle_ln_f32(float u)
 {
     uint32_t b = f32_bits(u);
     int e = (int)(b >> 23) - 126;                         /* u = m * 2^e, m in [0.5, 1) */
     float m = bits_f32((b & 0x007FFFFFu) | 0x3F000000u);
     if (m < 0.70710678f) { m = m * 2.0f; e -= 1; }
-    float a = m - 1.0f;
-    float d = m + 1.0f;
-    float s = a / d;
-    float z = s * s;
-    float p = 1.0f / 11.0f;
-    p = fmaf(p, z, 1.0f / 9.0f);
-    p = fmaf(p, z, 1.0f / 7.0f);
-    p = fmaf(p, z, 1.0f / 5.0f);
-    p = fmaf(p, z, 1.0f / 3.0f);
-    p = fmaf(p, z, 1.0f);
-    float sp = s * p;
-    float two_sp = 2.0f * sp;
-    return fmaf((float)e, 0.69314718f, two_sp);
+    float f = m - 1.0f;
+    float z = f * f;
+    float p = bits_f32(LN_POLY_BITS[7]);
+    for (int i = 6; i >= 0; --i) p = fmaf(p, f, bits_f32(LN_POLY_BITS[i]));
+    float t = f * z;
+    float h = 0.5f * z;
+    float r = fmaf(t, p, -h);
+    float lnm = f + r;
+    return fmaf((float)e, 0.69314718f, lnm);
 }
 
 /*
  * cos and sin of 2*pi*v for v in [0,1).  w = 4v counts quarter turns; k = nearest
  * integer (ties to even), t = w - k is exact with |t| <= 1/2, x = t*(pi/2) lies in
- * [-pi/4, pi/4] where the Taylor polynomials below are accurate to fp32 rounding.
+ * [-pi/4, pi/4] where the Taylor polynomials below (sin to x^9, cos to x^10) are accurate to
+ * fp32 rounding.
  */
 void oracle_cossin_2pi_f32(float v, float* c_out, float* s_out)
 {
@@ -95,16 +98,14 @@ void oracle_cossin_2pi_f32(float v, float* c_out, float* s_out)
     float x = t * 1.57079637f;
     float z = x * x;
 
-    float sp = -1.0f / 39916800.0f;            /* -1/11! */
-    sp = fmaf(sp, z, 1.0f / 362880.0f);        /*  1/9!  */
+    float sp = 1.0f / 362880.0f;               /*  1/9!  */
     sp = fmaf(sp, z, -1.0f / 5040.0f);         /* -1/7!  */
     sp = fmaf(sp, z, 1.0f / 120.0f);           /*  1/5!  */
     sp = fmaf(sp, z, -1.0f / 6.0f);            /* -1/3!  */
     sp = fmaf(sp, z, 1.0f);
     float sn = x * sp;
 
-    float cp = 1.0f / 479001600.0f;            /*  1/12! */
-    cp = fmaf(cp, z, -1.0f / 3628800.0f);      /* -1/10! */
+    float cp = -1.0f / 3628800.0f;             /* -1/10! */
     cp = fmaf(cp, z, 1.0f / 40320.0f);         /*  1/8!  */
     cp = fmaf(cp, z, -1.0f / 720.0f);          /* -1/6!  */
     cp = fmaf(cp, z, 1.0f / 24.0f);            /*  1/4!  */

@@ -53,18 +53,25 @@ def test_uniforms_are_exact_and_in_range():
     assert oracle.u_open(0xFFFFFFFF) == 1.0 and oracle.u_open(0) > 0.0
 
 
-def test_series_coefficients_are_fp32_roundings_of_the_fractions():
-    # ln(1 + tiny) and sin/cos at tiny arguments expose only the leading coefficients;
-    # the full table is checked through accuracy below.  Here: fp32(1/n) bit patterns
-    # that both implementations must use.
-    table = {3: 0x3EAAAAAB, 5: 0x3E4CCCCD, 7: 0x3E124925, 9: 0x3DE38E39, 11: 0x3DBA2E8C}
-    for n, bits in table.items():
-        assert np.float32(1.0) / np.float32(n) == np.uint32(bits).view(np.float32)
+def test_trig_coefficients_are_fp32_roundings_of_the_factorial_fractions():
+    # bit patterns that both implementations type in for sin (to x^9) and cos (to x^10)
     fact = {2: 0x3F000000, 3: 0x3E2AAAAB, 4: 0x3D2AAAAB, 5: 0x3C088889, 6: 0x3AB60B61,
-            7: 0x39500D01, 8: 0x37D00D01, 9: 0x3638EF1D, 10: 0x3493F27E, 11: 0x32D7322B,
-            12: 0x310F76C7}
+            7: 0x39500D01, 8: 0x37D00D01, 9: 0x3638EF1D, 10: 0x3493F27E}
     for n, bits in fact.items():
         assert np.float32(1.0) / np.float32(math.factorial(n)) == np.uint32(bits).view(np.float32)
+
+
+def test_ln_polynomial_is_a_fit_of_the_log_series_remainder():
+    # P(f) ~ (ln(1+f) - f + f^2/2) / f^3 on [sqrt(1/2)-1, sqrt(2)-1]: the stated coefficients must
+    # reproduce that function (an independent check of the table, in fp64)
+    bits = [0x3EAAAAA9, 0xBE800064, 0x3E4CD0A6, 0xBE2A6AA7, 0x3E116E25, 0xBE04D5F2, 0x3E022C8D, 0xBDA5EB80]
+    c = np.array(bits, dtype=np.uint32).view(np.float32).astype(np.float64)
+    f = np.linspace(math.sqrt(0.5) - 1, math.sqrt(2) - 1, 2001)
+    f = f[np.abs(f) > 1e-3]
+    want = (np.log1p(f) - f + f * f / 2) / f ** 3
+    got = sum(ck * f ** k for k, ck in enumerate(c))
+    assert np.abs(got - want).max() < 3e-6          # times |f|^3 <= 0.071: below 2e-7 in ln m
+    assert abs(c[0] - 1.0 / 3.0) < 1e-7
 
 
 def test_ln_against_libm():
@@ -77,8 +84,13 @@ def test_ln_against_libm():
         got = oracle.ln_f32(u)
         want = math.log(u)
         worst = max(worst, abs(got - want) / max(abs(want), 1e-6))
-    assert worst < 4e-7, worst
+    assert worst < 2e-7, worst
     assert oracle.ln_f32(1.0) == 0.0
+    # relative accuracy right below 1, where sqrt(-2 ln u) must stay real
+    for k in range(2**24 - 64, 2**24):
+        u = k / 2.0**24
+        assert oracle.ln_f32(u) < 0.0
+        assert abs(oracle.ln_f32(u) / math.log(u) - 1.0) < 2e-7
 
 
 def test_cossin_against_libm():
