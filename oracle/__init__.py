@@ -72,6 +72,11 @@ def _declare(L):
     L.oracle_gradient.argtypes = [_f32p, _f32p, C.c_uint32, C.c_uint32, C.c_double, _f64p]
     L.oracle_adam.argtypes = [_f64p, _f64p, _f64p, _f64p, C.c_uint32, C.c_uint32,
                               C.c_double, C.c_double, C.c_double, C.c_double]
+    L.oracle_ask_sigma.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, _f32p, _f32p, _f32p, _f32p]
+    L.oracle_gradient_sigma.argtypes = [_f32p, _f32p, C.c_uint32, C.c_uint32, _f64p, _f64p]
+    L.oracle_sigma_gradient.argtypes = [_f32p, _f32p, C.c_uint32, C.c_uint32, _f64p, _f64p]
+    L.oracle_sigma_update.argtypes = [_f64p, _f64p, C.c_uint32, C.c_double, C.c_double]
+    L.oracle_clipup.argtypes = [_f64p, _f64p, _f64p, C.c_uint32, C.c_double, C.c_double, C.c_double]
     L.oracle_mlp_forward.argtypes = [_f64p, C.c_uint32, _u32p, _f64p, _f64p, C.c_double]
     L.oracle_mlp_param_count.argtypes = [C.c_uint32, _u32p]
     L.oracle_mlp_param_count.restype = C.c_uint32
@@ -178,6 +183,43 @@ def adam(center, m, v, g, t, lr, beta1=0.9, beta2=0.999, adam_eps=1e-8):
     lib().oracle_adam(_p(c, _f64p), _p(mm, _f64p), _p(vv, _f64p), _p(gg, _f64p), c.shape[0], t,
                       lr, beta1, beta2, adam_eps)
     return c, mm, vv
+
+
+def ask_sigma(seed, generation, P, D, center, sigma, want_eps=True):
+    center = _f32(center); sigma = _f32(sigma)
+    theta = np.zeros((P, D), dtype=np.float32)
+    eps = np.zeros((P // 2, D), dtype=np.float32) if want_eps else None
+    lib().oracle_ask_sigma(seed, generation, P, D, _p(center, _f32p), _p(sigma, _f32p), _p(theta, _f32p),
+                           _p(eps, _f32p) if want_eps else None)
+    return theta, eps
+
+
+def gradient_sigma(u, eps, sigma):
+    u = _f32(u); eps = _f32(eps); H, D = eps.shape
+    sg = np.ascontiguousarray(sigma, dtype=np.float64); g = np.zeros(D, dtype=np.float64)
+    lib().oracle_gradient_sigma(_p(u, _f32p), _p(eps, _f32p), 2 * H, D, _p(sg, _f64p), _p(g, _f64p))
+    return g
+
+
+def sigma_gradient(u, eps, sigma):
+    u = _f32(u); eps = _f32(eps); H, D = eps.shape
+    sg = np.ascontiguousarray(sigma, dtype=np.float64); gs = np.zeros(D, dtype=np.float64)
+    lib().oracle_sigma_gradient(_p(u, _f32p), _p(eps, _f32p), 2 * H, D, _p(sg, _f64p), _p(gs, _f64p))
+    return gs
+
+
+def sigma_update(sigma, gs, lr_sigma, max_change):
+    sg = np.array(sigma, dtype=np.float64); g = np.ascontiguousarray(gs, dtype=np.float64)
+    lib().oracle_sigma_update(_p(sg, _f64p), _p(g, _f64p), sg.shape[0], float(lr_sigma), float(max_change))
+    return sg
+
+
+def clipup(center, velocity, g, lr, momentum, max_speed):
+    c = np.array(center, dtype=np.float64); v = np.array(velocity, dtype=np.float64)
+    gg = np.ascontiguousarray(g, dtype=np.float64)
+    lib().oracle_clipup(_p(c, _f64p), _p(v, _f64p), _p(gg, _f64p), c.shape[0], float(lr), float(momentum),
+                        float(max_speed))
+    return c, v
 
 
 # ---- policies ---------------------------------------------------------------------

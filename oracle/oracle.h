@@ -89,6 +89,29 @@ void oracle_gradient(const float* u, const float* eps, uint32_t P, uint32_t D,
 void oracle_adam(double* center, double* m, double* v, const double* g, uint32_t D,
                  uint32_t t, double lr, double beta1, double beta2, double adam_eps);
 
+/* ---- solver: per-dimension sigma and its PGPE update; ClipUp -------------------------- */
+
+/* ask with a sigma vector: theta[2j][d] = fma(+sigma[d], eps, center[d]), and the mirrored member. */
+void oracle_ask_sigma(uint64_t seed, uint32_t generation, uint32_t P, uint32_t D,
+                      const float* center, const float* sigma, float* theta, float* eps);
+
+/* g[d] = (sigma[d]/P) * sum_j (u[2j]-u[2j+1]) * eps[j][d]   (eps are the standard normals) */
+void oracle_gradient_sigma(const float* u, const float* eps, uint32_t P, uint32_t D,
+                           const double* sigma, double* g);
+
+/* PGPE sigma gradient with symmetric sampling and baseline b = mean(u):
+ * gs[d] = (1/H) * sum_j ((u[2j]+u[2j+1])/2 - b) * ((sigma[d] eps[j][d])^2 - sigma[d]^2) / sigma[d] */
+void oracle_sigma_gradient(const float* u, const float* eps, uint32_t P, uint32_t D,
+                           const double* sigma, double* gs);
+
+/* sigma[d] += lr_sigma * gs[d], then clipped to [sigma_old (1 - max_change), sigma_old (1 + max_change)] */
+void oracle_sigma_update(double* sigma, const double* gs, uint32_t D, double lr_sigma, double max_change);
+
+/* ClipUp (Toklu et al. 2020), ascent: v = momentum v + lr g/|g|; if |v| > max_speed, v is scaled
+ * back to that length; center += v. */
+void oracle_clipup(double* center, double* velocity, const double* g, uint32_t D,
+                   double lr, double momentum, double max_speed);
+
 /* ---- policies ------------------------------------------------------------------- */
 
 /* MLP: sizes[0..n_layers] (n_layers weight matrices). Flat parameters per layer:
