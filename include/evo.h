@@ -51,6 +51,8 @@ enum { EVO_NOISE_STORED = 0, EVO_NOISE_REGENERATED = 1 };
 enum { EVO_POLICY_NONE = 0, EVO_POLICY_MLP = 1, EVO_POLICY_CNN_28 = 2 };
 enum { EVO_TASK_NONE = 0, EVO_TASK_CARTPOLE = 1, EVO_TASK_TANH_LINEAR = 2, EVO_TASK_SUPERVISED = 3 };
 enum { EVO_ROLLOUT_AUTO = 0, EVO_ROLLOUT_GENERIC = 1, EVO_ROLLOUT_TILED = 2 };
+enum { EVO_OPT_ADAM = 0, EVO_OPT_CLIPUP = 1 };
+enum { EVO_SIGMA_CONSTANT = 0, EVO_SIGMA_PGPE = 1 };
 
 /* indices into evo_config.task_param for EVO_TASK_CARTPOLE */
 enum { EVO_CP_CART_MASS = 0, EVO_CP_POLE_MASS = 1, EVO_CP_POLE_HALF_LENGTH = 2, EVO_CP_GRAVITY = 3,
@@ -78,6 +80,12 @@ typedef struct evo_config {
     uint32_t trace_steps;          /* leading steps recorded when evo_rollout gets d_trace      */
     uint32_t rollout_kernel;       /* EVO_ROLLOUT_*: AUTO picks the tiled kernel when one fits  */
     float    task_param[16];       /* cart-pole: EVO_CP_* ; others unused                       */
+    uint32_t optimizer;            /* EVO_OPT_*: how the centre follows the ES gradient         */
+    float    clipup_momentum;      /* ClipUp: 0 selects 0.9                                     */
+    float    clipup_max_speed;     /* ClipUp: 0 selects 2 * lr                                  */
+    uint32_t sigma_mode;           /* EVO_SIGMA_*: keep sigma, or adapt it per dimension (PGPE) */
+    float    sigma_lr;             /* PGPE sigma step size, 0 selects 0.1                       */
+    float    sigma_max_change;     /* largest relative change of sigma per tell, 0 selects 0.2  */
 } evo_config;
 
 /* Bytes of device workspace a solver with this configuration needs.  Pure host function. */
@@ -124,7 +132,14 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
  *   t += 1;  m = b1 m + (1-b1) g;  v = b2 v + (1-b2) g^2
  *   center += lr * (m/(1-b1^t)) / (sqrt(v/(1-b2^t)) + adam_eps)          (ascent)
  * eps is the noise of the matching evo_ask (read back in STORED mode, recomputed from the
- * counters in REGENERATED mode).  Advances the generation.  A NaN in d_fitness[P] skips the
+ * counters in REGENERATED mode).  sigma is kept per dimension (all equal to cfg.sigma at
+ * start): ask uses sigma[d], and the gradient above is scaled by sigma[d].
+ * optimizer = EVO_OPT_CLIPUP replaces the Adam lines by ClipUp (the optimiser the paper's PGPE
+ * reference pairs it with, Section 5): vel = momentum vel + lr g/|g|; if |vel| > max_speed it is
+ * scaled back to that length; center += vel (vel lives in the first-moment buffer).
+ * sigma_mode = EVO_SIGMA_PGPE also adapts sigma (PGPE with symmetric sampling, Section 5):
+ *   gs[d] = (sigma[d]/H) * sum_j ((u[2j] + u[2j+1])/2) * (eps[j][d]^2 - 1)
+ *   sigma[d] += sigma_lr * gs[d], limited to a relative change of +-sigma_max_change per tell.  Advances the generation.  A NaN in d_fitness[P] skips the
  * update (centre, moments, t unchanged) and raises EVO_ERR_NONFINITE at the next
  * evo_sync_status.  Errors: BAD_ORDER (no ask since the last tell), INVALID_ARG, CUDA.
  */
@@ -148,6 +163,10 @@ evo_status evo_get_moments(evo_solver* s, const float** d_m, const float** d_v);
 evo_status evo_get_gradient(evo_solver* s, const float** d_g);
 evo_status evo_get_ranks  (evo_solver* s, const int32_t** d_rank, const float** d_u);
 evo_status evo_get_eps    (evo_solver* s, const float** d_eps);
+/* sigma[ldD] (fp32) in the workspace; evo_set_sigma copies D floats from a device pointer into
+ * it, asynchronously on the solver's stream (checkpoint / resume of an adapted sigma). */
+evo_status evo_get_sigma  (evo_solver* s, const float** d_sigma);
+evo_status evo_set_sigma  (evo_solver* s, const float* d_sigma);
 
 /* Checkpoint / resume: counters are (generation, Adam step).  evo_set_state copies D floats
  * from each non-NULL device pointer into the solver (asynchronously, on the solver's stream)

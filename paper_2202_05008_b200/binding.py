@@ -34,6 +34,8 @@ class EvoConfig(C.Structure):
         ("task_kind", C.c_uint32), ("episodes", C.c_uint32), ("horizon", C.c_uint32),
         ("batch", C.c_uint32), ("trace_steps", C.c_uint32), ("rollout_kernel", C.c_uint32),
         ("task_param", C.c_float * 16),
+        ("optimizer", C.c_uint32), ("clipup_momentum", C.c_float), ("clipup_max_speed", C.c_float),
+        ("sigma_mode", C.c_uint32), ("sigma_lr", C.c_float), ("sigma_max_change", C.c_float),
     ]
 
 
@@ -69,6 +71,8 @@ def load_library():
     L.evo_get_gradient.argtypes = [vp, C.POINTER(vp)]
     L.evo_get_ranks.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
     L.evo_get_eps.argtypes = [vp, C.POINTER(vp)]
+    L.evo_get_sigma.argtypes = [vp, C.POINTER(vp)]
+    L.evo_set_sigma.argtypes = [vp, vp]
     L.evo_get_counters.argtypes = [vp, u32p, u32p]
     L.evo_set_state.argtypes = [vp, vp, vp, vp, C.c_uint32, C.c_uint32]
     L.evo_sync_status.argtypes = [vp]
@@ -80,7 +84,7 @@ def load_library():
     L.evo_version.restype = C.c_uint32
     for name in ("evo_workspace_bytes", "evo_create", "evo_ask", "evo_rollout", "evo_tell",
                  "evo_destroy", "evo_set_batch", "evo_get_center", "evo_get_moments",
-                 "evo_get_gradient", "evo_get_ranks", "evo_get_eps", "evo_get_counters",
+                 "evo_get_gradient", "evo_get_ranks", "evo_get_eps", "evo_get_sigma", "evo_set_sigma", "evo_get_counters",
                  "evo_set_state", "evo_sync_status", "evo_launch_count"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -103,6 +107,8 @@ def make_config(w: W.Workload, *, trace_steps: int = 0, rollout_kernel: int = RO
     c.trace_steps, c.rollout_kernel = trace_steps, rollout_kernel
     for i, v in enumerate(w.task_param):
         c.task_param[i] = v
+    c.optimizer, c.clipup_momentum, c.clipup_max_speed = w.optimizer, w.clipup_momentum, w.clipup_max_speed
+    c.sigma_mode, c.sigma_lr, c.sigma_max_change = w.sigma_mode, w.sigma_lr, w.sigma_max_change
     return c
 
 
@@ -214,6 +220,15 @@ class Solver:
         if not p.value:
             return None
         return self._view_f32(p.value, self.P // 2, self.ldD)[:, :self.D]
+
+    def sigma(self) -> torch.Tensor:
+        p = C.c_void_p()
+        _check(self.lib.evo_get_sigma(self._h, C.byref(p)), "evo_get_sigma")
+        return self._view_f32(p.value, 1, self.ldD)[0, :self.D]
+
+    def set_sigma(self, sigma: torch.Tensor) -> None:
+        assert sigma.dtype == torch.float32 and sigma.is_cuda and sigma.is_contiguous() and sigma.numel() == self.D
+        _check(self.lib.evo_set_sigma(self._h, sigma.data_ptr()), "evo_set_sigma")
 
     def counters(self):
         g, t = C.c_uint32(), C.c_uint32()

@@ -34,6 +34,9 @@ static evo_status check_config(const evo_config* c)
     if (c->beta1 < 0.f || c->beta1 >= 1.f || c->beta2 < 0.f || c->beta2 >= 1.f || c->adam_eps < 0.f)
         return EVO_ERR_INVALID_ARG;
     if (c->rollout_kernel > EVO_ROLLOUT_TILED) return EVO_ERR_INVALID_ARG;
+    if (c->optimizer > EVO_OPT_CLIPUP || c->sigma_mode > EVO_SIGMA_PGPE) return EVO_ERR_INVALID_ARG;
+    if (c->clipup_momentum < 0.f || c->clipup_momentum >= 1.f || c->clipup_max_speed < 0.f) return EVO_ERR_INVALID_ARG;
+    if (c->sigma_lr < 0.f || c->sigma_max_change < 0.f || c->sigma_max_change >= 1.f) return EVO_ERR_INVALID_ARG;
     switch (c->task_kind) {
         case EVO_TASK_NONE: break;
         case EVO_TASK_CARTPOLE:
@@ -75,9 +78,12 @@ static evo_status make_layout(const evo_config& c, Layout* L)
     L->m = take(row);
     L->v = take(row);
     L->g = take(row);
+    L->sigma = take(row);
     L->u = take(P * sizeof(float));
     L->rank = take(P * sizeof(int32_t));
     L->grad_partial = take(2 * row * L->grad_splits);          // fp64 partial sums
+    L->sigma_partial = take(c.sigma_mode == EVO_SIGMA_PGPE ? row * L->grad_splits : 0);
+    L->norms = take(clipup_norm_doubles(ldD) * sizeof(double));
     L->fit_partial = take(P * L->n_eb * sizeof(float));
     L->task_const = take(kTlNx * (kTlNx + kTlNa) * sizeof(float));
     size_t cnn = 0;
@@ -120,6 +126,10 @@ evo_status evo_create(const evo_config* cfg_in, void* d_workspace, size_t worksp
     if (s->cfg.beta1 == 0.f) s->cfg.beta1 = 0.9f;
     if (s->cfg.beta2 == 0.f) s->cfg.beta2 = 0.999f;
     if (s->cfg.adam_eps == 0.f) s->cfg.adam_eps = 1e-8f;
+    if (s->cfg.clipup_momentum == 0.f) s->cfg.clipup_momentum = 0.9f;
+    if (s->cfg.clipup_max_speed == 0.f) s->cfg.clipup_max_speed = 2.f * s->cfg.lr;
+    if (s->cfg.sigma_lr == 0.f) s->cfg.sigma_lr = 0.1f;
+    if (s->cfg.sigma_max_change == 0.f) s->cfg.sigma_max_change = 0.2f;
     make_layout(s->cfg, &s->lay);
     if (workspace_bytes < s->lay.total) { delete s; return EVO_ERR_WORKSPACE; }
     s->ws = static_cast<char*>(d_workspace);
@@ -135,7 +145,8 @@ evo_status evo_create(const evo_config* cfg_in, void* d_workspace, size_t worksp
     const Layout& L = s->lay;
     int n = launch_init(s->stream, reinterpret_cast<float*>(s->ws + L.center),
                         reinterpret_cast<float*>(s->ws + L.m), reinterpret_cast<float*>(s->ws + L.v),
-                        reinterpret_cast<float*>(s->ws + L.g), L.ldD,
+                        reinterpret_cast<float*>(s->ws + L.g), reinterpret_cast<float*>(s->ws + L.sigma),
+                        s->cfg.sigma, s->cfg.param_dim, L.ldD,
                         reinterpret_cast<DeviceStatus*>(s->ws + L.status));
     if (n < 0) { delete s; return EVO_ERR_CUDA; }
     s->launches += n;
@@ -153,7 +164,8 @@ evo_status evo_ask(evo_solver* s, const float** d_theta, size_t* ld_theta)
     const Layout& L = s->lay;
     float* theta = reinterpret_cast<float*>(s->ws + L.theta);
     float* eps = s->cfg.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<float*>(s->ws + L.eps) : nullptr;
-    const int n = launch_ask(s->stream, reinterpret_cast<const float*>(s->ws + L.center), s->cfg.sigma,
+    const int n = launch_ask(s->stream, reinterpret_cast<const float*>(s->ws + L.center),
+                             reinterpret_cast<const float*>(s->ws + L.sigma),
                              s->k0, s->k1, s->generation, s->cfg.pop_size / 2, s->cfg.param_dim, L.ldD,
                              theta, eps);
     if (n < 0) return EVO_ERR_CUDA;
@@ -243,12 +255,23 @@ evo_status evo_tell(evo_solver* s, const float* d_fitness)
     s->launches += n;
     const float* eps = c.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<const float*>(s->ws + L.eps)
                                                         : nullptr;
-    n = launch_gradient_adam(s->stream, u, eps, s->k0, s->k1, s->generation, c.pop_size / 2, c.param_dim,
-                             L.ldD, L.grad_splits, reinterpret_cast<double*>(s->ws + L.grad_partial),
-                             c.sigma, c.lr, c.beta1, c.beta2, c.adam_eps,
-                             reinterpret_cast<float*>(s->ws + L.center),
-                             reinterpret_cast<float*>(s->ws + L.m), reinterpret_cast<float*>(s->ws + L.v),
-                             reinterpret_cast<float*>(s->ws + L.g), status);
+    TellArgs t;
+    t.u = u; t.eps = eps;
+    t.k0 = s->k0; t.k1 = s->k1; t.generation = s->generation;
+    t.H = c.pop_size / 2; t.D = c.param_dim; t.ldD = L.ldD; t.splits = L.grad_splits;
+    t.partial = reinterpret_cast<double*>(s->ws + L.grad_partial);
+    t.sigma_partial = c.sigma_mode == EVO_SIGMA_PGPE ? reinterpret_cast<float*>(s->ws + L.sigma_partial) : nullptr;
+    t.norms = reinterpret_cast<double*>(s->ws + L.norms);
+    t.sigma_vec = reinterpret_cast<float*>(s->ws + L.sigma);
+    t.lr = c.lr; t.beta1 = c.beta1; t.beta2 = c.beta2; t.adam_eps = c.adam_eps;
+    t.optimizer = c.optimizer; t.clipup_momentum = c.clipup_momentum; t.clipup_max_speed = c.clipup_max_speed;
+    t.sigma_lr = c.sigma_lr; t.sigma_max_change = c.sigma_max_change;
+    t.center = reinterpret_cast<float*>(s->ws + L.center);
+    t.m = reinterpret_cast<float*>(s->ws + L.m);
+    t.v = reinterpret_cast<float*>(s->ws + L.v);
+    t.g = reinterpret_cast<float*>(s->ws + L.g);
+    t.status = status;
+    n = launch_gradient_update(s->stream, t);
     if (n < 0) return EVO_ERR_CUDA;
     s->launches += n;
     s->asked = false;
@@ -298,6 +321,22 @@ evo_status evo_get_eps(evo_solver* s, const float** d_eps)
     if (!s || !d_eps) return EVO_ERR_INVALID_ARG;
     *d_eps = s->cfg.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<const float*>(s->ws + s->lay.eps)
                                                    : nullptr;
+    return EVO_OK;
+}
+
+evo_status evo_get_sigma(evo_solver* s, const float** d_sigma)
+{
+    if (!s || !d_sigma) return EVO_ERR_INVALID_ARG;
+    *d_sigma = reinterpret_cast<const float*>(s->ws + s->lay.sigma);
+    return EVO_OK;
+}
+
+evo_status evo_set_sigma(evo_solver* s, const float* d_sigma)
+{
+    if (!s || !d_sigma) return EVO_ERR_INVALID_ARG;
+    const size_t bytes = static_cast<size_t>(s->cfg.param_dim) * sizeof(float);
+    if (cudaMemcpyAsync(s->ws + s->lay.sigma, d_sigma, bytes, cudaMemcpyDeviceToDevice, s->stream) != cudaSuccess)
+        return EVO_ERR_CUDA;
     return EVO_OK;
 }
 
@@ -376,6 +415,6 @@ const char* evo_status_string(evo_status st)
     return "unknown status";
 }
 
-uint32_t evo_version(void) { return 100; }
+uint32_t evo_version(void) { return 101; }
 
 }  // extern "C"

@@ -39,24 +39,36 @@ struct RolloutMlpArgs {
 };
 
 struct Layout {                  // byte offsets into the workspace
-    size_t status, center, m, v, g, theta, eps, u, rank, grad_partial, fit_partial, task_const,
-           cnn_scratch, total;
+    size_t status, center, m, v, g, sigma, theta, eps, u, rank, grad_partial, sigma_partial, norms,
+           fit_partial, task_const, cnn_scratch, total;
     uint32_t ldD, grad_splits, n_eb, EB;
 };
 
 // ---- launchers (each returns the number of kernels it launched, or -1 on a launch error) ----
-int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, uint32_t ldD,
-                DeviceStatus* status);
+int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, float* sigma_vec,
+                float sigma, uint32_t D, uint32_t ldD, DeviceStatus* status);
 int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t k1, float* task_const);
-int launch_ask(cudaStream_t st, const float* center, float sigma, uint32_t k0, uint32_t k1,
+int launch_ask(cudaStream_t st, const float* center, const float* sigma_vec, uint32_t k0, uint32_t k1,
                uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, float* theta, float* eps);
 int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank, float* u,
                 DeviceStatus* status);
-int launch_gradient_adam(cudaStream_t st, const float* u, const float* eps /*NULL = regenerate*/,
-                         uint32_t k0, uint32_t k1, uint32_t generation, uint32_t H, uint32_t D,
-                         uint32_t ldD, uint32_t splits, double* partial, float sigma, float lr,
-                         float beta1, float beta2, float adam_eps, float* center, float* m, float* v,
-                         float* g, DeviceStatus* status);
+struct TellArgs {
+    const float* u;               // centred-rank weights [P]
+    const float* eps;             // stored noise, or NULL = regenerate from the counters
+    uint32_t k0, k1, generation, H, D, ldD, splits;
+    double* partial;              // [splits][ldD] fp64 partial sums of the centre gradient
+    float*  sigma_partial;        // [splits][ldD] fp32 partial sums of the sigma gradient, or NULL
+    double* norms;                // scratch for ClipUp's two vector norms
+    float*  sigma_vec;            // [ldD]
+    float   lr, beta1, beta2, adam_eps;
+    uint32_t optimizer;
+    float   clipup_momentum, clipup_max_speed;
+    float   sigma_lr, sigma_max_change;
+    float*  center; float* m; float* v; float* g;
+    DeviceStatus* status;
+};
+int launch_gradient_update(cudaStream_t st, const TellArgs& a);
+size_t clipup_norm_doubles(uint32_t ldD);
 uint32_t gradient_splits(uint32_t H, uint32_t ldD);
 
 int  launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a, uint32_t kernel_choice,

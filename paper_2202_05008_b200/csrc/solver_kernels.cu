@@ -9,17 +9,18 @@ namespace evo {
 // ------------------------------------------------------------------------------------------
 // init / task constants
 // ------------------------------------------------------------------------------------------
-__global__ void k_init(float* center, float* m, float* v, float* g, uint32_t ldD, DeviceStatus* status)
+__global__ void k_init(float* center, float* m, float* v, float* g, float* sigma_vec, float sigma,
+                       uint32_t D, uint32_t ldD, DeviceStatus* status)
 {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < ldD) { center[i] = 0.f; m[i] = 0.f; v[i] = 0.f; g[i] = 0.f; }
+    if (i < ldD) { center[i] = 0.f; m[i] = 0.f; v[i] = 0.f; g[i] = 0.f; sigma_vec[i] = (i < D) ? sigma : 0.f; }
     if (i == 0) { status->sticky = 0; status->nonfinite = 0; status->adam_step = 0; status->pad = 0; }
 }
 
-int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, uint32_t ldD,
-                DeviceStatus* status)
+int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, float* sigma_vec,
+                float sigma, uint32_t D, uint32_t ldD, DeviceStatus* status)
 {
-    k_init<<<(ldD + 255) / 256, 256, 0, st>>>(center, m, v, g, ldD, status);
+    k_init<<<(ldD + 255) / 256, 256, 0, st>>>(center, m, v, g, sigma_vec, sigma, D, ldD, status);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
@@ -56,14 +57,14 @@ int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t 
 constexpr uint32_t kAskPairsPerThread = 8;
 
 __global__ void __launch_bounds__(256)
-k_ask(const float* __restrict__ center, float sigma, PhiloxKey key, uint32_t generation,
+k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, PhiloxKey key, uint32_t generation,
       uint32_t H, uint32_t D, uint32_t ldD, float* __restrict__ theta, float* __restrict__ eps)
 {
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
     const uint32_t d0 = quad * 4u;
     const float4 c = reinterpret_cast<const float4*>(center)[quad];
-    const float nsigma = -sigma;
+    const float4 sg = reinterpret_cast<const float4*>(sigma_vec)[quad];      // one sigma per dimension
     const bool full = d0 + 4u <= D;
     for (uint32_t j = blockIdx.y * kAskPairsPerThread; j < H; j += gridDim.y * kAskPairsPerThread) {
         const uint32_t jend = min(j + kAskPairsPerThread, H);
@@ -75,10 +76,10 @@ k_ask(const float* __restrict__ center, float sigma, PhiloxKey key, uint32_t gen
                 if (d0 + 2u >= D) z.z = 0.f;
                 if (d0 + 3u >= D) z.w = 0.f;
             }
-            const float4 tp = make_float4(__fmaf_rn(sigma, z.x, c.x), __fmaf_rn(sigma, z.y, c.y),
-                                          __fmaf_rn(sigma, z.z, c.z), __fmaf_rn(sigma, z.w, c.w));
-            const float4 tm = make_float4(__fmaf_rn(nsigma, z.x, c.x), __fmaf_rn(nsigma, z.y, c.y),
-                                          __fmaf_rn(nsigma, z.z, c.z), __fmaf_rn(nsigma, z.w, c.w));
+            const float4 tp = make_float4(__fmaf_rn(sg.x, z.x, c.x), __fmaf_rn(sg.y, z.y, c.y),
+                                          __fmaf_rn(sg.z, z.z, c.z), __fmaf_rn(sg.w, z.w, c.w));
+            const float4 tm = make_float4(__fmaf_rn(-sg.x, z.x, c.x), __fmaf_rn(-sg.y, z.y, c.y),
+                                          __fmaf_rn(-sg.z, z.z, c.z), __fmaf_rn(-sg.w, z.w, c.w));
             float* row = theta + static_cast<size_t>(2u * jj) * ldD + d0;
             __stcs(reinterpret_cast<float4*>(row), tp);
             __stcs(reinterpret_cast<float4*>(row + ldD), tm);
@@ -87,13 +88,13 @@ k_ask(const float* __restrict__ center, float sigma, PhiloxKey key, uint32_t gen
     }
 }
 
-int launch_ask(cudaStream_t st, const float* center, float sigma, uint32_t k0, uint32_t k1,
+int launch_ask(cudaStream_t st, const float* center, const float* sigma_vec, uint32_t k0, uint32_t k1,
                uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, float* theta, float* eps)
 {
     const uint32_t quads = ldD / 4u;
     dim3 grid((quads + 255u) / 256u, (H + kAskPairsPerThread - 1u) / kAskPairsPerThread);
     if (grid.y > 65535u) grid.y = 65535u;
-    k_ask<<<grid, 256, 0, st>>>(center, sigma, PhiloxKey{k0, k1}, generation, H, D, ldD, theta, eps);
+    k_ask<<<grid, 256, 0, st>>>(center, sigma_vec, PhiloxKey{k0, k1}, generation, H, D, ldD, theta, eps);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
@@ -206,11 +207,21 @@ __device__ __forceinline__ void acc_fma(Acc4& a, double wd, const float4& e)
 constexpr int kGradThreads = 256;      // threads per block of the gradient kernel
 constexpr int kGradRows = 4;           // noise rows in flight per thread (multiple of 2)
 
-template <bool REGEN>
+// SIGMA also accumulates the PGPE sigma gradient sum_j ((u[2j]+u[2j+1])/2) (eps^2 - 1) in fp32 (a plain
+// step on sigma follows, which is not ill-conditioned like Adam's normalised step).
+__device__ __forceinline__ void sig_fma(float4& a, float sj, const float4& e)
+{
+    a.x = fmaf(sj, fmaf(e.x, e.x, -1.0f), a.x);
+    a.y = fmaf(sj, fmaf(e.y, e.y, -1.0f), a.y);
+    a.z = fmaf(sj, fmaf(e.z, e.z, -1.0f), a.z);
+    a.w = fmaf(sj, fmaf(e.w, e.w, -1.0f), a.w);
+}
+
+template <bool REGEN, bool SIGMA>
 __global__ void __launch_bounds__(kGradThreads)
 k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, PhiloxKey key,
                uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, uint32_t pairs_per_split,
-               double* __restrict__ partial, const DeviceStatus* status)
+               double* __restrict__ partial, float* __restrict__ sigma_partial, const DeviceStatus* status)
 {
     if (status->nonfinite) return;
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
@@ -218,20 +229,26 @@ k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, Philo
     const uint32_t j0 = blockIdx.y * pairs_per_split;
     const uint32_t j1 = min(H, j0 + pairs_per_split);
     Acc4 acc[2] = { {0., 0., 0., 0.}, {0., 0., 0., 0.} };
+    float4 sacc[2] = { make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f) };
     const float2* up = reinterpret_cast<const float2*>(u);
     uint32_t j = j0;
     for (; j + kGradRows <= j1; j += kGradRows) {
         float4 e[kGradRows];
         double w[kGradRows];
+        float sj[kGradRows];
 #pragma unroll
         for (int i = 0; i < kGradRows; ++i) {
             if (REGEN) e[i] = stream_normal4(key, 0u, generation, j + i, quad);
             else e[i] = __ldcs(reinterpret_cast<const float4*>(eps + static_cast<size_t>(j + i) * ldD) + quad);
             const float2 uu = __ldg(up + j + i);
             w[i] = static_cast<double>(uu.x) - static_cast<double>(uu.y);   // exact
+            sj[i] = 0.5f * (uu.x + uu.y);
         }
 #pragma unroll
-        for (int i = 0; i < kGradRows; ++i) acc_fma(acc[i & 1], w[i], e[i]);
+        for (int i = 0; i < kGradRows; ++i) {
+            acc_fma(acc[i & 1], w[i], e[i]);
+            if (SIGMA) sig_fma(sacc[i & 1], sj[i], e[i]);
+        }
     }
 #pragma unroll
     for (int i = 0; i < kGradRows - 1; ++i) {      // tail keeps the accumulator assignment j % 2
@@ -241,6 +258,7 @@ k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, Philo
             else e = __ldcs(reinterpret_cast<const float4*>(eps + static_cast<size_t>(j + i) * ldD) + quad);
             const float2 uu = __ldg(up + j + i);
             acc_fma(acc[i & 1], static_cast<double>(uu.x) - static_cast<double>(uu.y), e);
+            if (SIGMA) sig_fma(sacc[i & 1], 0.5f * (uu.x + uu.y), e);
         }
     }
     double r[4] = { acc[0].x + acc[1].x, acc[0].y + acc[1].y, acc[0].z + acc[1].z, acc[0].w + acc[1].w };
@@ -252,50 +270,159 @@ k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, Philo
     double2* out = reinterpret_cast<double2*>(partial + static_cast<size_t>(blockIdx.y) * ldD) + 2u * quad;
     out[0] = make_double2(r[0], r[1]);
     out[1] = make_double2(r[2], r[3]);
+    if (SIGMA) {
+        float4 sr = make_float4(sacc[0].x + sacc[1].x, sacc[0].y + sacc[1].y, sacc[0].z + sacc[1].z, sacc[0].w + sacc[1].w);
+        if (quad * 4u + 4u > D) {                  // padding columns carry no sigma signal
+            if (quad * 4u + 0u >= D) sr.x = 0.f;
+            if (quad * 4u + 1u >= D) sr.y = 0.f;
+            if (quad * 4u + 2u >= D) sr.z = 0.f;
+            if (quad * 4u + 3u >= D) sr.w = 0.f;
+        }
+        reinterpret_cast<float4*>(sigma_partial + static_cast<size_t>(blockIdx.y) * ldD)[quad] = sr;
+    }
 }
 
-// Sum the splits in order, scale, round the gradient to fp32 and take the Adam ascent step.
+// Sum the splits in order, scale by sigma[d]/P, round the gradient to fp32; then either take the
+// Adam ascent step (ADAM) or leave the step to the ClipUp kernels and emit this block's share of
+// |g|^2; finally adapt sigma if a sigma gradient was accumulated.
+template <bool ADAM>
 __global__ void __launch_bounds__(256)
-k_adam(const double* __restrict__ partial, uint32_t splits, uint32_t ldD, double scale, float lr,
-       float beta1, float beta2, float adam_eps, float* __restrict__ center, float* __restrict__ m,
-       float* __restrict__ v, float* __restrict__ g, const DeviceStatus* status)
+k_update(const double* __restrict__ partial, const float* __restrict__ sigma_partial, uint32_t splits,
+         uint32_t ldD, double inv_pop, float lr, float beta1, float beta2, float adam_eps,
+         float sigma_lr, float sigma_max_change, float inv_pairs, float* __restrict__ sigma_vec,
+         float* __restrict__ center, float* __restrict__ m, float* __restrict__ v, float* __restrict__ g,
+         double* __restrict__ norm_partial, const DeviceStatus* status)
 {
     if (status->nonfinite) return;
     __shared__ float corr[2];
-    if (threadIdx.x == 0) {
+    __shared__ double red[256];
+    if (ADAM && threadIdx.x == 0) {
         const double t = static_cast<double>(status->adam_step + 1u);
         corr[0] = static_cast<float>(1.0 / (1.0 - pow(static_cast<double>(beta1), t)));
         corr[1] = static_cast<float>(1.0 / (1.0 - pow(static_cast<double>(beta2), t)));
     }
     __syncthreads();
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool live = quad * 4u < ldD;
+    double gsq = 0.0;
+    if (live) {
+        double sum[4] = { 0., 0., 0., 0. };
+        for (uint32_t k = 0; k < splits; ++k) {
+            const double2* p = reinterpret_cast<const double2*>(partial + static_cast<size_t>(k) * ldD) + 2u * quad;
+            const double2 a = p[0], b = p[1];
+            sum[0] += a.x; sum[1] += a.y; sum[2] += b.x; sum[3] += b.y;
+        }
+        const float4 s4 = reinterpret_cast<const float4*>(sigma_vec)[quad];
+        float sg[4] = { s4.x, s4.y, s4.z, s4.w };
+        float gg[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            gg[i] = static_cast<float>(sum[i] * (static_cast<double>(sg[i]) * inv_pop));
+            gsq += static_cast<double>(gg[i]) * static_cast<double>(gg[i]);
+        }
+        reinterpret_cast<float4*>(g)[quad] = make_float4(gg[0], gg[1], gg[2], gg[3]);
+        if (ADAM) {
+            float4 c4 = reinterpret_cast<float4*>(center)[quad];
+            float4 m4 = reinterpret_cast<float4*>(m)[quad];
+            float4 v4 = reinterpret_cast<float4*>(v)[quad];
+            float cc[4] = { c4.x, c4.y, c4.z, c4.w }, mm[4] = { m4.x, m4.y, m4.z, m4.w },
+                  vv[4] = { v4.x, v4.y, v4.z, v4.w };
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                mm[i] = beta1 * mm[i] + (1.f - beta1) * gg[i];
+                vv[i] = beta2 * vv[i] + (1.f - beta2) * gg[i] * gg[i];
+                const float mhat = mm[i] * corr[0];
+                const float vhat = vv[i] * corr[1];
+                cc[i] += lr * mhat / (sqrtf(vhat) + adam_eps);
+            }
+            reinterpret_cast<float4*>(m)[quad] = make_float4(mm[0], mm[1], mm[2], mm[3]);
+            reinterpret_cast<float4*>(v)[quad] = make_float4(vv[0], vv[1], vv[2], vv[3]);
+            reinterpret_cast<float4*>(center)[quad] = make_float4(cc[0], cc[1], cc[2], cc[3]);
+        }
+        if (sigma_partial) {                            // PGPE sigma step with a relative-change limit
+            float ss[4] = { 0.f, 0.f, 0.f, 0.f };
+            for (uint32_t k = 0; k < splits; ++k) {
+                const float4 p = reinterpret_cast<const float4*>(sigma_partial + static_cast<size_t>(k) * ldD)[quad];
+                ss[0] += p.x; ss[1] += p.y; ss[2] += p.z; ss[3] += p.w;
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float gs = sg[i] * inv_pairs * ss[i];
+                const float lo = sg[i] * (1.f - sigma_max_change), hi = sg[i] * (1.f + sigma_max_change);
+                sg[i] = fminf(fmaxf(sg[i] + sigma_lr * gs, lo), hi);
+            }
+            reinterpret_cast<float4*>(sigma_vec)[quad] = make_float4(sg[0], sg[1], sg[2], sg[3]);
+        }
+    }
+    if (!ADAM) {                                        // fixed-order block sum of |g|^2
+        red[threadIdx.x] = gsq;
+        __syncthreads();
+        for (uint32_t off = 128; off > 0; off >>= 1) {
+            if (threadIdx.x < off) red[threadIdx.x] += red[threadIdx.x + off];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) norm_partial[blockIdx.x] = red[0];
+    }
+}
+
+// ClipUp, step 1: vel = momentum vel + lr g/|g| and this block's share of |vel|^2.
+// norm_partial: [0, nb) block sums of |g|^2 (in), [nb, 2nb) block sums of |vel|^2 (out).
+__global__ void __launch_bounds__(256)
+k_clipup_velocity(const float* __restrict__ g, float* __restrict__ vel, uint32_t ldD, float lr, float momentum,
+                  double* __restrict__ norm_partial, uint32_t nb, const DeviceStatus* status)
+{
+    if (status->nonfinite) return;
+    __shared__ double red[256];
+    __shared__ float inv_gnorm;
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+        for (uint32_t b = 0; b < nb; ++b) s += norm_partial[b];           // same order in every block
+        inv_gnorm = s > 0.0 ? static_cast<float>(1.0 / sqrt(s)) : 0.f;
+    }
+    __syncthreads();
+    const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
+    double vsq = 0.0;
+    if (quad * 4u < ldD) {
+        const float4 g4 = reinterpret_cast<const float4*>(g)[quad];
+        float4 v4 = reinterpret_cast<float4*>(vel)[quad];
+        const float k = lr * inv_gnorm;
+        v4.x = fmaf(momentum, v4.x, k * g4.x); v4.y = fmaf(momentum, v4.y, k * g4.y);
+        v4.z = fmaf(momentum, v4.z, k * g4.z); v4.w = fmaf(momentum, v4.w, k * g4.w);
+        reinterpret_cast<float4*>(vel)[quad] = v4;
+        vsq = static_cast<double>(v4.x) * v4.x + static_cast<double>(v4.y) * v4.y +
+              static_cast<double>(v4.z) * v4.z + static_cast<double>(v4.w) * v4.w;
+    }
+    red[threadIdx.x] = vsq;
+    __syncthreads();
+    for (uint32_t off = 128; off > 0; off >>= 1) {
+        if (threadIdx.x < off) red[threadIdx.x] += red[threadIdx.x + off];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) norm_partial[nb + blockIdx.x] = red[0];
+}
+
+// ClipUp, step 2: clip |vel| to max_speed and move the centre.
+__global__ void __launch_bounds__(256)
+k_clipup_apply(float* __restrict__ vel, float* __restrict__ center, uint32_t ldD, float max_speed,
+               const double* __restrict__ norm_partial, uint32_t nb, const DeviceStatus* status)
+{
+    if (status->nonfinite) return;
+    __shared__ float scale;
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+        for (uint32_t b = 0; b < nb; ++b) s += norm_partial[nb + b];
+        const double vn = sqrt(s);
+        scale = vn > static_cast<double>(max_speed) ? static_cast<float>(static_cast<double>(max_speed) / vn) : 1.0f;
+    }
+    __syncthreads();
+    const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
-    double sum[4] = { 0., 0., 0., 0. };
-    for (uint32_t k = 0; k < splits; ++k) {
-        const double2* p = reinterpret_cast<const double2*>(partial + static_cast<size_t>(k) * ldD) + 2u * quad;
-        const double2 a = p[0], b = p[1];
-        sum[0] += a.x; sum[1] += a.y; sum[2] += b.x; sum[3] += b.y;
-    }
-    float gg[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) gg[i] = static_cast<float>(sum[i] * scale);
+    float4 v4 = reinterpret_cast<float4*>(vel)[quad];
     float4 c4 = reinterpret_cast<float4*>(center)[quad];
-    float4 m4 = reinterpret_cast<float4*>(m)[quad];
-    float4 v4 = reinterpret_cast<float4*>(v)[quad];
-    float cc[4] = { c4.x, c4.y, c4.z, c4.w }, mm[4] = { m4.x, m4.y, m4.z, m4.w },
-          vv[4] = { v4.x, v4.y, v4.z, v4.w };
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        mm[i] = beta1 * mm[i] + (1.f - beta1) * gg[i];
-        vv[i] = beta2 * vv[i] + (1.f - beta2) * gg[i] * gg[i];
-        const float mhat = mm[i] * corr[0];
-        const float vhat = vv[i] * corr[1];
-        cc[i] += lr * mhat / (sqrtf(vhat) + adam_eps);
-    }
-    reinterpret_cast<float4*>(g)[quad] = make_float4(gg[0], gg[1], gg[2], gg[3]);
-    reinterpret_cast<float4*>(m)[quad] = make_float4(mm[0], mm[1], mm[2], mm[3]);
-    reinterpret_cast<float4*>(v)[quad] = make_float4(vv[0], vv[1], vv[2], vv[3]);
-    reinterpret_cast<float4*>(center)[quad] = make_float4(cc[0], cc[1], cc[2], cc[3]);
+    v4.x *= scale; v4.y *= scale; v4.z *= scale; v4.w *= scale;
+    c4.x += v4.x; c4.y += v4.y; c4.z += v4.z; c4.w += v4.w;
+    reinterpret_cast<float4*>(vel)[quad] = v4;
+    reinterpret_cast<float4*>(center)[quad] = c4;
 }
 
 // Closes a tell: the Adam step counter advances only if the update was applied.
@@ -321,30 +448,49 @@ uint32_t gradient_splits(uint32_t H, uint32_t ldD)
     return s;
 }
 
-int launch_gradient_adam(cudaStream_t st, const float* u, const float* eps, uint32_t k0, uint32_t k1,
-                         uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, uint32_t splits,
-                         double* partial, float sigma, float lr, float beta1, float beta2,
-                         float adam_eps, float* center, float* m, float* v, float* g,
-                         DeviceStatus* status)
+size_t clipup_norm_doubles(uint32_t ldD) { return 2u * ((ldD / 4u + 255u) / 256u); }
+
+template <bool REGEN, bool SIGMA>
+static void launch_grad(dim3 grid, cudaStream_t st, const TellArgs& a, uint32_t pps)
 {
-    const uint32_t quads = ldD / 4u;
-    const uint32_t pps = (H + splits - 1u) / splits;
-    const uint32_t used = (H + pps - 1u) / pps;        // splits that own at least one pair
+    k_grad_partial<REGEN, SIGMA><<<grid, kGradThreads, 0, st>>>(a.u, a.eps, PhiloxKey{a.k0, a.k1}, a.generation, a.H,
+                                                                a.D, a.ldD, pps, a.partial, a.sigma_partial, a.status);
+}
+
+int launch_gradient_update(cudaStream_t st, const TellArgs& a)
+{
+    const uint32_t quads = a.ldD / 4u;
+    const uint32_t pps = (a.H + a.splits - 1u) / a.splits;
+    const uint32_t used = (a.H + pps - 1u) / pps;      // splits that own at least one pair
     dim3 grid((quads + kGradThreads - 1u) / kGradThreads, used);
-    if (eps)
-        k_grad_partial<false><<<grid, kGradThreads, 0, st>>>(u, eps, PhiloxKey{k0, k1}, generation, H, D, ldD, pps,
-                                                    partial, status);
-    else
-        k_grad_partial<true><<<grid, kGradThreads, 0, st>>>(u, nullptr, PhiloxKey{k0, k1}, generation, H, D, ldD,
-                                                   pps, partial, status);
+    const bool sig = a.sigma_partial != nullptr;
+    if (a.eps) { if (sig) launch_grad<false, true>(grid, st, a, pps); else launch_grad<false, false>(grid, st, a, pps); }
+    else       { if (sig) launch_grad<true, true>(grid, st, a, pps);  else launch_grad<true, false>(grid, st, a, pps); }
     if (cudaGetLastError() != cudaSuccess) return -1;
-    const double scale = static_cast<double>(sigma) / static_cast<double>(2u * H);
-    k_adam<<<(quads + 255u) / 256u, 256, 0, st>>>(partial, used, ldD, scale, lr, beta1, beta2, adam_eps,
-                                                  center, m, v, g, status);
+    const double inv_pop = 1.0 / static_cast<double>(2u * a.H);
+    const float inv_pairs = 1.0f / static_cast<float>(a.H);
+    const uint32_t nb = (quads + 255u) / 256u;
+    int launches = 1;
+    if (a.optimizer == EVO_OPT_ADAM) {
+        k_update<true><<<nb, 256, 0, st>>>(a.partial, a.sigma_partial, used, a.ldD, inv_pop, a.lr, a.beta1, a.beta2,
+                                           a.adam_eps, a.sigma_lr, a.sigma_max_change, inv_pairs, a.sigma_vec,
+                                           a.center, a.m, a.v, a.g, a.norms, a.status);
+        if (cudaGetLastError() != cudaSuccess) return -1;
+        launches += 1;
+    } else {
+        k_update<false><<<nb, 256, 0, st>>>(a.partial, a.sigma_partial, used, a.ldD, inv_pop, a.lr, a.beta1, a.beta2,
+                                            a.adam_eps, a.sigma_lr, a.sigma_max_change, inv_pairs, a.sigma_vec,
+                                            a.center, a.m, a.v, a.g, a.norms, a.status);
+        if (cudaGetLastError() != cudaSuccess) return -1;
+        k_clipup_velocity<<<nb, 256, 0, st>>>(a.g, a.m, a.ldD, a.lr, a.clipup_momentum, a.norms, nb, a.status);
+        if (cudaGetLastError() != cudaSuccess) return -1;
+        k_clipup_apply<<<nb, 256, 0, st>>>(a.m, a.center, a.ldD, a.clipup_max_speed, a.norms, nb, a.status);
+        if (cudaGetLastError() != cudaSuccess) return -1;
+        launches += 3;
+    }
+    k_tell_finish<<<1, 1, 0, st>>>(a.status);
     if (cudaGetLastError() != cudaSuccess) return -1;
-    k_tell_finish<<<1, 1, 0, st>>>(status);
-    if (cudaGetLastError() != cudaSuccess) return -1;
-    return 3;
+    return launches + 1;
 }
 
 }  // namespace evo

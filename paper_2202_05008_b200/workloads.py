@@ -15,6 +15,8 @@ import numpy as np
 NOISE_STORED, NOISE_REGENERATED = 0, 1
 POLICY_NONE, POLICY_MLP, POLICY_CNN_28 = 0, 1, 2
 TASK_NONE, TASK_CARTPOLE, TASK_TANH_LINEAR, TASK_SUPERVISED = 0, 1, 2, 3
+OPT_ADAM, OPT_CLIPUP = 0, 1
+SIGMA_CONSTANT, SIGMA_PGPE = 0, 1
 
 CNN_PARAMS = 5994
 
@@ -38,6 +40,12 @@ class Workload:
     generations: int = 1
     # cart-pole: cart mass, pole mass, pole half length, gravity, dt, initial range
     task_param: Tuple[float, ...] = field(default_factory=tuple)
+    optimizer: int = OPT_ADAM
+    clipup_momentum: float = 0.0          # 0 = library default (0.9)
+    clipup_max_speed: float = 0.0         # 0 = library default (2 lr)
+    sigma_mode: int = SIGMA_CONSTANT
+    sigma_lr: float = 0.0                 # 0 = library default (0.1)
+    sigma_max_change: float = 0.0         # 0 = library default (0.2)
 
     @property
     def env_steps_per_generation(self) -> int:
