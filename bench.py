@@ -65,7 +65,9 @@ NCU_TRAFFIC_BYTES = {
     ("cfg2", "stored"): ("k_rollout_cartpole_ws", 4.797184e6),
     ("cfg2", "regenerated"): ("k_rollout_cartpole_ws", 4.797184e6),
     ("cfg3", "stored"): ("k_cnn_conv2_tc", 152.562176e6 + 3.476224e6),
-    ("cfg5", "stored"): ("k_ask", 32 * (3.161320e9 + 0.000144e9)),       # reduced-D capture scaled by D
+    ("cfg4", "stored"): ("k_rollout_mlp_tiled", 350.097920e6 + 4.999424e6),
+    ("cfg4", "regenerated"): ("k_rollout_mlp_tiled", 350.097920e6 + 4.999424e6),
+    ("cfg5", "stored"): ("k_ask", 32 * (3.161160e9 + 0.000273e9)),       # reduced-D capture scaled by D
 }
 
 

@@ -600,7 +600,7 @@ int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceSta
             return launch_one(k_rollout_mlp_tiled<5, 64, 64, 1, 8, 64, EVO_TASK_CARTPOLE, 1, 1, 4, 4, 1, 32>,
                               64, (2 * 5 + 64 + 64 + 1) * 8, st, a, status);
         case 2:
-            return launch_one(k_rollout_mlp_tiled<28, 128, 128, 8, 4, 128, EVO_TASK_TANH_LINEAR, 4, 4, 4, 4, 1, 16>,
+            return launch_one(k_rollout_mlp_tiled<28, 128, 128, 8, 4, 128, EVO_TASK_TANH_LINEAR, 4, 4, 8, 8, 1, 16>,
                               128, (2 * 36 + 128 + 128 + 8) * 4, st, a, status);
     }
     return -2;
