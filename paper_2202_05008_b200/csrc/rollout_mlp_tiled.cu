@@ -550,7 +550,10 @@ static const TiledShape kShapes[] = {
     { EVO_TASK_CARTPOLE, 5, 16, 16, 1, 1 },
     { EVO_TASK_CARTPOLE, 5, 64, 64, 1, 8 },
     { EVO_TASK_TANH_LINEAR, 28, 128, 128, 8, 4 },
+    { EVO_TASK_CARTPOLE, 5, 32, 32, 1, 8 },
+    { EVO_TASK_CARTPOLE, 5, 128, 128, 1, 8 },
 };
+static bool has_two_group_kernel(int shape) { return shape == 1 || shape == 3 || shape == 4; }
 
 int rollout_mlp_tiled_shape(uint32_t task, uint32_t n_layers, const uint32_t* sizes)
 {
@@ -563,11 +566,11 @@ int rollout_mlp_tiled_shape(uint32_t task, uint32_t n_layers, const uint32_t* si
     return -1;
 }
 
-// episodes per block; the 5-64-64-1 cart-pole shape switches to the warp-specialised kernel
+// episodes per block; the wider cart-pole shapes switch to the warp-specialised kernel
 // (two groups of 8) once a member has more than 8 episodes
 uint32_t rollout_mlp_tiled_eb(int shape, uint32_t episodes)
 {
-    if (shape == 1 && episodes > kShapes[1].EB) return 2u * kShapes[1].EB;
+    if (has_two_group_kernel(shape) && episodes > kShapes[shape].EB) return 2u * kShapes[shape].EB;
     return kShapes[shape].EB;
 }
 
@@ -588,9 +591,16 @@ int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceSta
 {
     const int shape = rollout_mlp_tiled_shape(a.task, a.n_layers, a.sizes);
     if (shape < 0) return -2;
-    if (shape == 1 && a.EB == 2u * kShapes[1].EB)
-        return launch_one(k_rollout_cartpole_ws<64, 64, 8, 64, 2, 1, 1, 4, 4, 1, 32>, 32 + 64 * 2,
-                          (2 * 5 + 64 + 2 * 64) * 8, st, a, status);
+    if (has_two_group_kernel(shape) && a.EB == 2u * kShapes[shape].EB) {
+        if (shape == 1)
+            return launch_one(k_rollout_cartpole_ws<64, 64, 8, 64, 2, 1, 1, 4, 4, 1, 32>, 32 + 64 * 2,
+                              (2 * 5 + 64 + 2 * 64) * 8, st, a, status);
+        if (shape == 3)
+            return launch_one(k_rollout_cartpole_ws<32, 32, 8, 32, 2, 1, 1, 4, 4, 1, 32>, 32 + 32 * 2,
+                              (2 * 5 + 32 + 2 * 32) * 8, st, a, status);
+        return launch_one(k_rollout_cartpole_ws<128, 128, 8, 128, 2, 1, 1, 4, 4, 1, 32>, 32 + 128 * 2,
+                          (2 * 5 + 128 + 2 * 128) * 8, st, a, status);
+    }
     if (a.EB != kShapes[shape].EB) return -2;
     switch (shape) {
         case 0:
@@ -602,6 +612,12 @@ int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceSta
         case 2:
             return launch_one(k_rollout_mlp_tiled<28, 128, 128, 8, 4, 128, EVO_TASK_TANH_LINEAR, 4, 4, 8, 8, 1, 16>,
                               128, (2 * 36 + 128 + 128 + 8) * 4, st, a, status);
+        case 3:
+            return launch_one(k_rollout_mlp_tiled<5, 32, 32, 1, 8, 32, EVO_TASK_CARTPOLE, 1, 1, 4, 4, 1, 32>,
+                              32, (2 * 5 + 32 + 32 + 1) * 8, st, a, status);
+        case 4:
+            return launch_one(k_rollout_mlp_tiled<5, 128, 128, 1, 8, 128, EVO_TASK_CARTPOLE, 1, 1, 4, 4, 1, 32>,
+                              128, (2 * 5 + 128 + 128 + 1) * 8, st, a, status);
     }
     return -2;
 }

@@ -1,0 +1,91 @@
+"""Edge cases of the C-ABI on a device: argument errors, minimal and odd sizes."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import rel_err, oracle_fitness
+from paper_2202_05008_b200 import Solver, EvoError, load_library, workloads as W
+from paper_2202_05008_b200.binding import make_config, ROLLOUT_TILED, ROLLOUT_GENERIC
+
+pytestmark = pytest.mark.gpu
+
+
+def test_create_rejects_small_workspace_and_unsupported_tiled_request():
+    lib = load_library()
+    cfg = make_config(W.CFG1)
+    n = C.c_size_t()
+    assert lib.evo_workspace_bytes(C.byref(cfg), C.byref(n)) == 0
+    ws = torch.empty(n.value + 256, dtype=torch.uint8, device="cuda")
+    ptr = (ws.data_ptr() + 255) // 256 * 256
+    h = C.c_void_p()
+    assert lib.evo_create(C.byref(cfg), ptr, n.value - 1, None, C.byref(h)) == 3      # workspace too small
+    assert lib.evo_create(C.byref(cfg), ptr + 4, n.value, None, C.byref(h)) == 1      # misaligned
+    # a shape without a compiled fast kernel: AUTO falls back to the generic kernel, TILED is refused at rollout
+    sizes = (5, 7, 3, 1)
+    w = W.CFG1.with_(layer_sizes=sizes, param_dim=W.mlp_param_count(sizes), horizon=10)
+    s = Solver(w, rollout_kernel=ROLLOUT_TILED)
+    s.ask()
+    with pytest.raises(EvoError) as e:
+        s.rollout()
+    assert e.value.code == 7
+    s.close()
+    torch.cuda.synchronize()
+
+
+def test_rollout_argument_errors():
+    lib = load_library()
+    s = Solver(W.CFG1.with_(horizon=10))
+    fit = torch.zeros(16, device="cuda")
+    assert lib.evo_rollout(s._h, None, fit.data_ptr(), None) == 2                     # no ask yet
+    s.ask()
+    assert lib.evo_rollout(s._h, None, None, None) == 1                               # no fitness buffer
+    theta = s.padded_rows(17)
+    assert lib.evo_rollout(s._h, theta.data_ptr() + 4, fit.data_ptr(), None) == 1     # misaligned matrix
+    trace = torch.zeros(16 * 10 * 4, device="cuda")
+    assert lib.evo_rollout(s._h, None, fit.data_ptr(), trace.data_ptr()) == 1         # trace_steps is 0
+    assert lib.evo_rollout(s._h, None, fit.data_ptr(), None) == 0
+    assert s.sync_status() == 0
+    s.close()
+
+
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_TILED])
+def test_smallest_population_single_step_single_episode(kernel):
+    w = W.CFG1.with_(pop_size=2, horizon=1, episodes=1)
+    s = Solver(w, trace_steps=1, rollout_kernel=kernel)
+    th = s.ask().cpu().numpy()
+    trace = torch.zeros(2, 1, 1, 4, device="cuda")
+    fit = s.rollout(trace=trace).cpu().numpy()
+    fit_o, tr_o = oracle_fitness(w, th, 0, 1, want_trace=True)
+    assert rel_err(fit, fit_o, floor=1.0) < 1e-3
+    assert np.abs(trace.cpu().numpy()[0, 0, 0] - tr_o[0][0, 0]).max() < 1e-5
+    s.tell(torch.tensor(fit, device="cuda"))
+    rank, u = (x.cpu().numpy() for x in s.ranks())
+    assert sorted(rank.tolist()) == [0, 1] and sorted(u.tolist()) == [-0.5, 0.5]
+    assert s.sync_status() == 0
+    s.close()
+
+
+def test_many_episodes_on_the_small_network():
+    w = W.CFG1.with_(episodes=100, horizon=20, pop_size=4)
+    s = Solver(w)
+    th = s.ask().cpu().numpy()
+    fit = s.rollout().cpu().numpy()
+    fit_o, _ = oracle_fitness(w, th, 0, 20)
+    assert rel_err(fit, fit_o, floor=1.0) < 1e-3
+    s.close()
+
+
+def test_cnn_single_image_batch():
+    w = W.CFG3.with_(pop_size=2, batch=1)
+    s = Solver(w)
+    images, labels = W.image_batch(w.seed, 0, 1)
+    s.set_batch(torch.tensor(images, device="cuda"), torch.tensor(labels, device="cuda"))
+    th = W.random_parameters(9, 2, W.CNN_PARAMS, scale=0.1)
+    arg = s.padded_rows(2); arg[:, :W.CNN_PARAMS] = torch.tensor(th, device="cuda")
+    fit = s.rollout(arg).cpu().numpy()
+    want = np.array([oracle.cnn_fitness(th[m], images, labels, True) for m in range(2)])
+    assert rel_err(fit, want, floor=1.0) < 1e-3 and s.sync_status() == 0
+    s.close()

@@ -103,6 +103,15 @@ def test_cfg2_shape_tiled_variants_and_ragged_episode_counts(episodes):
     _rollout_check(w, 60, list(range(6)), ROLLOUT_TILED, theta_np=theta)
 
 
+@pytest.mark.parametrize("hidden", [32, 128])
+@pytest.mark.parametrize("episodes", [3, 16, 21])
+def test_other_cartpole_widths_have_fast_kernels(hidden, episodes):
+    sizes = (5, hidden, hidden, 1)
+    w = W.CFG2.with_(pop_size=6, episodes=episodes, layer_sizes=sizes, param_dim=W.mlp_param_count(sizes))
+    theta = W.random_parameters(hidden, 6, w.param_dim, scale=0.25)
+    _rollout_check(w, 60, list(range(6)), ROLLOUT_TILED, theta_np=theta)
+
+
 def test_cfg1_shape_with_several_episodes():
     w = W.CFG1.with_(episodes=3)
     _rollout_check(w, 80, list(range(16)), ROLLOUT_TILED)
