@@ -22,6 +22,7 @@
 // on expiry the block records EVO_ERR_TIMEOUT, frees its TMEM and leaves.
 // Paper: Section 3 (supervised tasks are single-step tasks; ConvNet on 28x28 images).
 #include "internal.h"
+#include "async.cuh"
 #include <cuda_bf16.h>
 
 namespace evo {
@@ -29,11 +30,6 @@ namespace evo {
 // ------------------------------------------------------------------------------------------
 // PTX wrappers
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p)
-{
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
 // K-major operand without swizzle: 8-row x 16-byte core matrices; lbo = bytes between the core
 // matrices adjacent in K, sbo = bytes between 8-row groups adjacent in M (or N).
 __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
@@ -77,7 +73,6 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // 32 lanes x 16 consecutive 32-bit columns: thread = lane, r[i] = column i
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* r)
@@ -93,43 +88,10 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* r)
     for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(u[i]);
 }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
-}
-// Bounded wait.  try_wait is given a suspend-time hint, so a waiting warp sleeps in hardware
-// instead of taking issue slots from the warps that work; the loop re-arms it until the phase
-// completes or ~2^max_cycles_log2 SM clocks have passed.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t max_cycles_log2)
-{
-    uint32_t done;
-    asm volatile("{\n\t.reg .pred p;\n\t"
-                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                 "selp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    if (done) return true;
-    const long long t0 = clock64();
-    const long long limit = 1ll << max_cycles_log2;
-    for (;;) {
-        asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-                     "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(parity), "r"(20000u) : "memory");     // hint: 20 us
-        if (done) return true;
-        if (clock64() - t0 > limit) return false;
-    }
-}
-constexpr uint32_t kWaitIters = 31;        // log2 of the cycle budget of a wait: ~1 s
-
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
 }
 
 // Wait that cannot hang: after one time-out anywhere in the block every later wait returns at
@@ -138,7 +100,7 @@ __device__ __forceinline__ void wait_or_abort(volatile int* abort_flag, uint64_t
                                               DeviceStatus* status)
 {
     if (*abort_flag) return;
-    if (!mbar_wait_bounded(smem_u32(bar), parity, kWaitIters)) {
+    if (!mbar_wait_bounded(smem_u32(bar), parity, kWaitCyclesLog2)) {
         *abort_flag = 1;
         atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
     }
@@ -286,7 +248,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             mbar_init(smem_u32(&ctl.acc_free[i]), kC1EpiThreads / 32);
         }
         ctl.abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_init_fence();
     }
     __syncwarp();
     if (warp == 0) tmem_alloc(smem_u32(&ctl.tmem_slot), 512);
@@ -442,10 +404,7 @@ __device__ __forceinline__ void c2_wait(C2Smem& S, uint64_t* bar, uint32_t parit
 
 __device__ __forceinline__ void c2_load_pair(C2Smem& S, int buf, const unsigned char* src)
 {
-    const uint32_t bar = smem_u32(&S.full[buf]);
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(kPairBytes) : "memory");
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(smem_u32(S.a[buf])), "l"(src), "r"(kPairBytes), "r"(bar) : "memory");
+    bulk_copy_g2s(smem_u32(S.a[buf]), src, kPairBytes, smem_u32(&S.full[buf]));
 }
 
 // 13 MMAs (K = 16 each = two 5x5 taps x 8 channels) of one image pair into one accumulator.
@@ -482,7 +441,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&S.mma_done[i]), 1); mbar_init(smem_u32(&S.acc_free[i]), 4); }
         mbar_init(smem_u32(&S.item_ready), 1);
         S.abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_init_fence();
     }
     for (int k = tid; k < 256; k += kC2Threads) { S.wfT[k * 12 + 10] = 0.f; S.wfT[k * 12 + 11] = 0.f; }
     if (tid < 2) S.bfc[10 + tid] = 0.f;

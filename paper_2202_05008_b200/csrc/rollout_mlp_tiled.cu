@@ -15,6 +15,7 @@
 // Paper: Section 2 (roll-out loop, central seeds), Section 4 (get_actions over the population
 // with parameters as data; stateless task step; identical initial observations).
 #include "internal.h"
+#include "async.cuh"
 #include "noise.cuh"
 #include "tasks.cuh"
 
@@ -192,21 +193,6 @@ struct Dense {
 
 struct NoHook { __device__ __forceinline__ void operator()(int, const float*) const {} };
 
-// bounded wait on an mbarrier phase; returns false if it gave up
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t max_iter)
-{
-    for (uint32_t it = 0; it < max_iter; ++it) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                     "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
-        if (it > 64) __nanosleep(64);
-    }
-    return false;
-}
-
 template <int NIN, int H1, int H2, int NOUT, int EB, int THREADS, int TASK,
           int TI1, int S1, int TI2, int S2, int TI3, int S3>
 __global__ void __launch_bounds__(THREADS)
@@ -233,20 +219,11 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     const PhiloxKey key{ a.k0, a.k1 };
 
     // ---- parameter row: one bulk copy HBM -> shared memory ---------------------------------
-    const uint32_t bar = static_cast<uint32_t>(__cvta_generic_to_shared(&mbar));
-    const uint32_t bytes = a.ldD * 4u;
-    if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar));
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
+    const uint32_t bar = smem_u32(&mbar);
+    if (tid == 0) { mbar_init(bar, 1); mbar_init_fence(); }
     __syncthreads();
-    if (tid == 0) {
-        const float* src = a.theta + static_cast<size_t>(member) * a.ldD;
-        const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-    }
+    if (tid == 0)       // the member's whole parameter row in one bulk copy
+        bulk_copy_g2s(smem_u32(stage), a.theta + static_cast<size_t>(member) * a.ldD, a.ldD * 4u, bar);
 
     // ---- reset (overlaps the copy) -----------------------------------------------------------
     CartpoleConst cpc{};
@@ -274,11 +251,11 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     // one thread waits (bounded) and publishes the outcome, so the whole block takes one branch
     __shared__ int copy_ok;
     if (tid == 0) {
-        copy_ok = mbar_wait(bar, 0u, 1u << 22) ? 1 : 0;
+        copy_ok = mbar_wait_bounded(bar, 0u, kWaitCyclesLog2) ? 1 : 0;
         if (!copy_ok) {
             // the copy did not land in time: flag it, give it one more bounded chance, leave
             atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
-            mbar_wait(bar, 0u, 1u << 22);
+            mbar_wait_bounded(bar, 0u, kWaitCyclesLog2);
         }
     }
     __syncthreads();
@@ -415,20 +392,11 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
     const int nA = min(nE, EB), nB = nE - nA;                        // group sizes
     const PhiloxKey key{ a.k0, a.k1 };
 
-    const uint32_t bar = static_cast<uint32_t>(__cvta_generic_to_shared(&mbar));
-    const uint32_t bytes = a.ldD * 4u;
-    if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar));
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
+    const uint32_t bar = smem_u32(&mbar);
+    if (tid == 0) { mbar_init(bar, 1); mbar_init_fence(); }
     __syncthreads();
-    if (tid == 0) {
-        const float* src = a.theta + static_cast<size_t>(member) * a.ldD;
-        const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-    }
+    if (tid == 0)       // the member's whole parameter row in one bulk copy
+        bulk_copy_g2s(smem_u32(stage), a.theta + static_cast<size_t>(member) * a.ldD, a.ldD * 4u, bar);
     // seeded starts of both groups (lanes e < EB of the task warp keep the states in registers)
     const CartpoleConst cpc = cartpole_const(a.tp);
     CpState cps[2] = {};
@@ -448,10 +416,10 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
         }
     }
     if (tid == 0) {
-        copy_ok = mbar_wait(bar, 0u, 1u << 22) ? 1 : 0;
+        copy_ok = mbar_wait_bounded(bar, 0u, kWaitCyclesLog2) ? 1 : 0;
         if (!copy_ok) {
             atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
-            mbar_wait(bar, 0u, 1u << 22);
+            mbar_wait_bounded(bar, 0u, kWaitCyclesLog2);
         }
     }
     __syncthreads();
