@@ -238,7 +238,8 @@ def config_of(w, args, stored):
             "policy": "mlp " + "-".join(map(str, w.layer_sizes)) if w.layer_sizes else
                       ("cnn_28" if w.policy_kind == W.POLICY_CNN_28 else "none"),
             "episodes": w.episodes, "horizon": w.horizon, "batch": w.batch,
-            "noise": "stored" if stored else "regenerated", "parallelism": f"replicas x{args.gpus}",
+            "noise": "stored" if stored else "regenerated",
+            "parallelism": f"{'one population, pair shards' if args.sharded else 'replicas'} x{args.gpus}",
             "l2": "flushed between timed steps (256 MiB write, untimed)"}
 
 
@@ -260,9 +261,10 @@ def max_over_ranks(value_ms: float, device, world: int) -> float:
     return float(t.item())
 
 
-def whole_job_value(units_per_rank_step: float, world: int, ms_per_step: float) -> float:
-    """Aggregate throughput of all ranks (weak scaling: every rank does one full generation)."""
-    return world * units_per_rank_step / (ms_per_step * 1e-3)
+def whole_job_value(units_per_rank_step: float, world: int, ms_per_step: float, sharded: bool = False) -> float:
+    """Aggregate throughput of all ranks.  Replicas (weak scaling): every rank does one full
+    generation.  Pair shards (strong scaling): all ranks together do one generation."""
+    return (1 if sharded else world) * units_per_rank_step / (ms_per_step * 1e-3)
 
 
 # ------------------------------------------------------------------------------------------
@@ -271,7 +273,7 @@ def whole_job_value(units_per_rank_step: float, world: int, ms_per_step: float) 
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
-    from paper_2202_05008_b200 import Solver, workloads as W
+    from paper_2202_05008_b200 import Solver, sharded, workloads as W
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -284,9 +286,15 @@ def run_ours(args, w):
         dist.init_process_group("nccl", device_id=dev)
 
     stored = args.noise == "stored"
-    w_rank = w.with_(seed=rank_seed(w.seed, rank))      # independent replicas
-    s = Solver(w_rank, device=dev, noise_mode=W.NOISE_STORED if stored else W.NOISE_REGENERATED)
-    P, D = w.pop_size, w.param_dim
+    if args.sharded:                                    # one population, rank r owns a range of pairs
+        first_pair, n_pairs = sharded.shard_of(w.pop_size // 2, rank, world)
+        w_rank = w
+        s = Solver(w_rank, device=dev, noise_mode=W.NOISE_STORED if stored else W.NOISE_REGENERATED,
+                   shard_first_pair=first_pair, shard_pairs=n_pairs)
+    else:
+        w_rank = w.with_(seed=rank_seed(w.seed, rank))  # independent replicas
+        s = Solver(w_rank, device=dev, noise_mode=W.NOISE_STORED if stored else W.NOISE_REGENERATED)
+    P, D = s.P, w.param_dim                             # P = members this rank evaluates
     supervised = w.task_kind == W.TASK_SUPERVISED
     no_task = w.task_kind == W.TASK_NONE
     fitness = torch.empty(P, dtype=torch.float32, device=dev)
@@ -297,7 +305,17 @@ def run_ours(args, w):
             im, lb = W.image_batch(w_rank.seed, g, w.batch)
             batches.append((torch.tensor(im, device=dev), torch.tensor(lb, device=dev)))
     if no_task:
-        fits = [torch.tensor(W.synthetic_fitness(w_rank.seed, g, P), device=dev) for g in range(4)]
+        fits = [torch.tensor(W.synthetic_fitness(w_rank.seed, g, s.P_global), device=dev) for g in range(4)]
+        if args.sharded:
+            fits = [f[2 * first_pair:2 * (first_pair + n_pairs)].contiguous() for f in fits]
+
+    def tell(f):
+        if not args.sharded:
+            s.tell(f)
+            return
+        s.tell_begin(sharded.gather_fitness(f, world))
+        sharded.reduce_sums(*s.reduce_buffers(), world)
+        s.tell_end()
 
     def generation(i, ev=None):
         if ev: ev[0].record()
@@ -310,7 +328,7 @@ def run_ours(args, w):
         else:
             f = s.rollout(fitness=fitness)
         if ev: ev[2].record()
-        s.tell(f)
+        tell(f)
         if ev: ev[3].record()
 
     for i in range(args.warmup):
@@ -373,7 +391,7 @@ def run_ours(args, w):
             fitness.copy_(h_fits[i % 4], non_blocking=True)
         else:
             s.rollout(fitness=fitness)
-        s.tell(fitness)
+        tell(fitness)
         h_fit.copy_(fitness, non_blocking=True)
         h_center.copy_(s.center(), non_blocking=True)
         torch.cuda.current_stream().synchronize()
@@ -391,12 +409,12 @@ def run_ours(args, w):
 
     if rank == 0:
         metric, unit, units_per_gen = unit_of(w)
-        value = whole_job_value(units_per_gen, world, t_step_ms)
+        value = whole_job_value(units_per_gen, world, t_step_ms, args.sharded)
         peaks = measured_peaks()
         clocks = sampler.summary()
         sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
         max_mhz = clocks["sm_max_mhz"] or 1965
-        work = stage_work(w, stored)
+        work = stage_work(w.with_(pop_size=P) if args.sharded else w, stored)   # this rank's share
         alu_peak = sm_count * FP32_LANES_PER_SM * 2 * max_mhz * 1e6 / 1e12      # TFLOP/s fp32 FMA
         stages = {
             "ask": {"ms": t_ask, "GB/s": work["ask_bytes"] / (t_ask * 1e-3) / 1e9},
@@ -434,10 +452,10 @@ def run_ours(args, w):
                    "sample": sample}
         line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": t_step_ms, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "scaling": "strong" if args.sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": config_of(w, args, stored),
-                "generations_per_sec": world / (t_step_ms * 1e-3),
-                "e2e": {"value": whole_job_value(units_per_gen, world, e2e_ms), "unit": unit,
+                "generations_per_sec": (1 if args.sharded else world) / (t_step_ms * 1e-3),
+                "e2e": {"value": whole_job_value(units_per_gen, world, e2e_ms, args.sharded), "unit": unit,
                         "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
                 "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
                 "stages": stages, "cpu_baseline": cpu}
@@ -456,6 +474,9 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--noise", default="stored", choices=["stored", "regenerated"])
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing leg")
+    ap.add_argument("--sharded", action="store_true",
+                    help="one population split over the ranks by antithetic pairs (strong scaling) "
+                         "instead of independent replicas")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (experiments)")
     ap.add_argument("--dim", type=int, default=0, help="override the parameter count (cfg5 only)")
     args = ap.parse_args()

@@ -86,6 +86,8 @@ typedef struct evo_config {
     uint32_t sigma_mode;           /* EVO_SIGMA_*: keep sigma, or adapt it per dimension (PGPE) */
     float    sigma_lr;             /* PGPE sigma step size, 0 selects 0.1                       */
     float    sigma_max_change;     /* largest relative change of sigma per tell, 0 selects 0.2  */
+    uint32_t shard_first_pair;     /* multi-GPU: first antithetic pair this solver owns         */
+    uint32_t shard_pairs;          /* multi-GPU: pairs it owns; 0 = the whole population        */
 } evo_config;
 
 /* Bytes of device workspace a solver with this configuration needs.  Pure host function. */
@@ -139,11 +141,34 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
  * scaled back to that length; center += vel (vel lives in the first-moment buffer).
  * sigma_mode = EVO_SIGMA_PGPE also adapts sigma (PGPE with symmetric sampling, Section 5):
  *   gs[d] = (sigma[d]/H) * sum_j ((u[2j] + u[2j+1])/2) * (eps[j][d]^2 - 1)
- *   sigma[d] += sigma_lr * gs[d], limited to a relative change of +-sigma_max_change per tell.  Advances the generation.  A NaN in d_fitness[P] skips the
- * update (centre, moments, t unchanged) and raises EVO_ERR_NONFINITE at the next
- * evo_sync_status.  Errors: BAD_ORDER (no ask since the last tell), INVALID_ARG, CUDA.
+ *   sigma[d] += sigma_lr * gs[d], limited to a relative change of +-sigma_max_change per tell.
+ * Advances the generation.  A NaN in d_fitness[P] skips the update (centre, moments, sigma, t
+ * unchanged) and raises EVO_ERR_NONFINITE at the next evo_sync_status.  Not available on a
+ * sharded solver (shard_pairs > 0: EVO_ERR_UNSUPPORTED), which uses evo_tell_begin / _end.
+ * Errors: BAD_ORDER (no ask since the last tell), INVALID_ARG, UNSUPPORTED, CUDA.
  */
 evo_status evo_tell(evo_solver* s, const float* d_fitness);
+
+/*
+ * Sharded generation (paper Section 2, "Device Parallelism": the population is spread over the
+ * accelerators).  A solver created with shard_pairs > 0 owns pairs [shard_first_pair,
+ * shard_first_pair + shard_pairs) of a population of pop_size members: evo_ask returns only its
+ * 2*shard_pairs members (their noise comes from the global pair index, so no noise is ever
+ * exchanged), evo_rollout scores them into d_fitness[2*shard_pairs], and evo_tell is replaced by
+ *   evo_tell_begin(s, d_fitness_all)  d_fitness_all[pop_size] in global member order (the caller
+ *                                     all-gathers the shards' fitness): ranks all members, sums this
+ *                                     shard's pairs into the reduce buffers;
+ *   evo_get_reduce_buffers            device pointers of grad_sum[ldD] (fp64) and sigma_sum[ldD]
+ *                                     (fp32, NULL unless sigma adapts): the caller sums them over
+ *                                     the shards in place (all-reduce);
+ *   evo_tell_end(s)                   applies the optimiser step from the summed buffers.
+ * All shards end with the same centre provided the all-reduce delivers identical bits to all.
+ * A solver with shard_pairs == 0 may use the pair too (they then equal evo_tell).
+ * Errors: BAD_ORDER (begin without ask, end without begin), INVALID_ARG, CUDA.
+ */
+evo_status evo_tell_begin(evo_solver* s, const float* d_fitness_all);
+evo_status evo_get_reduce_buffers(evo_solver* s, double** d_grad_sum, float** d_sigma_sum, size_t* count);
+evo_status evo_tell_end(evo_solver* s);
 
 /* Frees the host handle.  Does not touch the workspace; does not synchronise. */
 evo_status evo_destroy(evo_solver* s);

@@ -36,6 +36,7 @@ class EvoConfig(C.Structure):
         ("task_param", C.c_float * 16),
         ("optimizer", C.c_uint32), ("clipup_momentum", C.c_float), ("clipup_max_speed", C.c_float),
         ("sigma_mode", C.c_uint32), ("sigma_lr", C.c_float), ("sigma_max_change", C.c_float),
+        ("shard_first_pair", C.c_uint32), ("shard_pairs", C.c_uint32),
     ]
 
 
@@ -64,6 +65,9 @@ def load_library():
     L.evo_ask.argtypes = [vp, C.POINTER(vp), szp]
     L.evo_rollout.argtypes = [vp, vp, vp, vp]
     L.evo_tell.argtypes = [vp, vp]
+    L.evo_tell_begin.argtypes = [vp, vp]
+    L.evo_get_reduce_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), szp]
+    L.evo_tell_end.argtypes = [vp]
     L.evo_destroy.argtypes = [vp]
     L.evo_set_batch.argtypes = [vp, vp, vp]
     L.evo_get_center.argtypes = [vp, C.POINTER(vp)]
@@ -82,7 +86,8 @@ def load_library():
     L.evo_status_string.argtypes = [C.c_int]
     L.evo_status_string.restype = C.c_char_p
     L.evo_version.restype = C.c_uint32
-    for name in ("evo_workspace_bytes", "evo_create", "evo_ask", "evo_rollout", "evo_tell",
+    for name in ("evo_workspace_bytes", "evo_create", "evo_ask", "evo_rollout", "evo_tell", "evo_tell_begin",
+                 "evo_get_reduce_buffers", "evo_tell_end",
                  "evo_destroy", "evo_set_batch", "evo_get_center", "evo_get_moments",
                  "evo_get_gradient", "evo_get_ranks", "evo_get_eps", "evo_get_sigma", "evo_set_sigma", "evo_get_counters",
                  "evo_set_state", "evo_sync_status", "evo_launch_count"):
@@ -92,7 +97,7 @@ def load_library():
 
 
 def make_config(w: W.Workload, *, trace_steps: int = 0, rollout_kernel: int = ROLLOUT_AUTO,
-                noise_mode: Optional[int] = None) -> EvoConfig:
+                noise_mode: Optional[int] = None, shard_first_pair: int = 0, shard_pairs: int = 0) -> EvoConfig:
     c = EvoConfig()
     c.struct_size = C.sizeof(EvoConfig)
     c.pop_size, c.param_dim, c.seed = w.pop_size, w.param_dim, w.seed
@@ -109,6 +114,7 @@ def make_config(w: W.Workload, *, trace_steps: int = 0, rollout_kernel: int = RO
         c.task_param[i] = v
     c.optimizer, c.clipup_momentum, c.clipup_max_speed = w.optimizer, w.clipup_momentum, w.clipup_max_speed
     c.sigma_mode, c.sigma_lr, c.sigma_max_change = w.sigma_mode, w.sigma_lr, w.sigma_max_change
+    c.shard_first_pair, c.shard_pairs = shard_first_pair, shard_pairs
     return c
 
 
@@ -138,7 +144,9 @@ class Solver:
             _check(self.lib.evo_create(C.byref(self.cfg), self._ws_ptr, self.workspace_bytes,
                                        self.stream.cuda_stream, C.byref(h)), "evo_create")
         self._h = h
-        self.P, self.D = workload.pop_size, workload.param_dim
+        # P = members this solver samples and evaluates (its shard); P_global = the population ranked
+        self.P_global = workload.pop_size
+        self.P, self.D = (2 * self.cfg.shard_pairs if self.cfg.shard_pairs else workload.pop_size), workload.param_dim
         self.ldD = (self.D + 31) // 32 * 32
         self._batch = None
 
@@ -163,8 +171,25 @@ class Solver:
         return fitness
 
     def tell(self, fitness: torch.Tensor) -> None:
-        assert fitness.dtype == torch.float32 and fitness.is_cuda and fitness.numel() == self.P
+        assert fitness.dtype == torch.float32 and fitness.is_cuda and fitness.numel() == self.P_global
         _check(self.lib.evo_tell(self._h, fitness.data_ptr()), "evo_tell")
+
+    # -- sharded tell: begin -> (caller sums the reduce buffers over the shards) -> end ------------
+    def tell_begin(self, fitness_all: torch.Tensor) -> None:
+        assert fitness_all.dtype == torch.float32 and fitness_all.is_cuda and fitness_all.numel() == self.P_global
+        _check(self.lib.evo_tell_begin(self._h, fitness_all.data_ptr()), "evo_tell_begin")
+
+    def reduce_buffers(self):
+        """(grad_sum fp64 [ldD], sigma_sum fp32 [ldD] or None): views to be summed over the shards in place."""
+        g, sg, n = C.c_void_p(), C.c_void_p(), C.c_size_t()
+        _check(self.lib.evo_get_reduce_buffers(self._h, C.byref(g), C.byref(sg), C.byref(n)), "evo_get_reduce_buffers")
+        off = g.value - self.workspace.data_ptr()
+        grad = self.workspace[off:off + n.value * 8].view(torch.float64)
+        sig = self._view_f32(sg.value, 1, n.value)[0] if sg.value else None
+        return grad, sig
+
+    def tell_end(self) -> None:
+        _check(self.lib.evo_tell_end(self._h), "evo_tell_end")
 
     def close(self) -> None:
         if getattr(self, "_h", None) is not None:
@@ -212,7 +237,7 @@ class Solver:
     def ranks(self):
         r, u = C.c_void_p(), C.c_void_p()
         _check(self.lib.evo_get_ranks(self._h, C.byref(r), C.byref(u)), "evo_get_ranks")
-        return self._view_i32(r.value, self.P), self._view_f32(u.value, 1, self.P)[0]
+        return self._view_i32(r.value, self.P_global), self._view_f32(u.value, 1, self.P_global)[0]
 
     def eps(self) -> Optional[torch.Tensor]:
         p = C.c_void_p()

@@ -16,6 +16,9 @@ struct evo_solver {
     cudaStream_t stream;
     uint32_t     generation;
     bool         asked;            // an ask without a matching tell is outstanding
+    bool         telling;          // evo_tell_begin done, evo_tell_end outstanding
+    uint32_t     local_pop;        // members this solver samples and evaluates (the shard's)
+    uint32_t     pair0;            // first global pair of the shard
     bool         ever_asked;
     const float*   d_images;
     const int32_t* d_labels;
@@ -37,6 +40,9 @@ static evo_status check_config(const evo_config* c)
     if (c->optimizer > EVO_OPT_CLIPUP || c->sigma_mode > EVO_SIGMA_PGPE) return EVO_ERR_INVALID_ARG;
     if (c->clipup_momentum < 0.f || c->clipup_momentum >= 1.f || c->clipup_max_speed < 0.f) return EVO_ERR_INVALID_ARG;
     if (c->sigma_lr < 0.f || c->sigma_max_change < 0.f || c->sigma_max_change >= 1.f) return EVO_ERR_INVALID_ARG;
+    if (c->shard_pairs > 0 &&
+        (c->shard_first_pair >= c->pop_size / 2u || c->shard_pairs > c->pop_size / 2u - c->shard_first_pair))
+        return EVO_ERR_INVALID_ARG;
     switch (c->task_kind) {
         case EVO_TASK_NONE: break;
         case EVO_TASK_CARTPOLE:
@@ -63,10 +69,12 @@ static evo_status check_config(const evo_config* c)
 
 static evo_status make_layout(const evo_config& c, Layout* L)
 {
-    const size_t P = c.pop_size, H = P / 2;
+    const size_t P = c.pop_size;                                        // global population (ranks)
+    const size_t Pl = c.shard_pairs ? 2u * c.shard_pairs : c.pop_size;   // members sampled / evaluated here
+    const size_t Hl = Pl / 2;
     const uint32_t ldD = static_cast<uint32_t>(align_up(c.param_dim, 32));
     L->ldD = ldD;
-    L->grad_splits = gradient_splits(static_cast<uint32_t>(H), ldD);
+    L->grad_splits = gradient_splits(static_cast<uint32_t>(Hl), ldD);
     L->EB = 1; L->n_eb = 1;
     if (c.task_kind == EVO_TASK_CARTPOLE || c.task_kind == EVO_TASK_TANH_LINEAR)
         rollout_mlp_plan(c, &L->EB, &L->n_eb);
@@ -83,18 +91,20 @@ static evo_status make_layout(const evo_config& c, Layout* L)
     L->rank = take(P * sizeof(int32_t));
     L->grad_partial = take(2 * row * L->grad_splits);          // fp64 partial sums
     L->sigma_partial = take(c.sigma_mode == EVO_SIGMA_PGPE ? row * L->grad_splits : 0);
+    L->grad_sum = take(2 * row);                                // fp64, summed over shards by the caller
+    L->sigma_sum = take(c.sigma_mode == EVO_SIGMA_PGPE ? row : 0);
     L->norms = take(clipup_norm_doubles(ldD) * sizeof(double));
-    L->fit_partial = take(P * L->n_eb * sizeof(float));
+    L->fit_partial = take(Pl * L->n_eb * sizeof(float));
     L->task_const = take(kTlNx * (kTlNx + kTlNa) * sizeof(float));
     size_t cnn = 0;
     if (c.task_kind == EVO_TASK_SUPERVISED) {
-        cnn = cnn_scratch_bytes(c.pop_size, c.batch);
-        const size_t tc = cnn_tc_scratch_bytes(c.pop_size, c.batch);
+        cnn = cnn_scratch_bytes(static_cast<uint32_t>(Pl), c.batch);
+        const size_t tc = cnn_tc_scratch_bytes(static_cast<uint32_t>(Pl), c.batch);
         if (tc > cnn) cnn = tc;
     }
     L->cnn_scratch = take(cnn);
-    L->theta = take(row * P);
-    L->eps = take(c.noise_mode == EVO_NOISE_STORED ? row * H : 0);
+    L->theta = take(row * Pl);
+    L->eps = take(c.noise_mode == EVO_NOISE_STORED ? row * Hl : 0);
     L->total = off;
     return EVO_OK;
 }
@@ -136,6 +146,9 @@ evo_status evo_create(const evo_config* cfg_in, void* d_workspace, size_t worksp
     s->stream = static_cast<cudaStream_t>(cuda_stream);
     s->generation = 0;
     s->asked = false;
+    s->telling = false;
+    s->local_pop = s->cfg.shard_pairs ? 2u * s->cfg.shard_pairs : s->cfg.pop_size;
+    s->pair0 = s->cfg.shard_pairs ? s->cfg.shard_first_pair : 0u;
     s->ever_asked = false;
     s->d_images = nullptr;
     s->d_labels = nullptr;
@@ -166,7 +179,7 @@ evo_status evo_ask(evo_solver* s, const float** d_theta, size_t* ld_theta)
     float* eps = s->cfg.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<float*>(s->ws + L.eps) : nullptr;
     const int n = launch_ask(s->stream, reinterpret_cast<const float*>(s->ws + L.center),
                              reinterpret_cast<const float*>(s->ws + L.sigma),
-                             s->k0, s->k1, s->generation, s->cfg.pop_size / 2, s->cfg.param_dim, L.ldD,
+                             s->k0, s->k1, s->generation, s->pair0, s->local_pop / 2, s->cfg.param_dim, L.ldD,
                              theta, eps);
     if (n < 0) return EVO_ERR_CUDA;
     s->launches += n;
@@ -204,9 +217,9 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
         if (d_trace) return EVO_ERR_UNSUPPORTED;
         // GENERIC selects the CUDA-core kernel, anything else the tensor-core path
         const int n = c.rollout_kernel == EVO_ROLLOUT_GENERIC
-            ? launch_rollout_cnn(s->stream, d_theta, L.ldD, c.pop_size, s->d_images, s->d_labels, c.batch,
+            ? launch_rollout_cnn(s->stream, d_theta, L.ldD, s->local_pop, s->d_images, s->d_labels, c.batch,
                                  s->ws + L.cnn_scratch, d_fitness)
-            : launch_rollout_cnn_tc(s->stream, d_theta, L.ldD, c.pop_size, s->d_images, s->d_labels, c.batch,
+            : launch_rollout_cnn_tc(s->stream, d_theta, L.ldD, s->local_pop, s->d_images, s->d_labels, c.batch,
                                     s->ws + L.cnn_scratch, d_fitness,
                                     reinterpret_cast<DeviceStatus*>(s->ws + L.status));
         if (n < 0) return n == -2 ? EVO_ERR_UNSUPPORTED : EVO_ERR_CUDA;
@@ -220,7 +233,7 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
     a.fit_partial = reinterpret_cast<float*>(s->ws + L.fit_partial);
     a.trace = d_trace;
     a.task_const = reinterpret_cast<const float*>(s->ws + L.task_const);
-    a.P = c.pop_size;
+    a.P = s->local_pop;
     a.ldD = L.ldD;
     a.n_layers = c.n_layers;
     a.max_width = 0;
@@ -241,24 +254,16 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
     return EVO_OK;
 }
 
-evo_status evo_tell(evo_solver* s, const float* d_fitness)
+static TellArgs tell_args(evo_solver* s)
 {
-    if (!s || !d_fitness) return EVO_ERR_INVALID_ARG;
-    if (!s->asked) return EVO_ERR_BAD_ORDER;
     const evo_config& c = s->cfg;
     const Layout& L = s->lay;
-    DeviceStatus* status = reinterpret_cast<DeviceStatus*>(s->ws + L.status);
-    float* u = reinterpret_cast<float*>(s->ws + L.u);
-    int n = launch_rank(s->stream, d_fitness, c.pop_size, reinterpret_cast<int32_t*>(s->ws + L.rank), u,
-                        status);
-    if (n < 0) return EVO_ERR_CUDA;
-    s->launches += n;
-    const float* eps = c.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<const float*>(s->ws + L.eps)
-                                                        : nullptr;
     TellArgs t;
-    t.u = u; t.eps = eps;
+    t.u = reinterpret_cast<const float*>(s->ws + L.u);
+    t.eps = c.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<const float*>(s->ws + L.eps) : nullptr;
     t.k0 = s->k0; t.k1 = s->k1; t.generation = s->generation;
-    t.H = c.pop_size / 2; t.D = c.param_dim; t.ldD = L.ldD; t.splits = L.grad_splits;
+    t.H = s->local_pop / 2; t.D = c.param_dim; t.ldD = L.ldD; t.splits = L.grad_splits;
+    t.pair0 = s->pair0; t.P = c.pop_size;
     t.partial = reinterpret_cast<double*>(s->ws + L.grad_partial);
     t.sigma_partial = c.sigma_mode == EVO_SIGMA_PGPE ? reinterpret_cast<float*>(s->ws + L.sigma_partial) : nullptr;
     t.norms = reinterpret_cast<double*>(s->ws + L.norms);
@@ -270,10 +275,67 @@ evo_status evo_tell(evo_solver* s, const float* d_fitness)
     t.m = reinterpret_cast<float*>(s->ws + L.m);
     t.v = reinterpret_cast<float*>(s->ws + L.v);
     t.g = reinterpret_cast<float*>(s->ws + L.g);
-    t.status = status;
+    t.status = reinterpret_cast<DeviceStatus*>(s->ws + L.status);
+    return t;
+}
+
+evo_status evo_tell(evo_solver* s, const float* d_fitness)
+{
+    if (!s || !d_fitness) return EVO_ERR_INVALID_ARG;
+    if (s->cfg.shard_pairs) return EVO_ERR_UNSUPPORTED;        // a shard needs the exchange in between
+    if (!s->asked || s->telling) return EVO_ERR_BAD_ORDER;
+    const Layout& L = s->lay;
+    const TellArgs t = tell_args(s);
+    int n = launch_rank(s->stream, d_fitness, s->cfg.pop_size, reinterpret_cast<int32_t*>(s->ws + L.rank),
+                        reinterpret_cast<float*>(s->ws + L.u), t.status);
+    if (n < 0) return EVO_ERR_CUDA;
+    s->launches += n;
     n = launch_gradient_update(s->stream, t);
     if (n < 0) return EVO_ERR_CUDA;
     s->launches += n;
+    s->asked = false;
+    s->generation += 1;
+    return EVO_OK;
+}
+
+evo_status evo_tell_begin(evo_solver* s, const float* d_fitness_all)
+{
+    if (!s || !d_fitness_all) return EVO_ERR_INVALID_ARG;
+    if (!s->asked || s->telling) return EVO_ERR_BAD_ORDER;
+    const Layout& L = s->lay;
+    const TellArgs t = tell_args(s);
+    int n = launch_rank(s->stream, d_fitness_all, s->cfg.pop_size, reinterpret_cast<int32_t*>(s->ws + L.rank),
+                        reinterpret_cast<float*>(s->ws + L.u), t.status);
+    if (n < 0) return EVO_ERR_CUDA;
+    s->launches += n;
+    n = launch_gradient_sums(s->stream, t, reinterpret_cast<double*>(s->ws + L.grad_sum),
+                             reinterpret_cast<float*>(s->ws + L.sigma_sum));
+    if (n < 0) return EVO_ERR_CUDA;
+    s->launches += n;
+    s->telling = true;
+    return EVO_OK;
+}
+
+evo_status evo_get_reduce_buffers(evo_solver* s, double** d_grad_sum, float** d_sigma_sum, size_t* count)
+{
+    if (!s || !d_grad_sum || !d_sigma_sum || !count) return EVO_ERR_INVALID_ARG;
+    *d_grad_sum = reinterpret_cast<double*>(s->ws + s->lay.grad_sum);
+    *d_sigma_sum = s->cfg.sigma_mode == EVO_SIGMA_PGPE ? reinterpret_cast<float*>(s->ws + s->lay.sigma_sum) : nullptr;
+    *count = s->lay.ldD;
+    return EVO_OK;
+}
+
+evo_status evo_tell_end(evo_solver* s)
+{
+    if (!s) return EVO_ERR_INVALID_ARG;
+    if (!s->telling) return EVO_ERR_BAD_ORDER;
+    const Layout& L = s->lay;
+    const TellArgs t = tell_args(s);
+    const int n = launch_update_from_sums(s->stream, t, reinterpret_cast<const double*>(s->ws + L.grad_sum),
+                                          reinterpret_cast<const float*>(s->ws + L.sigma_sum));
+    if (n < 0) return EVO_ERR_CUDA;
+    s->launches += n;
+    s->telling = false;
     s->asked = false;
     s->generation += 1;
     return EVO_OK;
@@ -370,6 +432,7 @@ evo_status evo_set_state(evo_solver* s, const float* d_center, const float* d_m,
     if (cudaStreamSynchronize(s->stream) != cudaSuccess) return EVO_ERR_CUDA;   // adam_step is a stack value
     s->generation = generation;
     s->asked = false;
+    s->telling = false;
     return EVO_OK;
 }
 
@@ -415,6 +478,6 @@ const char* evo_status_string(evo_status st)
     return "unknown status";
 }
 
-uint32_t evo_version(void) { return 101; }
+uint32_t evo_version(void) { return 102; }
 
 }  // extern "C"

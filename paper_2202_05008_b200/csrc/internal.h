@@ -39,7 +39,8 @@ struct RolloutMlpArgs {
 };
 
 struct Layout {                  // byte offsets into the workspace
-    size_t status, center, m, v, g, sigma, theta, eps, u, rank, grad_partial, sigma_partial, norms,
+    size_t status, center, m, v, g, sigma, theta, eps, u, rank, grad_partial, sigma_partial, grad_sum,
+           sigma_sum, norms,
            fit_partial, task_const, cnn_scratch, total;
     uint32_t ldD, grad_splits, n_eb, EB;
 };
@@ -49,13 +50,15 @@ int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, fl
                 float sigma, uint32_t D, uint32_t ldD, DeviceStatus* status);
 int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t k1, float* task_const);
 int launch_ask(cudaStream_t st, const float* center, const float* sigma_vec, uint32_t k0, uint32_t k1,
-               uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, float* theta, float* eps);
+               uint32_t generation, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* theta,
+               float* eps);
 int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank, float* u,
                 DeviceStatus* status);
 struct TellArgs {
     const float* u;               // centred-rank weights [P]
     const float* eps;             // stored noise, or NULL = regenerate from the counters
-    uint32_t k0, k1, generation, H, D, ldD, splits;
+    uint32_t k0, k1, generation, H, D, ldD, splits;   // H = pairs summed here (the shard's)
+    uint32_t pair0, P;            // first global pair of the shard; global population size
     double* partial;              // [splits][ldD] fp64 partial sums of the centre gradient
     float*  sigma_partial;        // [splits][ldD] fp32 partial sums of the sigma gradient, or NULL
     double* norms;                // scratch for ClipUp's two vector norms
@@ -68,6 +71,9 @@ struct TellArgs {
     DeviceStatus* status;
 };
 int launch_gradient_update(cudaStream_t st, const TellArgs& a);
+// the two halves of the sharded tell: partial sums -> reduce buffers; reduce buffers -> update
+int launch_gradient_sums(cudaStream_t st, const TellArgs& a, double* grad_sum, float* sigma_sum);
+int launch_update_from_sums(cudaStream_t st, const TellArgs& a, const double* grad_sum, const float* sigma_sum);
 size_t clipup_norm_doubles(uint32_t ldD);
 uint32_t gradient_splits(uint32_t H, uint32_t ldD);
 

@@ -58,7 +58,7 @@ constexpr uint32_t kAskPairsPerThread = 8;
 
 __global__ void __launch_bounds__(256)
 k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, PhiloxKey key, uint32_t generation,
-      uint32_t H, uint32_t D, uint32_t ldD, float* __restrict__ theta, float* __restrict__ eps)
+      uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* __restrict__ theta, float* __restrict__ eps)
 {
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
@@ -69,7 +69,7 @@ k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, Phi
     for (uint32_t j = blockIdx.y * kAskPairsPerThread; j < H; j += gridDim.y * kAskPairsPerThread) {
         const uint32_t jend = min(j + kAskPairsPerThread, H);
         for (uint32_t jj = j; jj < jend; ++jj) {
-            float4 z = stream_normal4(key, 0u, generation, jj, quad);
+            float4 z = stream_normal4(key, 0u, generation, pair0 + jj, quad);   // counters use the global pair
             if (!full) {                       // ragged tail and padding columns carry zeros
                 if (d0 + 0u >= D) z.x = 0.f;
                 if (d0 + 1u >= D) z.y = 0.f;
@@ -89,12 +89,13 @@ k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, Phi
 }
 
 int launch_ask(cudaStream_t st, const float* center, const float* sigma_vec, uint32_t k0, uint32_t k1,
-               uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, float* theta, float* eps)
+               uint32_t generation, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* theta,
+               float* eps)
 {
     const uint32_t quads = ldD / 4u;
     dim3 grid((quads + 255u) / 256u, (H + kAskPairsPerThread - 1u) / kAskPairsPerThread);
     if (grid.y > 65535u) grid.y = 65535u;
-    k_ask<<<grid, 256, 0, st>>>(center, sigma_vec, PhiloxKey{k0, k1}, generation, H, D, ldD, theta, eps);
+    k_ask<<<grid, 256, 0, st>>>(center, sigma_vec, PhiloxKey{k0, k1}, generation, pair0, H, D, ldD, theta, eps);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
@@ -220,8 +221,9 @@ __device__ __forceinline__ void sig_fma(float4& a, float sj, const float4& e)
 template <bool REGEN, bool SIGMA>
 __global__ void __launch_bounds__(kGradThreads)
 k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, PhiloxKey key,
-               uint32_t generation, uint32_t H, uint32_t D, uint32_t ldD, uint32_t pairs_per_split,
-               double* __restrict__ partial, float* __restrict__ sigma_partial, const DeviceStatus* status)
+               uint32_t generation, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD,
+               uint32_t pairs_per_split, double* __restrict__ partial, float* __restrict__ sigma_partial,
+               const DeviceStatus* status)
 {
     if (status->nonfinite) return;
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
@@ -230,7 +232,7 @@ k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, Philo
     const uint32_t j1 = min(H, j0 + pairs_per_split);
     Acc4 acc[2] = { {0., 0., 0., 0.}, {0., 0., 0., 0.} };
     float4 sacc[2] = { make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f) };
-    const float2* up = reinterpret_cast<const float2*>(u);
+    const float2* up = reinterpret_cast<const float2*>(u) + pair0;    // u is global, eps rows are the shard's
     uint32_t j = j0;
     for (; j + kGradRows <= j1; j += kGradRows) {
         float4 e[kGradRows];
@@ -238,7 +240,7 @@ k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, Philo
         float sj[kGradRows];
 #pragma unroll
         for (int i = 0; i < kGradRows; ++i) {
-            if (REGEN) e[i] = stream_normal4(key, 0u, generation, j + i, quad);
+            if (REGEN) e[i] = stream_normal4(key, 0u, generation, pair0 + j + i, quad);
             else e[i] = __ldcs(reinterpret_cast<const float4*>(eps + static_cast<size_t>(j + i) * ldD) + quad);
             const float2 uu = __ldg(up + j + i);
             w[i] = static_cast<double>(uu.x) - static_cast<double>(uu.y);   // exact
@@ -254,7 +256,7 @@ k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, Philo
     for (int i = 0; i < kGradRows - 1; ++i) {      // tail keeps the accumulator assignment j % 2
         if (j + i < j1) {
             float4 e;
-            if (REGEN) e = stream_normal4(key, 0u, generation, j + i, quad);
+            if (REGEN) e = stream_normal4(key, 0u, generation, pair0 + j + i, quad);
             else e = __ldcs(reinterpret_cast<const float4*>(eps + static_cast<size_t>(j + i) * ldD) + quad);
             const float2 uu = __ldg(up + j + i);
             acc_fma(acc[i & 1], static_cast<double>(uu.x) - static_cast<double>(uu.y), e);
@@ -453,11 +455,12 @@ size_t clipup_norm_doubles(uint32_t ldD) { return 2u * ((ldD / 4u + 255u) / 256u
 template <bool REGEN, bool SIGMA>
 static void launch_grad(dim3 grid, cudaStream_t st, const TellArgs& a, uint32_t pps)
 {
-    k_grad_partial<REGEN, SIGMA><<<grid, kGradThreads, 0, st>>>(a.u, a.eps, PhiloxKey{a.k0, a.k1}, a.generation, a.H,
-                                                                a.D, a.ldD, pps, a.partial, a.sigma_partial, a.status);
+    k_grad_partial<REGEN, SIGMA><<<grid, kGradThreads, 0, st>>>(a.u, a.eps, PhiloxKey{a.k0, a.k1}, a.generation, a.pair0,
+                                                                a.H, a.D, a.ldD, pps, a.partial, a.sigma_partial,
+                                                                a.status);
 }
 
-int launch_gradient_update(cudaStream_t st, const TellArgs& a)
+static int launch_partials(cudaStream_t st, const TellArgs& a, uint32_t* used_out)
 {
     const uint32_t quads = a.ldD / 4u;
     const uint32_t pps = (a.H + a.splits - 1u) / a.splits;
@@ -466,19 +469,27 @@ int launch_gradient_update(cudaStream_t st, const TellArgs& a)
     const bool sig = a.sigma_partial != nullptr;
     if (a.eps) { if (sig) launch_grad<false, true>(grid, st, a, pps); else launch_grad<false, false>(grid, st, a, pps); }
     else       { if (sig) launch_grad<true, true>(grid, st, a, pps);  else launch_grad<true, false>(grid, st, a, pps); }
-    if (cudaGetLastError() != cudaSuccess) return -1;
-    const double inv_pop = 1.0 / static_cast<double>(2u * a.H);
-    const float inv_pairs = 1.0f / static_cast<float>(a.H);
+    *used_out = used;
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+// optimiser step (and sigma step) from `splits` rows of partial sums
+static int launch_step(cudaStream_t st, const TellArgs& a, const double* partial, const float* sigma_partial,
+                       uint32_t splits)
+{
+    const uint32_t quads = a.ldD / 4u;
+    const double inv_pop = 1.0 / static_cast<double>(a.P);
+    const float inv_pairs = 2.0f / static_cast<float>(a.P);
     const uint32_t nb = (quads + 255u) / 256u;
-    int launches = 1;
+    int launches = 0;
     if (a.optimizer == EVO_OPT_ADAM) {
-        k_update<true><<<nb, 256, 0, st>>>(a.partial, a.sigma_partial, used, a.ldD, inv_pop, a.lr, a.beta1, a.beta2,
+        k_update<true><<<nb, 256, 0, st>>>(partial, sigma_partial, splits, a.ldD, inv_pop, a.lr, a.beta1, a.beta2,
                                            a.adam_eps, a.sigma_lr, a.sigma_max_change, inv_pairs, a.sigma_vec,
                                            a.center, a.m, a.v, a.g, a.norms, a.status);
         if (cudaGetLastError() != cudaSuccess) return -1;
         launches += 1;
     } else {
-        k_update<false><<<nb, 256, 0, st>>>(a.partial, a.sigma_partial, used, a.ldD, inv_pop, a.lr, a.beta1, a.beta2,
+        k_update<false><<<nb, 256, 0, st>>>(partial, sigma_partial, splits, a.ldD, inv_pop, a.lr, a.beta1, a.beta2,
                                             a.adam_eps, a.sigma_lr, a.sigma_max_change, inv_pairs, a.sigma_vec,
                                             a.center, a.m, a.v, a.g, a.norms, a.status);
         if (cudaGetLastError() != cudaSuccess) return -1;
@@ -491,6 +502,49 @@ int launch_gradient_update(cudaStream_t st, const TellArgs& a)
     k_tell_finish<<<1, 1, 0, st>>>(a.status);
     if (cudaGetLastError() != cudaSuccess) return -1;
     return launches + 1;
+}
+
+int launch_gradient_update(cudaStream_t st, const TellArgs& a)
+{
+    uint32_t used = 0;
+    const int n1 = launch_partials(st, a, &used);
+    if (n1 < 0) return -1;
+    const int n2 = launch_step(st, a, a.partial, a.sigma_partial, used);
+    return n2 < 0 ? -1 : n1 + n2;
+}
+
+// splits -> one row each, in split order (the buffers the caller sums across shards); a skipped
+// update (NaN fitness) leaves zeros so that the all-reduce still runs on defined values
+__global__ void __launch_bounds__(256)
+k_sum_splits(const double* __restrict__ partial, const float* __restrict__ sigma_partial, uint32_t splits,
+             uint32_t ldD, double* __restrict__ grad_sum, float* __restrict__ sigma_sum, const DeviceStatus* status)
+{
+    const uint32_t d = blockIdx.x * blockDim.x + threadIdx.x;
+    if (d >= ldD) return;
+    const bool skip = status->nonfinite != 0;
+    double s = 0.0;
+    float t = 0.f;
+    if (!skip) {
+        for (uint32_t k = 0; k < splits; ++k) s += partial[static_cast<size_t>(k) * ldD + d];
+        if (sigma_partial)
+            for (uint32_t k = 0; k < splits; ++k) t += sigma_partial[static_cast<size_t>(k) * ldD + d];
+    }
+    grad_sum[d] = s;
+    if (sigma_sum) sigma_sum[d] = t;
+}
+
+int launch_gradient_sums(cudaStream_t st, const TellArgs& a, double* grad_sum, float* sigma_sum)
+{
+    uint32_t used = 0;
+    if (launch_partials(st, a, &used) < 0) return -1;
+    k_sum_splits<<<(a.ldD + 255u) / 256u, 256, 0, st>>>(a.partial, a.sigma_partial, used, a.ldD, grad_sum,
+                                                        a.sigma_partial ? sigma_sum : nullptr, a.status);
+    return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
+int launch_update_from_sums(cudaStream_t st, const TellArgs& a, const double* grad_sum, const float* sigma_sum)
+{
+    return launch_step(st, a, grad_sum, a.sigma_partial ? sigma_sum : nullptr, 1u);
 }
 
 }  // namespace evo

@@ -50,3 +50,44 @@ def test_reference_arm_under_torchrun_prints_one_line_from_rank_zero():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["cpu_baseline"]["kind"] == "oracle"
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["value"] > 0
+
+
+def _exchange_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    from paper_2202_05008_b200 import sharded
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    H, D = 8, 5
+    first, n = sharded.shard_of(H, rank, world)
+    # member m has fitness 10 m; the shard holds members [2 first, 2 (first + n))
+    fit_local = torch.arange(2 * first, 2 * (first + n), dtype=torch.float32) * 10.0
+    fit_all = sharded.gather_fitness(fit_local, world)
+    grad = torch.full((D,), float(rank + 1), dtype=torch.float64)
+    sig = torch.full((D,), 0.5 * (rank + 1), dtype=torch.float32)
+    sharded.reduce_sums(grad, sig, world)
+    got = [None] * world
+    dist.all_gather_object(got, (first, n, fit_all.tolist(), grad.tolist(), sig.tolist()))
+    if rank == 0:
+        json.dump(got, open(out, "w"))
+    dist.destroy_process_group()
+
+
+def test_pair_shards_gather_fitness_in_member_order_and_sum_gradients(tmp_path):
+    out = str(tmp_path / "x.json")
+    port = 33500 + os.getpid() % 2000
+    mp.spawn(_exchange_worker, args=(2, port, out), nprocs=2, join=True)
+    r = json.load(open(out))
+    assert [(a[0], a[1]) for a in r] == [(0, 4), (4, 4)]
+    for a in r:                                            # every rank ends with the same values
+        assert a[2] == [10.0 * m for m in range(16)]
+        assert a[3] == [3.0] * 5 and a[4] == [1.5] * 5
+
+
+def test_shard_of_rejects_uneven_split():
+    sys.path.insert(0, ROOT)
+    from paper_2202_05008_b200 import sharded
+    import pytest
+    with pytest.raises(ValueError):
+        sharded.shard_of(10, 0, 4)
+    assert sharded.shard_of(12, 2, 4) == (6, 3)
