@@ -144,10 +144,29 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 # CPU oracle legs
 # ------------------------------------------------------------------------------------------
-def oracle_generation_sample(w, n_members, generation=0):
+def _oracle_member_rollout(w, generation):
+    """Returns f(row) -> fitness of one member through the oracle's rollout for this workload."""
+    import oracle
+    from paper_2202_05008_b200 import workloads as W
+    if w.task_kind == W.TASK_SUPERVISED:
+        images, labels = W.image_batch(w.seed, generation, w.batch)
+        return lambda row: oracle.cnn_fitness(row, images, labels, True)
+    if w.task_kind == W.TASK_CARTPOLE:
+        tp = w.task_param
+        p = oracle.cartpole_params(tp[0], tp[1], tp[2], tp[3], tp[4])
+        return lambda row: oracle.rollout_cartpole(row, w.layer_sizes, w.action_scale, p, tp[5], w.seed,
+                                                   generation, w.episodes, w.horizon)[0]
+    A, B = oracle.tanh_linear_constants(w.seed)
+    return lambda row: oracle.rollout_tanh_linear(row, w.layer_sizes, w.action_scale, A, B, w.seed,
+                                                  generation, w.episodes, w.horizon)[0]
+
+
+def oracle_generation_sample(w, n_members, generation=0, threads=1):
     """Times the oracle on ask + tell for the whole population (a column sample for very wide
     problems) and the rollout of n_members members; returns seconds for a full generation
-    extrapolated linearly (members and columns are independent)."""
+    extrapolated linearly (members and columns are independent).  threads > 1 spreads the
+    members' rollouts (unchanged oracle code, one member per call) over host threads; ask and
+    tell stay on one thread."""
     import oracle
     from paper_2202_05008_b200 import workloads as W
     P, D = w.pop_size, w.param_dim
@@ -161,22 +180,15 @@ def oracle_generation_sample(w, n_members, generation=0):
         full = np.zeros((n_members, D), dtype=np.float32)
         if cols == D:
             full[:] = theta[:n_members]
+        f = _oracle_member_rollout(w, generation)
         t0 = time.perf_counter()
-        if w.task_kind == W.TASK_SUPERVISED:
-            images, labels = W.image_batch(w.seed, generation, w.batch)
-            for m in range(n_members):
-                fitness[m] = oracle.cnn_fitness(full[m], images, labels, True)
-        elif w.task_kind == W.TASK_CARTPOLE:
-            tp = w.task_param
-            p = oracle.cartpole_params(tp[0], tp[1], tp[2], tp[3], tp[4])
-            for m in range(n_members):
-                fitness[m] = oracle.rollout_cartpole(full[m], w.layer_sizes, w.action_scale, p, tp[5],
-                                                     w.seed, generation, w.episodes, w.horizon)[0]
+        if threads > 1:
+            from concurrent.futures import ThreadPoolExecutor
+            with ThreadPoolExecutor(threads) as pool:      # the C oracle runs without the interpreter lock
+                fitness[:n_members] = list(pool.map(f, [full[m] for m in range(n_members)]))
         else:
-            A, B = oracle.tanh_linear_constants(w.seed)
             for m in range(n_members):
-                fitness[m] = oracle.rollout_tanh_linear(full[m], w.layer_sizes, w.action_scale, A, B,
-                                                        w.seed, generation, w.episodes, w.horizon)[0]
+                fitness[m] = f(full[m])
         t_roll = (time.perf_counter() - t0) * (P / n_members)
         n_done = n_members
     t0 = time.perf_counter()
@@ -274,6 +286,7 @@ def run_ours(args, w):
     import torch
     import torch.distributed as dist
     from paper_2202_05008_b200 import Solver, sharded, workloads as W
+    from paper_2202_05008_b200.binding import fma_probe
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -437,9 +450,12 @@ def run_ours(args, w):
                         "traffic": None}
         else:
             achieved = stages["rollout"]["TFLOP/s"]
+            fma_measured = fma_probe(dev)                 # register-only FMA chains, timed alone
             roofline = {"kernel": "k_rollout_mlp (tiled / warp-specialised)", "bound": "alu", "achieved": achieved, "peak": alu_peak,
                         "unit": "TFLOP/s", "frac": achieved / alu_peak,
                         "peak_source": f"{sm_count} SMs x 128 fp32 lanes x 2 x {max_mhz} MHz",
+                        "peak_measured": fma_measured, "frac_of_measured": achieved / fma_measured,
+                        "peak_measured_source": "evo_fma_probe (16 FMA chains per thread, best of 5 launches)",
                         "traffic": None}
         if traffic_entry is not None and (not no_task or roofline["kernel"] == traffic_entry[0]):
             roofline["traffic"] = traffic_entry[1]
@@ -450,6 +466,12 @@ def run_ours(args, w):
             t_cpu, sample = oracle_generation_sample(w, max(n, 1))
             cpu = {"value": units_per_gen / t_cpu, "unit": unit, "cores": 1, "kind": "oracle",
                    "sample": sample}
+            cores = len(os.sched_getaffinity(0))
+            if cores > 1 and not no_task:                  # same oracle, members spread over the host's cores
+                n_all = min(w.pop_size, max(n, 1) * cores)
+                t_all, sample_all = oracle_generation_sample(w, n_all, threads=cores)
+                cpu["all_cores"] = {"value": units_per_gen / t_all, "unit": unit, "cores": cores,
+                                    "sample": sample_all + f"; rollouts on {cores} threads"}
         line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": t_step_ms, "higher_is_better": True,
                 "scaling": "strong" if args.sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",

@@ -238,6 +238,19 @@ evo_status evo_es_gradient_static(const float* d_u, const float* d_eps, uint32_t
                                   uint32_t param_dim, size_t ld_eps, float sigma,
                                   float* d_gradient, void* cuda_stream);
 
+/*
+ * Measurement aid, not part of the method (the paper has no counterpart): launches
+ * blocks x threads threads that each run 16 independent chains of `iters` fp32 fused
+ * multiply-adds in registers and store one float to d_sink[blocks*threads] (device memory, caller
+ * owned).  *flops receives the floating-point operations of the launch (2 per FMA); dividing it
+ * by the launch's CUDA-event time gives the fp32 FMA rate this device really sustains, the
+ * denominator for kernels bound by plain fp32 arithmetic.  Asynchronous on cuda_stream.
+ * Errors: INVALID_ARG (NULL pointer, zero size, threads not a multiple of 32 or above 1024),
+ * CUDA (launch failed).
+ */
+evo_status evo_fma_probe(float* d_sink, uint32_t blocks, uint32_t threads, uint32_t iters,
+                         void* cuda_stream, uint64_t* flops);
+
 const char* evo_status_string(evo_status st);
 uint32_t    evo_version(void);            /* major*10000 + minor*100 + patch */
 

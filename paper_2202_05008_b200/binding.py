@@ -68,6 +68,7 @@ def load_library():
     L.evo_tell_begin.argtypes = [vp, vp]
     L.evo_get_reduce_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), szp]
     L.evo_tell_end.argtypes = [vp]
+    L.evo_fma_probe.argtypes = [vp, C.c_uint32, C.c_uint32, C.c_uint32, vp, C.POINTER(C.c_uint64)]
     L.evo_destroy.argtypes = [vp]
     L.evo_set_batch.argtypes = [vp, vp, vp]
     L.evo_get_center.argtypes = [vp, C.POINTER(vp)]
@@ -87,7 +88,7 @@ def load_library():
     L.evo_status_string.restype = C.c_char_p
     L.evo_version.restype = C.c_uint32
     for name in ("evo_workspace_bytes", "evo_create", "evo_ask", "evo_rollout", "evo_tell", "evo_tell_begin",
-                 "evo_get_reduce_buffers", "evo_tell_end",
+                 "evo_get_reduce_buffers", "evo_tell_end", "evo_fma_probe",
                  "evo_destroy", "evo_set_batch", "evo_get_center", "evo_get_moments",
                  "evo_get_gradient", "evo_get_ranks", "evo_get_eps", "evo_get_sigma", "evo_set_sigma", "evo_get_counters",
                  "evo_set_state", "evo_sync_status", "evo_launch_count"):
@@ -299,3 +300,27 @@ def es_gradient_static(u: torch.Tensor, eps: torch.Tensor, sigma: float,
         _check(lib.evo_es_gradient_static(u.data_ptr(), eps.data_ptr(), P, D, eps.stride(0), float(sigma),
                                           out.data_ptr(), st.cuda_stream), "evo_es_gradient_static")
     return out
+
+
+def fma_probe(device="cuda:0", iters: int = 1 << 14, repeats: int = 5, threads: int = 1024) -> float:
+    """Sustained fp32 FMA rate of `device` in TFLOP/s (best of `repeats` launches of
+    ``evo_fma_probe``, timed with CUDA events): the measured denominator for ALU-bound kernels."""
+    lib = load_library()
+    dev = torch.device(device)
+    with torch.cuda.device(dev):
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        blocks = sms * (2048 // threads) * 4
+        sink = torch.empty(blocks * threads, dtype=torch.float32, device=dev)
+        st = torch.cuda.current_stream(dev)
+        flops = C.c_uint64()
+        best = 0.0
+        for i in range(repeats + 2):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            _check(lib.evo_fma_probe(sink.data_ptr(), blocks, threads, iters, st.cuda_stream, C.byref(flops)),
+                   "evo_fma_probe")
+            e1.record(st)
+            e1.synchronize()
+            if i >= 2:                                   # two warm-up launches
+                best = max(best, flops.value / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+    return best

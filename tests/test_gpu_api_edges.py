@@ -89,3 +89,18 @@ def test_cnn_single_image_batch():
     want = np.array([oracle.cnn_fitness(th[m], images, labels, True) for m in range(2)])
     assert rel_err(fit, want, floor=1.0) < 1e-3 and s.sync_status() == 0
     s.close()
+
+
+def test_fma_probe_reports_a_plausible_fp32_rate_and_rejects_bad_shapes():
+    import ctypes as C
+    from paper_2202_05008_b200 import binding
+    rate = binding.fma_probe(iters=1 << 12, repeats=2)
+    assert 5.0 < rate < 200.0                          # TFLOP/s; nominal is about 74
+    lib = binding.load_library()
+    sink = torch.empty(1024, dtype=torch.float32, device="cuda")
+    flops = C.c_uint64()
+    assert lib.evo_fma_probe(sink.data_ptr(), 1, 48, 8, None, C.byref(flops)) == 1      # not a warp multiple
+    assert lib.evo_fma_probe(None, 1, 32, 8, None, C.byref(flops)) == 1
+    assert lib.evo_fma_probe(sink.data_ptr(), 1, 1024, 8, None, C.byref(flops)) == 0
+    torch.cuda.synchronize()
+    assert flops.value == 2 * 16 * 8 * 1024
