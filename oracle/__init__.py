@@ -13,7 +13,7 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = ["rng.c", "solver.c", "policy.c", "tasks.c"]
+_SRC = ["rng.c", "solver.c", "policy.c", "tasks.c", "seq2seq.c"]
 _LIB_PATH = os.path.join(_HERE, "liboracle.so")
 
 
@@ -82,6 +82,12 @@ def _declare(L):
     L.oracle_mlp_param_count.restype = C.c_uint32
     L.oracle_cnn_fitness.argtypes = [_f32p, _f32p, _i32p, C.c_uint32, C.c_int]
     L.oracle_cnn_fitness.restype = C.c_double
+    L.oracle_seq2seq_param_count.argtypes = [C.c_uint32]
+    L.oracle_seq2seq_param_count.restype = C.c_uint32
+    L.oracle_seq2seq_queries.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, _i32p, _i32p, _i32p]
+    L.oracle_seq2seq_fitness.argtypes = [_f32p, C.c_uint32, C.c_uint32, C.c_uint32, _i32p, _i32p, _i32p,
+                                         C.c_int, _f64p, _f64p]
+    L.oracle_seq2seq_fitness.restype = C.c_double
     L.oracle_cnn_logits.argtypes = [_f32p, _f32p, C.c_int, _f64p]
     L.oracle_bf16_round.argtypes = [C.c_float]; L.oracle_bf16_round.restype = C.c_float
     L.oracle_cartpole_reset.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_float, _f32p]
@@ -251,6 +257,32 @@ def cnn_logits(params, image, bf16_operands=True):
 
 
 def bf16_round(x): return float(lib().oracle_bf16_round(float(x)))
+
+
+def seq2seq_param_count(h): return int(lib().oracle_seq2seq_param_count(int(h)))
+
+
+def seq2seq_queries(seed, generation, B, nd):
+    """(encoder tokens [B][2nd+1], decoder input tokens [B][nd+1], targets [B][nd+1]), int32."""
+    enc = np.zeros((B, 2 * nd + 1), np.int32); dec = np.zeros((B, nd + 1), np.int32)
+    tgt = np.zeros((B, nd + 1), np.int32)
+    lib().oracle_seq2seq_queries(int(seed), int(generation), B, nd, _p(enc, _i32p), _p(dec, _i32p), _p(tgt, _i32p))
+    return enc, dec, tgt
+
+
+def seq2seq_fitness(params, h, nd, enc, dec, tgt, bf16_operands=True, want_logits=False):
+    """(fitness, accuracy[, logits [B][nd+1][12]]) of one member's LSTM encoder-decoder."""
+    p = _f32(params)
+    assert p.size == seq2seq_param_count(h)
+    enc = np.ascontiguousarray(enc, np.int32); dec = np.ascontiguousarray(dec, np.int32)
+    tgt = np.ascontiguousarray(tgt, np.int32)
+    B = enc.shape[0]
+    acc = np.zeros(1, np.float64)
+    logits = np.zeros((B, nd + 1, 12), np.float64) if want_logits else None
+    f = float(lib().oracle_seq2seq_fitness(_p(p, _f32p), h, nd, B, _p(enc, _i32p), _p(dec, _i32p), _p(tgt, _i32p),
+                                           int(bool(bf16_operands)), _p(acc, _f64p),
+                                           _p(logits, _f64p) if want_logits else None))
+    return (f, float(acc[0]), logits) if want_logits else (f, float(acc[0]))
 
 
 # ---- tasks ------------------------------------------------------------------------

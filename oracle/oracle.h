@@ -27,10 +27,13 @@
  * permutation and equals a sort; gradient against brute force from theta alone;
  * Adam against torch.optim.Adam; MLP against a numpy matmul; cart-pole energy and
  * momentum conservation, equilibria and small-angle period; tanh-linear recurrence
- * by hand; CNN against torch conv2d/max_pool2d/cross_entropy and the ln(10) case.
+ * by hand; CNN against torch conv2d/max_pool2d/cross_entropy and the ln(10) case; the LSTM
+ * seq2seq policy against torch.nn.LSTM + Linear + cross_entropy and the ln(12) case; its
+ * queries against integer addition.
  * Parity unpinned (conventions only, nothing external fixes them): counter/stream
  * layout of the random numbers, the sign order inside an antithetic pair, the
- * observation order, reward timing, flatten order of the CNN.
+ * observation order, reward timing, flatten order of the CNN, token codes and teacher forcing
+ * of the seq2seq task.
  */
 #ifndef ES_ORACLE_H
 #define ES_ORACLE_H
@@ -128,6 +131,18 @@ double oracle_cnn_fitness(const float* params /*5994*/, const float* images /*[B
 void oracle_cnn_logits(const float* params, const float* image /*[28][28]*/,
                        int bf16_operands, double logits[10]);
 float oracle_bf16_round(float x);
+
+/* LSTM encoder-decoder on the addition task (paper Section 3, "Seq2Seq Learning"); conventions in
+ * seq2seq.c.  Tokens: [B][2 nd + 1] encoder, [B][nd + 1] decoder inputs and targets.  Returns
+ * minus the mean cross-entropy over all answer positions; *accuracy (may be NULL) receives the
+ * fraction of positions whose arg-max token is right; logits_out (may be NULL) is [B][nd+1][12]. */
+uint32_t oracle_seq2seq_param_count(uint32_t h);
+void oracle_seq2seq_queries(uint64_t seed, uint32_t generation, uint32_t B, uint32_t nd,
+                            int32_t* enc_tokens, int32_t* dec_tokens, int32_t* targets);
+double oracle_seq2seq_fitness(const float* params, uint32_t h, uint32_t nd, uint32_t B,
+                              const int32_t* enc_tokens, const int32_t* dec_tokens,
+                              const int32_t* targets, int bf16_operands, double* accuracy,
+                              double* logits_out);
 
 /* ---- tasks ---------------------------------------------------------------------- */
 
