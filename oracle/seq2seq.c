@@ -15,9 +15,10 @@
  * Flat parameter order: enc.Wx[4h][12], enc.Wh[4h][h], enc.b[4h], dec.Wx, dec.Wh, dec.b,
  * out.W[12][h], out.b[12].
  *
- * bf16 reading: the two operands of the recurrent contraction Wh . h and of the read-out
- * out.W . h (weights and the hidden state) are rounded to bf16; everything else (the input
- * column Wx[:, token], biases, gates, cell state, softmax) is not rounded.
+ * bf16 reading: a cell's pre-activation is ONE contraction, [Wh | Wx | b] . [h; onehot(token); 1],
+ * and the read-out is another, out.W . h; the operands of both (Wh, Wx, b, out.W and the hidden
+ * state; the one-hot vector and the 1 are exact) are rounded to bf16.  The read-out bias, the
+ * gates, the cell state and the softmax are not rounded.
  */
 #include "oracle.h"
 
@@ -71,7 +72,7 @@ static void lstm_step(const float* Wx, const float* Wh, const float* b, uint32_t
         double acc = 0.0;
         for (uint32_t k = 0; k < h; ++k)
             acc += operand((double)Wh[(size_t)r * h + k], bf16) * operand(hs[k], bf16);
-        gates[r] = acc + (double)Wx[(size_t)r * VOCAB + token] + (double)b[r];
+        gates[r] = acc + operand((double)Wx[(size_t)r * VOCAB + token], bf16) + operand((double)b[r], bf16);
     }
     for (uint32_t k = 0; k < h; ++k) {
         const double ig = sigmoid(gates[k]);

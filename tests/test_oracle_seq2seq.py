@@ -44,13 +44,13 @@ def _torch_fitness(params, h, enc, dec, tgt, bf16=False):
             logits = hs @ ow.T + ob
     else:
         # step by step with LSTMCell-like algebra out of torch ops, rounding the operands of the
-        # recurrent and read-out products through torch's bfloat16
+        # cell's contraction (Wh, Wx, b, h) and of the read-out (out.W, h) through torch's bfloat16
         hcur = torch.zeros(B, h, dtype=torch.float64); c = torch.zeros(B, h, dtype=torch.float64)
         outs = []
         for phase, toks in ((0, enc), (1, dec)):
             wx, wh, b = cells[phase]
             for t in range(toks.shape[1]):
-                g = rnd(hcur) @ rnd(wh).T + wx[:, torch.tensor(toks[:, t], dtype=torch.long)].T + b
+                g = rnd(hcur) @ rnd(wh).T + rnd(wx)[:, torch.tensor(toks[:, t], dtype=torch.long)].T + rnd(b)
                 i, f, gg, og = g.split(h, dim=1)
                 c = torch.sigmoid(f) * c + torch.sigmoid(i) * torch.tanh(gg)
                 hcur = torch.sigmoid(og) * torch.tanh(c)
