@@ -48,8 +48,9 @@ typedef enum {
 } evo_status;
 
 enum { EVO_NOISE_STORED = 0, EVO_NOISE_REGENERATED = 1 };
-enum { EVO_POLICY_NONE = 0, EVO_POLICY_MLP = 1, EVO_POLICY_CNN_28 = 2 };
-enum { EVO_TASK_NONE = 0, EVO_TASK_CARTPOLE = 1, EVO_TASK_TANH_LINEAR = 2, EVO_TASK_SUPERVISED = 3 };
+enum { EVO_POLICY_NONE = 0, EVO_POLICY_MLP = 1, EVO_POLICY_CNN_28 = 2, EVO_POLICY_LSTM_SEQ2SEQ = 3 };
+enum { EVO_TASK_NONE = 0, EVO_TASK_CARTPOLE = 1, EVO_TASK_TANH_LINEAR = 2, EVO_TASK_SUPERVISED = 3,
+       EVO_TASK_SEQ2SEQ_ADD = 4 };
 enum { EVO_ROLLOUT_AUTO = 0, EVO_ROLLOUT_GENERIC = 1, EVO_ROLLOUT_TILED = 2 };
 enum { EVO_OPT_ADAM = 0, EVO_OPT_CLIPUP = 1 };
 enum { EVO_SIGMA_CONSTANT = 0, EVO_SIGMA_PGPE = 1 };
@@ -57,6 +58,9 @@ enum { EVO_SIGMA_CONSTANT = 0, EVO_SIGMA_PGPE = 1 };
 /* indices into evo_config.task_param for EVO_TASK_CARTPOLE */
 enum { EVO_CP_CART_MASS = 0, EVO_CP_POLE_MASS = 1, EVO_CP_POLE_HALF_LENGTH = 2, EVO_CP_GRAVITY = 3,
        EVO_CP_DT = 4, EVO_CP_INIT_RANGE = 5 };
+
+/* index into evo_config.task_param for EVO_TASK_SEQ2SEQ_ADD: digits per operand, 1..4 */
+enum { EVO_S2S_DIGITS = 0 };
 
 #define EVO_MAX_LAYERS 8
 
@@ -71,15 +75,15 @@ typedef struct evo_config {
     float    beta1, beta2, adam_eps;   /* 0 selects 0.9 / 0.999 / 1e-8                          */
     uint32_t policy_kind;          /* EVO_POLICY_*                                              */
     uint32_t n_layers;             /* MLP: number of weight matrices, 1..EVO_MAX_LAYERS         */
-    uint32_t layer_sizes[EVO_MAX_LAYERS + 1];  /* MLP widths, input first                       */
+    uint32_t layer_sizes[EVO_MAX_LAYERS + 1];  /* MLP widths, input first; LSTM: [0] = hidden   */
     float    action_scale;         /* MLP output = scale * tanh(.)                              */
     uint32_t task_kind;            /* EVO_TASK_*; NONE = caller computes fitness itself         */
     uint32_t episodes;             /* E >= 1 (control tasks)                                    */
     uint32_t horizon;              /* T >= 1 (control tasks)                                    */
-    uint32_t batch;                /* images per member (supervised task)                       */
+    uint32_t batch;                /* images (supervised) or queries (seq2seq) per member       */
     uint32_t trace_steps;          /* leading steps recorded when evo_rollout gets d_trace      */
     uint32_t rollout_kernel;       /* EVO_ROLLOUT_*: AUTO picks the tiled kernel when one fits  */
-    float    task_param[16];       /* cart-pole: EVO_CP_* ; others unused                       */
+    float    task_param[16];       /* cart-pole: EVO_CP_*; seq2seq: EVO_S2S_*; others unused    */
     uint32_t optimizer;            /* EVO_OPT_*: how the centre follows the ES gradient         */
     float    clipup_momentum;      /* ClipUp: 0 selects 0.9                                     */
     float    clipup_max_speed;     /* ClipUp: 0 selects 2 * lr                                  */

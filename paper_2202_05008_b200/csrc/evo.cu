@@ -62,6 +62,15 @@ static evo_status check_config(const evo_config* c)
             if (c->policy_kind != EVO_POLICY_CNN_28 || c->param_dim != kCnnParams || c->batch < 1)
                 return EVO_ERR_INVALID_ARG;
             break;
+        case EVO_TASK_SEQ2SEQ_ADD: {
+            const float nd = c->task_param[EVO_S2S_DIGITS];
+            if (c->policy_kind != EVO_POLICY_LSTM_SEQ2SEQ || !(nd >= 1.f) || nd != static_cast<float>(static_cast<uint32_t>(nd)))
+                return EVO_ERR_INVALID_ARG;
+            if (!s2s_supported(c->layer_sizes[0], static_cast<uint32_t>(nd), c->batch) ||
+                c->param_dim != s2s_param_count(c->layer_sizes[0]))
+                return EVO_ERR_INVALID_ARG;
+            break;
+        }
         default: return EVO_ERR_INVALID_ARG;
     }
     return EVO_OK;
@@ -102,7 +111,8 @@ static evo_status make_layout(const evo_config& c, Layout* L)
         const size_t tc = cnn_tc_scratch_bytes(static_cast<uint32_t>(Pl), c.batch);
         if (tc > cnn) cnn = tc;
     }
-    L->cnn_scratch = take(cnn);
+    if (c.task_kind == EVO_TASK_SEQ2SEQ_ADD) cnn = s2s_scratch_bytes(static_cast<uint32_t>(Pl), c.batch);
+    L->cnn_scratch = take(cnn);                                 // scratch of the single-step tasks
     L->theta = take(row * Pl);
     L->eps = take(c.noise_mode == EVO_NOISE_STORED ? row * Hl : 0);
     L->total = off;
@@ -227,6 +237,16 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
         return EVO_OK;
     }
     if (d_trace && c.trace_steps == 0) return EVO_ERR_INVALID_ARG;
+    if (c.task_kind == EVO_TASK_SEQ2SEQ_ADD) {
+        // d_trace, when given, receives the logits [P][batch][digits+1][12] (CUDA-core kernel)
+        const int n = launch_rollout_s2s(s->stream, d_theta, L.ldD, s->local_pop, c.layer_sizes[0],
+                                         static_cast<uint32_t>(c.task_param[EVO_S2S_DIGITS]), c.batch, s->k0, s->k1,
+                                         s->generation, c.rollout_kernel, s->ws + L.cnn_scratch, d_fitness, d_trace,
+                                         reinterpret_cast<DeviceStatus*>(s->ws + L.status));
+        if (n < 0) return n == -2 ? EVO_ERR_UNSUPPORTED : EVO_ERR_CUDA;
+        s->launches += n;
+        return EVO_OK;
+    }
     RolloutMlpArgs a;
     std::memset(&a, 0, sizeof(a));
     a.theta = d_theta;

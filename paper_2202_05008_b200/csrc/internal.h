@@ -91,4 +91,12 @@ int launch_rollout_cnn(cudaStream_t st, const float* theta, uint32_t ldD, uint32
                        const float* images, const int32_t* labels, uint32_t batch, void* scratch,
                        float* fitness);
 
+uint32_t s2s_param_count(uint32_t h);
+bool s2s_supported(uint32_t h, uint32_t nd, uint32_t B);
+size_t s2s_scratch_bytes(uint32_t P, uint32_t B);
+// logits (nullable): [P][B][nd+1][12], written by the CUDA-core kernel only
+int launch_rollout_s2s(cudaStream_t st, const float* theta, uint32_t ldD, uint32_t P, uint32_t h, uint32_t nd,
+                       uint32_t B, uint32_t k0, uint32_t k1, uint32_t generation, uint32_t kernel_choice,
+                       void* scratch, float* fitness, float* logits, DeviceStatus* status);
+
 }  // namespace evo

@@ -1,0 +1,544 @@
+// Sequence-to-sequence addition task with an LSTM encoder-decoder policy (paper Section 3,
+// "Seq2Seq Learning"): a single-step task whose fitness is minus the mean cross-entropy of the
+// answer digits over a batch of queries that every member sees.
+//
+// Conventions: tokens '0'..'9' -> 0..9, '+' -> 10, '=' -> 11; the encoder reads "a+b" (2 nd + 1
+// tokens), the decoder is fed '=' and then the true answer digits and must produce the nd + 1
+// digits of the sum; gate order (input, forget, cell, output); flat parameters enc.Wx[4h][12],
+// enc.Wh[4h][h], enc.b[4h], dec.*, out.W[12][h], out.b[12].  A cell's pre-activation is one
+// contraction [Wh | Wx | b] . [h; onehot(token); 1] with bf16 operands and fp32 accumulation; the
+// read-out out.W . h likewise.
+//
+//   k_s2s_simple  CUDA cores, one block per (member, 16 queries): the plain version.
+//   k_s2s_tc      tcgen05: one block per (member, 128 queries).  The member's [4h = 512] x [K = 144]
+//                 weight tile (bf16) stays in shared memory for a whole phase; the B operand is the
+//                 hidden state of the 128 queries plus their one-hot token and a constant 1, so
+//                 one chain of 9 MMAs per gate produces the complete pre-activation in TMEM.  The
+//                 queries are split into two halves of 64 whose steps alternate: while the
+//                 epilogue warps of one half apply the gate non-linearities and write the new
+//                 hidden state back into the B operand, the tensor cores work on the other half.
+//                 TMEM: 2 halves x 4 gates x 64 columns = 512.
+#include "internal.h"
+#include "async.cuh"
+#include "noise.cuh"
+#include "umma.cuh"
+
+namespace evo {
+
+constexpr int kVocab = 12;
+constexpr int kTokPlus = 10, kTokEq = 11;
+constexpr int kS2sMaxDigits = 4;
+constexpr int kS2sMaxTe = 2 * kS2sMaxDigits + 1, kS2sMaxTd = kS2sMaxDigits + 1;
+
+__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+// Query i of a generation: a, b uniform on [0, 10^nd) from the first two words of stream 6.
+__device__ __forceinline__ void s2s_query(PhiloxKey key, uint32_t generation, uint32_t i, uint32_t nd,
+                                          uint8_t* enc, uint8_t* dec, uint8_t* tgt)
+{
+    uint32_t range = 1;
+    for (uint32_t k = 0; k < nd; ++k) range *= 10u;
+    const uint4 w = philox4x32_10(i, 0u, generation, 6u, key);
+    const uint32_t a = __umulhi(w.x, range), b = __umulhi(w.y, range), sum = a + b;
+    uint32_t div = range / 10u;
+    for (uint32_t k = 0; k < nd; ++k, div /= 10u) {
+        enc[k] = static_cast<uint8_t>((a / div) % 10u);
+        enc[nd + 1 + k] = static_cast<uint8_t>((b / div) % 10u);
+    }
+    enc[nd] = kTokPlus;
+    div = range;
+    for (uint32_t k = 0; k <= nd; ++k, div /= 10u) tgt[k] = static_cast<uint8_t>((sum / div) % 10u);
+    dec[0] = kTokEq;
+    for (uint32_t k = 1; k <= nd; ++k) dec[k] = tgt[k - 1];
+}
+
+__device__ __forceinline__ float sigmoid_acc(float x) { return 1.0f / (1.0f + expf(-x)); }
+
+// cross-entropy of one position from its 12 logits
+__device__ __forceinline__ float token_loss(const float* lg, int target)
+{
+    float mx = lg[0];
+#pragma unroll
+    for (int o = 1; o < kVocab; ++o) mx = fmaxf(mx, lg[o]);
+    float se = 0.f;
+#pragma unroll
+    for (int o = 0; o < kVocab; ++o) se += expf(lg[o] - mx);
+    return (mx + logf(se)) - lg[target];
+}
+
+struct S2sArgs {
+    const float* theta; uint32_t ldD, P;
+    uint32_t h, nd, B;
+    uint32_t k0, k1, generation;
+    float* partial;              // [P][n_chunks] sums of token losses
+    uint32_t n_chunks;
+    float* logits;               // nullable: [P][B][nd+1][12] (simple kernel only)
+};
+
+// ------------------------------------------------------------------------------------------
+// CUDA-core version: thread = hidden unit, 16 queries per block, weights read through the caches.
+// ------------------------------------------------------------------------------------------
+constexpr int kSimpleQ = 16;
+
+__global__ void __launch_bounds__(128)
+k_s2s_simple(const S2sArgs a)
+{
+    __shared__ __align__(16) float hs[kSimpleQ][128];           // bf16-rounded hidden state
+    __shared__ float lg[kSimpleQ][kVocab];
+    __shared__ uint8_t enc[kSimpleQ][kS2sMaxTe], dec[kSimpleQ][kS2sMaxTd], tgt[kSimpleQ][kS2sMaxTd];
+    __shared__ float loss_s[kSimpleQ];
+    const uint32_t h = a.h, r = threadIdx.x, member = blockIdx.x, q0 = blockIdx.y * kSimpleQ;
+    const uint32_t nq = min(static_cast<uint32_t>(kSimpleQ), a.B - q0);
+    const uint32_t Te = 2 * a.nd + 1, Td = a.nd + 1;
+    const PhiloxKey key{a.k0, a.k1};
+    if (r < kSimpleQ) {
+        s2s_query(key, a.generation, q0 + min(r, nq - 1u), a.nd, enc[r], dec[r], tgt[r]);
+        loss_s[r] = 0.f;
+    }
+    for (uint32_t s = 0; s < kSimpleQ; ++s) hs[s][r] = 0.f;
+    float c[kSimpleQ];
+#pragma unroll
+    for (int s = 0; s < kSimpleQ; ++s) c[s] = 0.f;
+    const float* p = a.theta + static_cast<size_t>(member) * a.ldD;
+    const size_t cell = static_cast<size_t>(4) * h * kVocab + static_cast<size_t>(4) * h * h + 4u * h;
+    const float* oW = p + 2 * cell;
+    const float* ob = oW + static_cast<size_t>(kVocab) * h;
+    __syncthreads();
+
+    for (uint32_t t = 0; t < Te + Td; ++t) {
+        const bool decoding = t >= Te;
+        const float* Wx = p + (decoding ? cell : 0);
+        const float* Wh = Wx + static_cast<size_t>(4) * h * kVocab;
+        const float* bb = Wh + static_cast<size_t>(4) * h * h;
+        float acc[4][kSimpleQ];
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+#pragma unroll
+            for (int s = 0; s < kSimpleQ; ++s) acc[g][s] = 0.f;
+        if (r < h) {
+            for (uint32_t k = 0; k < h; k += 4) {
+                float4 w[4];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    w[g] = __ldg(reinterpret_cast<const float4*>(Wh + (static_cast<size_t>(g) * h + r) * h + k));
+                    w[g].x = bf16_round(w[g].x); w[g].y = bf16_round(w[g].y);
+                    w[g].z = bf16_round(w[g].z); w[g].w = bf16_round(w[g].w);
+                }
+#pragma unroll
+                for (int s = 0; s < kSimpleQ; ++s) {
+                    const float4 x = *reinterpret_cast<const float4*>(&hs[s][k]);
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        acc[g][s] = fmaf(w[g].x, x.x, acc[g][s]);
+                        acc[g][s] = fmaf(w[g].y, x.y, acc[g][s]);
+                        acc[g][s] = fmaf(w[g].z, x.z, acc[g][s]);
+                        acc[g][s] = fmaf(w[g].w, x.w, acc[g][s]);
+                    }
+                }
+            }
+        }
+        __syncthreads();                                       // every thread is done reading hs
+        if (r < h) {
+            float bias[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) bias[g] = bf16_round(bb[g * h + r]);
+#pragma unroll
+            for (int s = 0; s < kSimpleQ; ++s) {
+                const uint32_t tok = decoding ? dec[s][t - Te] : enc[s][t];
+                float pre[4];
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                    pre[g] = acc[g][s] + bf16_round(Wx[(static_cast<size_t>(g) * h + r) * kVocab + tok]) + bias[g];
+                const float ig = sigmoid_acc(pre[0]), fg = sigmoid_acc(pre[1]);
+                const float gg = tanhf(pre[2]), og = sigmoid_acc(pre[3]);
+                c[s] = fmaf(fg, c[s], ig * gg);
+                hs[s][r] = bf16_round(og * tanhf(c[s]));
+            }
+        }
+        __syncthreads();
+        if (decoding) {
+            for (uint32_t idx = r; idx < kSimpleQ * kVocab; idx += blockDim.x) {
+                const uint32_t s = idx / kVocab, o = idx % kVocab;
+                float v = 0.f;
+                for (uint32_t k = 0; k < h; ++k) v = fmaf(bf16_round(oW[o * h + k]), hs[s][k], v);
+                lg[s][o] = v + ob[o];
+                if (a.logits && s < nq)
+                    a.logits[((static_cast<size_t>(member) * a.B + q0 + s) * Td + (t - Te)) * kVocab + o] = lg[s][o];
+            }
+            __syncthreads();
+            if (r < nq) loss_s[r] += token_loss(lg[r], tgt[r][t - Te]);
+            __syncthreads();
+        }
+    }
+    if (r == 0) {
+        float total = 0.f;
+        for (uint32_t s = 0; s < nq; ++s) total += loss_s[s];
+        a.partial[static_cast<size_t>(member) * a.n_chunks + blockIdx.y] = total;
+    }
+}
+
+__global__ void k_s2s_finalize(const float* __restrict__ partial, uint32_t P, uint32_t n_chunks, float inv_count,
+                               float* __restrict__ fitness)
+{
+    const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= P) return;
+    float s = 0.f;
+    for (uint32_t t = 0; t < n_chunks; ++t) s += partial[static_cast<size_t>(m) * n_chunks + t];
+    fitness[m] = -s * inv_count;
+}
+
+// ------------------------------------------------------------------------------------------
+// tensor-core version (h = 128)
+// ------------------------------------------------------------------------------------------
+constexpr int kTcH = 128;
+constexpr int kTcQ = 128;                                  // queries per block: two halves of 64
+constexpr int kTcEpiThreads = 256;                         // warps 0-3: half 0, warps 4-7: half 1
+constexpr int kTcThreads = kTcEpiThreads + 32;             // + the MMA warp
+constexpr int kTcKBlocks = 18;                             // K = 128 (h) + 16 (one-hot, 1, padding) in groups of 8
+constexpr uint32_t kTcALbo = 64 * 128;                     // 64 row groups of 8 x 16 bytes between K groups
+constexpr uint32_t kTcBLbo = 16 * 128 + 16;                // 16 row groups, +16 bytes so that the 2-byte stores
+                                                           // of a warp (4 K groups) fall in distinct banks
+constexpr uint32_t kTcABytes = kTcKBlocks * kTcALbo;       // 147,456
+constexpr uint32_t kTcBBytes = kTcKBlocks * kTcBLbo;       // 37,152
+
+struct __align__(128) S2sSmem {
+    unsigned char A[kTcABytes];                            // [Wh | Wx | b | 0] as core matrices
+    unsigned char Bop[kTcBBytes];                          // [h; onehot; 1; 0] of the 128 queries
+    float oW[kVocab][kTcH];                                // read-out weights, bf16-rounded
+    float ob[kVocab];
+    float lg[2][64][kVocab + 1];
+    uint8_t enc[kTcQ][kS2sMaxTe + 1], dec[kTcQ][kS2sMaxTd + 1], tgt[kTcQ][kS2sMaxTd + 1];
+    float loss_w[8];
+    uint64_t full[2];                                      // the gates of a half are in TMEM
+    uint64_t hready[2];                                    // a half's B operand holds the next step's input
+    uint32_t tmem_slot;
+    volatile int abort;
+};
+
+// sigma(x) and tanh(x) from one special-function tanh each
+__device__ __forceinline__ float tanh_sfu(float x)
+{
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float sigmoid_ex2(float x)
+{
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * -1.4426950408889634f));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+    return r;
+}
+__device__ __forceinline__ float tanh_ex2(float x)
+{
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * 2.885390082f));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+    return fmaf(-2.0f, r, 1.0f);
+}
+
+// one phase's weights -> A operand (all threads of the block)
+__device__ __forceinline__ void s2s_stage_weights(S2sSmem& S, const float* __restrict__ cellp, uint32_t tid)
+{
+    const float* Wx = cellp;
+    const float* Wh = Wx + 4 * kTcH * kVocab;
+    const float* bb = Wh + 4 * kTcH * kTcH;
+    // Wh: 512 rows x 16 K groups; a thread converts 8 consecutive k of one row into one 16-byte row
+    constexpr uint32_t n_items = 512u * 16u;
+    for (uint32_t base = tid; base < n_items; base += 4u * kTcThreads) {
+        float4 v[4][2];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t idx = base + u * kTcThreads;
+            if (idx < n_items) {
+                const uint32_t m = idx & 511u, kb = idx >> 9;
+                const float4* src = reinterpret_cast<const float4*>(Wh + m * kTcH + kb * 8u);
+                v[u][0] = __ldg(src); v[u][1] = __ldg(src + 1);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t idx = base + u * kTcThreads;
+            if (idx < n_items) {
+                const uint32_t m = idx & 511u, kb = idx >> 9;
+                *reinterpret_cast<uint4*>(S.A + kb * kTcALbo + (m >> 3) * 128u + (m & 7u) * 16u) =
+                    make_uint4(pack_bf16(v[u][0].x, v[u][0].y), pack_bf16(v[u][0].z, v[u][0].w),
+                               pack_bf16(v[u][1].x, v[u][1].y), pack_bf16(v[u][1].z, v[u][1].w));
+            }
+        }
+    }
+    // K groups 16, 17: Wx[m][0..7] | Wx[m][8..11], b[m], 0, 0, 0
+    for (uint32_t m = tid; m < 512u; m += kTcThreads) {
+        const float* wx = Wx + m * kVocab;
+        *reinterpret_cast<uint4*>(S.A + 16u * kTcALbo + (m >> 3) * 128u + (m & 7u) * 16u) =
+            make_uint4(pack_bf16(wx[0], wx[1]), pack_bf16(wx[2], wx[3]), pack_bf16(wx[4], wx[5]), pack_bf16(wx[6], wx[7]));
+        *reinterpret_cast<uint4*>(S.A + 17u * kTcALbo + (m >> 3) * 128u + (m & 7u) * 16u) =
+            make_uint4(pack_bf16(wx[8], wx[9]), pack_bf16(wx[10], wx[11]), pack_bf16(bb[m], 0.f), 0u);
+    }
+}
+
+// one-hot (+ constant 1) rows of query n for the coming step
+__device__ __forceinline__ void s2s_write_onehot(S2sSmem& S, uint32_t n, uint32_t tok)
+{
+    uint32_t w[8];
+    const uint32_t one = (tok & 1u) ? 0x3F800000u : 0x00003F80u;  // bf16 1.0 in the upper / lower half
+#pragma unroll
+    for (uint32_t i = 0; i < 8u; ++i) w[i] = (i == (tok >> 1)) ? one : 0u;
+    w[6] |= 0x00003F80u;                                          // k = 12: the constant input of the bias
+    *reinterpret_cast<uint4*>(S.Bop + 16u * kTcBLbo + n * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+    *reinterpret_cast<uint4*>(S.Bop + 17u * kTcBLbo + n * 16u) = make_uint4(w[4], w[5], w[6], w[7]);
+}
+
+// barrier over the four epilogue warps of one half
+__device__ __forceinline__ void half_barrier(uint32_t half)
+{
+    if (half) asm volatile("bar.sync 2, 128;" ::: "memory");
+    else      asm volatile("bar.sync 1, 128;" ::: "memory");
+}
+
+template <bool SFU_TANH>
+__global__ void __launch_bounds__(kTcThreads, 1)
+k_s2s_tc(const S2sArgs a, DeviceStatus* status)
+{
+    extern __shared__ __align__(128) unsigned char s2s_smem_raw[];
+    S2sSmem& S = *reinterpret_cast<S2sSmem*>(s2s_smem_raw);
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31u;
+    const uint32_t Te = 2 * a.nd + 1, Td = a.nd + 1, T = Te + Td;
+    const uint32_t n_items = a.P * a.n_chunks;
+    const PhiloxKey key{a.k0, a.k1};
+    const size_t cell = static_cast<size_t>(4) * kTcH * kVocab + static_cast<size_t>(4) * kTcH * kTcH + 4u * kTcH;
+
+    if (tid == 0) {
+        mbar_init(smem_u32(&S.full[0]), 1); mbar_init(smem_u32(&S.full[1]), 1);
+        mbar_init(smem_u32(&S.hready[0]), 4); mbar_init(smem_u32(&S.hready[1]), 4);
+        S.abort = 0;
+        mbar_init_fence();
+    }
+    __syncwarp();
+    if (warp == 0) tmem_alloc(smem_u32(&S.tmem_slot), 512);
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = S.tmem_slot;
+
+    uint32_t n_full = 0u;                      // epilogue thread: completed waits on full[half]
+    uint32_t n_ready0 = 0u, n_ready1 = 0u;     // MMA thread: completed waits on hready[0], hready[1]
+    const uint32_t half = warp >> 2;           // epilogue warps: which 64 queries
+    const uint32_t r = tid & 127u;             // epilogue thread: hidden unit = TMEM lane
+
+    for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const uint32_t member = item / a.n_chunks, chunk = item % a.n_chunks;
+        const uint32_t q0 = chunk * kTcQ;
+        const uint32_t nq = min(static_cast<uint32_t>(kTcQ), a.B - q0);
+        const float* p = a.theta + static_cast<size_t>(member) * a.ldD;
+
+        // ---- per-item setup: queries, zero state, read-out weights, encoder weights ------------
+        if (tid < kTcQ) s2s_query(key, a.generation, q0 + min(tid, nq - 1u), a.nd, S.enc[tid], S.dec[tid], S.tgt[tid]);
+        for (uint32_t i = tid; i < 16u * kTcBLbo / 16u; i += kTcThreads)
+            reinterpret_cast<uint4*>(S.Bop)[i] = make_uint4(0u, 0u, 0u, 0u);
+        for (uint32_t i = tid; i < kVocab * kTcH; i += kTcThreads)
+            (&S.oW[0][0])[i] = bf16_round(p[2 * cell + i]);
+        if (tid < kVocab) S.ob[tid] = p[2 * cell + kVocab * kTcH + tid];
+        s2s_stage_weights(S, p, tid);
+        __syncthreads();                                        // tokens are there
+        if (tid < kTcQ) s2s_write_onehot(S, tid, S.enc[tid][0]);
+        fence_async_smem();
+        __syncthreads();
+
+        float c[64];
+#pragma unroll
+        for (int i = 0; i < 64; ++i) c[i] = 0.f;
+        float loss = 0.f;
+
+        for (uint32_t phase = 0; phase < 2u; ++phase) {
+            const uint32_t t0 = phase ? Te : 0u, t1 = phase ? T : Te;
+            if (phase) {
+                // every MMA of the encoder has been waited for by an epilogue warp: A may be replaced
+                __syncthreads();
+                s2s_stage_weights(S, p + cell, tid);
+                fence_async_smem();
+                __syncthreads();
+            }
+            if (warp == kTcEpiThreads / 32) {
+                // ================= MMA warp ============================================================
+                if (lane == 0) {
+                    constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
+                    const uint32_t a_base = smem_u32(S.A), b_base = smem_u32(S.Bop);
+                    for (uint32_t t = t0; t < t1; ++t)
+#pragma unroll
+                        for (uint32_t x = 0; x < 2u; ++x) {
+                            if (t > 0) {                         // step 0 reads the state the setup wrote
+                                uint32_t& n_ready = x ? n_ready1 : n_ready0;
+                                wait_or_abort(&S.abort, &S.hready[x], n_ready & 1u, status);
+                                ++n_ready;
+                            }
+                            tc_fence_after();
+#pragma unroll
+                            for (uint32_t g = 0; g < 4u; ++g)
+#pragma unroll
+                                for (uint32_t kk = 0; kk < kTcKBlocks / 2; ++kk) {
+                                    const uint64_t ad = umma_smem_desc(a_base + 2u * kk * kTcALbo + g * 16u * 128u, kTcALbo, 128u);
+                                    const uint64_t bd = umma_smem_desc(b_base + 2u * kk * kTcBLbo + x * 8u * 128u, kTcBLbo, 128u);
+                                    umma_bf16(tmem + x * 256u + g * 64u, ad, bd, idesc, kk);
+                                }
+                            umma_commit(smem_u32(&S.full[x]));
+                        }
+                }
+                __syncwarp();
+            } else {
+                // ================= epilogue warps ======================================================
+                const uint32_t tq = tmem + (static_cast<uint32_t>((warp & 3u) * 32u) << 16) + half * 256u;
+                for (uint32_t t = t0; t < t1; ++t) {
+                    wait_or_abort(&S.abort, &S.full[half], n_full & 1u, status);
+                    ++n_full;
+                    tc_fence_after();
+#pragma unroll
+                    for (uint32_t ch = 0; ch < 4u; ++ch) {
+                        uint32_t gi[16], gf[16], gg[16], go[16];
+                        tmem_ld16_issue(tq + 0u * 64u + ch * 16u, gi);
+                        tmem_ld16_issue(tq + 1u * 64u + ch * 16u, gf);
+                        tmem_ld16_issue(tq + 2u * 64u + ch * 16u, gg);
+                        tmem_ld16_issue(tq + 3u * 64u + ch * 16u, go);
+                        tmem_ld16_fence(gi); tmem_ld16_fence(gf); tmem_ld16_fence(gg); tmem_ld16_fence(go);
+                        // hidden unit r of query n sits at K group r/8, row n, element r%8
+                        unsigned char* dst = S.Bop + (r >> 3) * kTcBLbo + (half * 64u + ch * 16u) * 16u + (r & 7u) * 2u;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            float hv;
+                            if (SFU_TANH) {
+                                const float ig = fmaf(0.5f, tanh_sfu(0.5f * __uint_as_float(gi[j])), 0.5f);
+                                const float fg = fmaf(0.5f, tanh_sfu(0.5f * __uint_as_float(gf[j])), 0.5f);
+                                const float cg = tanh_sfu(__uint_as_float(gg[j]));
+                                const float og = fmaf(0.5f, tanh_sfu(0.5f * __uint_as_float(go[j])), 0.5f);
+                                c[ch * 16 + j] = fmaf(fg, c[ch * 16 + j], ig * cg);
+                                hv = og * tanh_sfu(c[ch * 16 + j]);
+                            } else {
+                                const float ig = sigmoid_ex2(__uint_as_float(gi[j]));
+                                const float fg = sigmoid_ex2(__uint_as_float(gf[j]));
+                                const float cg = tanh_ex2(__uint_as_float(gg[j]));
+                                const float og = sigmoid_ex2(__uint_as_float(go[j]));
+                                c[ch * 16 + j] = fmaf(fg, c[ch * 16 + j], ig * cg);
+                                hv = og * tanh_ex2(c[ch * 16 + j]);
+                            }
+                            *reinterpret_cast<__nv_bfloat16*>(dst + j * 16) = __float2bfloat16_rn(hv);
+                        }
+                    }
+                    // the coming step's token (none after the last step)
+                    if (t + 1u < T && r < 64u) {
+                        const uint32_t n = half * 64u + r;
+                        s2s_write_onehot(S, n, (t + 1u < Te) ? S.enc[n][t + 1u] : S.dec[n][t + 1u - Te]);
+                    }
+                    fence_async_smem();
+                    tc_fence_before();
+                    if (t >= Te) {
+                        // read-out on the CUDA cores from the state just written; the half's four warps
+                        // must all have written it
+                        half_barrier(half);
+                        if (t + 1u < T && lane == 0) mbar_arrive(smem_u32(&S.hready[half]));
+                        const uint32_t s = r & 63u, o0 = (r >> 6) * 6u;
+                        float acc[6] = { 0.f, 0.f, 0.f, 0.f, 0.f, 0.f };
+                        const unsigned char* hrow = S.Bop + (half * 64u + s) * 16u;
+#pragma unroll 4
+                        for (uint32_t kb = 0; kb < 16u; ++kb) {
+                            const uint4 hv = *reinterpret_cast<const uint4*>(hrow + kb * kTcBLbo);
+                            const uint32_t hw[4] = { hv.x, hv.y, hv.z, hv.w };
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float x0 = __uint_as_float(hw[i] << 16), x1 = __uint_as_float(hw[i] & 0xFFFF0000u);
+#pragma unroll
+                                for (int o = 0; o < 6; ++o) {
+                                    acc[o] = fmaf(S.oW[o0 + o][kb * 8u + 2 * i], x0, acc[o]);
+                                    acc[o] = fmaf(S.oW[o0 + o][kb * 8u + 2 * i + 1], x1, acc[o]);
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int o = 0; o < 6; ++o) S.lg[half][s][o0 + o] = acc[o] + S.ob[o0 + o];
+                        half_barrier(half);
+                        if (r < 64u && half * 64u + r < nq)
+                            loss += token_loss(S.lg[half][r], S.tgt[half * 64u + r][t - Te]);
+                        // the next epilogue overwrites the state: everyone must be done reading it
+                        half_barrier(half);
+                    } else {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&S.hready[half]));
+                    }
+                }
+            }
+        }
+        // ---- the item's loss: fixed-order sum over the 4 warps that hold query losses -----------
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, off);
+        if (warp < 8u && lane == 0) S.loss_w[warp] = loss;
+        __syncthreads();
+        if (tid == 0)
+            a.partial[static_cast<size_t>(member) * a.n_chunks + chunk] =
+                (S.loss_w[0] + S.loss_w[1]) + (S.loss_w[4] + S.loss_w[5]);
+        __syncthreads();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+uint32_t s2s_param_count(uint32_t h)
+{
+    return 2u * (4u * h * kVocab + 4u * h * h + 4u * h) + kVocab * h + kVocab;
+}
+
+bool s2s_supported(uint32_t h, uint32_t nd, uint32_t B)
+{
+    return h >= 32 && h <= 128 && h % 32 == 0 && nd >= 1 && nd <= kS2sMaxDigits && B >= 1;
+}
+
+static uint32_t s2s_chunks(uint32_t B, bool tc) { return tc ? (B + kTcQ - 1) / kTcQ : (B + kSimpleQ - 1) / kSimpleQ; }
+
+size_t s2s_scratch_bytes(uint32_t P, uint32_t B)
+{
+    return static_cast<size_t>(P) * s2s_chunks(B, false) * sizeof(float);     // the finer split bounds both
+}
+
+int launch_rollout_s2s(cudaStream_t st, const float* theta, uint32_t ldD, uint32_t P, uint32_t h, uint32_t nd,
+                       uint32_t B, uint32_t k0, uint32_t k1, uint32_t generation, uint32_t kernel_choice,
+                       void* scratch, float* fitness, float* logits, DeviceStatus* status)
+{
+    const bool want_tc = kernel_choice != EVO_ROLLOUT_GENERIC;
+    if (want_tc && (h != kTcH || logits)) {
+        if (kernel_choice == EVO_ROLLOUT_TILED) return -2;       // asked for explicitly, not available
+    }
+    const bool tc = want_tc && h == kTcH && !logits;
+    S2sArgs a;
+    a.theta = theta; a.ldD = ldD; a.P = P; a.h = h; a.nd = nd; a.B = B;
+    a.k0 = k0; a.k1 = k1; a.generation = generation;
+    a.partial = static_cast<float*>(scratch);
+    a.n_chunks = s2s_chunks(B, tc);
+    a.logits = logits;
+    if (tc) {
+        static int sm_count = 0;
+        if (sm_count == 0) {
+            int dev = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+            if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+        }
+        if (cudaFuncSetAttribute(k_s2s_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(sizeof(S2sSmem))) != cudaSuccess) return -1;
+        const uint32_t items = P * a.n_chunks;
+        const uint32_t grid = items < static_cast<uint32_t>(sm_count) ? items : static_cast<uint32_t>(sm_count);
+        k_s2s_tc<false><<<grid, kTcThreads, sizeof(S2sSmem), st>>>(a, status);
+    } else {
+        dim3 grid(P, a.n_chunks);
+        k_s2s_simple<<<grid, 128, 0, st>>>(a);
+    }
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    const float inv = 1.0f / (static_cast<float>(B) * static_cast<float>(nd + 1));
+    k_s2s_finalize<<<(P + 255u) / 256u, 256, 0, st>>>(a.partial, P, a.n_chunks, inv, fitness);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return 2;
+}
+
+}  // namespace evo

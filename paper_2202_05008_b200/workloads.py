@@ -13,8 +13,8 @@ from typing import Tuple
 import numpy as np
 
 NOISE_STORED, NOISE_REGENERATED = 0, 1
-POLICY_NONE, POLICY_MLP, POLICY_CNN_28 = 0, 1, 2
-TASK_NONE, TASK_CARTPOLE, TASK_TANH_LINEAR, TASK_SUPERVISED = 0, 1, 2, 3
+POLICY_NONE, POLICY_MLP, POLICY_CNN_28, POLICY_LSTM_SEQ2SEQ = 0, 1, 2, 3
+TASK_NONE, TASK_CARTPOLE, TASK_TANH_LINEAR, TASK_SUPERVISED, TASK_SEQ2SEQ_ADD = 0, 1, 2, 3, 4
 OPT_ADAM, OPT_CLIPUP = 0, 1
 SIGMA_CONSTANT, SIGMA_PGPE = 0, 1
 
@@ -38,7 +38,7 @@ class Workload:
     horizon: int = 1
     batch: int = 0
     generations: int = 1
-    # cart-pole: cart mass, pole mass, pole half length, gravity, dt, initial range
+    # cart-pole: cart mass, pole mass, pole half length, gravity, dt, initial range; seq2seq: digits
     task_param: Tuple[float, ...] = field(default_factory=tuple)
     optimizer: int = OPT_ADAM
     clipup_momentum: float = 0.0          # 0 = library default (0.9)
@@ -49,7 +49,7 @@ class Workload:
 
     @property
     def env_steps_per_generation(self) -> int:
-        if self.task_kind == TASK_SUPERVISED:
+        if self.task_kind in (TASK_SUPERVISED, TASK_SEQ2SEQ_ADD):
             return self.pop_size * self.batch
         if self.task_kind == TASK_NONE:
             return 0
@@ -81,7 +81,19 @@ CFG4 = Workload("cfg4_tanh_linear_pop4096", 4096, 21256, seed=2, policy_kind=POL
 CFG5 = Workload("cfg5_update_sweep_pop16384", 16384, 1 << 20, seed=3, sigma=0.02,
                 generations=1)
 
-CONFIGS = {"cfg1": CFG1, "cfg2": CFG2, "cfg3": CFG3, "cfg4": CFG4, "cfg5": CFG5}
+
+
+def seq2seq_param_count(h: int) -> int:
+    return 2 * (4 * h * 12 + 4 * h * h + 4 * h) + 12 * h + 12
+
+
+# the paper's seq2seq example (Section 3): LSTM encoder-decoder, 3-digit addition, a network of
+# "hundreds of thousands of parameters" -> hidden width 128 gives 145,932
+SEQ2SEQ = Workload("seq2seq_add_lstm128_pop1024", 1024, seq2seq_param_count(128), seed=4,
+                   policy_kind=POLICY_LSTM_SEQ2SEQ, layer_sizes=(128,), task_kind=TASK_SEQ2SEQ_ADD,
+                   batch=128, generations=20, task_param=(3.0,))
+
+CONFIGS = {"cfg1": CFG1, "cfg2": CFG2, "cfg3": CFG3, "cfg4": CFG4, "cfg5": CFG5, "seq2seq": SEQ2SEQ}
 
 assert mlp_param_count(CFG1.layer_sizes) == CFG1.param_dim
 assert mlp_param_count(CFG2.layer_sizes) == CFG2.param_dim

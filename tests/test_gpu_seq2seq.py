@@ -1,0 +1,110 @@
+"""Parity of the seq2seq roll-out (paper Section 3, "Seq2Seq Learning") with the oracle, through the
+C-ABI: the CUDA-core kernel (any hidden width, logits visible) and the tcgen05 kernel (h = 128)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2202_05008_b200 import Solver, workloads as W
+from paper_2202_05008_b200.binding import ROLLOUT_AUTO, ROLLOUT_GENERIC, ROLLOUT_TILED
+
+pytestmark = pytest.mark.gpu
+
+# Both sides round the operands of the contractions to bf16 at the same points; what is left is
+# fp32 accumulation order and the rare hidden-state element that rounds to the neighbouring bf16
+# value (2^-9 relative) because the kernel's fp32 activation differs from the oracle's fp64 one in
+# the last bits.  Averaged over the batch that stays well below 1e-3 on the fitness.
+FIT_TOL = 1e-3
+
+
+def _workload(h, nd, B, P, sigma=0.3, seed=11):
+    return W.SEQ2SEQ.with_(pop_size=P, param_dim=W.seq2seq_param_count(h), layer_sizes=(h,), batch=B,
+                           task_param=(float(nd),), sigma=sigma, seed=seed)
+
+
+def _oracle_fits(w, theta, generation, want_logits=False):
+    h, nd = w.layer_sizes[0], int(w.task_param[0])
+    enc, dec, tgt = oracle.seq2seq_queries(w.seed, generation, w.batch, nd)
+    return [oracle.seq2seq_fitness(row, h, nd, enc, dec, tgt, True, want_logits=want_logits) for row in theta]
+
+
+@pytest.mark.parametrize("h,nd,B", [(32, 2, 20), (64, 1, 16), (128, 3, 9)])
+def test_cuda_core_kernel_matches_oracle_with_logits(h, nd, B):
+    w = _workload(h, nd, B, P=4)
+    s = Solver(w, rollout_kernel=ROLLOUT_GENERIC, trace_steps=1)
+    theta = s.ask().cpu().numpy()
+    logits = torch.zeros(w.pop_size, B, nd + 1, 12, device="cuda")
+    fit = s.rollout(trace=logits).cpu().numpy()
+    want = _oracle_fits(w, theta, 0, want_logits=True)
+    assert s.sync_status() == 0
+    for m in range(w.pop_size):
+        assert np.max(np.abs(logits[m].cpu().numpy() - want[m][2])) < 2e-2
+        assert abs(fit[m] - want[m][0]) < FIT_TOL
+    # the typical element agrees far better than the worst one
+    assert np.median(np.abs(logits[0].cpu().numpy() - want[0][2])) < 1e-4
+
+
+@pytest.mark.parametrize("B", [128, 100, 200])
+def test_tensor_core_kernel_matches_oracle(B):
+    w = _workload(128, 3, B, P=6, sigma=0.1)
+    s = Solver(w, rollout_kernel=ROLLOUT_TILED)
+    theta = s.ask().cpu().numpy()
+    fit = s.rollout().cpu().numpy()
+    assert s.sync_status() == 0
+    want = _oracle_fits(w, theta, 0)
+    for m in range(w.pop_size):
+        assert abs(fit[m] - want[m][0]) < FIT_TOL, (m, fit[m], want[m][0])
+    assert np.std(fit) > 1e-3                                    # members really differ
+
+
+def test_tensor_core_and_cuda_core_kernels_agree_and_repeat():
+    w = _workload(128, 3, 128, P=150, sigma=0.05)                # more items than SMs: blocks loop
+    a = Solver(w, rollout_kernel=ROLLOUT_TILED)
+    b = Solver(w, rollout_kernel=ROLLOUT_GENERIC)
+    a.ask(); b.ask()
+    fa = a.rollout().clone(); fa2 = a.rollout().clone(); fb = b.rollout().clone()
+    assert torch.equal(fa, fa2)
+    assert float((fa - fb).abs().max()) < FIT_TOL
+    assert a.sync_status() == 0 and b.sync_status() == 0
+
+
+def test_zero_parameters_and_generation_dependence():
+    w = _workload(128, 3, 128, P=2, sigma=0.1)
+    s = Solver(w)
+    s.ask()
+    zero = s.padded_rows(2); zero.zero_()
+    fit = s.rollout(theta=zero).cpu().numpy()
+    assert np.max(np.abs(fit + math.log(12))) < 1e-6
+    f0 = s.rollout().clone()
+    s.tell(f0)
+    s.ask()
+    f1 = s.rollout().clone()
+    assert not torch.equal(f0, f1)                               # new centre and new queries
+    assert s.sync_status() == 0
+
+
+def test_second_generation_uses_that_generations_queries():
+    w = _workload(128, 2, 64, P=4, sigma=0.1)
+    s = Solver(w)
+    s.ask(); s.tell(s.rollout())
+    theta = s.ask().cpu().numpy()
+    fit = s.rollout().cpu().numpy()
+    want = _oracle_fits(w, theta, 1)
+    for m in range(w.pop_size):
+        assert abs(fit[m] - want[m][0]) < FIT_TOL
+
+
+def test_config_errors():
+    from paper_2202_05008_b200 import EvoError
+    with pytest.raises(EvoError):
+        Solver(_workload(128, 3, 128, P=2).with_(param_dim=1000))
+    with pytest.raises(EvoError):
+        Solver(_workload(48, 3, 128, P=2))                        # width not a multiple of 32
+    with pytest.raises(EvoError):
+        Solver(_workload(128, 5, 128, P=2))                       # more digits than supported
+    s = Solver(_workload(64, 3, 128, P=2), rollout_kernel=ROLLOUT_TILED)
+    s.ask()
+    with pytest.raises(EvoError):
+        s.rollout()                                               # the tensor-core kernel needs h = 128
