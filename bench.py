@@ -42,6 +42,9 @@ def rollout_flops_per_env_step(w):
     from paper_2202_05008_b200 import workloads as W
     if w.task_kind == W.TASK_SUPERVISED:
         return 645120.0                       # conv1 230,400 + conv2 409,600 + fc 5,120 (2 x MAC)
+    if w.task_kind == W.TASK_SEQ2SEQ_ADD:         # per query: every LSTM step + the read-out steps
+        h, nd = w.layer_sizes[0], int(w.task_param[0])
+        return 2.0 * ((3 * nd + 2) * 4 * h * (h + 12 + 1) + (nd + 1) * 12 * h)
     macs = mlp_macs(w.layer_sizes)
     if w.task_kind == W.TASK_TANH_LINEAR:
         macs += 28 * 28 + 28 * 8              # the task's own x' = tanh(Ax + Ba)
@@ -156,6 +159,10 @@ def _oracle_member_rollout(w, generation):
         p = oracle.cartpole_params(tp[0], tp[1], tp[2], tp[3], tp[4])
         return lambda row: oracle.rollout_cartpole(row, w.layer_sizes, w.action_scale, p, tp[5], w.seed,
                                                    generation, w.episodes, w.horizon)[0]
+    if w.task_kind == W.TASK_SEQ2SEQ_ADD:
+        h, nd = w.layer_sizes[0], int(w.task_param[0])
+        enc, dec, tgt = oracle.seq2seq_queries(w.seed, generation, w.batch, nd)
+        return lambda row: oracle.seq2seq_fitness(row, h, nd, enc, dec, tgt, True)[0]
     A, B = oracle.tanh_linear_constants(w.seed)
     return lambda row: oracle.rollout_tanh_linear(row, w.layer_sizes, w.action_scale, A, B, w.seed,
                                                   generation, w.episodes, w.horizon)[0]
@@ -245,10 +252,12 @@ def run_reference(args, w):
 def config_of(w, args, stored):
     from paper_2202_05008_b200 import workloads as W
     task = {W.TASK_NONE: "none", W.TASK_CARTPOLE: "cartpole_swingup", W.TASK_TANH_LINEAR: "tanh_linear",
-            W.TASK_SUPERVISED: "supervised_28x28"}[w.task_kind]
+            W.TASK_SUPERVISED: "supervised_28x28", W.TASK_SEQ2SEQ_ADD: "seq2seq_addition"}[w.task_kind]
     return {"workload": w.name, "pop_size": w.pop_size, "param_dim": w.param_dim, "task": task,
-            "policy": "mlp " + "-".join(map(str, w.layer_sizes)) if w.layer_sizes else
-                      ("cnn_28" if w.policy_kind == W.POLICY_CNN_28 else "none"),
+            "policy": "mlp " + "-".join(map(str, w.layer_sizes)) if w.policy_kind == W.POLICY_MLP else
+                      {W.POLICY_CNN_28: "cnn_28",
+                       W.POLICY_LSTM_SEQ2SEQ: f"lstm_encoder_decoder h={w.layer_sizes[0] if w.layer_sizes else 0}"
+                       }.get(w.policy_kind, "none"),
             "episodes": w.episodes, "horizon": w.horizon, "batch": w.batch,
             "noise": "stored" if stored else "regenerated",
             "parallelism": f"{'one population, pair shards' if args.sharded else 'replicas'} x{args.gpus}",
@@ -442,9 +451,10 @@ def run_ours(args, w):
                         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                         "traffic": None}
-        elif supervised:
+        elif supervised or w.task_kind == W.TASK_SEQ2SEQ_ADD:
             achieved = stages["rollout"]["TFLOP/s"]
-            roofline = {"kernel": "k_cnn_conv1_tc + k_cnn_conv2_tc", "bound": "tensor", "achieved": achieved,
+            roofline = {"kernel": "k_cnn_conv1_tc + k_cnn_conv2_tc" if supervised else "k_s2s_tc",
+                        "bound": "tensor", "achieved": achieved,
                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                         "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"],
                         "traffic": None}
@@ -493,7 +503,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "seq2seq"])
     ap.add_argument("--noise", default="stored", choices=["stored", "regenerated"])
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing leg")
     ap.add_argument("--sharded", action="store_true",

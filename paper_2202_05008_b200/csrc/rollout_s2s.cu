@@ -22,6 +22,7 @@
 #include "async.cuh"
 #include "noise.cuh"
 #include "umma.cuh"
+#include <cuda_fp16.h>
 
 namespace evo {
 
@@ -193,18 +194,19 @@ __global__ void k_s2s_finalize(const float* __restrict__ partial, uint32_t P, ui
 constexpr int kTcH = 128;
 constexpr int kTcQ = 128;                                  // queries per block: two halves of 64
 constexpr int kTcEpiThreads = 256;                         // warps 0-3: half 0, warps 4-7: half 1
-constexpr int kTcThreads = kTcEpiThreads + 32;             // + the MMA warp
+constexpr int kTcThreads = kTcEpiThreads + 64;             // + one MMA warp per half
 constexpr int kTcKBlocks = 18;                             // K = 128 (h) + 16 (one-hot, 1, padding) in groups of 8
 constexpr uint32_t kTcALbo = 64 * 128;                     // 64 row groups of 8 x 16 bytes between K groups
 constexpr uint32_t kTcBLbo = 16 * 128 + 16;                // 16 row groups, +16 bytes so that the 2-byte stores
                                                            // of a warp (4 K groups) fall in distinct banks
 constexpr uint32_t kTcABytes = kTcKBlocks * kTcALbo;       // 147,456
 constexpr uint32_t kTcBBytes = kTcKBlocks * kTcBLbo;       // 37,152
+constexpr uint32_t kTcCellFloats = 4 * kTcH * kVocab + 4 * kTcH * kTcH + 4 * kTcH;   // one LSTM cell
 
 struct __align__(128) S2sSmem {
     unsigned char A[kTcABytes];                            // [Wh | Wx | b | 0] as core matrices
     unsigned char Bop[kTcBBytes];                          // [h; onehot; 1; 0] of the 128 queries
-    float oW[kVocab][kTcH];                                // read-out weights, bf16-rounded
+    float oW[16][kVocab][8];                               // read-out weights [K group][token][k], bf16-rounded
     float ob[kVocab];
     float lg[2][64][kVocab + 1];
     uint8_t enc[kTcQ][kS2sMaxTe + 1], dec[kTcQ][kS2sMaxTd + 1], tgt[kTcQ][kS2sMaxTd + 1];
@@ -215,29 +217,59 @@ struct __align__(128) S2sSmem {
     volatile int abort;
 };
 
-// sigma(x) and tanh(x) from one special-function tanh each
-__device__ __forceinline__ float tanh_sfu(float x)
+// two tanh at once on the special-function unit, in and out as packed fp16 (relative error 2^-11,
+// the same class as the fp32 approximation)
+__device__ __forceinline__ uint32_t tanh_h2(uint32_t x)
 {
-    float y;
-    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    uint32_t y;
+    asm("tanh.approx.f16x2 %0, %1;" : "=r"(y) : "r"(x));
     return y;
 }
-__device__ __forceinline__ float sigmoid_ex2(float x)
+__device__ __forceinline__ uint32_t pack_h2(float lo, float hi)
 {
-    float e, r;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * -1.4426950408889634f));
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
-    return r;
+    uint32_t y;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(y) : "f"(hi), "f"(lo));
+    return y;
 }
-__device__ __forceinline__ float tanh_ex2(float x)
+__device__ __forceinline__ float2 unpack_h2(uint32_t v)
 {
-    float e, r;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * 2.885390082f));
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
-    return fmaf(-2.0f, r, 1.0f);
+    return __half22float2(*reinterpret_cast<const __half2*>(&v));
+}
+// 0.5 t + 0.5 on both halves: sigma(x) from t = tanh(x / 2)
+__device__ __forceinline__ uint32_t half_plus_half_h2(uint32_t t)
+{
+    uint32_t y;
+    asm("fma.rn.f16x2 %0, %1, %2, %2;" : "=r"(y) : "r"(t), "r"(0x38003800u));
+    return y;
+}
+__device__ __forceinline__ uint32_t mul_h2(uint32_t a, uint32_t b)
+{
+    uint32_t y;
+    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(y) : "r"(a), "r"(b));
+    return y;
+}
+// two fp32 fused multiply-adds in one instruction
+__device__ __forceinline__ void ffma2(float2& acc, float2 a, float2 b)
+{
+    asm("fma.rn.f32x2 %0, %1, %2, %0;"
+        : "+l"(*reinterpret_cast<unsigned long long*>(&acc))
+        : "l"(*reinterpret_cast<const unsigned long long*>(&a)), "l"(*reinterpret_cast<const unsigned long long*>(&b)));
+}
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t p;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(p));
+    return p != 0;
+}
+// asks the L2 to fetch `bytes` (multiple of 16) starting at a 16-byte aligned address
+__device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(__cvta_generic_to_global(p)), "r"(bytes) : "memory");
 }
 
-// one phase's weights -> A operand (all threads of the block)
+// One cell's weights -> A operand (all threads of the block).  The rows of the input, forget and
+// output gates are halved (exact in bf16) so that their sigma(x) = 0.5 tanh(x / 2) + 0.5 needs no
+// scaling of the accumulator.
 __device__ __forceinline__ void s2s_stage_weights(S2sSmem& S, const float* __restrict__ cellp, uint32_t tid)
 {
     const float* Wx = cellp;
@@ -245,35 +277,40 @@ __device__ __forceinline__ void s2s_stage_weights(S2sSmem& S, const float* __res
     const float* bb = Wh + 4 * kTcH * kTcH;
     // Wh: 512 rows x 16 K groups; a thread converts 8 consecutive k of one row into one 16-byte row
     constexpr uint32_t n_items = 512u * 16u;
-    for (uint32_t base = tid; base < n_items; base += 4u * kTcThreads) {
-        float4 v[4][2];
+    constexpr int U = 8;
+#pragma unroll 1
+    for (uint32_t base = tid; base < n_items; base += U * kTcThreads) {
+        float4 v[U][2];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const uint32_t idx = base + u * kTcThreads;
-            if (idx < n_items) {
-                const uint32_t m = idx & 511u, kb = idx >> 9;
-                const float4* src = reinterpret_cast<const float4*>(Wh + m * kTcH + kb * 8u);
-                v[u][0] = __ldg(src); v[u][1] = __ldg(src + 1);
-            }
+        for (int u = 0; u < U; ++u) {
+            const uint32_t idx = min(base + u * kTcThreads, n_items - 1u);
+            const uint32_t m = idx & 511u, kb = idx >> 9;
+            const float4* src = reinterpret_cast<const float4*>(Wh + m * kTcH + kb * 8u);
+            v[u][0] = __ldg(src); v[u][1] = __ldg(src + 1);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
             const uint32_t idx = base + u * kTcThreads;
             if (idx < n_items) {
                 const uint32_t m = idx & 511u, kb = idx >> 9;
+                const float sc = ((m >> 7) == 2u) ? 1.0f : 0.5f;
                 *reinterpret_cast<uint4*>(S.A + kb * kTcALbo + (m >> 3) * 128u + (m & 7u) * 16u) =
-                    make_uint4(pack_bf16(v[u][0].x, v[u][0].y), pack_bf16(v[u][0].z, v[u][0].w),
-                               pack_bf16(v[u][1].x, v[u][1].y), pack_bf16(v[u][1].z, v[u][1].w));
+                    make_uint4(pack_bf16(sc * v[u][0].x, sc * v[u][0].y), pack_bf16(sc * v[u][0].z, sc * v[u][0].w),
+                               pack_bf16(sc * v[u][1].x, sc * v[u][1].y), pack_bf16(sc * v[u][1].z, sc * v[u][1].w));
             }
         }
     }
     // K groups 16, 17: Wx[m][0..7] | Wx[m][8..11], b[m], 0, 0, 0
     for (uint32_t m = tid; m < 512u; m += kTcThreads) {
-        const float* wx = Wx + m * kVocab;
+        const float4* wx = reinterpret_cast<const float4*>(Wx + m * kVocab);        // 48-byte rows
+        const float4 w0 = __ldg(wx), w1 = __ldg(wx + 1), w2 = __ldg(wx + 2);
+        const float sc = ((m >> 7) == 2u) ? 1.0f : 0.5f;
+        const float bias = sc * __ldg(bb + m);
         *reinterpret_cast<uint4*>(S.A + 16u * kTcALbo + (m >> 3) * 128u + (m & 7u) * 16u) =
-            make_uint4(pack_bf16(wx[0], wx[1]), pack_bf16(wx[2], wx[3]), pack_bf16(wx[4], wx[5]), pack_bf16(wx[6], wx[7]));
+            make_uint4(pack_bf16(sc * w0.x, sc * w0.y), pack_bf16(sc * w0.z, sc * w0.w),
+                       pack_bf16(sc * w1.x, sc * w1.y), pack_bf16(sc * w1.z, sc * w1.w));
         *reinterpret_cast<uint4*>(S.A + 17u * kTcALbo + (m >> 3) * 128u + (m & 7u) * 16u) =
-            make_uint4(pack_bf16(wx[8], wx[9]), pack_bf16(wx[10], wx[11]), pack_bf16(bb[m], 0.f), 0u);
+            make_uint4(pack_bf16(sc * w2.x, sc * w2.y), pack_bf16(sc * w2.z, sc * w2.w), pack_bf16(bias, 0.f), 0u);
     }
 }
 
@@ -296,7 +333,6 @@ __device__ __forceinline__ void half_barrier(uint32_t half)
     else      asm volatile("bar.sync 1, 128;" ::: "memory");
 }
 
-template <bool SFU_TANH>
 __global__ void __launch_bounds__(kTcThreads, 1)
 k_s2s_tc(const S2sArgs a, DeviceStatus* status)
 {
@@ -306,7 +342,6 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
     const uint32_t Te = 2 * a.nd + 1, Td = a.nd + 1, T = Te + Td;
     const uint32_t n_items = a.P * a.n_chunks;
     const PhiloxKey key{a.k0, a.k1};
-    const size_t cell = static_cast<size_t>(4) * kTcH * kVocab + static_cast<size_t>(4) * kTcH * kTcH + 4u * kTcH;
 
     if (tid == 0) {
         mbar_init(smem_u32(&S.full[0]), 1); mbar_init(smem_u32(&S.full[1]), 1);
@@ -322,10 +357,11 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
     tc_fence_after();
     const uint32_t tmem = S.tmem_slot;
 
-    uint32_t n_full = 0u;                      // epilogue thread: completed waits on full[half]
-    uint32_t n_ready0 = 0u, n_ready1 = 0u;     // MMA thread: completed waits on hready[0], hready[1]
-    const uint32_t half = warp >> 2;           // epilogue warps: which 64 queries
+    uint32_t n_wait = 0u;                      // completed waits: full[half] (epilogue) / hready[x] (MMA warp)
+    const bool is_mma = warp >= kTcEpiThreads / 32;
+    const uint32_t half = is_mma ? warp - kTcEpiThreads / 32 : warp >> 2;   // which 64 queries this warp serves
     const uint32_t r = tid & 127u;             // epilogue thread: hidden unit = TMEM lane
+    uint32_t staged_chunk = 0xFFFFFFFFu;
 
     for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
         const uint32_t member = item / a.n_chunks, chunk = item % a.n_chunks;
@@ -334,12 +370,26 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
         const float* p = a.theta + static_cast<size_t>(member) * a.ldD;
 
         // ---- per-item setup: queries, zero state, read-out weights, encoder weights ------------
-        if (tid < kTcQ) s2s_query(key, a.generation, q0 + min(tid, nq - 1u), a.nd, S.enc[tid], S.dec[tid], S.tgt[tid]);
+        if (chunk != staged_chunk) {
+            if (tid < kTcQ) s2s_query(key, a.generation, q0 + min(tid, nq - 1u), a.nd, S.enc[tid], S.dec[tid], S.tgt[tid]);
+            staged_chunk = chunk;
+        }
+        if (is_mma) {                                            // the decoder's weights will be wanted next
+            const char* next = reinterpret_cast<const char*>(p + kTcCellFloats);
+            constexpr uint32_t piece = kTcCellFloats * 4u / 64u;       // 4,512 bytes per lane of the two warps
+            prefetch_l2(next + ((warp - kTcEpiThreads / 32) * 32u + lane) * piece, piece);
+        }
         for (uint32_t i = tid; i < 16u * kTcBLbo / 16u; i += kTcThreads)
             reinterpret_cast<uint4*>(S.Bop)[i] = make_uint4(0u, 0u, 0u, 0u);
-        for (uint32_t i = tid; i < kVocab * kTcH; i += kTcThreads)
-            (&S.oW[0][0])[i] = bf16_round(p[2 * cell + i]);
-        if (tid < kVocab) S.ob[tid] = p[2 * cell + kVocab * kTcH + tid];
+        for (uint32_t i = tid; i < kVocab * 16u; i += kTcThreads) {       // (token, K group) -> 8 weights
+            const uint32_t o = i >> 4, kb = i & 15u;
+            const float4* src = reinterpret_cast<const float4*>(p + 2u * kTcCellFloats + o * kTcH + kb * 8u);
+            const float4 w0 = __ldg(src), w1 = __ldg(src + 1);
+            float* dst = S.oW[kb][o];
+            dst[0] = bf16_round(w0.x); dst[1] = bf16_round(w0.y); dst[2] = bf16_round(w0.z); dst[3] = bf16_round(w0.w);
+            dst[4] = bf16_round(w1.x); dst[5] = bf16_round(w1.y); dst[6] = bf16_round(w1.z); dst[7] = bf16_round(w1.w);
+        }
+        if (tid < kVocab) S.ob[tid] = p[2u * kTcCellFloats + kVocab * kTcH + tid];
         s2s_stage_weights(S, p, tid);
         __syncthreads();                                        // tokens are there
         if (tid < kTcQ) s2s_write_onehot(S, tid, S.enc[tid][0]);
@@ -356,42 +406,46 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
             if (phase) {
                 // every MMA of the encoder has been waited for by an epilogue warp: A may be replaced
                 __syncthreads();
-                s2s_stage_weights(S, p + cell, tid);
+                s2s_stage_weights(S, p + kTcCellFloats, tid);
                 fence_async_smem();
                 __syncthreads();
-            }
-            if (warp == kTcEpiThreads / 32) {
-                // ================= MMA warp ============================================================
-                if (lane == 0) {
-                    constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
-                    const uint32_t a_base = smem_u32(S.A), b_base = smem_u32(S.Bop);
-                    for (uint32_t t = t0; t < t1; ++t)
-#pragma unroll
-                        for (uint32_t x = 0; x < 2u; ++x) {
-                            if (t > 0) {                         // step 0 reads the state the setup wrote
-                                uint32_t& n_ready = x ? n_ready1 : n_ready0;
-                                wait_or_abort(&S.abort, &S.hready[x], n_ready & 1u, status);
-                                ++n_ready;
-                            }
-                            tc_fence_after();
-#pragma unroll
-                            for (uint32_t g = 0; g < 4u; ++g)
-#pragma unroll
-                                for (uint32_t kk = 0; kk < kTcKBlocks / 2; ++kk) {
-                                    const uint64_t ad = umma_smem_desc(a_base + 2u * kk * kTcALbo + g * 16u * 128u, kTcALbo, 128u);
-                                    const uint64_t bd = umma_smem_desc(b_base + 2u * kk * kTcBLbo + x * 8u * 128u, kTcBLbo, 128u);
-                                    umma_bf16(tmem + x * 256u + g * 64u, ad, bd, idesc, kk);
-                                }
-                            umma_commit(smem_u32(&S.full[x]));
-                        }
+                if (is_mma && item + gridDim.x < n_items) {     // the next item's encoder cell
+                    const uint32_t nm = (item + gridDim.x) / a.n_chunks;
+                    const char* next = reinterpret_cast<const char*>(a.theta + static_cast<size_t>(nm) * a.ldD);
+                    constexpr uint32_t piece = kTcCellFloats * 4u / 64u;
+                    prefetch_l2(next + ((warp - kTcEpiThreads / 32) * 32u + lane) * piece, piece);
                 }
-                __syncwarp();
+            }
+            if (is_mma) {
+                // ================= MMA warp of one half (the whole warp walks the loop) ================
+                constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
+                const uint32_t a_base = smem_u32(S.A), b_base = smem_u32(S.Bop) + half * 8u * 128u;
+                const uint32_t d_base = tmem + half * 256u;
+                for (uint32_t t = t0; t < t1; ++t) {
+                    if (t > 0) {                                 // step 0 reads the state the setup wrote
+                        wait_or_abort(&S.abort, &S.hready[half], n_wait & 1u, status);
+                        ++n_wait;
+                    }
+                    tc_fence_after();
+                    if (elect_one()) {
+#pragma unroll
+                        for (uint32_t g = 0; g < 4u; ++g)
+#pragma unroll
+                            for (uint32_t kk = 0; kk < kTcKBlocks / 2; ++kk) {
+                                const uint64_t ad = umma_smem_desc(a_base + 2u * kk * kTcALbo + g * 16u * 128u, kTcALbo, 128u);
+                                const uint64_t bd = umma_smem_desc(b_base + 2u * kk * kTcBLbo, kTcBLbo, 128u);
+                                umma_bf16(d_base + g * 64u, ad, bd, idesc, kk);
+                            }
+                        umma_commit(smem_u32(&S.full[half]));
+                    }
+                    __syncwarp();
+                }
             } else {
                 // ================= epilogue warps ======================================================
                 const uint32_t tq = tmem + (static_cast<uint32_t>((warp & 3u) * 32u) << 16) + half * 256u;
                 for (uint32_t t = t0; t < t1; ++t) {
-                    wait_or_abort(&S.abort, &S.full[half], n_full & 1u, status);
-                    ++n_full;
+                    wait_or_abort(&S.abort, &S.full[half], n_wait & 1u, status);
+                    ++n_wait;
                     tc_fence_after();
 #pragma unroll
                     for (uint32_t ch = 0; ch < 4u; ++ch) {
@@ -404,24 +458,20 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                         // hidden unit r of query n sits at K group r/8, row n, element r%8
                         unsigned char* dst = S.Bop + (r >> 3) * kTcBLbo + (half * 64u + ch * 16u) * 16u + (r & 7u) * 2u;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            float hv;
-                            if (SFU_TANH) {
-                                const float ig = fmaf(0.5f, tanh_sfu(0.5f * __uint_as_float(gi[j])), 0.5f);
-                                const float fg = fmaf(0.5f, tanh_sfu(0.5f * __uint_as_float(gf[j])), 0.5f);
-                                const float cg = tanh_sfu(__uint_as_float(gg[j]));
-                                const float og = fmaf(0.5f, tanh_sfu(0.5f * __uint_as_float(go[j])), 0.5f);
-                                c[ch * 16 + j] = fmaf(fg, c[ch * 16 + j], ig * cg);
-                                hv = og * tanh_sfu(c[ch * 16 + j]);
-                            } else {
-                                const float ig = sigmoid_ex2(__uint_as_float(gi[j]));
-                                const float fg = sigmoid_ex2(__uint_as_float(gf[j]));
-                                const float cg = tanh_ex2(__uint_as_float(gg[j]));
-                                const float og = sigmoid_ex2(__uint_as_float(go[j]));
-                                c[ch * 16 + j] = fmaf(fg, c[ch * 16 + j], ig * cg);
-                                hv = og * tanh_ex2(c[ch * 16 + j]);
-                            }
-                            *reinterpret_cast<__nv_bfloat16*>(dst + j * 16) = __float2bfloat16_rn(hv);
+                        for (int j = 0; j < 16; j += 2) {
+                            // the accumulators of the i, f, o gates already hold x / 2
+                            const float2 ig = unpack_h2(half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(gi[j]), __uint_as_float(gi[j + 1])))));
+                            const float2 fg = unpack_h2(half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(gf[j]), __uint_as_float(gf[j + 1])))));
+                            const float2 cg = unpack_h2(tanh_h2(pack_h2(__uint_as_float(gg[j]), __uint_as_float(gg[j + 1]))));
+                            const uint32_t og = half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(go[j]), __uint_as_float(go[j + 1]))));
+                            float& c0 = c[ch * 16 + j];
+                            float& c1 = c[ch * 16 + j + 1];
+                            c0 = fmaf(fg.x, c0, ig.x * cg.x);
+                            c1 = fmaf(fg.y, c1, ig.y * cg.y);
+                            const float2 hv = unpack_h2(mul_h2(og, tanh_h2(pack_h2(c0, c1))));
+                            const uint32_t hb = pack_bf16(hv.x, hv.y);
+                            *reinterpret_cast<uint16_t*>(dst + j * 16) = static_cast<uint16_t>(hb & 0xFFFFu);
+                            *reinterpret_cast<uint16_t*>(dst + j * 16 + 16) = static_cast<uint16_t>(hb >> 16);
                         }
                     }
                     // the coming step's token (none after the last step)
@@ -432,29 +482,35 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                     fence_async_smem();
                     tc_fence_before();
                     if (t >= Te) {
-                        // read-out on the CUDA cores from the state just written; the half's four warps
-                        // must all have written it
+                        // read-out on the CUDA cores from the state just written (all four warps of the
+                        // half must have written it), while the tensor cores work on the next step
                         half_barrier(half);
                         if (t + 1u < T && lane == 0) mbar_arrive(smem_u32(&S.hready[half]));
                         const uint32_t s = r & 63u, o0 = (r >> 6) * 6u;
-                        float acc[6] = { 0.f, 0.f, 0.f, 0.f, 0.f, 0.f };
+                        float2 acc[6];
+#pragma unroll
+                        for (int o = 0; o < 6; ++o) acc[o] = make_float2(0.f, 0.f);
                         const unsigned char* hrow = S.Bop + (half * 64u + s) * 16u;
-#pragma unroll 4
+#pragma unroll 2
                         for (uint32_t kb = 0; kb < 16u; ++kb) {
                             const uint4 hv = *reinterpret_cast<const uint4*>(hrow + kb * kTcBLbo);
                             const uint32_t hw[4] = { hv.x, hv.y, hv.z, hv.w };
+                            float2 x[4];
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const float x0 = __uint_as_float(hw[i] << 16), x1 = __uint_as_float(hw[i] & 0xFFFF0000u);
+                            for (int i = 0; i < 4; ++i)
+                                x[i] = make_float2(__uint_as_float(hw[i] << 16), __uint_as_float(hw[i] & 0xFFFF0000u));
 #pragma unroll
-                                for (int o = 0; o < 6; ++o) {
-                                    acc[o] = fmaf(S.oW[o0 + o][kb * 8u + 2 * i], x0, acc[o]);
-                                    acc[o] = fmaf(S.oW[o0 + o][kb * 8u + 2 * i + 1], x1, acc[o]);
-                                }
+                            for (int o = 0; o < 6; ++o) {
+                                const float4 w0 = *reinterpret_cast<const float4*>(&S.oW[kb][o0 + o][0]);
+                                const float4 w1 = *reinterpret_cast<const float4*>(&S.oW[kb][o0 + o][4]);
+                                ffma2(acc[o], make_float2(w0.x, w0.y), x[0]);
+                                ffma2(acc[o], make_float2(w0.z, w0.w), x[1]);
+                                ffma2(acc[o], make_float2(w1.x, w1.y), x[2]);
+                                ffma2(acc[o], make_float2(w1.z, w1.w), x[3]);
                             }
                         }
 #pragma unroll
-                        for (int o = 0; o < 6; ++o) S.lg[half][s][o0 + o] = acc[o] + S.ob[o0 + o];
+                        for (int o = 0; o < 6; ++o) S.lg[half][s][o0 + o] = (acc[o].x + acc[o].y) + S.ob[o0 + o];
                         half_barrier(half);
                         if (r < 64u && half * 64u + r < nq)
                             loss += token_loss(S.lg[half][r], S.tgt[half * 64u + r][t - Te]);
@@ -525,11 +581,11 @@ int launch_rollout_s2s(cudaStream_t st, const float* theta, uint32_t ldD, uint32
             if (cudaGetDevice(&dev) != cudaSuccess) return -1;
             if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
         }
-        if (cudaFuncSetAttribute(k_s2s_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(k_s2s_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(sizeof(S2sSmem))) != cudaSuccess) return -1;
         const uint32_t items = P * a.n_chunks;
         const uint32_t grid = items < static_cast<uint32_t>(sm_count) ? items : static_cast<uint32_t>(sm_count);
-        k_s2s_tc<false><<<grid, kTcThreads, sizeof(S2sSmem), st>>>(a, status);
+        k_s2s_tc<<<grid, kTcThreads, sizeof(S2sSmem), st>>>(a, status);
     } else {
         dim3 grid(P, a.n_chunks);
         k_s2s_simple<<<grid, 128, 0, st>>>(a);
