@@ -194,7 +194,7 @@ __global__ void k_s2s_finalize(const float* __restrict__ partial, uint32_t P, ui
 constexpr int kTcH = 128;
 constexpr int kTcQ = 128;                                  // queries per block: two halves of 64
 constexpr int kTcEpiThreads = 256;                         // warps 0-3: half 0, warps 4-7: half 1
-constexpr int kTcThreads = kTcEpiThreads + 64;             // + one MMA warp per half
+constexpr int kTcThreads = kTcEpiThreads + 32;             // + the MMA warp
 constexpr int kTcKBlocks = 18;                             // K = 128 (h) + 16 (one-hot, 1, padding) in groups of 8
 constexpr uint32_t kTcALbo = 64 * 128;                     // 64 row groups of 8 x 16 bytes between K groups
 constexpr uint32_t kTcBLbo = 16 * 128 + 16;                // 16 row groups, +16 bytes so that the 2-byte stores
@@ -208,9 +208,9 @@ struct __align__(128) S2sSmem {
     unsigned char Bop[kTcBBytes];                          // [h; onehot; 1; 0] of the 128 queries
     float oW[16][kVocab][8];                               // read-out weights [K group][token][k], bf16-rounded
     float ob[kVocab];
-    float lg[2][64][kVocab + 1];
+    float lg[kS2sMaxTd][kTcQ][kVocab];                     // logits of every answer position
     uint8_t enc[kTcQ][kS2sMaxTe + 1], dec[kTcQ][kS2sMaxTd + 1], tgt[kTcQ][kS2sMaxTd + 1];
-    float loss_w[8];
+    float loss_w[kTcThreads / 32];
     uint64_t full[2];                                      // the gates of a half are in TMEM
     uint64_t hready[2];                                    // a half's B operand holds the next step's input
     uint32_t tmem_slot;
@@ -275,7 +275,10 @@ __device__ __forceinline__ void s2s_stage_weights(S2sSmem& S, const float* __res
     const float* Wx = cellp;
     const float* Wh = Wx + 4 * kTcH * kVocab;
     const float* bb = Wh + 4 * kTcH * kTcH;
-    // Wh: 512 rows x 16 K groups; a thread converts 8 consecutive k of one row into one 16-byte row
+    // Wh: 512 rows x 16 K groups; a thread converts 8 consecutive k of one row into one 16-byte row.
+    // Within a warp the 8 lanes of a quarter take the 8 rows of a row group (so the 16-byte stores
+    // of a quarter-warp fall in distinct banks) and the 4 quarters take 4 adjacent K groups (so a
+    // load instruction touches one 128-byte line per row).
     constexpr uint32_t n_items = 512u * 16u;
     constexpr int U = 8;
 #pragma unroll 1
@@ -284,7 +287,7 @@ __device__ __forceinline__ void s2s_stage_weights(S2sSmem& S, const float* __res
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const uint32_t idx = min(base + u * kTcThreads, n_items - 1u);
-            const uint32_t m = idx & 511u, kb = idx >> 9;
+            const uint32_t m = (idx >> 7) * 8u + (idx & 7u), kb = ((idx >> 5) & 3u) * 4u + ((idx >> 3) & 3u);
             const float4* src = reinterpret_cast<const float4*>(Wh + m * kTcH + kb * 8u);
             v[u][0] = __ldg(src); v[u][1] = __ldg(src + 1);
         }
@@ -292,7 +295,7 @@ __device__ __forceinline__ void s2s_stage_weights(S2sSmem& S, const float* __res
         for (int u = 0; u < U; ++u) {
             const uint32_t idx = base + u * kTcThreads;
             if (idx < n_items) {
-                const uint32_t m = idx & 511u, kb = idx >> 9;
+                const uint32_t m = (idx >> 7) * 8u + (idx & 7u), kb = ((idx >> 5) & 3u) * 4u + ((idx >> 3) & 3u);
                 const float sc = ((m >> 7) == 2u) ? 1.0f : 0.5f;
                 *reinterpret_cast<uint4*>(S.A + kb * kTcALbo + (m >> 3) * 128u + (m & 7u) * 16u) =
                     make_uint4(pack_bf16(sc * v[u][0].x, sc * v[u][0].y), pack_bf16(sc * v[u][0].z, sc * v[u][0].w),
@@ -357,9 +360,9 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
     tc_fence_after();
     const uint32_t tmem = S.tmem_slot;
 
-    uint32_t n_wait = 0u;                      // completed waits: full[half] (epilogue) / hready[x] (MMA warp)
+    uint32_t n_wait = 0u, n_wait1 = 0u;        // completed waits: full[half] (epilogue) / hready[0], hready[1] (MMA warp)
     const bool is_mma = warp >= kTcEpiThreads / 32;
-    const uint32_t half = is_mma ? warp - kTcEpiThreads / 32 : warp >> 2;   // which 64 queries this warp serves
+    const uint32_t half = (warp >> 2) & 1u;    // epilogue warps: which 64 queries
     const uint32_t r = tid & 127u;             // epilogue thread: hidden unit = TMEM lane
     uint32_t staged_chunk = 0xFFFFFFFFu;
 
@@ -376,8 +379,8 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
         }
         if (is_mma) {                                            // the decoder's weights will be wanted next
             const char* next = reinterpret_cast<const char*>(p + kTcCellFloats);
-            constexpr uint32_t piece = kTcCellFloats * 4u / 64u;       // 4,512 bytes per lane of the two warps
-            prefetch_l2(next + ((warp - kTcEpiThreads / 32) * 32u + lane) * piece, piece);
+            constexpr uint32_t piece = kTcCellFloats * 4u / 32u;       // 9,024 bytes per lane
+            prefetch_l2(next + lane * piece, piece);
         }
         for (uint32_t i = tid; i < 16u * kTcBLbo / 16u; i += kTcThreads)
             reinterpret_cast<uint4*>(S.Bop)[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -412,33 +415,38 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                 if (is_mma && item + gridDim.x < n_items) {     // the next item's encoder cell
                     const uint32_t nm = (item + gridDim.x) / a.n_chunks;
                     const char* next = reinterpret_cast<const char*>(a.theta + static_cast<size_t>(nm) * a.ldD);
-                    constexpr uint32_t piece = kTcCellFloats * 4u / 64u;
-                    prefetch_l2(next + ((warp - kTcEpiThreads / 32) * 32u + lane) * piece, piece);
+                    constexpr uint32_t piece = kTcCellFloats * 4u / 32u;
+                    prefetch_l2(next + lane * piece, piece);
                 }
             }
             if (is_mma) {
-                // ================= MMA warp of one half (the whole warp walks the loop) ================
+                // ================= MMA warp (the whole warp walks the loop, one lane issues) ===========
+                // The halves alternate, so that one half's MMAs run while the other half's gates are
+                // being applied.
                 constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
-                const uint32_t a_base = smem_u32(S.A), b_base = smem_u32(S.Bop) + half * 8u * 128u;
-                const uint32_t d_base = tmem + half * 256u;
+                const uint32_t a_base = smem_u32(S.A), b_base = smem_u32(S.Bop);
                 for (uint32_t t = t0; t < t1; ++t) {
-                    if (t > 0) {                                 // step 0 reads the state the setup wrote
-                        wait_or_abort(&S.abort, &S.hready[half], n_wait & 1u, status);
-                        ++n_wait;
-                    }
-                    tc_fence_after();
-                    if (elect_one()) {
 #pragma unroll
-                        for (uint32_t g = 0; g < 4u; ++g)
+                    for (uint32_t x = 0; x < 2u; ++x) {
+                        if (t > 0) {                             // step 0 reads the state the setup wrote
+                            uint32_t& n = x ? n_wait1 : n_wait;
+                            wait_or_abort(&S.abort, &S.hready[x], n & 1u, status);
+                            ++n;
+                        }
+                        tc_fence_after();
+                        if (elect_one()) {
 #pragma unroll
-                            for (uint32_t kk = 0; kk < kTcKBlocks / 2; ++kk) {
-                                const uint64_t ad = umma_smem_desc(a_base + 2u * kk * kTcALbo + g * 16u * 128u, kTcALbo, 128u);
-                                const uint64_t bd = umma_smem_desc(b_base + 2u * kk * kTcBLbo, kTcBLbo, 128u);
-                                umma_bf16(d_base + g * 64u, ad, bd, idesc, kk);
-                            }
-                        umma_commit(smem_u32(&S.full[half]));
+                            for (uint32_t g = 0; g < 4u; ++g)
+#pragma unroll
+                                for (uint32_t kk = 0; kk < kTcKBlocks / 2; ++kk) {
+                                    const uint64_t ad = umma_smem_desc(a_base + 2u * kk * kTcALbo + g * 16u * 128u, kTcALbo, 128u);
+                                    const uint64_t bd = umma_smem_desc(b_base + 2u * kk * kTcBLbo + x * 8u * 128u, kTcBLbo, 128u);
+                                    umma_bf16(tmem + x * 256u + g * 64u, ad, bd, idesc, kk);
+                                }
+                            umma_commit(smem_u32(&S.full[x]));
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
                 }
             } else {
                 // ================= epilogue warps ======================================================
@@ -447,25 +455,32 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                     wait_or_abort(&S.abort, &S.full[half], n_wait & 1u, status);
                     ++n_wait;
                     tc_fence_after();
+                    // 8 chunks of 8 queries; the loads of the next chunk are in flight while this one
+                    // is worked on (two register sets)
+                    uint32_t g0[2][8], g1[2][8], g2[2][8], g3[2][8];
+                    tmem_ld8_issue(tq + 0u * 64u, g0[0]); tmem_ld8_issue(tq + 1u * 64u, g1[0]);
+                    tmem_ld8_issue(tq + 2u * 64u, g2[0]); tmem_ld8_issue(tq + 3u * 64u, g3[0]);
+                    tmem_ld8x4_fence(g0[0], g1[0], g2[0], g3[0]);
 #pragma unroll
-                    for (uint32_t ch = 0; ch < 4u; ++ch) {
-                        uint32_t gi[16], gf[16], gg[16], go[16];
-                        tmem_ld16_issue(tq + 0u * 64u + ch * 16u, gi);
-                        tmem_ld16_issue(tq + 1u * 64u + ch * 16u, gf);
-                        tmem_ld16_issue(tq + 2u * 64u + ch * 16u, gg);
-                        tmem_ld16_issue(tq + 3u * 64u + ch * 16u, go);
-                        tmem_ld16_fence(gi); tmem_ld16_fence(gf); tmem_ld16_fence(gg); tmem_ld16_fence(go);
+                    for (uint32_t ch = 0; ch < 8u; ++ch) {
+                        const uint32_t cur = ch & 1u, nxt = cur ^ 1u;
+                        if (ch + 1u < 8u) {
+                            tmem_ld8_issue(tq + 0u * 64u + (ch + 1u) * 8u, g0[nxt]);
+                            tmem_ld8_issue(tq + 1u * 64u + (ch + 1u) * 8u, g1[nxt]);
+                            tmem_ld8_issue(tq + 2u * 64u + (ch + 1u) * 8u, g2[nxt]);
+                            tmem_ld8_issue(tq + 3u * 64u + (ch + 1u) * 8u, g3[nxt]);
+                        }
                         // hidden unit r of query n sits at K group r/8, row n, element r%8
-                        unsigned char* dst = S.Bop + (r >> 3) * kTcBLbo + (half * 64u + ch * 16u) * 16u + (r & 7u) * 2u;
+                        unsigned char* dst = S.Bop + (r >> 3) * kTcBLbo + (half * 64u + ch * 8u) * 16u + (r & 7u) * 2u;
 #pragma unroll
-                        for (int j = 0; j < 16; j += 2) {
+                        for (int j = 0; j < 8; j += 2) {
                             // the accumulators of the i, f, o gates already hold x / 2
-                            const float2 ig = unpack_h2(half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(gi[j]), __uint_as_float(gi[j + 1])))));
-                            const float2 fg = unpack_h2(half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(gf[j]), __uint_as_float(gf[j + 1])))));
-                            const float2 cg = unpack_h2(tanh_h2(pack_h2(__uint_as_float(gg[j]), __uint_as_float(gg[j + 1]))));
-                            const uint32_t og = half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(go[j]), __uint_as_float(go[j + 1]))));
-                            float& c0 = c[ch * 16 + j];
-                            float& c1 = c[ch * 16 + j + 1];
+                            const float2 ig = unpack_h2(half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(g0[cur][j]), __uint_as_float(g0[cur][j + 1])))));
+                            const float2 fg = unpack_h2(half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(g1[cur][j]), __uint_as_float(g1[cur][j + 1])))));
+                            const float2 cg = unpack_h2(tanh_h2(pack_h2(__uint_as_float(g2[cur][j]), __uint_as_float(g2[cur][j + 1]))));
+                            const uint32_t og = half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(g3[cur][j]), __uint_as_float(g3[cur][j + 1]))));
+                            float& c0 = c[ch * 8 + j];
+                            float& c1 = c[ch * 8 + j + 1];
                             c0 = fmaf(fg.x, c0, ig.x * cg.x);
                             c1 = fmaf(fg.y, c1, ig.y * cg.y);
                             const float2 hv = unpack_h2(mul_h2(og, tanh_h2(pack_h2(c0, c1))));
@@ -473,6 +488,7 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                             *reinterpret_cast<uint16_t*>(dst + j * 16) = static_cast<uint16_t>(hb & 0xFFFFu);
                             *reinterpret_cast<uint16_t*>(dst + j * 16 + 16) = static_cast<uint16_t>(hb >> 16);
                         }
+                        if (ch + 1u < 8u) tmem_ld8x4_fence(g0[nxt], g1[nxt], g2[nxt], g3[nxt]);
                     }
                     // the coming step's token (none after the last step)
                     if (t + 1u < T && r < 64u) {
@@ -491,7 +507,7 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
 #pragma unroll
                         for (int o = 0; o < 6; ++o) acc[o] = make_float2(0.f, 0.f);
                         const unsigned char* hrow = S.Bop + (half * 64u + s) * 16u;
-#pragma unroll 2
+#pragma unroll 4
                         for (uint32_t kb = 0; kb < 16u; ++kb) {
                             const uint4 hv = *reinterpret_cast<const uint4*>(hrow + kb * kTcBLbo);
                             const uint32_t hw[4] = { hv.x, hv.y, hv.z, hv.w };
@@ -510,10 +526,7 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                             }
                         }
 #pragma unroll
-                        for (int o = 0; o < 6; ++o) S.lg[half][s][o0 + o] = (acc[o].x + acc[o].y) + S.ob[o0 + o];
-                        half_barrier(half);
-                        if (r < 64u && half * 64u + r < nq)
-                            loss += token_loss(S.lg[half][r], S.tgt[half * 64u + r][t - Te]);
+                        for (int o = 0; o < 6; ++o) S.lg[t - Te][half * 64u + s][o0 + o] = (acc[o].x + acc[o].y) + S.ob[o0 + o];
                         // the next epilogue overwrites the state: everyone must be done reading it
                         half_barrier(half);
                     } else {
@@ -523,14 +536,21 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                 }
             }
         }
-        // ---- the item's loss: fixed-order sum over the 4 warps that hold query losses -----------
+        // ---- the item's loss: cross-entropy of every (position, query), summed in a fixed order ----
+        __syncthreads();
+        for (uint32_t idx = tid; idx < Td * kTcQ; idx += kTcThreads) {
+            const uint32_t pos = idx / kTcQ, q = idx % kTcQ;
+            if (q < nq) loss += token_loss(S.lg[pos][q], S.tgt[q][pos]);
+        }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, off);
-        if (warp < 8u && lane == 0) S.loss_w[warp] = loss;
+        if (lane == 0) S.loss_w[warp] = loss;
         __syncthreads();
-        if (tid == 0)
-            a.partial[static_cast<size_t>(member) * a.n_chunks + chunk] =
-                (S.loss_w[0] + S.loss_w[1]) + (S.loss_w[4] + S.loss_w[5]);
+        if (tid == 0) {
+            float total = 0.f;
+            for (int w = 0; w < kTcThreads / 32; ++w) total += S.loss_w[w];
+            a.partial[static_cast<size_t>(member) * a.n_chunks + chunk] = total;
+        }
         __syncthreads();
     }
 
