@@ -10,19 +10,25 @@
 // read-out out.W . h likewise.
 //
 //   k_s2s_simple  CUDA cores, one block per (member, 16 queries): the plain version.
-//   k_s2s_tc      tcgen05: one block per (member, 128 queries).  The member's [4h = 512] x [K = 144]
-//                 weight tile (bf16) stays in shared memory for a whole phase; the B operand is the
-//                 hidden state of the 128 queries plus their one-hot token and a constant 1, so
-//                 one chain of 9 MMAs per gate produces the complete pre-activation in TMEM.  The
-//                 queries are split into two halves of 64 whose steps alternate: while the
-//                 epilogue warps of one half apply the gate non-linearities and write the new
-//                 hidden state back into the B operand, the tensor cores work on the other half.
-//                 TMEM: 2 halves x 4 gates x 64 columns = 512.
+//   k_s2s_tc      tcgen05, one block per (member, 128 queries), one block per SM.  The member's
+//                 [4h = 512] x [K = 144] weight tile (bf16, 144 KB) stays in shared memory for a
+//                 whole phase (encoder, then decoder); the B operand is the hidden state of the 128
+//                 queries plus their one-hot token and a constant 1, so one chain of 9 MMAs per gate
+//                 produces the complete pre-activation in TMEM (2 halves x 4 gates x 64 columns =
+//                 all 512 columns).  The queries are two halves of 64 whose steps alternate: while
+//                 the epilogue warps of one half apply the gate non-linearities (thread = hidden
+//                 unit = TMEM lane, cell state in registers) and write the new hidden state straight
+//                 back into the B operand, the tensor cores work on the other half.  The rows of the
+//                 sigmoid gates are halved when staged, so every non-linearity is one tanh of the
+//                 special-function unit; that unit (5 tanh per cell and step) is what bounds the
+//                 kernel, not the tensor cores.  The decoder's read-out runs on the CUDA cores from
+//                 the B operand while the next step's MMAs are in flight; its logits are kept and
+//                 the cross-entropy is taken once per item.  The next cell's weights are prefetched
+//                 into L2 while the current phase computes.  Every wait is bounded.
 #include "internal.h"
 #include "async.cuh"
 #include "noise.cuh"
 #include "umma.cuh"
-#include <cuda_fp16.h>
 
 namespace evo {
 
@@ -193,7 +199,11 @@ __global__ void k_s2s_finalize(const float* __restrict__ partial, uint32_t P, ui
 // ------------------------------------------------------------------------------------------
 constexpr int kTcH = 128;
 constexpr int kTcQ = 128;                                  // queries per block: two halves of 64
-constexpr int kTcEpiThreads = 256;                         // warps 0-3: half 0, warps 4-7: half 1
+constexpr int kTcSub = 1;                                  // warps per TMEM lane quarter and half: each takes 64 / kTcSub queries
+constexpr int kTcHalfThreads = 128 * kTcSub;
+constexpr int kTcEpiThreads = 2 * kTcHalfThreads;          // half 0's warps first, then half 1's
+constexpr int kTcCols = 64 / kTcSub;                       // queries per epilogue thread
+constexpr int kTcOutPerThread = kVocab * 64 / kTcHalfThreads;   // read-out: tokens per thread
 constexpr int kTcThreads = kTcEpiThreads + 32;             // + the MMA warp
 constexpr int kTcKBlocks = 18;                             // K = 128 (h) + 16 (one-hot, 1, padding) in groups of 8
 constexpr uint32_t kTcALbo = 64 * 128;                     // 64 row groups of 8 x 16 bytes between K groups
@@ -217,35 +227,10 @@ struct __align__(128) S2sSmem {
     volatile int abort;
 };
 
-// two tanh at once on the special-function unit, in and out as packed fp16 (relative error 2^-11,
-// the same class as the fp32 approximation)
-__device__ __forceinline__ uint32_t tanh_h2(uint32_t x)
+__device__ __forceinline__ float tanh_sfu(float x)
 {
-    uint32_t y;
-    asm("tanh.approx.f16x2 %0, %1;" : "=r"(y) : "r"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_h2(float lo, float hi)
-{
-    uint32_t y;
-    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(y) : "f"(hi), "f"(lo));
-    return y;
-}
-__device__ __forceinline__ float2 unpack_h2(uint32_t v)
-{
-    return __half22float2(*reinterpret_cast<const __half2*>(&v));
-}
-// 0.5 t + 0.5 on both halves: sigma(x) from t = tanh(x / 2)
-__device__ __forceinline__ uint32_t half_plus_half_h2(uint32_t t)
-{
-    uint32_t y;
-    asm("fma.rn.f16x2 %0, %1, %2, %2;" : "=r"(y) : "r"(t), "r"(0x38003800u));
-    return y;
-}
-__device__ __forceinline__ uint32_t mul_h2(uint32_t a, uint32_t b)
-{
-    uint32_t y;
-    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(y) : "r"(a), "r"(b));
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 // two fp32 fused multiply-adds in one instruction
@@ -332,8 +317,8 @@ __device__ __forceinline__ void s2s_write_onehot(S2sSmem& S, uint32_t n, uint32_
 // barrier over the four epilogue warps of one half
 __device__ __forceinline__ void half_barrier(uint32_t half)
 {
-    if (half) asm volatile("bar.sync 2, 128;" ::: "memory");
-    else      asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (half) asm volatile("bar.sync 2, %0;" :: "n"(kTcHalfThreads) : "memory");
+    else      asm volatile("bar.sync 1, %0;" :: "n"(kTcHalfThreads) : "memory");
 }
 
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -348,7 +333,7 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
 
     if (tid == 0) {
         mbar_init(smem_u32(&S.full[0]), 1); mbar_init(smem_u32(&S.full[1]), 1);
-        mbar_init(smem_u32(&S.hready[0]), 4); mbar_init(smem_u32(&S.hready[1]), 4);
+        mbar_init(smem_u32(&S.hready[0]), kTcHalfThreads / 32); mbar_init(smem_u32(&S.hready[1]), kTcHalfThreads / 32);
         S.abort = 0;
         mbar_init_fence();
     }
@@ -362,7 +347,8 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
 
     uint32_t n_wait = 0u, n_wait1 = 0u;        // completed waits: full[half] (epilogue) / hready[0], hready[1] (MMA warp)
     const bool is_mma = warp >= kTcEpiThreads / 32;
-    const uint32_t half = (warp >> 2) & 1u;    // epilogue warps: which 64 queries
+    const uint32_t half = (tid / kTcHalfThreads) & 1u;          // epilogue warps: which 64 queries
+    const uint32_t sub = (tid % kTcHalfThreads) >> 7;           // ... and which kTcCols of them
     const uint32_t r = tid & 127u;             // epilogue thread: hidden unit = TMEM lane
     uint32_t staged_chunk = 0xFFFFFFFFu;
 
@@ -399,9 +385,9 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
         fence_async_smem();
         __syncthreads();
 
-        float c[64];
+        float c[kTcCols];
 #pragma unroll
-        for (int i = 0; i < 64; ++i) c[i] = 0.f;
+        for (int i = 0; i < kTcCols; ++i) c[i] = 0.f;
         float loss = 0.f;
 
         for (uint32_t phase = 0; phase < 2u; ++phase) {
@@ -450,62 +436,72 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                 }
             } else {
                 // ================= epilogue warps ======================================================
-                const uint32_t tq = tmem + (static_cast<uint32_t>((warp & 3u) * 32u) << 16) + half * 256u;
+                const uint32_t tq = tmem + (static_cast<uint32_t>((warp & 3u) * 32u) << 16) + half * 256u + sub * kTcCols;
                 for (uint32_t t = t0; t < t1; ++t) {
                     wait_or_abort(&S.abort, &S.full[half], n_wait & 1u, status);
                     ++n_wait;
                     tc_fence_after();
-                    // 8 chunks of 8 queries; the loads of the next chunk are in flight while this one
+                    // chunks of 8 queries; the loads of the next chunk are in flight while this one
                     // is worked on (two register sets)
                     uint32_t g0[2][8], g1[2][8], g2[2][8], g3[2][8];
                     tmem_ld8_issue(tq + 0u * 64u, g0[0]); tmem_ld8_issue(tq + 1u * 64u, g1[0]);
                     tmem_ld8_issue(tq + 2u * 64u, g2[0]); tmem_ld8_issue(tq + 3u * 64u, g3[0]);
                     tmem_ld8x4_fence(g0[0], g1[0], g2[0], g3[0]);
 #pragma unroll
-                    for (uint32_t ch = 0; ch < 8u; ++ch) {
+                    for (uint32_t ch = 0; ch < kTcCols / 8u; ++ch) {
                         const uint32_t cur = ch & 1u, nxt = cur ^ 1u;
-                        if (ch + 1u < 8u) {
+                        if (ch + 1u < kTcCols / 8u) {
                             tmem_ld8_issue(tq + 0u * 64u + (ch + 1u) * 8u, g0[nxt]);
                             tmem_ld8_issue(tq + 1u * 64u + (ch + 1u) * 8u, g1[nxt]);
                             tmem_ld8_issue(tq + 2u * 64u + (ch + 1u) * 8u, g2[nxt]);
                             tmem_ld8_issue(tq + 3u * 64u + (ch + 1u) * 8u, g3[nxt]);
                         }
                         // hidden unit r of query n sits at K group r/8, row n, element r%8
-                        unsigned char* dst = S.Bop + (r >> 3) * kTcBLbo + (half * 64u + ch * 8u) * 16u + (r & 7u) * 2u;
+                        unsigned char* dst = S.Bop + (r >> 3) * kTcBLbo + (half * 64u + sub * kTcCols + ch * 8u) * 16u + (r & 7u) * 2u;
 #pragma unroll
                         for (int j = 0; j < 8; j += 2) {
                             // the accumulators of the i, f, o gates already hold x / 2
-                            const float2 ig = unpack_h2(half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(g0[cur][j]), __uint_as_float(g0[cur][j + 1])))));
-                            const float2 fg = unpack_h2(half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(g1[cur][j]), __uint_as_float(g1[cur][j + 1])))));
-                            const float2 cg = unpack_h2(tanh_h2(pack_h2(__uint_as_float(g2[cur][j]), __uint_as_float(g2[cur][j + 1]))));
-                            const uint32_t og = half_plus_half_h2(tanh_h2(pack_h2(__uint_as_float(g3[cur][j]), __uint_as_float(g3[cur][j + 1]))));
-                            float& c0 = c[ch * 8 + j];
-                            float& c1 = c[ch * 8 + j + 1];
-                            c0 = fmaf(fg.x, c0, ig.x * cg.x);
-                            c1 = fmaf(fg.y, c1, ig.y * cg.y);
-                            const float2 hv = unpack_h2(mul_h2(og, tanh_h2(pack_h2(c0, c1))));
+                            float2 hv;
+                            {
+                                const float ig = fmaf(0.5f, tanh_sfu(__uint_as_float(g0[cur][j])), 0.5f);
+                                const float fg = fmaf(0.5f, tanh_sfu(__uint_as_float(g1[cur][j])), 0.5f);
+                                const float cg = tanh_sfu(__uint_as_float(g2[cur][j]));
+                                const float og = fmaf(0.5f, tanh_sfu(__uint_as_float(g3[cur][j])), 0.5f);
+                                float& c0 = c[ch * 8 + j];
+                                c0 = fmaf(fg, c0, ig * cg);
+                                hv.x = og * tanh_sfu(c0);
+                            }
+                            {
+                                const float ig = fmaf(0.5f, tanh_sfu(__uint_as_float(g0[cur][j + 1])), 0.5f);
+                                const float fg = fmaf(0.5f, tanh_sfu(__uint_as_float(g1[cur][j + 1])), 0.5f);
+                                const float cg = tanh_sfu(__uint_as_float(g2[cur][j + 1]));
+                                const float og = fmaf(0.5f, tanh_sfu(__uint_as_float(g3[cur][j + 1])), 0.5f);
+                                float& c1 = c[ch * 8 + j + 1];
+                                c1 = fmaf(fg, c1, ig * cg);
+                                hv.y = og * tanh_sfu(c1);
+                            }
                             const uint32_t hb = pack_bf16(hv.x, hv.y);
                             *reinterpret_cast<uint16_t*>(dst + j * 16) = static_cast<uint16_t>(hb & 0xFFFFu);
                             *reinterpret_cast<uint16_t*>(dst + j * 16 + 16) = static_cast<uint16_t>(hb >> 16);
                         }
-                        if (ch + 1u < 8u) tmem_ld8x4_fence(g0[nxt], g1[nxt], g2[nxt], g3[nxt]);
+                        if (ch + 1u < kTcCols / 8u) tmem_ld8x4_fence(g0[nxt], g1[nxt], g2[nxt], g3[nxt]);
                     }
                     // the coming step's token (none after the last step)
-                    if (t + 1u < T && r < 64u) {
+                    if (t + 1u < T && sub == 0u && r < 64u) {
                         const uint32_t n = half * 64u + r;
                         s2s_write_onehot(S, n, (t + 1u < Te) ? S.enc[n][t + 1u] : S.dec[n][t + 1u - Te]);
                     }
                     fence_async_smem();
                     tc_fence_before();
                     if (t >= Te) {
-                        // read-out on the CUDA cores from the state just written (all four warps of the
+                        // read-out on the CUDA cores from the state just written (all warps of the
                         // half must have written it), while the tensor cores work on the next step
                         half_barrier(half);
                         if (t + 1u < T && lane == 0) mbar_arrive(smem_u32(&S.hready[half]));
-                        const uint32_t s = r & 63u, o0 = (r >> 6) * 6u;
-                        float2 acc[6];
+                        const uint32_t s = tid & 63u, o0 = ((tid % kTcHalfThreads) >> 6) * kTcOutPerThread;
+                        float2 acc[kTcOutPerThread];
 #pragma unroll
-                        for (int o = 0; o < 6; ++o) acc[o] = make_float2(0.f, 0.f);
+                        for (int o = 0; o < kTcOutPerThread; ++o) acc[o] = make_float2(0.f, 0.f);
                         const unsigned char* hrow = S.Bop + (half * 64u + s) * 16u;
 #pragma unroll 4
                         for (uint32_t kb = 0; kb < 16u; ++kb) {
@@ -516,7 +512,7 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                             for (int i = 0; i < 4; ++i)
                                 x[i] = make_float2(__uint_as_float(hw[i] << 16), __uint_as_float(hw[i] & 0xFFFF0000u));
 #pragma unroll
-                            for (int o = 0; o < 6; ++o) {
+                            for (int o = 0; o < kTcOutPerThread; ++o) {
                                 const float4 w0 = *reinterpret_cast<const float4*>(&S.oW[kb][o0 + o][0]);
                                 const float4 w1 = *reinterpret_cast<const float4*>(&S.oW[kb][o0 + o][4]);
                                 ffma2(acc[o], make_float2(w0.x, w0.y), x[0]);
@@ -526,7 +522,7 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
                             }
                         }
 #pragma unroll
-                        for (int o = 0; o < 6; ++o) S.lg[t - Te][half * 64u + s][o0 + o] = (acc[o].x + acc[o].y) + S.ob[o0 + o];
+                        for (int o = 0; o < kTcOutPerThread; ++o) S.lg[t - Te][half * 64u + s][o0 + o] = (acc[o].x + acc[o].y) + S.ob[o0 + o];
                         // the next epilogue overwrites the state: everyone must be done reading it
                         half_barrier(half);
                     } else {
