@@ -46,3 +46,13 @@ def test_cnn_cross_entropy_goes_down_on_a_fixed_batch():
     first, last = _improves(hist)
     assert last > first + 0.02, (first, last)                      # -loss rises from about -ln 10
     s.close()
+
+
+def test_seq2seq_cross_entropy_goes_down_from_log_vocab():
+    """One-digit addition with the LSTM encoder-decoder (tcgen05 kernel): from the zero centre
+    (fitness -ln 12) the population mean has to rise clearly within 60 generations."""
+    w = W.SEQ2SEQ.with_(pop_size=256, task_param=(1.0,), sigma=0.05, lr=0.02)
+    _, hist = run(w, 60)
+    assert abs(hist[0][0] + np.log(12)) < 0.02
+    assert hist[-1][0] > hist[0][0] + 0.4
+    assert hist[-1][0] > -1.9
