@@ -13,7 +13,7 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = ["rng.c", "solver.c", "policy.c", "tasks.c", "seq2seq.c"]
+_SRC = ["rng.c", "solver.c", "policy.c", "tasks.c", "seq2seq.c", "paint.c"]
 _LIB_PATH = os.path.join(_HERE, "liboracle.so")
 
 
@@ -82,6 +82,11 @@ def _declare(L):
     L.oracle_mlp_param_count.restype = C.c_uint32
     L.oracle_cnn_fitness.argtypes = [_f32p, _f32p, _i32p, C.c_uint32, C.c_int]
     L.oracle_cnn_fitness.restype = C.c_double
+    L.oracle_paint_inside.argtypes = [_f32p, C.c_float, C.c_float]
+    L.oracle_paint_inside.restype = C.c_int
+    L.oracle_paint_render.argtypes = [_f32p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_double, _f64p]
+    L.oracle_paint_fitness.argtypes = [_f32p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_double, _f32p, _f64p]
+    L.oracle_paint_fitness.restype = C.c_double
     L.oracle_seq2seq_param_count.argtypes = [C.c_uint32]
     L.oracle_seq2seq_param_count.restype = C.c_uint32
     L.oracle_seq2seq_queries.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, _i32p, _i32p, _i32p]
@@ -257,6 +262,27 @@ def cnn_logits(params, image, bf16_operands=True):
 
 
 def bf16_round(x): return float(lib().oracle_bf16_round(float(x)))
+
+
+def paint_inside(tri6, px, py):
+    t = _f32(tri6)
+    return bool(lib().oracle_paint_inside(_p(t, _f32p), float(px), float(py)))
+
+
+def paint_render(params, W, H, background=0.0):
+    """Canvas [H][W][3] (fp64) of the triangles in `params` ([N][10] raw numbers)."""
+    p = _f32(params).reshape(-1)
+    canvas = np.zeros((H, W, 3), np.float64)
+    lib().oracle_paint_render(_p(p, _f32p), p.size // 10, W, H, float(background), _p(canvas, _f64p))
+    return canvas
+
+
+def paint_fitness(params, W, H, target, background=0.0):
+    p = _f32(params).reshape(-1); t = _f32(target)
+    assert t.shape == (H, W, 3)
+    canvas = np.zeros((H, W, 3), np.float64)
+    return float(lib().oracle_paint_fitness(_p(p, _f32p), p.size // 10, W, H, float(background),
+                                            _p(t, _f32p), _p(canvas, _f64p)))
 
 
 def seq2seq_param_count(h): return int(lib().oracle_seq2seq_param_count(int(h)))

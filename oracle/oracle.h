@@ -29,7 +29,8 @@
  * momentum conservation, equilibria and small-angle period; tanh-linear recurrence
  * by hand; CNN against torch conv2d/max_pool2d/cross_entropy and the ln(10) case; the LSTM
  * seq2seq policy against torch.nn.LSTM + Linear + cross_entropy and the ln(12) case; its
- * queries against integer addition.
+ * queries against integer addition; the triangle painter against hand-counted coverage, closed-form
+ * blending, vertex-order invariance and a barycentric rasteriser.
  * Parity unpinned (conventions only, nothing external fixes them): counter/stream
  * layout of the random numbers, the sign order inside an antithetic pair, the
  * observation order, reward timing, flatten order of the CNN, token codes and teacher forcing
@@ -143,6 +144,14 @@ double oracle_seq2seq_fitness(const float* params, uint32_t h, uint32_t nd, uint
                               const int32_t* enc_tokens, const int32_t* dec_tokens,
                               const int32_t* targets, int bf16_operands, double* accuracy,
                               double* logits_out);
+
+/* Triangle painting (paper Section 3, "Concrete and Abstract Painting"); conventions in paint.c.
+ * params: n_triangles x (x0 y0 x1 y1 x2 y2 r g b a); canvas and target are [H][W][3]. */
+int  oracle_paint_inside(const float tri[6], float px, float py);
+void oracle_paint_render(const float* params, uint32_t n_triangles, uint32_t W, uint32_t H,
+                         double background, double* canvas);
+double oracle_paint_fitness(const float* params, uint32_t n_triangles, uint32_t W, uint32_t H,
+                            double background, const float* target, double* canvas /* scratch, output */);
 
 /* ---- tasks ---------------------------------------------------------------------- */
 
