@@ -13,9 +13,11 @@
  * Which pixels a triangle covers is an integer decision, so it is DEFINED in fp32, each step a
  * single correctly rounded operation: u = fmaf(0.5f, v, 0.5f) clamped; for an edge from a to b,
  * e(p) = (bx - ax) * (py - ay) - (by - ay) * (px - ax) with the two differences, the two products
- * and the final difference each rounded once; p is inside when the three edge values are all >= 0 or
- * all <= 0; a triangle whose own third vertex has edge value 0 (no area) paints nothing.  Colours
- * and compositing are plain real arithmetic (fp64 here).
+ * and the final difference each rounded once; p is inside when it lies in the closed bounding box of
+ * the three vertices and the three edge values are all >= 0 or all <= 0; a triangle whose own third
+ * vertex has edge value 0 (no area) paints nothing.  (The bounding box keeps a needle-thin triangle,
+ * whose three edge lines nearly coincide, from claiming pixels far beyond its tips through rounding.)
+ * Colours and compositing are plain real arithmetic (fp64 here).
  */
 #include "oracle.h"
 
@@ -46,6 +48,8 @@ int oracle_paint_inside(const float tri[6], float px, float py)
     const float x1 = unit_f32(tri[2]), y1 = unit_f32(tri[3]);
     const float x2 = unit_f32(tri[4]), y2 = unit_f32(tri[5]);
     if (edge_f32(x0, y0, x1, y1, x2, y2) == 0.0f) return 0;
+    if (px < fminf(x0, fminf(x1, x2)) || px > fmaxf(x0, fmaxf(x1, x2))) return 0;
+    if (py < fminf(y0, fminf(y1, y2)) || py > fmaxf(y0, fmaxf(y1, y2))) return 0;
     const float e0 = edge_f32(x0, y0, x1, y1, px, py);
     const float e1 = edge_f32(x1, y1, x2, y2, px, py);
     const float e2 = edge_f32(x2, y2, x0, y0, px, py);

@@ -131,3 +131,15 @@ def test_single_pixel_inside_decision_is_taken_in_fp32():
             assert not inside
             hits += 1
     assert hits > 20
+
+
+def test_needle_triangle_stays_inside_its_bounding_box():
+    # nearly collinear vertices: without the bounding box, rounding could let pixels on the
+    # extension of the needle pass the three edge tests
+    t = tri((0.30, 0.30), (0.50, 0.50), (0.40, 0.4000001), (1, 1, 1), 1.0)
+    c = oracle.paint_render(t[None], 200, 200)[:, :, 0]
+    ys, xs = np.nonzero(c)
+    if len(xs):
+        assert xs.min() >= 0.30 * 200 - 1 and xs.max() <= 0.50 * 200 and ys.min() >= 0.30 * 200 - 1 and ys.max() <= 0.50 * 200
+    for px, py in ((0.7, 0.7), (0.1, 0.1), (0.9, 0.9000001)):
+        assert not oracle.paint_inside(t[:6], px, py)
