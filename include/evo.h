@@ -50,7 +50,7 @@ typedef enum {
 enum { EVO_NOISE_STORED = 0, EVO_NOISE_REGENERATED = 1 };
 enum { EVO_POLICY_NONE = 0, EVO_POLICY_MLP = 1, EVO_POLICY_CNN_28 = 2, EVO_POLICY_LSTM_SEQ2SEQ = 3 };
 enum { EVO_TASK_NONE = 0, EVO_TASK_CARTPOLE = 1, EVO_TASK_TANH_LINEAR = 2, EVO_TASK_SUPERVISED = 3,
-       EVO_TASK_SEQ2SEQ_ADD = 4 };
+       EVO_TASK_SEQ2SEQ_ADD = 4, EVO_TASK_PAINT = 5 };
 enum { EVO_ROLLOUT_AUTO = 0, EVO_ROLLOUT_GENERIC = 1, EVO_ROLLOUT_TILED = 2 };
 enum { EVO_OPT_ADAM = 0, EVO_OPT_CLIPUP = 1 };
 enum { EVO_SIGMA_CONSTANT = 0, EVO_SIGMA_PGPE = 1 };
@@ -61,6 +61,10 @@ enum { EVO_CP_CART_MASS = 0, EVO_CP_POLE_MASS = 1, EVO_CP_POLE_HALF_LENGTH = 2, 
 
 /* index into evo_config.task_param for EVO_TASK_SEQ2SEQ_ADD: digits per operand, 1..4 */
 enum { EVO_S2S_DIGITS = 0 };
+
+/* indices into evo_config.task_param for EVO_TASK_PAINT: canvas width and height in pixels, grey
+ * level of the empty canvas */
+enum { EVO_PAINT_WIDTH = 0, EVO_PAINT_HEIGHT = 1, EVO_PAINT_BACKGROUND = 2 };
 
 #define EVO_MAX_LAYERS 8
 
@@ -83,7 +87,7 @@ typedef struct evo_config {
     uint32_t batch;                /* images (supervised) or queries (seq2seq) per member       */
     uint32_t trace_steps;          /* leading steps recorded when evo_rollout gets d_trace      */
     uint32_t rollout_kernel;       /* EVO_ROLLOUT_*: AUTO picks the tiled kernel when one fits  */
-    float    task_param[16];       /* cart-pole: EVO_CP_*; seq2seq: EVO_S2S_*; others unused    */
+    float    task_param[16];       /* EVO_CP_* / EVO_S2S_* / EVO_PAINT_* by task; else unused   */
     uint32_t optimizer;            /* EVO_OPT_*: how the centre follows the ES gradient         */
     float    clipup_momentum;      /* ClipUp: 0 selects 0.9                                     */
     float    clipup_max_speed;     /* ClipUp: 0 selects 2 * lr                                  */
@@ -123,7 +127,10 @@ evo_status evo_ask(evo_solver* s, const float** d_theta, size_t* ld_theta);
  * caller matrix must be [P][ldD] with the same pitch, 16-byte aligned) and writes
  * d_fitness[P] (fp32).  Control tasks: E episodes of T steps per member from seeded initial
  * states shared by all members; fitness = mean episode return.  Supervised task: fitness =
- * -mean cross-entropy on the batch bound with evo_set_batch.
+ * -mean cross-entropy on the batch bound with evo_set_batch.  Seq2seq task: -mean cross-entropy of
+ * the answer digits on `batch` queries the library draws itself.  Painting task (policy NONE: the
+ * parameter row is param_dim / 10 triangles x0 y0 x1 y1 x2 y2 r g b a): -mean squared distance of
+ * the painted canvas to the image bound with evo_set_target.
  * d_trace: NULL, or [P][E][trace_steps][state_dim] floats receiving the post-step task state
  * (state_dim = 4 cart-pole: x, x', theta, theta'; 28 tanh-linear).
  * Errors: BAD_ORDER (d_theta NULL before any ask; supervised without a batch), INVALID_ARG,
@@ -183,6 +190,12 @@ evo_status evo_destroy(evo_solver* s);
  * provide data and labels).  d_images [batch][28][28] fp32, d_labels [batch] int32 in 0..9;
  * both stay owned by the caller and must outlive the rollouts that use them. */
 evo_status evo_set_batch(evo_solver* s, const float* d_images, const int32_t* d_labels);
+
+/* Painting task (paper Section 3, "Concrete and Abstract Painting"): bind the target image,
+ * d_target [height][width][3] fp32 in [0,1], owned by the caller, alive during the rollouts.  With
+ * this task evo_rollout's d_trace, when given (trace_steps > 0), receives every member's canvas
+ * [P][height][width][3].  Errors: INVALID_ARG (NULL), UNSUPPORTED (other task). */
+evo_status evo_set_target(evo_solver* s, const float* d_target);
 
 /* Device pointers into the workspace (valid for the solver's lifetime): centre, Adam moments,
  * last gradient (each [ldD] floats, padding zero); ranks [P] int32 and centred-rank weights

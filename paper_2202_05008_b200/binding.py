@@ -68,6 +68,7 @@ def load_library():
     L.evo_tell_begin.argtypes = [vp, vp]
     L.evo_get_reduce_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), szp]
     L.evo_tell_end.argtypes = [vp]
+    L.evo_set_target.argtypes = [vp, vp]
     L.evo_fma_probe.argtypes = [vp, C.c_uint32, C.c_uint32, C.c_uint32, vp, C.POINTER(C.c_uint64)]
     L.evo_destroy.argtypes = [vp]
     L.evo_set_batch.argtypes = [vp, vp, vp]
@@ -88,7 +89,7 @@ def load_library():
     L.evo_status_string.restype = C.c_char_p
     L.evo_version.restype = C.c_uint32
     for name in ("evo_workspace_bytes", "evo_create", "evo_ask", "evo_rollout", "evo_tell", "evo_tell_begin",
-                 "evo_get_reduce_buffers", "evo_tell_end", "evo_fma_probe",
+                 "evo_get_reduce_buffers", "evo_tell_end", "evo_fma_probe", "evo_set_target",
                  "evo_destroy", "evo_set_batch", "evo_get_center", "evo_get_moments",
                  "evo_get_gradient", "evo_get_ranks", "evo_get_eps", "evo_get_sigma", "evo_set_sigma", "evo_get_counters",
                  "evo_set_state", "evo_sync_status", "evo_launch_count"):
@@ -205,6 +206,12 @@ class Solver:
         assert labels.dtype == torch.int32 and labels.is_cuda and labels.is_contiguous()
         self._batch = (images, labels)           # keep alive
         _check(self.lib.evo_set_batch(self._h, images.data_ptr(), labels.data_ptr()), "evo_set_batch")
+
+    def set_target(self, target: torch.Tensor) -> None:
+        """Painting task: the image [H][W][3] (fp32, device) every member's canvas is compared with."""
+        assert target.dtype == torch.float32 and target.is_cuda and target.is_contiguous()
+        self._target = target                    # keep alive
+        _check(self.lib.evo_set_target(self._h, target.data_ptr()), "evo_set_target")
 
     def padded_rows(self, rows: int) -> torch.Tensor:
         """A zeroed [rows][ldD] device matrix with the pitch evo_rollout expects."""

@@ -22,6 +22,7 @@ struct evo_solver {
     bool         ever_asked;
     const float*   d_images;
     const int32_t* d_labels;
+    const float*   d_target;
     uint64_t     launches;
     uint32_t     k0, k1;
 };
@@ -71,6 +72,16 @@ static evo_status check_config(const evo_config* c)
                 return EVO_ERR_INVALID_ARG;
             break;
         }
+        case EVO_TASK_PAINT: {
+            const float w = c->task_param[EVO_PAINT_WIDTH], h = c->task_param[EVO_PAINT_HEIGHT];
+            const float bg = c->task_param[EVO_PAINT_BACKGROUND];
+            if (c->policy_kind != EVO_POLICY_NONE || !(w >= 1.f) || !(h >= 1.f) || !(w <= 4096.f) || !(h <= 4096.f) ||
+                w != static_cast<float>(static_cast<uint32_t>(w)) || h != static_cast<float>(static_cast<uint32_t>(h)) ||
+                !(bg >= 0.f) || !(bg <= 1.f))
+                return EVO_ERR_INVALID_ARG;
+            if (!paint_supported(c->param_dim, static_cast<uint32_t>(w), static_cast<uint32_t>(h))) return EVO_ERR_INVALID_ARG;
+            break;
+        }
         default: return EVO_ERR_INVALID_ARG;
     }
     return EVO_OK;
@@ -112,6 +123,9 @@ static evo_status make_layout(const evo_config& c, Layout* L)
         if (tc > cnn) cnn = tc;
     }
     if (c.task_kind == EVO_TASK_SEQ2SEQ_ADD) cnn = s2s_scratch_bytes(static_cast<uint32_t>(Pl), c.batch);
+    if (c.task_kind == EVO_TASK_PAINT)
+        cnn = paint_scratch_bytes(static_cast<uint32_t>(Pl), static_cast<uint32_t>(c.task_param[EVO_PAINT_WIDTH]),
+                                  static_cast<uint32_t>(c.task_param[EVO_PAINT_HEIGHT]));
     L->cnn_scratch = take(cnn);                                 // scratch of the single-step tasks
     L->theta = take(row * Pl);
     L->eps = take(c.noise_mode == EVO_NOISE_STORED ? row * Hl : 0);
@@ -162,6 +176,7 @@ evo_status evo_create(const evo_config* cfg_in, void* d_workspace, size_t worksp
     s->ever_asked = false;
     s->d_images = nullptr;
     s->d_labels = nullptr;
+    s->d_target = nullptr;
     s->launches = 0;
     s->k0 = static_cast<uint32_t>(s->cfg.seed & 0xFFFFFFFFull);
     s->k1 = static_cast<uint32_t>(s->cfg.seed >> 32);
@@ -210,6 +225,14 @@ evo_status evo_set_batch(evo_solver* s, const float* d_images, const int32_t* d_
     return EVO_OK;
 }
 
+evo_status evo_set_target(evo_solver* s, const float* d_target)
+{
+    if (!s || !d_target) return EVO_ERR_INVALID_ARG;
+    if (s->cfg.task_kind != EVO_TASK_PAINT) return EVO_ERR_UNSUPPORTED;
+    s->d_target = d_target;
+    return EVO_OK;
+}
+
 evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, float* d_trace)
 {
     if (!s || !d_fitness) return EVO_ERR_INVALID_ARG;
@@ -237,6 +260,17 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
         return EVO_OK;
     }
     if (d_trace && c.trace_steps == 0) return EVO_ERR_INVALID_ARG;
+    if (c.task_kind == EVO_TASK_PAINT) {
+        if (!s->d_target) return EVO_ERR_BAD_ORDER;
+        const int n = launch_rollout_paint(s->stream, d_theta, L.ldD, s->local_pop, c.param_dim,
+                                           static_cast<uint32_t>(c.task_param[EVO_PAINT_WIDTH]),
+                                           static_cast<uint32_t>(c.task_param[EVO_PAINT_HEIGHT]),
+                                           c.task_param[EVO_PAINT_BACKGROUND], s->d_target, s->ws + L.cnn_scratch,
+                                           d_fitness, d_trace);
+        if (n < 0) return EVO_ERR_CUDA;
+        s->launches += n;
+        return EVO_OK;
+    }
     if (c.task_kind == EVO_TASK_SEQ2SEQ_ADD) {
         // d_trace, when given, receives the logits [P][batch][digits+1][12] (CUDA-core kernel)
         const int n = launch_rollout_s2s(s->stream, d_theta, L.ldD, s->local_pop, c.layer_sizes[0],

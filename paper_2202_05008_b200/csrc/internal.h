@@ -99,4 +99,11 @@ int launch_rollout_s2s(cudaStream_t st, const float* theta, uint32_t ldD, uint32
                        uint32_t B, uint32_t k0, uint32_t k1, uint32_t generation, uint32_t kernel_choice,
                        void* scratch, float* fitness, float* logits, DeviceStatus* status);
 
+bool paint_supported(uint32_t param_dim, uint32_t W, uint32_t H);
+size_t paint_scratch_bytes(uint32_t P, uint32_t W, uint32_t H);
+// canvas (nullable): [P][H][W][3]
+int launch_rollout_paint(cudaStream_t st, const float* theta, uint32_t ldD, uint32_t P, uint32_t param_dim,
+                         uint32_t W, uint32_t H, float background, const float* target, void* scratch,
+                         float* fitness, float* canvas);
+
 }  // namespace evo

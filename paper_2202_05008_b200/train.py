@@ -17,11 +17,16 @@ from .binding import Solver
 
 def run(workload: W.Workload, generations: int, device="cuda:0", log_every: int = 0,
         fixed_batch: bool = False, initial_center: Optional[torch.Tensor] = None,
-        **cfg_kw) -> Tuple[Solver, List[Tuple[float, float]]]:
+        target: Optional[torch.Tensor] = None, **cfg_kw) -> Tuple[Solver, List[Tuple[float, float]]]:
     """Runs `generations` generations; returns the solver and [(mean fitness, best fitness)]."""
     s = Solver(workload, device=device, **cfg_kw)
     if initial_center is not None:
         s.set_state(center=initial_center.to(s.device).contiguous())
+    if workload.task_kind == W.TASK_PAINT:
+        if target is None:
+            width, height = int(workload.task_param[0]), int(workload.task_param[1])
+            target = torch.tensor(W.paint_target(workload.seed, width, height), device=s.device)
+        s.set_target(target)
     history = []
     fitness = torch.empty(workload.pop_size, dtype=torch.float32, device=s.device)
     for g in range(generations):

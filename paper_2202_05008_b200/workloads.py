@@ -14,7 +14,7 @@ import numpy as np
 
 NOISE_STORED, NOISE_REGENERATED = 0, 1
 POLICY_NONE, POLICY_MLP, POLICY_CNN_28, POLICY_LSTM_SEQ2SEQ = 0, 1, 2, 3
-TASK_NONE, TASK_CARTPOLE, TASK_TANH_LINEAR, TASK_SUPERVISED, TASK_SEQ2SEQ_ADD = 0, 1, 2, 3, 4
+TASK_NONE, TASK_CARTPOLE, TASK_TANH_LINEAR, TASK_SUPERVISED, TASK_SEQ2SEQ_ADD, TASK_PAINT = 0, 1, 2, 3, 4, 5
 OPT_ADAM, OPT_CLIPUP = 0, 1
 SIGMA_CONSTANT, SIGMA_PGPE = 0, 1
 
@@ -51,6 +51,8 @@ class Workload:
     def env_steps_per_generation(self) -> int:
         if self.task_kind in (TASK_SUPERVISED, TASK_SEQ2SEQ_ADD):
             return self.pop_size * self.batch
+        if self.task_kind == TASK_PAINT:
+            return self.pop_size                 # one painted canvas per member
         if self.task_kind == TASK_NONE:
             return 0
         return self.pop_size * self.episodes * self.horizon
@@ -93,7 +95,30 @@ SEQ2SEQ = Workload("seq2seq_add_lstm128_pop1024", 1024, seq2seq_param_count(128)
                    policy_kind=POLICY_LSTM_SEQ2SEQ, layer_sizes=(128,), task_kind=TASK_SEQ2SEQ_ADD,
                    batch=128, generations=20, task_param=(3.0,))
 
-CONFIGS = {"cfg1": CFG1, "cfg2": CFG2, "cfg3": CFG3, "cfg4": CFG4, "cfg5": CFG5, "seq2seq": SEQ2SEQ}
+# the paper's painting example (Section 3): a canvas of semi-transparent triangles fitted to an
+# image; task parameters = canvas width, height, background grey level
+PAINT = Workload("paint_64_triangles_128x128_pop1024", 1024, 10 * 64, seed=5, sigma=0.1, lr=0.02,
+                 task_kind=TASK_PAINT, generations=20, task_param=(128.0, 128.0, 0.0))
+
+
+def paint_target(seed: int, width: int, height: int) -> np.ndarray:
+    """Synthetic target image [H][W][3] fp32 in [0,1]: a few soft colour blobs and one hard-edged
+    bar on a dark ground (stands in for the photographs the paper's example fits)."""
+    rng = np.random.default_rng([seed, 0x7061696E74])
+    y, x = np.meshgrid((np.arange(height) + 0.5) / height, (np.arange(width) + 0.5) / width, indexing="ij")
+    img = np.full((height, width, 3), 0.05, np.float64)
+    for _ in range(6):
+        cx, cy, rad = rng.random(), rng.random(), 0.08 + 0.25 * rng.random()
+        colour = rng.random(3)
+        blob = np.exp(-((x - cx) ** 2 + (y - cy) ** 2) / (2 * rad * rad))
+        img += blob[:, :, None] * colour[None, None, :] * 0.6
+    x0, x1 = sorted(rng.random(2)); y0 = rng.random() * 0.8
+    bar = (x >= x0) & (x <= x1) & (y >= y0) & (y <= y0 + 0.1)
+    img[bar] = rng.random(3)
+    return np.clip(img, 0.0, 1.0).astype(np.float32)
+
+
+CONFIGS = {"cfg1": CFG1, "cfg2": CFG2, "cfg3": CFG3, "cfg4": CFG4, "cfg5": CFG5, "seq2seq": SEQ2SEQ, "paint": PAINT}
 
 assert mlp_param_count(CFG1.layer_sizes) == CFG1.param_dim
 assert mlp_param_count(CFG2.layer_sizes) == CFG2.param_dim
