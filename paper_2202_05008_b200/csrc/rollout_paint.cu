@@ -58,8 +58,10 @@ struct PaintArgs {
 __global__ void __launch_bounds__(kPaintThreads)
 k_paint(const PaintArgs a)
 {
-    __shared__ __align__(16) PaintTri tri[kPaintMaxTriangles];
-    __shared__ uint16_t keep[kPaintMaxTriangles];      // indices of the triangles that touch the tile, in order
+    // sized by the launch: n_tri records, then n_tri indices of the triangles that touch the tile, in order
+    extern __shared__ __align__(16) unsigned char paint_smem[];
+    PaintTri* tri = reinterpret_cast<PaintTri*>(paint_smem);
+    uint16_t* keep = reinterpret_cast<uint16_t*>(paint_smem + sizeof(PaintTri) * a.n_tri);
     __shared__ uint32_t n_keep;
     __shared__ uint32_t warp_count[kPaintThreads / 32];
     __shared__ float warp_sum[kPaintThreads / 32];
@@ -219,7 +221,8 @@ int launch_rollout_paint(cudaStream_t st, const float* theta, uint32_t ldD, uint
     a.tiles_x = (W + kPaintTileW - 1) / kPaintTileW; a.tiles_y = (H + kPaintTileH - 1) / kPaintTileH;
     const uint32_t tiles = a.tiles_x * a.tiles_y;
     dim3 grid(P, tiles);
-    k_paint<<<grid, kPaintThreads, 0, st>>>(a);
+    const size_t smem = (sizeof(PaintTri) + sizeof(uint16_t)) * a.n_tri;       // at most 33 KB
+    k_paint<<<grid, kPaintThreads, smem, st>>>(a);
     if (cudaGetLastError() != cudaSuccess) return -1;
     const float inv = 1.0f / (3.0f * static_cast<float>(W) * static_cast<float>(H));
     k_paint_finalize<<<(P + 255u) / 256u, 256, 0, st>>>(a.partial, P, tiles, inv, fitness);
