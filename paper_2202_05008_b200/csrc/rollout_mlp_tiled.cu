@@ -16,6 +16,7 @@
 // with parameters as data; stateless task step; identical initial observations).
 #include "internal.h"
 #include "async.cuh"
+#include "fp32x2.cuh"
 #include "noise.cuh"
 #include "tasks.cuh"
 
@@ -147,19 +148,44 @@ struct Dense {
                                         float scale, Hook&& hook) const
     {
         float acc[N];
+        if constexpr (TI % 2 == 0) {
+            // rows in pairs: one paired FMA updates rows 2j and 2j+1 of an episode
+            float2 acc2[TI / 2][EB];
 #pragma unroll
-        for (int r = 0; r < TI; ++r)
+            for (int j = 0; j < TI / 2; ++j)
 #pragma unroll
-            for (int e = 0; e < EB; ++e) acc[r * EB + e] = bias[r];
+                for (int e = 0; e < EB; ++e) acc2[j][e] = make_float2(bias[2 * j], bias[2 * j + 1]);
 #pragma unroll
-        for (int k = 0; k < KS; ++k) {
-            float a[EB];
-            EpVec<EB>::load(in + (k * S + s) * LD, a);     // lane s takes inputs s, s+S, ... (no bank conflicts)
-            hook(k * S + s, a);
+            for (int k = 0; k < KS; ++k) {
+                float a[EB];
+                EpVec<EB>::load(in + (k * S + s) * LD, a);     // lane s takes inputs s, s+S, ... (no bank conflicts)
+                hook(k * S + s, a);
+#pragma unroll
+                for (int e = 0; e < EB; ++e) {
+                    const float2 aa = make_float2(a[e], a[e]);
+#pragma unroll
+                    for (int j = 0; j < TI / 2; ++j) ffma2(acc2[j][e], make_float2(w[2 * j][k], w[2 * j + 1][k]), aa);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < TI / 2; ++j)
+#pragma unroll
+                for (int e = 0; e < EB; ++e) { acc[(2 * j) * EB + e] = acc2[j][e].x; acc[(2 * j + 1) * EB + e] = acc2[j][e].y; }
+        } else {
 #pragma unroll
             for (int r = 0; r < TI; ++r)
 #pragma unroll
-                for (int e = 0; e < EB; ++e) acc[r * EB + e] = fmaf(w[r][k], a[e], acc[r * EB + e]);
+                for (int e = 0; e < EB; ++e) acc[r * EB + e] = bias[r];
+#pragma unroll
+            for (int k = 0; k < KS; ++k) {
+                float a[EB];
+                EpVec<EB>::load(in + (k * S + s) * LD, a);     // lane s takes inputs s, s+S, ... (no bank conflicts)
+                hook(k * S + s, a);
+#pragma unroll
+                for (int r = 0; r < TI; ++r)
+#pragma unroll
+                    for (int e = 0; e < EB; ++e) acc[r * EB + e] = fmaf(w[r][k], a[e], acc[r * EB + e]);
+            }
         }
         int offset;
         if constexpr (PERM) { reduce_lanes_perm<TI, EB, S>(acc); offset = row_mask<S>(s, TI) * EB; }

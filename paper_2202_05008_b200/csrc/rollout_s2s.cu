@@ -29,6 +29,7 @@
 #include "async.cuh"
 #include "noise.cuh"
 #include "umma.cuh"
+#include "fp32x2.cuh"
 
 namespace evo {
 
@@ -232,13 +233,6 @@ __device__ __forceinline__ float tanh_sfu(float x)
     float y;
     asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-}
-// two fp32 fused multiply-adds in one instruction
-__device__ __forceinline__ void ffma2(float2& acc, float2 a, float2 b)
-{
-    asm("fma.rn.f32x2 %0, %1, %2, %0;"
-        : "+l"(*reinterpret_cast<unsigned long long*>(&acc))
-        : "l"(*reinterpret_cast<const unsigned long long*>(&a)), "l"(*reinterpret_cast<const unsigned long long*>(&b)));
 }
 __device__ __forceinline__ bool elect_one()
 {
