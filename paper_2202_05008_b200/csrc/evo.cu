@@ -532,6 +532,6 @@ const char* evo_status_string(evo_status st)
     return "unknown status";
 }
 
-uint32_t evo_version(void) { return 102; }
+uint32_t evo_version(void) { return 103; }
 
 }  // extern "C"
