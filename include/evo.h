@@ -210,10 +210,13 @@ evo_status evo_get_eps    (evo_solver* s, const float** d_eps);
 evo_status evo_get_sigma  (evo_solver* s, const float** d_sigma);
 evo_status evo_set_sigma  (evo_solver* s, const float* d_sigma);
 
-/* Checkpoint / resume: counters are (generation, Adam step).  evo_set_state copies D floats
- * from each non-NULL device pointer into the solver (asynchronously, on the solver's stream)
- * and sets the counters; the Adam step is read back from the device by evo_get_counters,
- * which therefore synchronises the stream. */
+/* Checkpoint / resume: counters are (generation, Adam step).  Both live in device memory and are
+ * advanced by the kernel that closes a tell, so evo_ask / evo_rollout / evo_tell pass nothing to
+ * their kernels that changes from one generation to the next: a sequence ask -> rollout -> tell
+ * captured into a CUDA graph (on the solver's stream, which must not be the legacy default stream)
+ * can be replayed, each replay being one more generation.  evo_set_state copies D floats from each
+ * non-NULL device pointer into the solver and sets the counters; evo_get_counters reads them back;
+ * both therefore synchronise the stream (do not call them while capturing). */
 evo_status evo_get_counters(evo_solver* s, uint32_t* generation, uint32_t* adam_step);
 evo_status evo_set_state(evo_solver* s, const float* d_center, const float* d_m, const float* d_v,
                          uint32_t generation, uint32_t adam_step);

@@ -193,6 +193,20 @@ class Solver:
     def tell_end(self) -> None:
         _check(self.lib.evo_tell_end(self._h), "evo_tell_end")
 
+    def capture_generation(self, fitness: torch.Tensor) -> "torch.cuda.CUDAGraph":
+        """Captures ask -> rollout -> tell into a CUDA graph; every ``replay()`` is one generation
+        (the counters that select the random streams live on the device).  The solver must have
+        been created on a non-default stream; the fitness of the last replay is left in ``fitness``."""
+        if self.stream.cuda_stream == 0:
+            raise ValueError("graph capture needs a solver created with stream=torch.cuda.Stream()")
+        assert fitness.dtype == torch.float32 and fitness.is_cuda and fitness.numel() == self.P
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=self.stream):
+            self.ask()
+            self.rollout(fitness=fitness)
+            self.tell(fitness)
+        return graph
+
     def close(self) -> None:
         if getattr(self, "_h", None) is not None:
             self.lib.evo_destroy(self._h)

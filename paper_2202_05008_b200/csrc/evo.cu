@@ -204,7 +204,7 @@ evo_status evo_ask(evo_solver* s, const float** d_theta, size_t* ld_theta)
     float* eps = s->cfg.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<float*>(s->ws + L.eps) : nullptr;
     const int n = launch_ask(s->stream, reinterpret_cast<const float*>(s->ws + L.center),
                              reinterpret_cast<const float*>(s->ws + L.sigma),
-                             s->k0, s->k1, s->generation, s->pair0, s->local_pop / 2, s->cfg.param_dim, L.ldD,
+                             s->k0, s->k1, reinterpret_cast<const DeviceStatus*>(s->ws + L.status), s->pair0, s->local_pop / 2, s->cfg.param_dim, L.ldD,
                              theta, eps);
     if (n < 0) return EVO_ERR_CUDA;
     s->launches += n;
@@ -275,7 +275,7 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
         // d_trace, when given, receives the logits [P][batch][digits+1][12] (CUDA-core kernel)
         const int n = launch_rollout_s2s(s->stream, d_theta, L.ldD, s->local_pop, c.layer_sizes[0],
                                          static_cast<uint32_t>(c.task_param[EVO_S2S_DIGITS]), c.batch, s->k0, s->k1,
-                                         s->generation, c.rollout_kernel, s->ws + L.cnn_scratch, d_fitness, d_trace,
+                                         c.rollout_kernel, s->ws + L.cnn_scratch, d_fitness, d_trace,
                                          reinterpret_cast<DeviceStatus*>(s->ws + L.status));
         if (n < 0) return n == -2 ? EVO_ERR_UNSUPPORTED : EVO_ERR_CUDA;
         s->launches += n;
@@ -299,7 +299,7 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
     a.task = c.task_kind;
     a.E = c.episodes; a.T = c.horizon; a.EB = L.EB; a.n_eb = L.n_eb;
     a.trace_T = c.trace_steps < c.horizon ? c.trace_steps : c.horizon;
-    a.k0 = s->k0; a.k1 = s->k1; a.generation = s->generation;
+    a.k0 = s->k0; a.k1 = s->k1;
     std::memcpy(a.tp, c.task_param, sizeof(a.tp));
     const int n = launch_rollout_mlp(s->stream, a, c.rollout_kernel, d_fitness,
                                      reinterpret_cast<DeviceStatus*>(s->ws + L.status));
@@ -315,7 +315,7 @@ static TellArgs tell_args(evo_solver* s)
     TellArgs t;
     t.u = reinterpret_cast<const float*>(s->ws + L.u);
     t.eps = c.noise_mode == EVO_NOISE_STORED ? reinterpret_cast<const float*>(s->ws + L.eps) : nullptr;
-    t.k0 = s->k0; t.k1 = s->k1; t.generation = s->generation;
+    t.k0 = s->k0; t.k1 = s->k1;
     t.H = s->local_pop / 2; t.D = c.param_dim; t.ldD = L.ldD; t.splits = L.grad_splits;
     t.pair0 = s->pair0; t.P = c.pop_size;
     t.partial = reinterpret_cast<double*>(s->ws + L.grad_partial);
@@ -463,8 +463,9 @@ evo_status evo_get_counters(evo_solver* s, uint32_t* generation, uint32_t* adam_
     if (cudaMemcpyAsync(&h, s->ws + s->lay.status, sizeof(h), cudaMemcpyDeviceToHost, s->stream) != cudaSuccess)
         return EVO_ERR_CUDA;
     if (cudaStreamSynchronize(s->stream) != cudaSuccess) return EVO_ERR_CUDA;
-    *generation = s->generation;
+    *generation = h.generation;
     *adam_step = h.adam_step;
+    s->generation = h.generation;                 // host mirror (informative only)
     return EVO_OK;
 }
 
@@ -480,10 +481,12 @@ evo_status evo_set_state(evo_solver* s, const float* d_center, const float* d_m,
         return EVO_ERR_CUDA;
     if (d_v && cudaMemcpyAsync(s->ws + L.v, d_v, bytes, cudaMemcpyDeviceToDevice, s->stream) != cudaSuccess)
         return EVO_ERR_CUDA;
-    if (cudaMemcpyAsync(s->ws + L.status + offsetof(DeviceStatus, adam_step), &adam_step, sizeof(uint32_t),
+    static_assert(offsetof(DeviceStatus, generation) == offsetof(DeviceStatus, adam_step) + sizeof(uint32_t), "adjacent counters");
+    const uint32_t counters[2] = { adam_step, generation };
+    if (cudaMemcpyAsync(s->ws + L.status + offsetof(DeviceStatus, adam_step), counters, sizeof(counters),
                         cudaMemcpyHostToDevice, s->stream) != cudaSuccess)
         return EVO_ERR_CUDA;
-    if (cudaStreamSynchronize(s->stream) != cudaSuccess) return EVO_ERR_CUDA;   // adam_step is a stack value
+    if (cudaStreamSynchronize(s->stream) != cudaSuccess) return EVO_ERR_CUDA;   // the counters are a stack value
     s->generation = generation;
     s->asked = false;
     s->telling = false;

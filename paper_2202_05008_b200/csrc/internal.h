@@ -13,7 +13,7 @@ struct DeviceStatus {
     uint32_t sticky;        // OR of (1u << evo_status) for conditions raised on the device
     uint32_t nonfinite;     // set by the rank kernel of the current tell, cleared by its finish
     uint32_t adam_step;     // t
-    uint32_t pad;
+    uint32_t generation;    // counter word of every random stream; advanced by the kernel that closes a tell
 };
 
 constexpr uint32_t kTlNx = 28;   // tanh-linear task: state width
@@ -33,7 +33,7 @@ struct RolloutMlpArgs {
     uint32_t task;
     uint32_t E, T, EB, n_eb;     // episodes, horizon, episodes per block, blocks per member
     uint32_t trace_T;
-    uint32_t k0, k1, generation;
+    uint32_t k0, k1;             // the generation is read from the device status by the kernels
     float    tp[16];
     uint32_t weights_in_smem;
 };
@@ -50,14 +50,14 @@ int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, fl
                 float sigma, uint32_t D, uint32_t ldD, DeviceStatus* status);
 int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t k1, float* task_const);
 int launch_ask(cudaStream_t st, const float* center, const float* sigma_vec, uint32_t k0, uint32_t k1,
-               uint32_t generation, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* theta,
+               const DeviceStatus* status, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* theta,
                float* eps);
 int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank, float* u,
                 DeviceStatus* status);
 struct TellArgs {
     const float* u;               // centred-rank weights [P]
     const float* eps;             // stored noise, or NULL = regenerate from the counters
-    uint32_t k0, k1, generation, H, D, ldD, splits;   // H = pairs summed here (the shard's)
+    uint32_t k0, k1, H, D, ldD, splits;   // H = pairs summed here (the shard's)
     uint32_t pair0, P;            // first global pair of the shard; global population size
     double* partial;              // [splits][ldD] fp64 partial sums of the centre gradient
     float*  sigma_partial;        // [splits][ldD] fp32 partial sums of the sigma gradient, or NULL
@@ -96,7 +96,7 @@ bool s2s_supported(uint32_t h, uint32_t nd, uint32_t B);
 size_t s2s_scratch_bytes(uint32_t P, uint32_t B);
 // logits (nullable): [P][B][nd+1][12], written by the CUDA-core kernel only
 int launch_rollout_s2s(cudaStream_t st, const float* theta, uint32_t ldD, uint32_t P, uint32_t h, uint32_t nd,
-                       uint32_t B, uint32_t k0, uint32_t k1, uint32_t generation, uint32_t kernel_choice,
+                       uint32_t B, uint32_t k0, uint32_t k1, uint32_t kernel_choice,
                        void* scratch, float* fitness, float* logits, DeviceStatus* status);
 
 bool paint_supported(uint32_t param_dim, uint32_t W, uint32_t H);

@@ -21,7 +21,7 @@ namespace evo {
 constexpr int kGenericThreads = 128;
 
 __global__ void __launch_bounds__(kGenericThreads)
-k_rollout_mlp_generic(const RolloutMlpArgs a)
+k_rollout_mlp_generic(const RolloutMlpArgs a, const DeviceStatus* __restrict__ status)
 {
     extern __shared__ __align__(16) float smem[];
     const uint32_t member = blockIdx.x, eb = blockIdx.y;
@@ -30,6 +30,7 @@ k_rollout_mlp_generic(const RolloutMlpArgs a)
     const uint32_t EB = a.EB;
     const uint32_t tid = threadIdx.x;
     const PhiloxKey key{ a.k0, a.k1 };
+    const uint32_t generation = status->generation;
 
     uint32_t n_params = 0;
     for (uint32_t l = 0; l < a.n_layers; ++l) n_params += a.sizes[l + 1] * a.sizes[l] + a.sizes[l + 1];
@@ -61,7 +62,7 @@ k_rollout_mlp_generic(const RolloutMlpArgs a)
     if (a.task == EVO_TASK_CARTPOLE) {
         cpc = cartpole_const(a.tp);
         if (tid < nE) {
-            cps = cartpole_reset(key, a.generation, e0 + tid, a.tp[EVO_CP_INIT_RANGE]);
+            cps = cartpole_reset(key, generation, e0 + tid, a.tp[EVO_CP_INIT_RANGE]);
             float sn, cs;
             sincosf(cps.th, &sn, &cs);
             obs[0 * EB + tid] = cps.x;  obs[1 * EB + tid] = cps.xd;
@@ -71,7 +72,7 @@ k_rollout_mlp_generic(const RolloutMlpArgs a)
     } else {
         for (uint32_t item = tid; item < (kTlNx / 4) * nE; item += blockDim.x) {
             const uint32_t q = item / nE, e = item % nE;
-            const float4 z = stream_normal4(key, 1u, a.generation, e0 + e, q);
+            const float4 z = stream_normal4(key, 1u, generation, e0 + e, q);
             obs[(4 * q + 0) * EB + e] = z.x; obs[(4 * q + 1) * EB + e] = z.y;
             obs[(4 * q + 2) * EB + e] = z.z; obs[(4 * q + 3) * EB + e] = z.w;
         }
@@ -241,7 +242,7 @@ int launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a_in, uint32_t ker
         if (cudaFuncSetAttribute(k_rollout_mlp_generic, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(bytes)) != cudaSuccess) return -1;
         dim3 grid(a.P, a.n_eb);
-        k_rollout_mlp_generic<<<grid, kGenericThreads, bytes, st>>>(a);
+        k_rollout_mlp_generic<<<grid, kGenericThreads, bytes, st>>>(a, status);
         if (cudaGetLastError() != cudaSuccess) return -1;
         launches += 1;
     }

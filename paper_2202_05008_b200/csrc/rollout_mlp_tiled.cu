@@ -258,7 +258,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     if (CART) {
         cpc = cartpole_const(a.tp);
         if (tid < EB) {
-            cps = cartpole_reset(key, a.generation, e0 + min(tid, nE - 1), a.tp[EVO_CP_INIT_RANGE]);
+            cps = cartpole_reset(key, status->generation, e0 + min(tid, nE - 1), a.tp[EVO_CP_INIT_RANGE]);
             float sn, cs;
             sincos_fast(cps.th, sn, cs);
             obs0[0 * EB + tid] = cps.x;  obs0[1 * EB + tid] = cps.xd;
@@ -268,7 +268,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     } else {
         for (int item = tid; item < (kTlNx / 4) * EB; item += THREADS) {
             const int q = item / EB, e = item % EB;
-            const float4 z = stream_normal4(key, 1u, a.generation, e0 + min(e, nE - 1), q);
+            const float4 z = stream_normal4(key, 1u, status->generation, e0 + min(e, nE - 1), q);
             obs0[(4 * q + 0) * EB + e] = z.x; obs0[(4 * q + 1) * EB + e] = z.y;
             obs0[(4 * q + 2) * EB + e] = z.z; obs0[(4 * q + 3) * EB + e] = z.w;
         }
@@ -432,7 +432,7 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
         for (int g = 0; g < 2; ++g) {
             const int ng = g ? nB : nA;
             const uint32_t ep = e0 + g * EB + min(tid, max(ng, 1) - 1);
-            cps[g] = cartpole_reset(key, a.generation, min(ep, a.E - 1u), a.tp[EVO_CP_INIT_RANGE]);
+            cps[g] = cartpole_reset(key, status->generation, min(ep, a.E - 1u), a.tp[EVO_CP_INIT_RANGE]);
             float sn, cs;
             sincos_fast(cps[g].th, sn, cs);
             float* o = obs + g * NIN * EB;

@@ -77,7 +77,8 @@ __device__ __forceinline__ float token_loss(const float* lg, int target)
 struct S2sArgs {
     const float* theta; uint32_t ldD, P;
     uint32_t h, nd, B;
-    uint32_t k0, k1, generation;
+    uint32_t k0, k1;
+    const DeviceStatus* status;  // holds the generation counter
     float* partial;              // [P][n_chunks] sums of token losses
     uint32_t n_chunks;
     float* logits;               // nullable: [P][B][nd+1][12] (simple kernel only)
@@ -100,7 +101,7 @@ k_s2s_simple(const S2sArgs a)
     const uint32_t Te = 2 * a.nd + 1, Td = a.nd + 1;
     const PhiloxKey key{a.k0, a.k1};
     if (r < kSimpleQ) {
-        s2s_query(key, a.generation, q0 + min(r, nq - 1u), a.nd, enc[r], dec[r], tgt[r]);
+        s2s_query(key, a.status->generation, q0 + min(r, nq - 1u), a.nd, enc[r], dec[r], tgt[r]);
         loss_s[r] = 0.f;
     }
     for (uint32_t s = 0; s < kSimpleQ; ++s) hs[s][r] = 0.f;
@@ -354,7 +355,7 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
 
         // ---- per-item setup: queries, zero state, read-out weights, encoder weights ------------
         if (chunk != staged_chunk) {
-            if (tid < kTcQ) s2s_query(key, a.generation, q0 + min(tid, nq - 1u), a.nd, S.enc[tid], S.dec[tid], S.tgt[tid]);
+            if (tid < kTcQ) s2s_query(key, a.status->generation, q0 + min(tid, nq - 1u), a.nd, S.enc[tid], S.dec[tid], S.tgt[tid]);
             staged_chunk = chunk;
         }
         if (is_mma) {                                            // the decoder's weights will be wanted next
@@ -570,7 +571,7 @@ size_t s2s_scratch_bytes(uint32_t P, uint32_t B)
 }
 
 int launch_rollout_s2s(cudaStream_t st, const float* theta, uint32_t ldD, uint32_t P, uint32_t h, uint32_t nd,
-                       uint32_t B, uint32_t k0, uint32_t k1, uint32_t generation, uint32_t kernel_choice,
+                       uint32_t B, uint32_t k0, uint32_t k1, uint32_t kernel_choice,
                        void* scratch, float* fitness, float* logits, DeviceStatus* status)
 {
     const bool want_tc = kernel_choice != EVO_ROLLOUT_GENERIC;
@@ -580,7 +581,7 @@ int launch_rollout_s2s(cudaStream_t st, const float* theta, uint32_t ldD, uint32
     const bool tc = want_tc && h == kTcH && !logits;
     S2sArgs a;
     a.theta = theta; a.ldD = ldD; a.P = P; a.h = h; a.nd = nd; a.B = B;
-    a.k0 = k0; a.k1 = k1; a.generation = generation;
+    a.k0 = k0; a.k1 = k1; a.status = status;
     a.partial = static_cast<float*>(scratch);
     a.n_chunks = s2s_chunks(B, tc);
     a.logits = logits;

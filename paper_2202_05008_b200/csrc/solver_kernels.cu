@@ -14,7 +14,7 @@ __global__ void k_init(float* center, float* m, float* v, float* g, float* sigma
 {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < ldD) { center[i] = 0.f; m[i] = 0.f; v[i] = 0.f; g[i] = 0.f; sigma_vec[i] = (i < D) ? sigma : 0.f; }
-    if (i == 0) { status->sticky = 0; status->nonfinite = 0; status->adam_step = 0; status->pad = 0; }
+    if (i == 0) { status->sticky = 0; status->nonfinite = 0; status->adam_step = 0; status->generation = 0; }
 }
 
 int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, float* sigma_vec,
@@ -57,11 +57,12 @@ int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t 
 constexpr uint32_t kAskPairsPerThread = 8;
 
 __global__ void __launch_bounds__(256)
-k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, PhiloxKey key, uint32_t generation,
-      uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* __restrict__ theta, float* __restrict__ eps)
+k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, PhiloxKey key,
+      const DeviceStatus* __restrict__ status, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* __restrict__ theta, float* __restrict__ eps)
 {
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
+    const uint32_t generation = status->generation;
     const uint32_t d0 = quad * 4u;
     const float4 c = reinterpret_cast<const float4*>(center)[quad];
     const float4 sg = reinterpret_cast<const float4*>(sigma_vec)[quad];      // one sigma per dimension
@@ -89,13 +90,13 @@ k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, Phi
 }
 
 int launch_ask(cudaStream_t st, const float* center, const float* sigma_vec, uint32_t k0, uint32_t k1,
-               uint32_t generation, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* theta,
+               const DeviceStatus* status, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* theta,
                float* eps)
 {
     const uint32_t quads = ldD / 4u;
     dim3 grid((quads + 255u) / 256u, (H + kAskPairsPerThread - 1u) / kAskPairsPerThread);
     if (grid.y > 65535u) grid.y = 65535u;
-    k_ask<<<grid, 256, 0, st>>>(center, sigma_vec, PhiloxKey{k0, k1}, generation, pair0, H, D, ldD, theta, eps);
+    k_ask<<<grid, 256, 0, st>>>(center, sigma_vec, PhiloxKey{k0, k1}, status, pair0, H, D, ldD, theta, eps);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
@@ -221,13 +222,14 @@ __device__ __forceinline__ void sig_fma(float4& a, float sj, const float4& e)
 template <bool REGEN, bool SIGMA>
 __global__ void __launch_bounds__(kGradThreads)
 k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, PhiloxKey key,
-               uint32_t generation, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD,
+               uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD,
                uint32_t pairs_per_split, double* __restrict__ partial, float* __restrict__ sigma_partial,
                const DeviceStatus* status)
 {
     if (status->nonfinite) return;
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
+    const uint32_t generation = status->generation;
     const uint32_t j0 = blockIdx.y * pairs_per_split;
     const uint32_t j1 = min(H, j0 + pairs_per_split);
     Acc4 acc[2] = { {0., 0., 0., 0.}, {0., 0., 0., 0.} };
@@ -427,7 +429,8 @@ k_clipup_apply(float* __restrict__ vel, float* __restrict__ center, uint32_t ldD
     reinterpret_cast<float4*>(center)[quad] = c4;
 }
 
-// Closes a tell: the Adam step counter advances only if the update was applied.
+// Closes a tell: the Adam step counter advances only if the update was applied; the generation
+// counter (the random streams of the next ask and roll-out) always does.
 __global__ void k_tell_finish(DeviceStatus* status)
 {
     if (status->nonfinite) {
@@ -436,6 +439,7 @@ __global__ void k_tell_finish(DeviceStatus* status)
     } else {
         status->adam_step += 1u;
     }
+    status->generation += 1u;
 }
 
 uint32_t gradient_splits(uint32_t H, uint32_t ldD)
@@ -455,7 +459,7 @@ size_t clipup_norm_doubles(uint32_t ldD) { return 2u * ((ldD / 4u + 255u) / 256u
 template <bool REGEN, bool SIGMA>
 static void launch_grad(dim3 grid, cudaStream_t st, const TellArgs& a, uint32_t pps)
 {
-    k_grad_partial<REGEN, SIGMA><<<grid, kGradThreads, 0, st>>>(a.u, a.eps, PhiloxKey{a.k0, a.k1}, a.generation, a.pair0,
+    k_grad_partial<REGEN, SIGMA><<<grid, kGradThreads, 0, st>>>(a.u, a.eps, PhiloxKey{a.k0, a.k1}, a.pair0,
                                                                 a.H, a.D, a.ldD, pps, a.partial, a.sigma_partial,
                                                                 a.status);
 }

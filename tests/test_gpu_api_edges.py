@@ -104,3 +104,27 @@ def test_fma_probe_reports_a_plausible_fp32_rate_and_rejects_bad_shapes():
     assert lib.evo_fma_probe(sink.data_ptr(), 1, 1024, 8, None, C.byref(flops)) == 0
     torch.cuda.synchronize()
     assert flops.value == 2 * 16 * 8 * 1024
+
+
+def test_graph_replay_of_a_generation_matches_plain_calls():
+    """ask -> rollout -> tell captured once and replayed must walk through the same generations
+    (same noise, same episode seeds, same centre) as the three calls made one by one."""
+    w = W.CFG1.with_(pop_size=32)
+    plain = Solver(w)
+    for _ in range(4):
+        plain.ask()
+        plain.tell(plain.rollout())
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        g = Solver(w, stream=side)
+        fit = torch.empty(w.pop_size, device="cuda")
+        g.ask(); g.tell(g.rollout(fitness=fit))                  # generation 0 by hand (also warms up)
+        graph = g.capture_generation(fit)                         # capturing does not run anything
+        for _ in range(3):
+            graph.replay()
+        side.synchronize()
+    assert g.counters() == plain.counters() == (4, 4)
+    assert torch.equal(g.center(), plain.center())
+    assert g.sync_status() == 0
+    with pytest.raises(ValueError):
+        plain.capture_generation(fit)                             # default stream cannot be captured
