@@ -440,6 +440,35 @@ def run_ours(args, w):
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
     e2e_ms = max_over_ranks(e2e_ms, dev, world)
 
+    # ---- optional: the same generation replayed from a CUDA graph (no host launch cost) ---------
+    graph_ms = None
+    if args.graph and not args.sharded and not no_task:
+        side = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(side):
+            sg = Solver(w_rank, device=dev, stream=side,
+                        noise_mode=W.NOISE_STORED if stored else W.NOISE_REGENERATED)
+            if supervised:
+                sg.set_batch(*batches[0])
+            if w.task_kind == W.TASK_PAINT:
+                sg.set_target(d_target)
+            gfit = torch.empty(P, dtype=torch.float32, device=dev)
+            for _ in range(max(args.warmup, 3)):
+                sg.ask(); sg.rollout(fitness=gfit); sg.tell(gfit)
+            graph = sg.capture_generation(gfit)
+            gev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+            graph.replay()
+            side.synchronize()
+            for i in range(args.steps):
+                flush.fill_(i & 255)
+                gev[i][0].record(side)
+                graph.replay()
+                gev[i][1].record(side)
+            side.synchronize()
+            if sg.sync_status() != 0:
+                raise SystemExit("bench.py: device status not ok after the graph replays")
+            graph_ms = max_over_ranks(sum(a.elapsed_time(b) for a, b in gev), dev, world) / args.steps
+            sg.close()
+
     if rank == 0:
         metric, unit, units_per_gen = unit_of(w)
         value = whole_job_value(units_per_gen, world, t_step_ms, args.sharded)
@@ -505,6 +534,9 @@ def run_ours(args, w):
                         "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
                 "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
                 "stages": stages, "cpu_baseline": cpu}
+        if graph_ms is not None:
+            line["graph_replay"] = {"ms_per_step": graph_ms, "value": whole_job_value(units_per_gen, world, graph_ms),
+                                    "unit": unit, "note": "ask -> rollout -> tell captured once, replayed per step"}
         print(json.dumps(line))
     s.close()
     if world > 1:
@@ -523,6 +555,8 @@ def main():
     ap.add_argument("--sharded", action="store_true",
                     help="one population split over the ranks by antithetic pairs (strong scaling) "
                          "instead of independent replicas")
+    ap.add_argument("--graph", action="store_true",
+                    help="also time the generation replayed from a CUDA graph (extra key graph_replay)")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (experiments)")
     ap.add_argument("--dim", type=int, default=0, help="override the parameter count (cfg5 only)")
     args = ap.parse_args()
