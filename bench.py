@@ -394,7 +394,8 @@ def run_ours(args, w):
     t_ask = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
     t_roll = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
     t_tell = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
-    t_total_ms = sum(e[0].elapsed_time(e[3]) for e in events)
+    per_step = sorted(e[0].elapsed_time(e[3]) for e in events)
+    t_total_ms = sum(per_step)
     t_step_ms = max_over_ranks(t_total_ms, dev, world) / args.steps
 
     # ---- end to end: host-resident centre in, fitness and centre out, every step -----------
@@ -530,6 +531,8 @@ def run_ours(args, w):
                 "scaling": "strong" if args.sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": config_of(w, args, stored),
                 "generations_per_sec": (1 if args.sharded else world) / (t_step_ms * 1e-3),
+                "ms_per_step_median": per_step[len(per_step) // 2], "ms_per_step_best": per_step[0],
+                "sm_count": sm_count,
                 "e2e": {"value": whole_job_value(units_per_gen, world, e2e_ms, args.sharded), "unit": unit,
                         "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
                 "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
