@@ -208,10 +208,11 @@ constexpr int kTcCols = 64 / kTcSub;                       // queries per epilog
 constexpr int kTcOutPerThread = kVocab * 64 / kTcHalfThreads;   // read-out: tokens per thread
 constexpr int kTcThreads = kTcEpiThreads + 32;             // + the MMA warp
 constexpr int kTcKBlocks = 18;                             // K = 128 (h) + 16 (one-hot, 1, padding) in groups of 8
-constexpr uint32_t kTcALbo = 64 * 128;                     // 64 row groups of 8 x 16 bytes between K groups
+constexpr uint32_t kTcALbo = 64 * 128 + 16;                // 64 row groups of 8 x 16 bytes between K groups, +16 bytes
+                                                           // (bank spread of the staging stores)
 constexpr uint32_t kTcBLbo = 16 * 128 + 16;                // 16 row groups, +16 bytes so that the 2-byte stores
                                                            // of a warp (4 K groups) fall in distinct banks
-constexpr uint32_t kTcABytes = kTcKBlocks * kTcALbo;       // 147,456
+constexpr uint32_t kTcABytes = kTcKBlocks * kTcALbo;       // 147,744
 constexpr uint32_t kTcBBytes = kTcKBlocks * kTcBLbo;       // 37,152
 constexpr uint32_t kTcCellFloats = 4 * kTcH * kVocab + 4 * kTcH * kTcH + 4 * kTcH;   // one LSTM cell
 
@@ -255,31 +256,46 @@ __device__ __forceinline__ void s2s_stage_weights(S2sSmem& S, const float* __res
     const float* Wx = cellp;
     const float* Wh = Wx + 4 * kTcH * kVocab;
     const float* bb = Wh + 4 * kTcH * kTcH;
-    // Wh: 512 rows x 16 K groups; a thread converts 8 consecutive k of one row into one 16-byte row.
-    // Within a warp the 8 lanes of a quarter take the 8 rows of a row group (so the 16-byte stores
-    // of a quarter-warp fall in distinct banks) and the 4 quarters take 4 adjacent K groups (so a
-    // load instruction touches one 128-byte line per row).
-    constexpr uint32_t n_items = 512u * 16u;
-    constexpr int U = 8;
+    // Wh: 64 groups of 8 rows x 128 k.  A warp reads a whole row with one fully coalesced 128-bit
+    // load per lane (lane l gets k = 4l .. 4l+3), 8 rows per group, two groups at a time.  A
+    // 16-byte row of a core matrix (8 k) is the data of an even/odd lane pair, so the pair swaps
+    // halves: the even lane ends with rows 0-3 of its K group, the odd lane with rows 4-7, and each
+    // stores them as 128-bit words (the K-group pitch is padded by 16 bytes so that the four K
+    // groups of a quarter-warp fall in distinct banks).
+    const uint32_t warp = tid >> 5, lane = tid & 31u;
+    const bool odd = lane & 1u;
+    constexpr uint32_t kWarps = kTcThreads / 32, G = 2;
 #pragma unroll 1
-    for (uint32_t base = tid; base < n_items; base += U * kTcThreads) {
-        float4 v[U][2];
+    for (uint32_t mg0 = warp * G; mg0 < 64u; mg0 += kWarps * G) {
+        float4 v[G][8];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t idx = min(base + u * kTcThreads, n_items - 1u);
-            const uint32_t m = (idx >> 7) * 8u + (idx & 7u), kb = ((idx >> 5) & 3u) * 4u + ((idx >> 3) & 3u);
-            const float4* src = reinterpret_cast<const float4*>(Wh + m * kTcH + kb * 8u);
-            v[u][0] = __ldg(src); v[u][1] = __ldg(src + 1);
-        }
+        for (uint32_t g = 0; g < G; ++g)
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t idx = base + u * kTcThreads;
-            if (idx < n_items) {
-                const uint32_t m = (idx >> 7) * 8u + (idx & 7u), kb = ((idx >> 5) & 3u) * 4u + ((idx >> 3) & 3u);
-                const float sc = ((m >> 7) == 2u) ? 1.0f : 0.5f;
-                *reinterpret_cast<uint4*>(S.A + kb * kTcALbo + (m >> 3) * 128u + (m & 7u) * 16u) =
-                    make_uint4(pack_bf16(sc * v[u][0].x, sc * v[u][0].y), pack_bf16(sc * v[u][0].z, sc * v[u][0].w),
-                               pack_bf16(sc * v[u][1].x, sc * v[u][1].y), pack_bf16(sc * v[u][1].z, sc * v[u][1].w));
+            for (uint32_t r = 0; r < 8u; ++r) {
+                const uint32_t mg = min(mg0 + g, 63u);
+                v[g][r] = __ldg(reinterpret_cast<const float4*>(Wh + (mg * 8u + r) * kTcH) + lane);
+            }
+#pragma unroll
+        for (uint32_t g = 0; g < G; ++g) {
+            const uint32_t mg = mg0 + g;
+            if (mg < 64u) {
+                const float sc = ((mg >> 4) == 2u) ? 1.0f : 0.5f;       // 16 row groups per gate
+                uint32_t w0[8], w1[8];
+#pragma unroll
+                for (uint32_t r = 0; r < 8u; ++r) {
+                    w0[r] = pack_bf16(sc * v[g][r].x, sc * v[g][r].y);
+                    w1[r] = pack_bf16(sc * v[g][r].z, sc * v[g][r].w);
+                }
+                unsigned char* dst = S.A + (lane >> 1) * kTcALbo + mg * 128u + (odd ? 64u : 0u);
+#pragma unroll
+                for (uint32_t i = 0; i < 4u; ++i) {
+                    const uint32_t got0 = __shfl_xor_sync(0xffffffffu, odd ? w0[i] : w0[i + 4], 1);
+                    const uint32_t got1 = __shfl_xor_sync(0xffffffffu, odd ? w1[i] : w1[i + 4], 1);
+                    const uint32_t keep0 = odd ? w0[i + 4] : w0[i], keep1 = odd ? w1[i + 4] : w1[i];
+                    // the even lane's words are k 0-3 of the K group, the odd lane's k 4-7
+                    *reinterpret_cast<uint4*>(dst + i * 16u) =
+                        odd ? make_uint4(got0, got1, keep0, keep1) : make_uint4(keep0, keep1, got0, got1);
+                }
             }
         }
     }
