@@ -237,7 +237,8 @@ def run_reference(args, w):
     if rank != 0:
         return
     metric, unit, units_per_gen = unit_of(w)
-    n = members_for_budget(w, 1.0)
+    # per-step sample sized so that warm-up + timed steps take about two minutes in all
+    n = members_for_budget(w, min(1.0, 120.0 / max(1, args.warmup + args.steps)))
     times, sample = [], ""
     for i in range(args.warmup + args.steps):
         t, sample = oracle_generation_sample(w, max(n, 1), generation=i)
