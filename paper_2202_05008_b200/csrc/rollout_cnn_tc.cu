@@ -382,11 +382,14 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         // both accumulators start out free
         if (lane == 0) { mbar_arrive(smem_u32(&S.acc_free[0])); mbar_arrive(smem_u32(&S.acc_free[1])); }
         uint32_t gp = 0, done_par = 0;
-        for (;;) {
-            if (tid == 0) {                          // one thread decides, so the whole team takes one branch
-                const uint32_t next = atomicAdd(work_counter, 1u);
-                S.item = S.abort ? kNoItem : next;
-            }
+        // Items are equal in cost, so every block takes one contiguous range of them: consecutive
+        // items belong to the same member almost always, and a member's weights are staged only
+        // when the member changes.
+        const uint32_t item_end = static_cast<uint32_t>((static_cast<uint64_t>(blockIdx.x) + 1u) * n_items / gridDim.x);
+        uint32_t staged_member = 0xFFFFFFFFu;
+        for (uint32_t next = static_cast<uint32_t>(static_cast<uint64_t>(blockIdx.x) * n_items / gridDim.x);; ++next) {
+            if (tid == 0)                            // one thread decides, so the whole team takes one branch
+                S.item = (S.abort || next >= item_end) ? kNoItem : next;
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
             const uint32_t item = S.item;
             if (item >= n_items) break;
@@ -404,6 +407,8 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 
             // ---- weights: coalesced reads, then the operand layouts are built from shared memory ----
             float* raw = &S.p2[0][0];                               // 3,200 floats of scratch
+            if (member != staged_member) {
+            staged_member = member;
             {   // conv2 weights (offset 208) and linear weights (offset 3424) start 16-byte aligned
                 const float4* w2v = reinterpret_cast<const float4*>(prm + 208u);
                 const float4* wfv = reinterpret_cast<const float4*>(prm + 3424u);
@@ -443,6 +448,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             }
             fence_async_smem();
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+            }
             if (tid == 0) { S.n = n; __threadfence_block(); mbar_arrive(smem_u32(&S.item_ready)); }
 
             // After the 2x2 max (lanes ^1 = x parity, ^16 = y parity) done as a reduce-scatter, this
