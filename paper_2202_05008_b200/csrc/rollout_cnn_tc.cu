@@ -210,43 +210,48 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             const uint32_t gp = tile * 128u + row;                     // my pooled pixel = my TMEM lane
             const bool pix_ok = gp < n_pooled;
             const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
+            const size_t pix_off = pooled1_offset(0u, n_pairs, img, py, px);     // + member * member_stride
+            const size_t member_stride = static_cast<size_t>(n_pairs) * (12u * 2u * 12u);
 
             for (uint32_t gm = 0; gm < n_gm; ++gm, ++u) {
                 const uint32_t buf = u & 1u;
                 wait_or_abort(&ctl.abort, &ctl.mma_done[buf], (u >> 1) & 1u, status);
                 tc_fence_after();
-                const uint32_t t0 = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + buf * 256u;
-#pragma unroll 1
-                for (uint32_t chunk = 2u * half; chunk < 2u * half + 2u; ++chunk) {   // 16 filters = 2 members at a time
-                    uint32_t r0[16], r1[16], r2[16], r3[16];
-                    tmem_ld16_issue(t0 + 0u * 64u + chunk * 16u, r0);
-                    tmem_ld16_issue(t0 + 1u * 64u + chunk * 16u, r1);
-                    tmem_ld16_issue(t0 + 2u * 64u + chunk * 16u, r2);
-                    tmem_ld16_issue(t0 + 3u * 64u + chunk * 16u, r3);
-                    tmem_ld16_fence(r0); tmem_ld16_fence(r1); tmem_ld16_fence(r2); tmem_ld16_fence(r3);
-                    if (chunk == 2u * half + 1u) {                        // my part of the accumulator is in registers
+                const uint32_t t0 = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + buf * 256u + half * 32u;
+                // My four members of the unit, one at a time: the 8 filters of a member under the four
+                // pooling windows are 4 x 8 columns.  The loads of the next member are in flight while
+                // this one is pooled and stored (two register buffers).
+                uint32_t ra[4][8], rb[4][8];
+#pragma unroll
+                for (int w = 0; w < 4; ++w) tmem_ld8_issue(t0 + w * 64u, ra[w]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t (&cur)[4][8] = (j & 1) ? rb : ra;
+                    uint32_t (&nxt)[4][8] = (j & 1) ? ra : rb;
+                    tmem_ld8x4_fence(cur[0], cur[1], cur[2], cur[3]);
+                    if (j < 3) {
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) tmem_ld8_issue(t0 + w * 64u + (j + 1) * 8u, nxt[w]);
+                    } else {                                             // my part of the accumulator is in registers
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&ctl.acc_free[buf]));
                     }
-                    const uint32_t m0 = gm * 8u + chunk * 2u;            // first of the two members
-                    const float* bb = bias + m0 * 8u;
-                    uint32_t o[8];
+                    const uint32_t m = gm * 8u + half * 4u + j;
+                    const float4 b0 = *reinterpret_cast<const float4*>(bias + m * 8u);
+                    const float4 b1 = *reinterpret_cast<const float4*>(bias + m * 8u + 4u);
+                    const float bb[8] = { b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w };
+                    uint32_t o[4];
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const float v0 = fmaxf(fmaxf(__uint_as_float(r0[2 * c]), __uint_as_float(r1[2 * c])),
-                                               fmaxf(__uint_as_float(r2[2 * c]), __uint_as_float(r3[2 * c])));
-                        const float v1 = fmaxf(fmaxf(__uint_as_float(r0[2 * c + 1]), __uint_as_float(r1[2 * c + 1])),
-                                               fmaxf(__uint_as_float(r2[2 * c + 1]), __uint_as_float(r3[2 * c + 1])));
+                    for (int c = 0; c < 4; ++c) {
+                        const float v0 = fmaxf(fmaxf(__uint_as_float(cur[0][2 * c]), __uint_as_float(cur[1][2 * c])),
+                                               fmaxf(__uint_as_float(cur[2][2 * c]), __uint_as_float(cur[3][2 * c])));
+                        const float v1 = fmaxf(fmaxf(__uint_as_float(cur[0][2 * c + 1]), __uint_as_float(cur[1][2 * c + 1])),
+                                               fmaxf(__uint_as_float(cur[2][2 * c + 1]), __uint_as_float(cur[3][2 * c + 1])));
                         o[c] = pack_bf16(fmaxf(v0 + bb[2 * c], 0.f), fmaxf(v1 + bb[2 * c + 1], 0.f));
                     }
-                    if (pix_ok) {
-                        if (m0 < n_members)
-                            pooled1[pooled1_offset(group0 + m0, n_pairs, img, py, px)] = make_uint4(o[0], o[1], o[2], o[3]);
-                        if (m0 + 1u < n_members)
-                            pooled1[pooled1_offset(group0 + m0 + 1u, n_pairs, img, py, px)] = make_uint4(o[4], o[5], o[6], o[7]);
-                    }
-                    __syncwarp();
+                    if (pix_ok && m < n_members)
+                        pooled1[pix_off + static_cast<size_t>(group0 + m) * member_stride] = make_uint4(o[0], o[1], o[2], o[3]);
                 }
                 if (has_next && gm == stage_after) {
                     // the other A buffer was last read by the previous tile, whose accumulators have all
