@@ -62,6 +62,14 @@ __device__ __forceinline__ size_t pooled1_offset(uint32_t member, uint32_t n_pai
     return (((static_cast<size_t>(member) * n_pairs + (image >> 1)) * 12 + py) * 2 + (image & 1u)) * 12 + px;
 }
 
+// max of three values in one instruction (the 3-input form of max.f32)
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 // 6x6 image patch under one pooled pixel (zero for rows past the batch)
 __device__ __forceinline__ void c1_load_patch(const float* __restrict__ images, uint32_t gp, uint32_t n_pooled,
                                               float (&patch)[36])
@@ -241,14 +249,18 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     const float4 b0 = *reinterpret_cast<const float4*>(bias + m * 8u);
                     const float4 b1 = *reinterpret_cast<const float4*>(bias + m * 8u + 4u);
                     const float bb[8] = { b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w };
+                    // relu(max4 + b) = max(max4, -b) + b: two 3-input max and one add per value
                     uint32_t o[4];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const float v0 = fmaxf(fmaxf(__uint_as_float(cur[0][2 * c]), __uint_as_float(cur[1][2 * c])),
-                                               fmaxf(__uint_as_float(cur[2][2 * c]), __uint_as_float(cur[3][2 * c])));
-                        const float v1 = fmaxf(fmaxf(__uint_as_float(cur[0][2 * c + 1]), __uint_as_float(cur[1][2 * c + 1])),
-                                               fmaxf(__uint_as_float(cur[2][2 * c + 1]), __uint_as_float(cur[3][2 * c + 1])));
-                        o[c] = pack_bf16(fmaxf(v0 + bb[2 * c], 0.f), fmaxf(v1 + bb[2 * c + 1], 0.f));
+                        float v[2];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int k = 2 * c + h;
+                            const float m3 = fmax3(__uint_as_float(cur[0][k]), __uint_as_float(cur[1][k]), __uint_as_float(cur[2][k]));
+                            v[h] = fmax3(m3, __uint_as_float(cur[3][k]), -bb[k]) + bb[k];
+                        }
+                        o[c] = pack_bf16(v[0], v[1]);
                     }
                     if (pix_ok && m < n_members)
                         pooled1[pix_off + static_cast<size_t>(group0 + m) * member_stride] = make_uint4(o[0], o[1], o[2], o[3]);
