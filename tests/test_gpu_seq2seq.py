@@ -70,6 +70,25 @@ def test_tensor_core_and_cuda_core_kernels_agree_and_repeat():
     assert a.sync_status() == 0 and b.sync_status() == 0
 
 
+def test_bench_size_workload_sampled_members():
+    """The workload bench.py times (P = 1024, 128 queries, h = 128) in its launch configuration:
+    members sampled across the population (first, last, and the block-loop boundaries at multiples
+    of the SM count) against the oracle one by one; every fitness finite and below zero."""
+    w = W.SEQ2SEQ
+    s = Solver(w)
+    theta = s.ask()
+    fit = s.rollout().cpu().numpy()
+    assert s.sync_status() == 0
+    assert np.all(np.isfinite(fit)) and np.all(fit < 0.0)
+    h, nd = w.layer_sizes[0], int(w.task_param[0])
+    enc, dec, tgt = oracle.seq2seq_queries(w.seed, 0, w.batch, nd)
+    sm = torch.cuda.get_device_properties(0).multi_processor_count
+    for m in sorted({0, 1, sm - 1, sm, 2 * sm + 1, w.pop_size // 2, w.pop_size - 1}):
+        row = theta[m].cpu().numpy()
+        want = oracle.seq2seq_fitness(row, h, nd, enc, dec, tgt, True)[0]
+        assert abs(fit[m] - want) < FIT_TOL, (m, fit[m], want)
+
+
 def test_zero_parameters_and_generation_dependence():
     w = _workload(128, 3, 128, P=2, sigma=0.1)
     s = Solver(w)
