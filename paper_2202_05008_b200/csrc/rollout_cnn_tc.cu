@@ -297,14 +297,16 @@ constexpr int kC2Threads = kC2EpiThreads + 32;
 constexpr int kPairsPerItem = 16;
 constexpr uint32_t kPairBytes = 12 * 2 * 12 * 16;        // 4608
 constexpr int kC2Bufs = 4;
-constexpr int kP2Stride = 257;                           // odd pitch: image rows fall in distinct banks
+constexpr int kP2Stride = 258;                           // bf16 elements; 129 words: image rows fall in distinct banks
 constexpr uint32_t kNoItem = 0xFFFFFFFFu;
 
 struct __align__(128) C2Smem {
     unsigned char a[kC2Bufs][kPairBytes];                // pooled image pairs (ring)
     unsigned char b[26 * 2 * 128];                       // W2 as core matrices (tap, filter group)
     float wfT[256 * 12];                                 // linear layer transposed [k][class], bf16-rounded
-    float p2[2 * kPairsPerItem][kP2Stride];              // pooled-2 activations of the item's images
+    __align__(16) __nv_bfloat16 p2[2 * kPairsPerItem][kP2Stride];   // pooled-2 activations of the item's images (they are
+                                                         // bf16 operands of the linear layer anyway; half the size lets
+                                                         // four blocks share an SM)
     float logit[2 * kPairsPerItem][12];
     float b2[16];
     float bfc[12];
@@ -423,7 +425,8 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     c2_load_pair(S, (gp + i) % kC2Bufs, src + static_cast<size_t>(i) * kPairBytes);
 
             // ---- weights: coalesced reads, then the operand layouts are built from shared memory ----
-            float* raw = &S.p2[0][0];                               // 3,200 floats of scratch
+            float* raw = reinterpret_cast<float*>(&S.p2[0][0]);     // 3,200 floats of scratch
+            static_assert(sizeof(S.p2) >= 3200 * sizeof(float), "weight scratch fits in the activation buffer");
             if (member != staged_member) {
             staged_member = member;
             {   // conv2 weights (offset 208) and linear weights (offset 3424) start 16-byte aligned
@@ -504,10 +507,9 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                         r[c] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 16));
                     }
                     // activation index inside the item: (pixel, channel), channel innermost
-                    float* dst = S.p2[2 * i + im] + (py * 4 + px) * 16 + c0;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        dst[j] = __bfloat162float(__float2bfloat16_rn(fmaxf(r[j] + bias4[j], 0.f)));
+                    uint32_t* dst = reinterpret_cast<uint32_t*>(&S.p2[2 * i + im][(py * 4 + px) * 16 + c0]);
+                    dst[0] = pack_bf16(fmaxf(r[0] + bias4[0], 0.f), fmaxf(r[1] + bias4[1], 0.f));
+                    dst[1] = pack_bf16(fmaxf(r[2] + bias4[2], 0.f), fmaxf(r[3] + bias4[3], 0.f));
                 }
             }
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
@@ -520,19 +522,24 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 #pragma unroll
                 for (int j = 0; j < 12; ++j) acc[j] = 0.f;
                 if (lane < 2 * n) {
-                    const float* x = S.p2[lane] + 64 * warp;
+                    const uint32_t* x2 = reinterpret_cast<const uint32_t*>(&S.p2[lane][64 * warp]);   // two inputs per word
                     const float* wr = S.wfT + 64 * warp * 12;
-#pragma unroll 4
-                    for (int k = 0; k < 64; ++k) {
-                        const float xv = x[k];
-                        const float4 w0 = *reinterpret_cast<const float4*>(wr + k * 12);
-                        const float4 w1 = *reinterpret_cast<const float4*>(wr + k * 12 + 4);
-                        const float4 w2 = *reinterpret_cast<const float4*>(wr + k * 12 + 8);
-                        acc[0] = fmaf(w0.x, xv, acc[0]); acc[1] = fmaf(w0.y, xv, acc[1]);
-                        acc[2] = fmaf(w0.z, xv, acc[2]); acc[3] = fmaf(w0.w, xv, acc[3]);
-                        acc[4] = fmaf(w1.x, xv, acc[4]); acc[5] = fmaf(w1.y, xv, acc[5]);
-                        acc[6] = fmaf(w1.z, xv, acc[6]); acc[7] = fmaf(w1.w, xv, acc[7]);
-                        acc[8] = fmaf(w2.x, xv, acc[8]); acc[9] = fmaf(w2.y, xv, acc[9]);
+#pragma unroll 2
+                    for (int k2 = 0; k2 < 32; ++k2) {
+                        const uint32_t pair = x2[k2];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const float xv = __uint_as_float(h ? (pair & 0xFFFF0000u) : (pair << 16));
+                            const float* wk = wr + (2 * k2 + h) * 12;
+                            const float4 w0 = *reinterpret_cast<const float4*>(wk);
+                            const float4 w1 = *reinterpret_cast<const float4*>(wk + 4);
+                            const float4 w2 = *reinterpret_cast<const float4*>(wk + 8);
+                            acc[0] = fmaf(w0.x, xv, acc[0]); acc[1] = fmaf(w0.y, xv, acc[1]);
+                            acc[2] = fmaf(w0.z, xv, acc[2]); acc[3] = fmaf(w0.w, xv, acc[3]);
+                            acc[4] = fmaf(w1.x, xv, acc[4]); acc[5] = fmaf(w1.y, xv, acc[5]);
+                            acc[6] = fmaf(w1.z, xv, acc[6]); acc[7] = fmaf(w1.w, xv, acc[7]);
+                            acc[8] = fmaf(w2.x, xv, acc[8]); acc[9] = fmaf(w2.y, xv, acc[9]);
+                        }
                     }
                 }
                 float4* pw = reinterpret_cast<float4*>(part + (warp * 32 + lane) * 12);
@@ -627,7 +634,7 @@ int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uin
     const int c2_bytes = static_cast<int>(sizeof(C2Smem));
     if (cudaFuncSetAttribute(k_cnn_conv2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, c2_bytes) != cudaSuccess) return -1;
     const uint32_t n_items = P * ipm;
-    const uint32_t g2 = min(n_items, static_cast<uint32_t>(sm_count) * 3u);      // 3 blocks of ~72 KB per SM
+    const uint32_t g2 = min(n_items, static_cast<uint32_t>(sm_count) * 4u);      // 4 blocks of ~55 KB per SM
     k_cnn_conv2_tc<<<g2, kC2Threads, c2_bytes, st>>>(theta, ldD, P, pooled1, labels, batch, ipm, partial, counter, status);
     if (cudaGetLastError() != cudaSuccess) return -1;
     k_cnn_tc_finalize<<<(P + 255u) / 256u, 256, 0, st>>>(partial, P, ipm, batch, fitness);
