@@ -268,6 +268,11 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 if (has_next && gm == stage_after) {
                     // the other A buffer was last read by the previous tile, whose accumulators have all
                     // been waited for: refill it for the next tile
+                    // keep the conversion of the patch here: hoisted to the loads at the top of the tile it
+                    // would make every warp wait there for the images instead of letting them land under
+                    // the epilogues
+#pragma unroll
+                    for (int i = 0; i < 36; ++i) asm volatile("" : "+f"(patch[i]));
                     if (half) c1_stage_rows(Asm + ((ti + 1u) & 1u) * kC1SmemA, row, 1, patch);
                     else      c1_stage_rows(Asm + ((ti + 1u) & 1u) * kC1SmemA, row, 0, patch);
                     fence_async_smem();
