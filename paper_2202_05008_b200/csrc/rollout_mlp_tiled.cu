@@ -426,6 +426,7 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
     // seeded starts of both groups (lanes e < EB of the task warp keep the states in registers)
     const CartpoleConst cpc = cartpole_const(a.tp);
     CpState cps[2] = {};
+    float snc[2] = { 0.f, 0.f }, csc[2] = { 1.f, 1.f };    // sin/cos of the pole angle, carried from the observation
     float ret[2] = { 0.f, 0.f };
     if (tid < EB) {
 #pragma unroll
@@ -435,6 +436,7 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
             cps[g] = cartpole_reset(key, status->generation, min(ep, a.E - 1u), a.tp[EVO_CP_INIT_RANGE]);
             float sn, cs;
             sincos_fast(cps[g].th, sn, cs);
+            snc[g] = sn; csc[g] = cs;
             float* o = obs + g * NIN * EB;
             o[0 * EB + tid] = cps[g].x;  o[1 * EB + tid] = cps[g].xd;
             o[2 * EB + tid] = cs;        o[3 * EB + tid] = sn;
@@ -504,9 +506,10 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
             for (int off = EB; off < 32; off <<= 1) pre += __shfl_xor_sync(0xffffffffu, pre, off);
             const float force = a.action_scale * tanh_fast(pre + b3);
             if (tid < EB) {
-                cps[g] = cartpole_step_fast(cpc, cps[g], force);
+                cps[g] = cartpole_step_fast_sc(cpc, cps[g], force, snc[g], csc[g]);
                 float sn, cs;
                 sincos_fast(cps[g].th, sn, cs);
+                snc[g] = sn; csc[g] = cs;
                 ret[g] += cs * __expf(-cps[g].x * cps[g].x);       // reward on the post-step state
                 float* o = obs + g * NIN * EB;
                 o[0 * EB + tid] = cps[g].x;  o[1 * EB + tid] = cps[g].xd;

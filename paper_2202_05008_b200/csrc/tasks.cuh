@@ -103,10 +103,10 @@ __device__ __forceinline__ void sincos_fast(float th, float& sn, float& cs)
     sn = (q >= 2) ? -b : b;
 }
 
-__device__ __forceinline__ CpState cartpole_deriv_fast(const CartpoleConst& c, const CpState& s, float force)
+// derivative with sin/cos of s.th supplied by the caller
+__device__ __forceinline__ CpState cartpole_deriv_fast_sc(const CartpoleConst& c, const CpState& s, float force,
+                                                          float sn, float cs)
 {
-    float sn, cs;
-    sincos_fast(s.th, sn, cs);
     const float tmp = fmaf(c.pole_mass_length * s.thd * s.thd, sn, force) * c.inv_total;
     const float den = c.length * fmaf(-c.pole_mass * c.inv_total * cs, cs, 4.0f / 3.0f);
     const float th_acc = __fdividef(fmaf(c.gravity, sn, -cs * tmp), den);
@@ -114,10 +114,20 @@ __device__ __forceinline__ CpState cartpole_deriv_fast(const CartpoleConst& c, c
     return CpState{ s.xd, x_acc, s.thd, th_acc };
 }
 
-__device__ __forceinline__ CpState cartpole_step_fast(const CartpoleConst& c, const CpState& s, float force)
+__device__ __forceinline__ CpState cartpole_deriv_fast(const CartpoleConst& c, const CpState& s, float force)
+{
+    float sn, cs;
+    sincos_fast(s.th, sn, cs);
+    return cartpole_deriv_fast_sc(c, s, force, sn, cs);
+}
+
+// RK4 step; (sn, cs) = sin/cos of s.th, which a caller that has just computed the observation of s
+// already holds (the first stage then needs no sin/cos of its own; same arithmetic, same bits)
+__device__ __forceinline__ CpState cartpole_step_fast_sc(const CartpoleConst& c, const CpState& s, float force,
+                                                         float sn, float cs)
 {
     const float h = c.dt;
-    const CpState k1 = cartpole_deriv_fast(c, s, force);
+    const CpState k1 = cartpole_deriv_fast_sc(c, s, force, sn, cs);
     const CpState k2 = cartpole_deriv_fast(c, cp_axpy(s, 0.5f * h, k1), force);
     const CpState k3 = cartpole_deriv_fast(c, cp_axpy(s, 0.5f * h, k2), force);
     const CpState k4 = cartpole_deriv_fast(c, cp_axpy(s, h, k3), force);
@@ -128,6 +138,13 @@ __device__ __forceinline__ CpState cartpole_step_fast(const CartpoleConst& c, co
     n.th  = fmaf(w, (k1.th  + k4.th)  + 2.0f * (k2.th  + k3.th),  s.th);
     n.thd = fmaf(w, (k1.thd + k4.thd) + 2.0f * (k2.thd + k3.thd), s.thd);
     return n;
+}
+
+__device__ __forceinline__ CpState cartpole_step_fast(const CartpoleConst& c, const CpState& s, float force)
+{
+    float sn, cs;
+    sincos_fast(s.th, sn, cs);
+    return cartpole_step_fast_sc(c, s, force, sn, cs);
 }
 
 }  // namespace evo
