@@ -127,10 +127,25 @@ __device__ __forceinline__ CpState cartpole_step_fast_sc(const CartpoleConst& c,
                                                          float sn, float cs)
 {
     const float h = c.dt;
+    // sin/cos at the inner stages by rotating (sn, cs) through the stage's small angle increment d
+    // (Taylor to d^7 / d^8: error < 3e-6 even at |d| = 1, i.e. a pole speed of 100 rad/s at dt = 0.01)
+    auto stage = [&](const CpState& q, float d) {
+        const float z = d * d;
+        float sd = fmaf(z, -1.98412698e-4f, 8.33333333e-3f);
+        sd = fmaf(sd, z, -1.66666667e-1f);
+        sd = fmaf(sd * z, d, d);
+        float cd = fmaf(z, 2.48015873e-5f, -1.38888889e-3f);
+        cd = fmaf(cd, z, 4.16666667e-2f);
+        cd = fmaf(cd, z, -0.5f);
+        cd = fmaf(cd, z, 1.0f);
+        const float s2 = fmaf(sn, cd, cs * sd);
+        const float c2 = fmaf(cs, cd, -sn * sd);
+        return cartpole_deriv_fast_sc(c, q, force, s2, c2);
+    };
     const CpState k1 = cartpole_deriv_fast_sc(c, s, force, sn, cs);
-    const CpState k2 = cartpole_deriv_fast(c, cp_axpy(s, 0.5f * h, k1), force);
-    const CpState k3 = cartpole_deriv_fast(c, cp_axpy(s, 0.5f * h, k2), force);
-    const CpState k4 = cartpole_deriv_fast(c, cp_axpy(s, h, k3), force);
+    const CpState k2 = stage(cp_axpy(s, 0.5f * h, k1), 0.5f * h * k1.th);
+    const CpState k3 = stage(cp_axpy(s, 0.5f * h, k2), 0.5f * h * k2.th);
+    const CpState k4 = stage(cp_axpy(s, h, k3), h * k3.th);
     const float w = h * (1.0f / 6.0f);
     CpState n;
     n.x   = fmaf(w, (k1.x   + k4.x)   + 2.0f * (k2.x   + k3.x),   s.x);
