@@ -254,6 +254,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     // ---- reset (overlaps the copy) -----------------------------------------------------------
     CartpoleConst cpc{};
     CpState cps{};
+    float snc = 0.f, csc = 1.f;             // sin/cos of the pole angle, carried from the observation
     float ret = 0.f;                        // cart-pole: lane e of warp 0; tanh-linear: see below
     if (CART) {
         cpc = cartpole_const(a.tp);
@@ -261,6 +262,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
             cps = cartpole_reset(key, status->generation, e0 + min(tid, nE - 1), a.tp[EVO_CP_INIT_RANGE]);
             float sn, cs;
             sincos_fast(cps.th, sn, cs);
+            snc = sn; csc = cs;
             obs0[0 * EB + tid] = cps.x;  obs0[1 * EB + tid] = cps.xd;
             obs0[2 * EB + tid] = cs;     obs0[3 * EB + tid] = sn;
             obs0[4 * EB + tid] = cps.thd;
@@ -331,9 +333,10 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
                 L3.template run<true>(h2, actb, a.action_scale, NoHook{});
                 __syncwarp();
                 if (tid < EB) {
-                    cps = cartpole_step_fast(cpc, cps, actb[tid]);
+                    cps = cartpole_step_fast_sc(cpc, cps, actb[tid], snc, csc);
                     float sn, cs;
                     sincos_fast(cps.th, sn, cs);
+                    snc = sn; csc = cs;
                     ret += cs * __expf(-cps.x * cps.x);       // reward on the post-step state
                     obs[0 * EB + tid] = cps.x;  obs[1 * EB + tid] = cps.xd;
                     obs[2 * EB + tid] = cs;     obs[3 * EB + tid] = sn;
