@@ -54,6 +54,11 @@ enum { EVO_TASK_NONE = 0, EVO_TASK_CARTPOLE = 1, EVO_TASK_TANH_LINEAR = 2, EVO_T
 enum { EVO_ROLLOUT_AUTO = 0, EVO_ROLLOUT_GENERIC = 1, EVO_ROLLOUT_TILED = 2 };
 enum { EVO_OPT_ADAM = 0, EVO_OPT_CLIPUP = 1 };
 enum { EVO_SIGMA_CONSTANT = 0, EVO_SIGMA_PGPE = 1 };
+/* evo_config.debug_flags.  DROP_PARAM_COPY: the control-task roll-out kernels do not start the
+ * asynchronous copy of a member's parameter row, so the bounded wait for it must run out: every
+ * block raises EVO_ERR_TIMEOUT, writes NaN as its return and leaves (nothing is left in flight).
+ * It exists so that the time-out path can be tested without disturbing the device. */
+enum { EVO_DEBUG_DROP_PARAM_COPY = 1 };
 
 /* indices into evo_config.task_param for EVO_TASK_CARTPOLE */
 enum { EVO_CP_CART_MASS = 0, EVO_CP_POLE_MASS = 1, EVO_CP_POLE_HALF_LENGTH = 2, EVO_CP_GRAVITY = 3,
@@ -72,7 +77,7 @@ typedef struct evo_config {
     uint32_t struct_size;          /* sizeof(evo_config), checked                               */
     uint32_t pop_size;             /* P, even, >= 2                                             */
     uint64_t seed;                 /* Philox key of every random stream of this solver          */
-    uint32_t param_dim;            /* D >= 1                                                    */
+    uint32_t param_dim;            /* D, 1 .. 2^30                                              */
     uint32_t noise_mode;           /* EVO_NOISE_*: keep eps[H][ldD] from ask, or recompute it   */
     float    sigma;                /* > 0, constant                                             */
     float    lr;                   /* Adam step size                                            */
@@ -85,7 +90,7 @@ typedef struct evo_config {
     uint32_t episodes;             /* E >= 1 (control tasks)                                    */
     uint32_t horizon;              /* T >= 1 (control tasks)                                    */
     uint32_t batch;                /* images (supervised) or queries (seq2seq) per member       */
-    uint32_t trace_steps;          /* leading steps recorded when evo_rollout gets d_trace      */
+    uint32_t trace_steps;          /* leading steps recorded when evo_rollout gets d_trace, <= T */
     uint32_t rollout_kernel;       /* EVO_ROLLOUT_*: AUTO picks the tiled kernel when one fits  */
     float    task_param[16];       /* EVO_CP_* / EVO_S2S_* / EVO_PAINT_* by task; else unused   */
     uint32_t optimizer;            /* EVO_OPT_*: how the centre follows the ES gradient         */
@@ -96,6 +101,9 @@ typedef struct evo_config {
     float    sigma_max_change;     /* largest relative change of sigma per tell, 0 selects 0.2  */
     uint32_t shard_first_pair;     /* multi-GPU: first antithetic pair this solver owns         */
     uint32_t shard_pairs;          /* multi-GPU: pairs it owns; 0 = the whole population        */
+    uint32_t wait_cycles_log2;     /* a device-side wait gives up after 2^n SM clocks and raises
+                                      EVO_ERR_TIMEOUT; 0 selects 31 (about a second), else 10..40 */
+    uint32_t debug_flags;          /* EVO_DEBUG_* bits, 0 in production                          */
 } evo_config;
 
 /* Bytes of device workspace a solver with this configuration needs.  Pure host function. */
@@ -131,8 +139,9 @@ evo_status evo_ask(evo_solver* s, const float** d_theta, size_t* ld_theta);
  * the answer digits on `batch` queries the library draws itself.  Painting task (policy NONE: the
  * parameter row is param_dim / 10 triangles x0 y0 x1 y1 x2 y2 r g b a): -mean squared distance of
  * the painted canvas to the image bound with evo_set_target.
- * d_trace: NULL, or [P][E][trace_steps][state_dim] floats receiving the post-step task state
- * (state_dim = 4 cart-pole: x, x', theta, theta'; 28 tanh-linear).
+ * d_trace: NULL, or [P][E][trace_steps][state_dim] floats (16-byte aligned) receiving the
+ * post-step task state of the first trace_steps steps (state_dim = 4 cart-pole: x, x', theta,
+ * theta'; 28 tanh-linear); control tasks require trace_steps <= horizon at evo_create.
  * Errors: BAD_ORDER (d_theta NULL before any ask; supervised without a batch), INVALID_ARG,
  * UNSUPPORTED (task NONE), CUDA.
  */
@@ -245,7 +254,8 @@ evo_status evo_launch_count(evo_solver* s, uint64_t* launches);
  *     must use evo_create / evo_tell with a caller workspace.
  *   - The device that owns the buffers must be current.  The first call on each device looks
  *     up the array's device address (no allocation); make that first call outside of any
- *     stream capture.  No call allocates, frees or synchronises.
+ *     stream capture.  No call allocates, frees or synchronises.  The address is cached per
+ *     device for the life of the process: do not call again on a device after cudaDeviceReset.
  *   - All calls on a device share the one array, which keeps whatever the previous call left;
  *     each call overwrites every word it reads back, so nothing needs clearing.  Two calls
  *     whose kernels may overlap on the GPU (different streams, or the same stream from two
@@ -258,21 +268,8 @@ evo_status evo_es_gradient_static(const float* d_u, const float* d_eps, uint32_t
                                   uint32_t param_dim, size_t ld_eps, float sigma,
                                   float* d_gradient, void* cuda_stream);
 
-/*
- * Measurement aid, not part of the method (the paper has no counterpart): launches
- * blocks x threads threads that each run 16 independent chains of `iters` fp32 fused
- * multiply-adds in registers and store one float to d_sink[blocks*threads] (device memory, caller
- * owned).  *flops receives the floating-point operations of the launch (2 per FMA); dividing it
- * by the launch's CUDA-event time gives the fp32 FMA rate this device really sustains, the
- * denominator for kernels bound by plain fp32 arithmetic.  Asynchronous on cuda_stream.
- * Errors: INVALID_ARG (NULL pointer, zero size, threads not a multiple of 32 or above 1024),
- * CUDA (launch failed).
- */
-evo_status evo_fma_probe(float* d_sink, uint32_t blocks, uint32_t threads, uint32_t iters,
-                         void* cuda_stream, uint64_t* flops);
-
 const char* evo_status_string(evo_status st);
-uint32_t    evo_version(void);            /* major*10000 + minor*100 + patch */
+uint32_t    evo_version(void);            /* major*10000 + minor*100 + patch: 1.1.0 = 10100 */
 
 #ifdef __cplusplus
 }

@@ -21,6 +21,7 @@ EVO_MAX_LAYERS = 8
 STATUS = {0: "EVO_OK", 1: "EVO_ERR_INVALID_ARG", 2: "EVO_ERR_BAD_ORDER", 3: "EVO_ERR_WORKSPACE",
           4: "EVO_ERR_CUDA", 5: "EVO_ERR_NONFINITE", 6: "EVO_ERR_TIMEOUT", 7: "EVO_ERR_UNSUPPORTED"}
 ROLLOUT_AUTO, ROLLOUT_GENERIC, ROLLOUT_TILED = 0, 1, 2
+DEBUG_DROP_PARAM_COPY = 1
 
 
 class EvoConfig(C.Structure):
@@ -37,6 +38,7 @@ class EvoConfig(C.Structure):
         ("optimizer", C.c_uint32), ("clipup_momentum", C.c_float), ("clipup_max_speed", C.c_float),
         ("sigma_mode", C.c_uint32), ("sigma_lr", C.c_float), ("sigma_max_change", C.c_float),
         ("shard_first_pair", C.c_uint32), ("shard_pairs", C.c_uint32),
+        ("wait_cycles_log2", C.c_uint32), ("debug_flags", C.c_uint32),
     ]
 
 
@@ -69,7 +71,6 @@ def load_library():
     L.evo_get_reduce_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), szp]
     L.evo_tell_end.argtypes = [vp]
     L.evo_set_target.argtypes = [vp, vp]
-    L.evo_fma_probe.argtypes = [vp, C.c_uint32, C.c_uint32, C.c_uint32, vp, C.POINTER(C.c_uint64)]
     L.evo_destroy.argtypes = [vp]
     L.evo_set_batch.argtypes = [vp, vp, vp]
     L.evo_get_center.argtypes = [vp, C.POINTER(vp)]
@@ -89,7 +90,7 @@ def load_library():
     L.evo_status_string.restype = C.c_char_p
     L.evo_version.restype = C.c_uint32
     for name in ("evo_workspace_bytes", "evo_create", "evo_ask", "evo_rollout", "evo_tell", "evo_tell_begin",
-                 "evo_get_reduce_buffers", "evo_tell_end", "evo_fma_probe", "evo_set_target",
+                 "evo_get_reduce_buffers", "evo_tell_end", "evo_set_target",
                  "evo_destroy", "evo_set_batch", "evo_get_center", "evo_get_moments",
                  "evo_get_gradient", "evo_get_ranks", "evo_get_eps", "evo_get_sigma", "evo_set_sigma", "evo_get_counters",
                  "evo_set_state", "evo_sync_status", "evo_launch_count"):
@@ -99,7 +100,8 @@ def load_library():
 
 
 def make_config(w: W.Workload, *, trace_steps: int = 0, rollout_kernel: int = ROLLOUT_AUTO,
-                noise_mode: Optional[int] = None, shard_first_pair: int = 0, shard_pairs: int = 0) -> EvoConfig:
+                noise_mode: Optional[int] = None, shard_first_pair: int = 0, shard_pairs: int = 0,
+                wait_cycles_log2: int = 0, debug_flags: int = 0) -> EvoConfig:
     c = EvoConfig()
     c.struct_size = C.sizeof(EvoConfig)
     c.pop_size, c.param_dim, c.seed = w.pop_size, w.param_dim, w.seed
@@ -117,6 +119,7 @@ def make_config(w: W.Workload, *, trace_steps: int = 0, rollout_kernel: int = RO
     c.optimizer, c.clipup_momentum, c.clipup_max_speed = w.optimizer, w.clipup_momentum, w.clipup_max_speed
     c.sigma_mode, c.sigma_lr, c.sigma_max_change = w.sigma_mode, w.sigma_lr, w.sigma_max_change
     c.shard_first_pair, c.shard_pairs = shard_first_pair, shard_pairs
+    c.wait_cycles_log2, c.debug_flags = wait_cycles_log2, debug_flags
     return c
 
 
@@ -321,27 +324,3 @@ def es_gradient_static(u: torch.Tensor, eps: torch.Tensor, sigma: float,
         _check(lib.evo_es_gradient_static(u.data_ptr(), eps.data_ptr(), P, D, eps.stride(0), float(sigma),
                                           out.data_ptr(), st.cuda_stream), "evo_es_gradient_static")
     return out
-
-
-def fma_probe(device="cuda:0", iters: int = 1 << 14, repeats: int = 5, threads: int = 1024) -> float:
-    """Sustained fp32 FMA rate of `device` in TFLOP/s (best of `repeats` launches of
-    ``evo_fma_probe``, timed with CUDA events): the measured denominator for ALU-bound kernels."""
-    lib = load_library()
-    dev = torch.device(device)
-    with torch.cuda.device(dev):
-        sms = torch.cuda.get_device_properties(dev).multi_processor_count
-        blocks = sms * (2048 // threads) * 4
-        sink = torch.empty(blocks * threads, dtype=torch.float32, device=dev)
-        st = torch.cuda.current_stream(dev)
-        flops = C.c_uint64()
-        best = 0.0
-        for i in range(repeats + 2):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(st)
-            _check(lib.evo_fma_probe(sink.data_ptr(), blocks, threads, iters, st.cuda_stream, C.byref(flops)),
-                   "evo_fma_probe")
-            e1.record(st)
-            e1.synchronize()
-            if i >= 2:                                   # two warm-up launches
-                best = max(best, flops.value / (e0.elapsed_time(e1) * 1e-3) / 1e12)
-    return best

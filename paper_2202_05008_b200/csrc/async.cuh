@@ -37,8 +37,9 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void* src
 
 // Bounded wait.  try_wait is given a suspend-time hint, so a waiting warp sleeps in hardware
 // instead of taking issue slots from the warps that work; the loop re-arms it until the phase
-// completes or ~2^max_cycles_log2 SM clocks have passed.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t max_cycles_log2)
+// completes or ~2^(*max_cycles_log2) SM clocks have passed (the limit lives in the device status
+// block, so a test can make it short).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, const uint32_t* max_cycles_log2)
 {
     uint32_t done;
     asm volatile("{\n\t.reg .pred p;\n\t"
@@ -47,7 +48,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
                  : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     if (done) return true;
     const long long t0 = clock64();
-    const long long limit = 1ll << max_cycles_log2;
+    const long long limit = 1ll << *max_cycles_log2;      // read only once the wait has to sleep
     for (;;) {
         asm volatile("{\n\t.reg .pred p;\n\t"
                      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
@@ -57,6 +58,5 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
         if (clock64() - t0 > limit) return false;
     }
 }
-constexpr uint32_t kWaitCyclesLog2 = 31;      // ~1 s at 2 GHz
 
 }  // namespace evo

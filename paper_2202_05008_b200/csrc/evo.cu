@@ -25,6 +25,7 @@ struct evo_solver {
     const float*   d_target;
     uint64_t     launches;
     uint32_t     k0, k1;
+    bool         rollout_prepared;  // per-kernel attributes are set by the solver's first roll-out only
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -33,6 +34,7 @@ static evo_status check_config(const evo_config* c)
 {
     if (!c || c->struct_size != sizeof(evo_config)) return EVO_ERR_INVALID_ARG;
     if (c->pop_size < 2 || (c->pop_size & 1u) || c->param_dim < 1) return EVO_ERR_INVALID_ARG;
+    if (c->param_dim > kMaxParamDim) return EVO_ERR_INVALID_ARG;      // the row pitch must fit 32 bits
     if (!(c->sigma > 0.f) || !std::isfinite(c->sigma) || !std::isfinite(c->lr)) return EVO_ERR_INVALID_ARG;
     if (c->noise_mode > EVO_NOISE_REGENERATED) return EVO_ERR_INVALID_ARG;
     if (c->beta1 < 0.f || c->beta1 >= 1.f || c->beta2 < 0.f || c->beta2 >= 1.f || c->adam_eps < 0.f)
@@ -41,6 +43,8 @@ static evo_status check_config(const evo_config* c)
     if (c->optimizer > EVO_OPT_CLIPUP || c->sigma_mode > EVO_SIGMA_PGPE) return EVO_ERR_INVALID_ARG;
     if (c->clipup_momentum < 0.f || c->clipup_momentum >= 1.f || c->clipup_max_speed < 0.f) return EVO_ERR_INVALID_ARG;
     if (c->sigma_lr < 0.f || c->sigma_max_change < 0.f || c->sigma_max_change >= 1.f) return EVO_ERR_INVALID_ARG;
+    if (c->wait_cycles_log2 != 0 && (c->wait_cycles_log2 < 10 || c->wait_cycles_log2 > 40)) return EVO_ERR_INVALID_ARG;
+    if (c->debug_flags & ~static_cast<uint32_t>(EVO_DEBUG_DROP_PARAM_COPY)) return EVO_ERR_INVALID_ARG;
     if (c->shard_pairs > 0 &&
         (c->shard_first_pair >= c->pop_size / 2u || c->shard_pairs > c->pop_size / 2u - c->shard_first_pair))
         return EVO_ERR_INVALID_ARG;
@@ -50,6 +54,7 @@ static evo_status check_config(const evo_config* c)
         case EVO_TASK_TANH_LINEAR:
             if (c->policy_kind != EVO_POLICY_MLP) return EVO_ERR_INVALID_ARG;
             if (c->episodes < 1 || c->horizon < 1) return EVO_ERR_INVALID_ARG;
+            if (c->trace_steps > c->horizon) return EVO_ERR_INVALID_ARG;   // the trace pitch is trace_steps
             if (!rollout_mlp_supported(*c)) return EVO_ERR_INVALID_ARG;
             if (c->task_kind == EVO_TASK_CARTPOLE) {
                 const float* tp = c->task_param;
@@ -164,6 +169,7 @@ evo_status evo_create(const evo_config* cfg_in, void* d_workspace, size_t worksp
     if (s->cfg.clipup_max_speed == 0.f) s->cfg.clipup_max_speed = 2.f * s->cfg.lr;
     if (s->cfg.sigma_lr == 0.f) s->cfg.sigma_lr = 0.1f;
     if (s->cfg.sigma_max_change == 0.f) s->cfg.sigma_max_change = 0.2f;
+    if (s->cfg.wait_cycles_log2 == 0) s->cfg.wait_cycles_log2 = 31;       // ~1 s at 2 GHz
     make_layout(s->cfg, &s->lay);
     if (workspace_bytes < s->lay.total) { delete s; return EVO_ERR_WORKSPACE; }
     s->ws = static_cast<char*>(d_workspace);
@@ -178,6 +184,7 @@ evo_status evo_create(const evo_config* cfg_in, void* d_workspace, size_t worksp
     s->d_labels = nullptr;
     s->d_target = nullptr;
     s->launches = 0;
+    s->rollout_prepared = false;
     s->k0 = static_cast<uint32_t>(s->cfg.seed & 0xFFFFFFFFull);
     s->k1 = static_cast<uint32_t>(s->cfg.seed >> 32);
     const Layout& L = s->lay;
@@ -185,7 +192,8 @@ evo_status evo_create(const evo_config* cfg_in, void* d_workspace, size_t worksp
                         reinterpret_cast<float*>(s->ws + L.m), reinterpret_cast<float*>(s->ws + L.v),
                         reinterpret_cast<float*>(s->ws + L.g), reinterpret_cast<float*>(s->ws + L.sigma),
                         s->cfg.sigma, s->cfg.param_dim, L.ldD,
-                        reinterpret_cast<DeviceStatus*>(s->ws + L.status));
+                        reinterpret_cast<DeviceStatus*>(s->ws + L.status), s->cfg.wait_cycles_log2,
+                        s->cfg.debug_flags);
     if (n < 0) { delete s; return EVO_ERR_CUDA; }
     s->launches += n;
     n = launch_task_constants(s->stream, s->cfg.task_kind, s->k0, s->k1,
@@ -260,6 +268,7 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
         return EVO_OK;
     }
     if (d_trace && c.trace_steps == 0) return EVO_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_trace) & 15u) return EVO_ERR_INVALID_ARG;   // written with 128-bit stores
     if (c.task_kind == EVO_TASK_PAINT) {
         if (!s->d_target) return EVO_ERR_BAD_ORDER;
         const int n = launch_rollout_paint(s->stream, d_theta, L.ldD, s->local_pop, c.param_dim,
@@ -301,9 +310,11 @@ evo_status evo_rollout(evo_solver* s, const float* d_theta, float* d_fitness, fl
     a.trace_T = c.trace_steps < c.horizon ? c.trace_steps : c.horizon;
     a.k0 = s->k0; a.k1 = s->k1;
     std::memcpy(a.tp, c.task_param, sizeof(a.tp));
+    a.attr_done = s->rollout_prepared ? 1u : 0u;
     const int n = launch_rollout_mlp(s->stream, a, c.rollout_kernel, d_fitness,
                                      reinterpret_cast<DeviceStatus*>(s->ws + L.status));
     if (n < 0) return n == -2 ? EVO_ERR_UNSUPPORTED : EVO_ERR_CUDA;
+    s->rollout_prepared = true;
     s->launches += n;
     return EVO_OK;
 }
@@ -535,6 +546,6 @@ const char* evo_status_string(evo_status st)
     return "unknown status";
 }
 
-uint32_t evo_version(void) { return 103; }
+uint32_t evo_version(void) { return 10100; }   // 1.1.0
 
 }  // extern "C"

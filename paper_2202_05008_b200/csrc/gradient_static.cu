@@ -18,7 +18,9 @@ constexpr size_t kStaticScratchDoubles = EVO_STATIC_SCRATCH_BYTES / sizeof(doubl
 static __device__ __align__(256) double g_static_scratch[kStaticScratchDoubles];
 
 // In host code the name above is only a handle for the runtime, not a device address; the
-// address each device maps it to is looked up once per device and cached here.
+// address each device maps it to is looked up once per device and cached here.  The cached
+// address belongs to the device's primary context: after cudaDeviceReset it is stale, so a
+// process that resets a device must not call this entry point on it again.
 constexpr int kMaxDevices = 64;
 static double*    g_scratch_ptr[kMaxDevices] = {};
 static std::mutex g_scratch_mutex;
@@ -89,8 +91,9 @@ extern "C" evo_status evo_es_gradient_static(const float* d_u, const float* d_ep
     if (!d_u || !d_eps || !d_gradient) return EVO_ERR_INVALID_ARG;
     if (pop_size < 2 || (pop_size & 1u) || param_dim < 1 || ld_eps < param_dim) return EVO_ERR_INVALID_ARG;
     const uint32_t H = pop_size / 2u;
+    // the size check comes first and in 64 bits: rounding a huge param_dim up must not wrap to 0
+    if ((static_cast<size_t>(param_dim) + 31u) / 32u * 32u > kStaticScratchDoubles) return EVO_ERR_WORKSPACE;
     const uint32_t ldS = (param_dim + 31u) / 32u * 32u;             // row pitch inside the scratch
-    if (static_cast<size_t>(ldS) > kStaticScratchDoubles) return EVO_ERR_WORKSPACE;
     // as many splits as the plan for this shape wants, but no more than the fixed array holds
     uint32_t splits = gradient_splits(H, ldS);
     const size_t fit = kStaticScratchDoubles / ldS;

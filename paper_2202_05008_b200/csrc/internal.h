@@ -14,11 +14,14 @@ struct DeviceStatus {
     uint32_t nonfinite;     // set by the rank kernel of the current tell, cleared by its finish
     uint32_t adam_step;     // t
     uint32_t generation;    // counter word of every random stream; advanced by the kernel that closes a tell
+    uint32_t wait_cycles_log2;  // every bounded device-side wait gives up after 2^this SM clocks
+    uint32_t debug_flags;   // EVO_DEBUG_* bits of the configuration
 };
 
 constexpr uint32_t kTlNx = 28;   // tanh-linear task: state width
 constexpr uint32_t kTlNa = 8;    // tanh-linear task: action width
 constexpr uint32_t kCnnParams = 5994;
+constexpr uint32_t kMaxParamDim = 1u << 30;   // keeps ldD = round_up(D, 32) and 4 * ldD inside 32 bits
 
 struct RolloutMlpArgs {
     const float* theta;          // [P][ldD]
@@ -36,6 +39,7 @@ struct RolloutMlpArgs {
     uint32_t k0, k1;             // the generation is read from the device status by the kernels
     float    tp[16];
     uint32_t weights_in_smem;
+    uint32_t attr_done;          // the kernel's dynamic shared-memory limit was raised by an earlier launch of this solver
 };
 
 struct Layout {                  // byte offsets into the workspace
@@ -47,7 +51,8 @@ struct Layout {                  // byte offsets into the workspace
 
 // ---- launchers (each returns the number of kernels it launched, or -1 on a launch error) ----
 int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, float* sigma_vec,
-                float sigma, uint32_t D, uint32_t ldD, DeviceStatus* status);
+                float sigma, uint32_t D, uint32_t ldD, DeviceStatus* status, uint32_t wait_cycles_log2,
+                uint32_t debug_flags);
 int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t k1, float* task_const);
 int launch_ask(cudaStream_t st, const float* center, const float* sigma_vec, uint32_t k0, uint32_t k1,
                const DeviceStatus* status, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* theta,

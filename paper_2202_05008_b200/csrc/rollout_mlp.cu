@@ -239,7 +239,8 @@ int launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a_in, uint32_t ker
         a.weights_in_smem = 1;
         if (bytes > 200u * 1024u) { a.weights_in_smem = 0; bytes = generic_smem_bytes(a, false); }
         if (bytes > 200u * 1024u) return -2;
-        if (cudaFuncSetAttribute(k_rollout_mlp_generic, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (!a.attr_done &&
+            cudaFuncSetAttribute(k_rollout_mlp_generic, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(bytes)) != cudaSuccess) return -1;
         dim3 grid(a.P, a.n_eb);
         k_rollout_mlp_generic<<<grid, kGenericThreads, bytes, st>>>(a, status);

@@ -248,7 +248,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     const uint32_t bar = smem_u32(&mbar);
     if (tid == 0) { mbar_init(bar, 1); mbar_init_fence(); }
     __syncthreads();
-    if (tid == 0)       // the member's whole parameter row in one bulk copy
+    if (tid == 0 && !(status->debug_flags & EVO_DEBUG_DROP_PARAM_COPY))   // the member's whole parameter row in one bulk copy
         bulk_copy_g2s(smem_u32(stage), a.theta + static_cast<size_t>(member) * a.ldD, a.ldD * 4u, bar);
 
     // ---- reset (overlaps the copy) -----------------------------------------------------------
@@ -279,11 +279,14 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     // one thread waits (bounded) and publishes the outcome, so the whole block takes one branch
     __shared__ int copy_ok;
     if (tid == 0) {
-        copy_ok = mbar_wait_bounded(bar, 0u, kWaitCyclesLog2) ? 1 : 0;
+        copy_ok = mbar_wait_bounded(bar, 0u, &status->wait_cycles_log2) ? 1 : 0;
         if (!copy_ok) {
-            // the copy did not land in time: flag it, give it one more bounded chance, leave
+            // the copy did not land in time: flag it, give it one more bounded chance (so that it is
+            // not still writing into shared memory that the next block gets), and leave a NaN as
+            // this block's return: the member's fitness is then NaN and tell skips the update
             atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
-            mbar_wait_bounded(bar, 0u, kWaitCyclesLog2);
+            mbar_wait_bounded(bar, 0u, &status->wait_cycles_log2);
+            a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = __int_as_float(0x7FC00000);
         }
     }
     __syncthreads();
@@ -427,7 +430,7 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
     const uint32_t bar = smem_u32(&mbar);
     if (tid == 0) { mbar_init(bar, 1); mbar_init_fence(); }
     __syncthreads();
-    if (tid == 0)       // the member's whole parameter row in one bulk copy
+    if (tid == 0 && !(status->debug_flags & EVO_DEBUG_DROP_PARAM_COPY))   // the member's whole parameter row in one bulk copy
         bulk_copy_g2s(smem_u32(stage), a.theta + static_cast<size_t>(member) * a.ldD, a.ldD * 4u, bar);
     // seeded starts of both groups (lanes e < EB of the task warp keep the states in registers)
     const CartpoleConst cpc = cartpole_const(a.tp);
@@ -450,10 +453,11 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
         }
     }
     if (tid == 0) {
-        copy_ok = mbar_wait_bounded(bar, 0u, kWaitCyclesLog2) ? 1 : 0;
-        if (!copy_ok) {
+        copy_ok = mbar_wait_bounded(bar, 0u, &status->wait_cycles_log2) ? 1 : 0;
+        if (!copy_ok) {                                   // as in k_rollout_mlp_tiled
             atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
-            mbar_wait_bounded(bar, 0u, kWaitCyclesLog2);
+            mbar_wait_bounded(bar, 0u, &status->wait_cycles_log2);
+            a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = __int_as_float(0x7FC00000);
         }
     }
     __syncthreads();
@@ -583,7 +587,8 @@ static int launch_one(K kernel, int threads, size_t act_floats, cudaStream_t st,
 {
     const size_t bytes = (static_cast<size_t>(a.ldD) + act_floats) * sizeof(float);
     if (bytes > 220u * 1024u) return -2;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) != cudaSuccess)
+    if (!a.attr_done &&
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) != cudaSuccess)
         return -1;
     dim3 grid(a.P, a.n_eb);
     kernel<<<grid, threads, bytes, st>>>(a, status);

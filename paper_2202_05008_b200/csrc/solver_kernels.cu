@@ -10,17 +10,23 @@ namespace evo {
 // init / task constants
 // ------------------------------------------------------------------------------------------
 __global__ void k_init(float* center, float* m, float* v, float* g, float* sigma_vec, float sigma,
-                       uint32_t D, uint32_t ldD, DeviceStatus* status)
+                       uint32_t D, uint32_t ldD, DeviceStatus* status, uint32_t wait_cycles_log2,
+                       uint32_t debug_flags)
 {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < ldD) { center[i] = 0.f; m[i] = 0.f; v[i] = 0.f; g[i] = 0.f; sigma_vec[i] = (i < D) ? sigma : 0.f; }
-    if (i == 0) { status->sticky = 0; status->nonfinite = 0; status->adam_step = 0; status->generation = 0; }
+    if (i == 0) {
+        status->sticky = 0; status->nonfinite = 0; status->adam_step = 0; status->generation = 0;
+        status->wait_cycles_log2 = wait_cycles_log2; status->debug_flags = debug_flags;
+    }
 }
 
 int launch_init(cudaStream_t st, float* center, float* m, float* v, float* g, float* sigma_vec,
-                float sigma, uint32_t D, uint32_t ldD, DeviceStatus* status)
+                float sigma, uint32_t D, uint32_t ldD, DeviceStatus* status, uint32_t wait_cycles_log2,
+                uint32_t debug_flags)
 {
-    k_init<<<(ldD + 255) / 256, 256, 0, st>>>(center, m, v, g, sigma_vec, sigma, D, ldD, status);
+    k_init<<<(ldD + 255) / 256, 256, 0, st>>>(center, m, v, g, sigma_vec, sigma, D, ldD, status,
+                                              wait_cycles_log2, debug_flags);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

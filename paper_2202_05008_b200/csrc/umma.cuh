@@ -78,7 +78,7 @@ __device__ __forceinline__ void wait_or_abort(volatile int* abort_flag, uint64_t
                                               DeviceStatus* status)
 {
     if (*abort_flag) return;
-    if (!mbar_wait_bounded(smem_u32(bar), parity, kWaitCyclesLog2)) {
+    if (!mbar_wait_bounded(smem_u32(bar), parity, &status->wait_cycles_log2)) {
         *abort_flag = 1;
         atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
     }

@@ -60,6 +60,16 @@ def test_bad_configs_are_rejected(lib):
                dict(layer_sizes=(4, 16, 16, 1)), dict(episodes=0)):
         cfg = make_config(w.with_(**kw))
         assert lib.evo_workspace_bytes(C.byref(cfg), C.byref(n)) == 1, kw
+    # the row pitch must fit 32 bits; the trace covers at most the horizon; the wait limit and the
+    # debug bits are range-checked
+    assert lib.evo_workspace_bytes(C.byref(make_config(pk.workloads.CFG5.with_(param_dim=(1 << 30) + 1))), C.byref(n)) == 1
+    assert lib.evo_workspace_bytes(C.byref(make_config(pk.workloads.CFG5.with_(param_dim=0xFFFFFFF0))), C.byref(n)) == 1
+    assert lib.evo_workspace_bytes(C.byref(make_config(w, trace_steps=w.horizon + 1)), C.byref(n)) == 1
+    assert lib.evo_workspace_bytes(C.byref(make_config(w, trace_steps=w.horizon)), C.byref(n)) == 0
+    assert lib.evo_workspace_bytes(C.byref(make_config(w, wait_cycles_log2=9)), C.byref(n)) == 1
+    assert lib.evo_workspace_bytes(C.byref(make_config(w, wait_cycles_log2=41)), C.byref(n)) == 1
+    assert lib.evo_workspace_bytes(C.byref(make_config(w, wait_cycles_log2=16, debug_flags=1)), C.byref(n)) == 0
+    assert lib.evo_workspace_bytes(C.byref(make_config(w, debug_flags=2)), C.byref(n)) == 1
     assert lib.evo_workspace_bytes(None, C.byref(n)) == 1
     assert lib.evo_workspace_bytes(C.byref(make_config(w)), None) == 1
     # create without a workspace / with a misaligned one fails before any CUDA call
@@ -68,7 +78,7 @@ def test_bad_configs_are_rejected(lib):
     assert lib.evo_create(C.byref(make_config(w)), 0x1001, 1 << 20, None, C.byref(h)) == 1
     assert lib.evo_ask(None, None, None) == 1 and lib.evo_tell(None, None) == 1
     assert lib.evo_status_string(5).decode().startswith("non-finite")
-    assert lib.evo_version() >= 100
+    assert lib.evo_version() == 10100                     # 1.1.0 as major*10000 + minor*100 + patch
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

@@ -49,6 +49,42 @@ def test_rollout_argument_errors():
     assert lib.evo_rollout(s._h, None, fit.data_ptr(), None) == 0
     assert s.sync_status() == 0
     s.close()
+    # the trace is written with 128-bit stores: a pointer that is only 4-byte aligned is refused
+    s = Solver(W.CFG1.with_(horizon=10), trace_steps=10)
+    s.ask()
+    trace = torch.zeros(16 * 10 * 4 + 4, device="cuda")
+    assert lib.evo_rollout(s._h, None, fit.data_ptr(), trace.data_ptr() + 4) == 1
+    assert lib.evo_rollout(s._h, None, fit.data_ptr(), trace.data_ptr()) == 0
+    assert s.sync_status() == 0
+    s.close()
+
+
+@pytest.mark.parametrize("w", [W.CFG1.with_(horizon=5), W.CFG2.with_(pop_size=4, horizon=5),
+                               W.CFG4.with_(pop_size=4, horizon=5)])
+def test_a_device_wait_that_runs_out_raises_timeout_and_leaves_the_solver_usable(w):
+    """The failure path of the bounded waits, made to happen without disturbing the device: with
+    EVO_DEBUG_DROP_PARAM_COPY the roll-out blocks never start the copy they wait for, and with a
+    limit of 2^16 clocks the wait gives up after ~30 us.  Every block must return by itself, raise
+    EVO_ERR_TIMEOUT and report NaN; evo_sync_status must report the condition once and clear it; a
+    tell on that fitness must skip the update (NaN fitness)."""
+    from paper_2202_05008_b200.binding import DEBUG_DROP_PARAM_COPY
+    s = Solver(w, wait_cycles_log2=16, debug_flags=DEBUG_DROP_PARAM_COPY)
+    s.ask()
+    fit = s.rollout()
+    assert s.sync_status() == 6                        # EVO_ERR_TIMEOUT, reported ...
+    assert s.sync_status() == 0                        # ... once
+    assert bool(torch.isnan(fit).all())
+    c0 = s.center().clone()
+    s.tell(fit)
+    assert s.sync_status() == 5                        # NaN fitness: update skipped
+    assert torch.equal(s.center(), c0) and s.counters() == (1, 0)
+    s.close()
+    # the same configuration without the flag runs normally afterwards on the same device
+    s = Solver(w, wait_cycles_log2=22)
+    s.ask()
+    fit = s.rollout()
+    assert s.sync_status() == 0 and bool(torch.isfinite(fit).all())
+    s.close()
 
 
 @pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_TILED])
@@ -92,16 +128,17 @@ def test_cnn_single_image_batch():
 
 
 def test_fma_probe_reports_a_plausible_fp32_rate_and_rejects_bad_shapes():
+    """The probe is bench.py's measurement aid (its own shared object beside bench.py)."""
     import ctypes as C
-    from paper_2202_05008_b200 import binding
-    rate = binding.fma_probe(iters=1 << 12, repeats=2)
+    import bench
+    rate = bench.fma_probe(iters=1 << 12, repeats=2)
     assert 5.0 < rate < 200.0                          # TFLOP/s; nominal is about 74
-    lib = binding.load_library()
+    lib = bench._probe
     sink = torch.empty(1024, dtype=torch.float32, device="cuda")
     flops = C.c_uint64()
-    assert lib.evo_fma_probe(sink.data_ptr(), 1, 48, 8, None, C.byref(flops)) == 1      # not a warp multiple
-    assert lib.evo_fma_probe(None, 1, 32, 8, None, C.byref(flops)) == 1
-    assert lib.evo_fma_probe(sink.data_ptr(), 1, 1024, 8, None, C.byref(flops)) == 0
+    assert lib.bench_fma_probe(sink.data_ptr(), 1, 48, 8, None, C.byref(flops)) == 1      # not a warp multiple
+    assert lib.bench_fma_probe(None, 1, 32, 8, None, C.byref(flops)) == 1
+    assert lib.bench_fma_probe(sink.data_ptr(), 1, 1024, 8, None, C.byref(flops)) == 0
     torch.cuda.synchronize()
     assert flops.value == 2 * 16 * 8 * 1024
 

@@ -50,6 +50,24 @@ def test_cnn_random_large_parameters_ragged_batch(kernel):
     _run(w, theta_np=W.random_parameters(5, 4, W.CNN_PARAMS, scale=0.2), kernel=kernel)
 
 
+def test_cnn_tensor_core_path_against_the_unrounded_oracle():
+    """Against the fp64 oracle with NO bf16 rounding (the mode pinned to torch's conv2d): the bound
+    is the kernel's own 1e-3 plus the gap between the two oracle modes, which a CPU test pins
+    (tests/test_oracle_bf16_gap.py), so the rounding points the kernel shares with the bf16 oracle
+    are bounded by something the kernel did not shape."""
+    w = W.CFG3.with_(pop_size=16, batch=256)
+    s = Solver(w)
+    images, labels = W.image_batch(w.seed, 0, w.batch)
+    s.set_batch(torch.tensor(images, device="cuda"), torch.tensor(labels, device="cuda"))
+    theta = s.ask().cpu().numpy()
+    fit = s.rollout().cpu().numpy()
+    assert s.sync_status() == 0
+    members = [0, 1, 7, 8, 15]
+    want = np.array([oracle.cnn_fitness(theta[m], images, labels, False) for m in members])
+    assert rel_err(fit[members], want, floor=1.0) < 2e-3
+    s.close()
+
+
 def test_cnn_more_than_one_member_group_and_tiny_batch():
     # 70 members = two conv1 groups (64 + 6); batch 3 = one full pair and one half pair
     w = W.CFG3.with_(pop_size=70, batch=3)

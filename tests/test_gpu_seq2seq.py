@@ -59,6 +59,23 @@ def test_tensor_core_kernel_matches_oracle(B):
     assert np.std(fit) > 1e-3                                    # members really differ
 
 
+@pytest.mark.parametrize("kernel", [ROLLOUT_TILED, ROLLOUT_GENERIC])
+def test_kernels_against_the_unrounded_oracle(kernel):
+    """Against the fp64 oracle with NO bf16 rounding (the mode pinned to torch.nn.LSTM): bound =
+    the kernel's 1e-3 plus the gap between the two oracle modes pinned on the CPU
+    (tests/test_oracle_bf16_gap.py), so the rounding points are not only checked against an oracle
+    that rounds at the same places."""
+    w = _workload(128, 3, 128, P=4, sigma=0.1)
+    s = Solver(w, rollout_kernel=kernel)
+    theta = s.ask().cpu().numpy()
+    fit = s.rollout().cpu().numpy()
+    assert s.sync_status() == 0
+    enc, dec, tgt = oracle.seq2seq_queries(w.seed, 0, w.batch, 3)
+    for m in range(w.pop_size):
+        want = oracle.seq2seq_fitness(theta[m], 128, 3, enc, dec, tgt, False)[0]
+        assert abs(fit[m] - want) / max(abs(want), 1.0) < 2e-3, (m, fit[m], want)
+
+
 def test_tensor_core_and_cuda_core_kernels_agree_and_repeat():
     w = _workload(128, 3, 128, P=150, sigma=0.05)                # more items than SMs: blocks loop
     a = Solver(w, rollout_kernel=ROLLOUT_TILED)

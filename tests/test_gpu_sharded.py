@@ -51,6 +51,74 @@ def test_sharded_cartpole_generations_match_unsharded(world, noise):
     assert all(s.sync_status() == 0 for s in shards) and full.sync_status() == 0
 
 
+def _sharded_generation_by_hand(shards, fit_all=None):
+    """ask -> rollout -> tell on every shard in turn, the two exchanges done by hand: fitness shards
+    concatenated in member order, reduce buffers summed and handed back to every shard."""
+    thetas = [s.ask() for s in shards]
+    if fit_all is None:
+        fit_all = torch.cat([s.rollout().clone() for s in shards])
+    for s in shards:
+        s.tell_begin(fit_all)
+    bufs = [s.reduce_buffers() for s in shards]
+    g = torch.stack([b[0] for b in bufs]).sum(0)
+    for s, b in zip(shards, bufs):
+        b[0].copy_(g)
+        s.tell_end()
+    return thetas, fit_all
+
+
+@pytest.mark.parametrize("world", [2, 8])
+def test_sharded_large_population_tanh_linear_matches_unsharded(world):
+    """The large-population control configuration (4,096 members, MLP 28-128-128-8, 4 episodes) in
+    pair shards, horizon cut to 50 steps: rows and fitness bit-equal to the unsharded solver, centre
+    within 1e-6, shards bit-identical among themselves."""
+    w = W.CFG4.with_(horizon=50)
+    full = binding.Solver(w)
+    theta_full = full.ask()
+    fit_full = full.rollout().clone()
+    full.tell(fit_full)
+    shards = _shards(w, world)
+    thetas, fit_all = _sharded_generation_by_hand(shards)
+    per = w.pop_size // world
+    for r in (0, world - 1):                                        # first and last shard's rows
+        assert torch.equal(thetas[r], theta_full[r * per:(r + 1) * per])
+    assert torch.equal(fit_all, fit_full)
+    c_full = full.center().cpu().numpy()
+    for s in shards:
+        assert rel_err(s.center().cpu().numpy(), c_full) < 1e-6
+    for s in shards[1:]:
+        assert torch.equal(s.center(), shards[0].center())
+    assert all(s.sync_status() == 0 for s in shards) and full.sync_status() == 0
+    for s in shards:
+        s.close()
+    full.close()
+
+
+@pytest.mark.parametrize("world", [2, 8])
+def test_sharded_update_sweep_with_regenerated_noise_matches_unsharded(world):
+    """The update-bandwidth configuration (16,384 members, no task, regenerated noise) at a reduced
+    parameter count (D = 8,200, not a multiple of 32): every shard recomputes the noise of its own
+    pairs from the global pair index in ask and again in tell."""
+    w = W.CFG5.with_(param_dim=8200)
+    full = binding.Solver(w, noise_mode=W.NOISE_REGENERATED)
+    shards = _shards(w, world, noise_mode=W.NOISE_REGENERATED)
+    per = w.pop_size // world
+    for gen in range(2):
+        fit = torch.tensor(W.synthetic_fitness(w.seed, gen, w.pop_size), device="cuda")
+        theta_full = full.ask()
+        full.tell(fit)
+        thetas, _ = _sharded_generation_by_hand(shards, fit_all=fit)
+        for r in (0, world // 2, world - 1):
+            assert torch.equal(thetas[r], theta_full[r * per:(r + 1) * per])
+        assert rel_err(shards[0].center().cpu().numpy(), full.center().cpu().numpy()) < 1e-6
+        for s in shards[1:]:
+            assert torch.equal(s.center(), shards[0].center())
+    assert all(s.sync_status() == 0 for s in shards) and full.sync_status() == 0
+    for s in shards:
+        s.close()
+    full.close()
+
+
 def test_sharded_sigma_adaptation_and_clipup_match_oracle():
     w = W.CFG1.with_(pop_size=32, optimizer=W.OPT_CLIPUP, sigma_mode=W.SIGMA_PGPE,
                             sigma_lr=0.2, sigma_max_change=0.2, lr=0.15, clipup_max_speed=0.3)
