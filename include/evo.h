@@ -54,11 +54,13 @@ enum { EVO_TASK_NONE = 0, EVO_TASK_CARTPOLE = 1, EVO_TASK_TANH_LINEAR = 2, EVO_T
 enum { EVO_ROLLOUT_AUTO = 0, EVO_ROLLOUT_GENERIC = 1, EVO_ROLLOUT_TILED = 2 };
 enum { EVO_OPT_ADAM = 0, EVO_OPT_CLIPUP = 1 };
 enum { EVO_SIGMA_CONSTANT = 0, EVO_SIGMA_PGPE = 1 };
-/* evo_config.debug_flags.  DROP_PARAM_COPY: the control-task roll-out kernels do not start the
- * asynchronous copy of a member's parameter row, so the bounded wait for it must run out: every
- * block raises EVO_ERR_TIMEOUT, writes NaN as its return and leaves (nothing is left in flight).
- * It exists so that the time-out path can be tested without disturbing the device. */
-enum { EVO_DEBUG_DROP_PARAM_COPY = 1 };
+/* evo_config.debug_flags.  DROP_COMPLETION: the control-task roll-out kernels leave out the
+ * asynchronous completion their first bounded wait depends on (the copy of a member's parameter
+ * row; in the tensor-core kernel the commit of the first batch of MMAs), so that wait must run
+ * out: every block raises EVO_ERR_TIMEOUT, reports NaN as its return and leaves by itself, with
+ * nothing left in flight.  It exists so that the time-out path can be tested without disturbing
+ * the device. */
+enum { EVO_DEBUG_DROP_COMPLETION = 1 };
 
 /* indices into evo_config.task_param for EVO_TASK_CARTPOLE */
 enum { EVO_CP_CART_MASS = 0, EVO_CP_POLE_MASS = 1, EVO_CP_POLE_HALF_LENGTH = 2, EVO_CP_GRAVITY = 3,

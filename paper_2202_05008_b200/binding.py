@@ -21,7 +21,7 @@ EVO_MAX_LAYERS = 8
 STATUS = {0: "EVO_OK", 1: "EVO_ERR_INVALID_ARG", 2: "EVO_ERR_BAD_ORDER", 3: "EVO_ERR_WORKSPACE",
           4: "EVO_ERR_CUDA", 5: "EVO_ERR_NONFINITE", 6: "EVO_ERR_TIMEOUT", 7: "EVO_ERR_UNSUPPORTED"}
 ROLLOUT_AUTO, ROLLOUT_GENERIC, ROLLOUT_TILED = 0, 1, 2
-DEBUG_DROP_PARAM_COPY = 1
+DEBUG_DROP_COMPLETION = 1
 
 
 class EvoConfig(C.Structure):

@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libevo.so")
-SOURCES = ["evo.cu", "solver_kernels.cu", "rollout_mlp.cu", "rollout_mlp_tiled.cu", "rollout_cnn.cu", "rollout_cnn_tc.cu", "gradient_static.cu", "rollout_s2s.cu", "rollout_paint.cu"]
+SOURCES = ["evo.cu", "solver_kernels.cu", "rollout_mlp.cu", "rollout_mlp_tiled.cu", "rollout_tl_tc.cu", "rollout_cnn.cu", "rollout_cnn_tc.cu", "gradient_static.cu", "rollout_s2s.cu", "rollout_paint.cu"]
 HEADERS = ["internal.h", "noise.cuh", "tasks.cuh", "async.cuh", "umma.cuh", "fp32x2.cuh", os.path.join("..", "..", "include", "evo.h")]
 
 

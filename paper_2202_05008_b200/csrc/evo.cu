@@ -44,7 +44,7 @@ static evo_status check_config(const evo_config* c)
     if (c->clipup_momentum < 0.f || c->clipup_momentum >= 1.f || c->clipup_max_speed < 0.f) return EVO_ERR_INVALID_ARG;
     if (c->sigma_lr < 0.f || c->sigma_max_change < 0.f || c->sigma_max_change >= 1.f) return EVO_ERR_INVALID_ARG;
     if (c->wait_cycles_log2 != 0 && (c->wait_cycles_log2 < 10 || c->wait_cycles_log2 > 40)) return EVO_ERR_INVALID_ARG;
-    if (c->debug_flags & ~static_cast<uint32_t>(EVO_DEBUG_DROP_PARAM_COPY)) return EVO_ERR_INVALID_ARG;
+    if (c->debug_flags & ~static_cast<uint32_t>(EVO_DEBUG_DROP_COMPLETION)) return EVO_ERR_INVALID_ARG;
     if (c->shard_pairs > 0 &&
         (c->shard_first_pair >= c->pop_size / 2u || c->shard_pairs > c->pop_size / 2u - c->shard_first_pair))
         return EVO_ERR_INVALID_ARG;

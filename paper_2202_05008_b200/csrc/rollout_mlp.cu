@@ -192,6 +192,8 @@ bool rollout_mlp_supported(const evo_config& cfg)
 int rollout_mlp_tiled_shape(uint32_t task, uint32_t n_layers, const uint32_t* sizes);
 uint32_t rollout_mlp_tiled_eb(int shape, uint32_t episodes);
 int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus* status);
+bool rollout_tl_tc_supported(const RolloutMlpArgs& a);
+int launch_rollout_tl_tc(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus* status);
 
 static bool use_tiled(uint32_t task, uint32_t n_layers, const uint32_t* sizes, uint32_t choice)
 {
@@ -230,7 +232,12 @@ int launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a_in, uint32_t ker
     int launches = 0;
     const bool tiled_ok = rollout_mlp_tiled_shape(a.task, a.n_layers, a.sizes) >= 0;
     if (kernel_choice == EVO_ROLLOUT_TILED && !tiled_ok) return -2;
-    if (tiled_ok && kernel_choice != EVO_ROLLOUT_GENERIC) {
+    if (kernel_choice == EVO_ROLLOUT_AUTO && rollout_tl_tc_supported(a)) {
+        // the large tanh-linear policy: wide layers on the tensor cores (TILED keeps the fp32-pipe kernel)
+        const int r = launch_rollout_tl_tc(st, a, status);
+        if (r < 0) return r;
+        launches += r;
+    } else if (tiled_ok && kernel_choice != EVO_ROLLOUT_GENERIC) {
         const int r = launch_rollout_mlp_tiled(st, a, status);
         if (r < 0) return r;
         launches += r;

@@ -248,7 +248,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     const uint32_t bar = smem_u32(&mbar);
     if (tid == 0) { mbar_init(bar, 1); mbar_init_fence(); }
     __syncthreads();
-    if (tid == 0 && !(status->debug_flags & EVO_DEBUG_DROP_PARAM_COPY))   // the member's whole parameter row in one bulk copy
+    if (tid == 0 && !(status->debug_flags & EVO_DEBUG_DROP_COMPLETION))   // the member's whole parameter row in one bulk copy
         bulk_copy_g2s(smem_u32(stage), a.theta + static_cast<size_t>(member) * a.ldD, a.ldD * 4u, bar);
 
     // ---- reset (overlaps the copy) -----------------------------------------------------------
@@ -430,7 +430,7 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
     const uint32_t bar = smem_u32(&mbar);
     if (tid == 0) { mbar_init(bar, 1); mbar_init_fence(); }
     __syncthreads();
-    if (tid == 0 && !(status->debug_flags & EVO_DEBUG_DROP_PARAM_COPY))   // the member's whole parameter row in one bulk copy
+    if (tid == 0 && !(status->debug_flags & EVO_DEBUG_DROP_COMPLETION))   // the member's whole parameter row in one bulk copy
         bulk_copy_g2s(smem_u32(stage), a.theta + static_cast<size_t>(member) * a.ldD, a.ldD * 4u, bar);
     // seeded starts of both groups (lanes e < EB of the task warp keep the states in registers)
     const CartpoleConst cpc = cartpole_const(a.tp);

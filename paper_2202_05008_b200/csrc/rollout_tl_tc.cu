@@ -1,0 +1,422 @@
+// Large-population control roll-out (tanh-linear task, MLP 28-128-128-8) on the tensor cores.
+//
+// A member's two wide layers are the A operands of tcgen05.mma and stay on chip for all T steps:
+// W (128 x K) as two fp16 parts, w = hi + lo with hi = fp16(w) and lo = fp16(w - hi) (22 mantissa
+// bits together; every product of two fp16 numbers is exact and sums accumulate in fp32, so the
+// layer is as accurate as an fp32 FMA chain).  The hi part of W2 and both parts of W1 live in
+// tensor memory, the lo part of W2 in shared memory.  The B operand of a layer is the activation
+// block of the member's four episodes, also as two fp16 parts set side by side, N = 8 columns
+// [hi(e0..e3) | lo(e0..e3)]: one MMA with A = W_part then yields W_part . a_hi and W_part . a_lo at once
+// and the epilogue adds the two column groups, so all four cross terms are kept and a layer costs
+// two MMAs per 16 inputs.
+//
+// One block per SM runs four TEAMS of 128 threads; a team owns one (member, episode block) at a
+// time, 128 columns of tensor memory and its own mbarrier.  Thread r of a team is row r of the
+// hidden layers (tensor-memory lane r).  Every warp of a team issues its own share of a layer's
+// MMAs (one elected lane each: a single thread can only start an MMA every ~50 clocks) into its own
+// 8-column accumulator and commits to the team's mbarrier; the epilogue reads the four
+// accumulators, adds bias, applies tanh, splits into fp16 parts and writes the next B operand with
+// one 16-byte store per thread.  The narrow layers (action 128 -> 8, task dynamics 36 -> 28) run on
+// the fp32 pipe with the hidden layer in fp32.  While one team waits for its MMAs or sits in an
+// epilogue the other three use the SM: the per-step chain of a member (two MMA batches, four
+// tanh layers) is latency, and four members per SM overlap it.
+//
+// Paper: Section 2 (roll-out loop, central seeds), Section 4 (get_actions over the population with
+// parameters as data; stateless task step; identical initial observations for all members).
+#include "internal.h"
+#include "umma.cuh"
+#include "noise.cuh"
+
+#include <cuda_fp16.h>
+
+namespace evo {
+namespace tl {
+
+constexpr int kH = 128;                 // hidden width = MMA M
+constexpr int kNx = 28, kNa = 8;        // task state and action widths
+constexpr int kK1 = 32;                 // layer-1 inputs padded to two K steps of 16
+constexpr int kEB = 4;                  // episodes per team item
+constexpr int kTeams = 4, kTeamThreads = 128, kThreads = kTeams * kTeamThreads;
+// tensor-memory columns of a team
+constexpr uint32_t kColW2hi = 0, kColW1hi = 64, kColW1lo = 80, kColAcc = 96, kColsTeam = 128;
+// offsets in the flat parameter row
+constexpr int kOffW1 = 0, kOffB1 = kH * kNx, kOffW2 = kOffB1 + kH, kOffB2 = kOffW2 + kH * kH,
+              kOffW3 = kOffB2 + kH, kOffB3 = kOffW3 + kNa * kH;
+static_assert(kOffB3 + kNa == 21256, "parameter layout of the 28-128-128-8 policy");
+constexpr int kH2Pitch = kH + 16;       // h2 rows in shared memory, 4 floats of skew per 32
+
+struct TeamSmem {
+    alignas(128) unsigned char w2lo[kH * kH * 2];    // fp16, K-major 8x8 core matrices (A operand)
+    alignas(128) unsigned char b1[kK1 * 16];         // layer-1 B operand: [k][hi e0..3 | lo e0..3] fp16
+    alignas(128) unsigned char b2[kH * 16];          // layer-2 B operand
+    alignas(16) float h2[kEB][kH2Pitch];             // second hidden layer, fp32, [episode][unit]
+    alignas(16) float x[kEB][32];                    // task state, fp32
+    alignas(16) float act[kEB][kNa];                 // action, fp32
+    alignas(8) uint64_t bar;                         // MMA batches of this team
+    float ret[kEB];
+    int abort;
+};
+struct Smem {
+    TeamSmem team[kTeams];
+    alignas(16) float dyn[kNx][36];                  // [A | B] of the task, row i = output i
+    alignas(8) uint64_t drain_bar;
+    uint32_t tmem_slot;
+};
+
+__host__ __device__ constexpr uint32_t idesc_f16(uint32_t M, uint32_t N, bool b_mn_major)
+{
+    // c = f32, a = b = f16, A K-major (or tensor memory), B as given
+    return (1u << 4) | (b_mn_major ? (1u << 16) : 0u) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 :: "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* u)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "r"(taddr), "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 32 lanes x 32 consecutive columns (the four accumulators of a team): thread = lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* r)
+{
+    uint32_t u[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+                   "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
+                   "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
+                   "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
+}
+
+// tanh(x) = 1 - 2/(exp(2x)+1) on the special-function unit; absolute error ~2e-7
+__device__ __forceinline__ float tanh_sfu(float x)
+{
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * 2.885390082f));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+    return fmaf(-2.0f, r, 1.0f);
+}
+
+// x = hi + lo with both parts fp16 (round to nearest)
+__device__ __forceinline__ void split_f16(float x, __half& hi, __half& lo)
+{
+    hi = __float2half_rn(x);
+    lo = __float2half_rn(x - __half2float(hi));
+}
+__device__ __forceinline__ uint32_t pack_h2(__half a, __half b)      // a in the low half
+{
+    return static_cast<uint32_t>(__half_as_ushort(a)) | (static_cast<uint32_t>(__half_as_ushort(b)) << 16);
+}
+
+__device__ __forceinline__ void team_sync(int team)
+{
+    asm volatile("bar.sync %0, %1;" :: "r"(1 + team), "n"(kTeamThreads) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    Smem& S = *reinterpret_cast<Smem*>(smem_raw);
+    const int tid = threadIdx.x;
+    const int team = tid / kTeamThreads, r = tid % kTeamThreads;     // r = hidden unit = tensor-memory lane
+    const int w = r / 32, l = r % 32;                                // team-local warp and lane
+    TeamSmem& T = S.team[team];
+    const PhiloxKey key{ a.k0, a.k1 };
+
+    // ---- block set-up: task matrices, barriers, tensor memory ---------------------------------------
+    for (int i = tid; i < kNx * 36; i += kThreads) {
+        const int row = i / 36, col = i % 36;
+        S.dyn[row][col] = col < kNx ? a.task_const[row * kNx + col] : a.task_const[kNx * kNx + row * kNa + (col - kNx)];
+    }
+    for (int i = r; i < kK1 * 16 / 4; i += kTeamThreads) reinterpret_cast<uint32_t*>(T.b1)[i] = 0u;   // rows 28..31 stay zero
+    if (r == 0) { mbar_init(smem_u32(&T.bar), 4); mbar_init_fence(); T.abort = 0; }
+    if (tid == 0) { mbar_init(smem_u32(&S.drain_bar), kTeams * 4); mbar_init_fence(); }
+    if (tid < 32) tmem_alloc(smem_u32(&S.tmem_slot), 512);
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tm = S.tmem_slot + static_cast<uint32_t>(team) * kColsTeam;   // the team's columns
+    const uint32_t tm_lane = tm + (static_cast<uint32_t>(w * 32) << 16);          // this warp's lanes
+    const uint32_t bar = smem_u32(&T.bar);
+    uint32_t parity = 0;
+
+    // operand descriptors of this warp's MMAs (only lane 0 issues)
+    constexpr uint32_t kIdesc = idesc_f16(kH, 8, true);
+    //   layer 1: warp w takes part (w & 1) of W1 and K step (w >> 1)
+    const uint32_t l1_a = tm + ((w & 1) ? kColW1lo : kColW1hi) + 8u * static_cast<uint32_t>(w >> 1);
+    const uint64_t l1_b = umma_smem_desc(smem_u32(T.b1) + static_cast<uint32_t>(w >> 1) * 256u, 128u, 128u);
+    //   layer 2: warp w takes K steps 2w and 2w+1, both parts of W2
+    const uint32_t l2_a0 = tm + kColW2hi + 8u * static_cast<uint32_t>(2 * w);
+    const uint64_t l2_b0 = umma_smem_desc(smem_u32(T.b2) + static_cast<uint32_t>(2 * w) * 256u, 128u, 128u);
+    const uint64_t l2_b1 = umma_smem_desc(smem_u32(T.b2) + static_cast<uint32_t>(2 * w + 1) * 256u, 128u, 128u);
+    const uint64_t l2_s0 = umma_smem_desc(smem_u32(T.w2lo) + static_cast<uint32_t>(2 * w) * 256u, 128u, 2048u);
+    const uint64_t l2_s1 = umma_smem_desc(smem_u32(T.w2lo) + static_cast<uint32_t>(2 * w + 1) * 256u, 128u, 2048u);
+    const uint32_t acc_w = tm + kColAcc + 8u * static_cast<uint32_t>(w);
+    const bool drop_first_commit = (status->debug_flags & EVO_DEBUG_DROP_COMPLETION) != 0u;
+
+    // the narrow layers use another thread mapping: warp = episode, lane = (action o, input quarter q)
+    // for the action layer and lane = output i for the task dynamics
+    const int e = w, o = l & 7, q = l >> 3, di = min(l, kNx - 1);
+    const bool tracing = a.trace != nullptr;
+    volatile int* const aborted = &T.abort;
+
+    const uint32_t items = a.P * a.n_eb;
+    for (uint32_t item = blockIdx.x * kTeams + team; item < items; item += gridDim.x * kTeams) {
+        const uint32_t member = item / a.n_eb, eb = item % a.n_eb;
+        const uint32_t e0 = eb * kEB;
+        const int nE = min(static_cast<uint32_t>(kEB), a.E - e0);
+        const float* th = a.theta + static_cast<size_t>(member) * a.ldD;
+
+        // ---- the member's weights: registers -> tensor memory / shared memory ---------------------
+        {   // W1 row r (28 inputs, padded with zeros to 32): both parts into tensor memory
+            float wrow[kK1];
+#pragma unroll
+            for (int c = 0; c < kNx / 4; ++c) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(th + kOffW1 + r * kNx) + c);
+                wrow[4 * c] = v.x; wrow[4 * c + 1] = v.y; wrow[4 * c + 2] = v.z; wrow[4 * c + 3] = v.w;
+            }
+#pragma unroll
+            for (int k = kNx; k < kK1; ++k) wrow[k] = 0.f;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t hi[8], lo[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    __half h0, l0, h1, l1;
+                    split_f16(wrow[16 * c + 2 * i], h0, l0);
+                    split_f16(wrow[16 * c + 2 * i + 1], h1, l1);
+                    hi[i] = pack_h2(h0, h1); lo[i] = pack_h2(l0, l1);
+                }
+                tmem_st8(tm_lane + kColW1hi + 8u * c, hi);
+                tmem_st8(tm_lane + kColW1lo + 8u * c, lo);
+            }
+        }
+#pragma unroll 1
+        for (int c = 0; c < kH / 16; ++c) {   // W2 row r, 16 inputs at a time: hi -> tensor memory, lo -> shared memory
+            float wv[16];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(th + kOffW2 + r * kH + 16 * c) + j);
+                wv[4 * j] = v.x; wv[4 * j + 1] = v.y; wv[4 * j + 2] = v.z; wv[4 * j + 3] = v.w;
+            }
+            uint32_t hi[8], lo[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                __half h0, l0, h1, l1;
+                split_f16(wv[2 * i], h0, l0);
+                split_f16(wv[2 * i + 1], h1, l1);
+                hi[i] = pack_h2(h0, h1); lo[i] = pack_h2(l0, l1);
+            }
+            tmem_st8(tm_lane + kColW2hi + 8u * c, hi);
+            // core matrix (row group r/8, K chunk): 8 rows x 16 bytes; K chunks 128 B apart, row groups 2048 B
+            unsigned char* dst = T.w2lo + (r >> 3) * 2048 + (2 * c) * 128 + (r & 7) * 16;
+            *reinterpret_cast<uint4*>(dst) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            *reinterpret_cast<uint4*>(dst + 128) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        }
+        tmem_st_wait();
+        const float bias1 = __ldg(th + kOffB1 + r), bias2 = __ldg(th + kOffB2 + r);
+        float w3[32];                           // action layer: row o, inputs 32q .. 32q+31
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float4 v = __ldg(reinterpret_cast<const float4*>(th + kOffW3 + o * kH + 32 * q) + j);
+            w3[4 * j] = v.x; w3[4 * j + 1] = v.y; w3[4 * j + 2] = v.z; w3[4 * j + 3] = v.w;
+        }
+        const float bias3 = __ldg(th + kOffB3 + o);
+
+        // ---- reset: seeded start states, the same for every member ----------------------------------
+        if (r < kEB * (kNx / 4)) {
+            const int ee = r / (kNx / 4), qq = r % (kNx / 4);
+            const float4 z = stream_normal4(key, 1u, status->generation, e0 + min(ee, nE - 1), qq);
+            const float zs[4] = { z.x, z.y, z.z, z.w };
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                __half hi, lo;
+                split_f16(zs[j], hi, lo);
+                T.x[ee][4 * qq + j] = zs[j];
+                reinterpret_cast<__half*>(T.b1 + (4 * qq + j) * 16)[ee] = hi;
+                reinterpret_cast<__half*>(T.b1 + (4 * qq + j) * 16)[4 + ee] = lo;
+            }
+        }
+        fence_async_smem();
+        tc_fence_before();
+        team_sync(team);
+        float xcur = T.x[e][di];                // this thread's state component (lanes 28..31 mirror 27)
+        float ret = 0.f;
+
+        // ---- time loop ----------------------------------------------------------------------------------
+        for (uint32_t t = 0; t < a.T; ++t) {
+            // layer 1: one MMA per warp
+            if (l == 0 && !*aborted) {
+                tc_fence_after();
+                mma_f16_ts(acc_w, l1_a, l1_b, kIdesc, 0u);
+                if (!(drop_first_commit && t == 0u)) umma_commit(bar);
+            }
+            __syncwarp();
+            wait_or_abort(&T.abort, &T.bar, parity, status); parity ^= 1u;
+            tc_fence_after();
+            {
+                float v[32];
+                tmem_ld32(tm_lane + kColAcc, v);
+                uint32_t pk[4];
+                __half hh[kEB], hl[kEB];
+#pragma unroll
+                for (int ee = 0; ee < kEB; ++ee) {
+                    const float pre = bias1 + ((v[ee] + v[4 + ee]) + (v[8 + ee] + v[12 + ee])) +
+                                      ((v[16 + ee] + v[20 + ee]) + (v[24 + ee] + v[28 + ee]));
+                    split_f16(tanh_sfu(pre), hh[ee], hl[ee]);
+                }
+                pk[0] = pack_h2(hh[0], hh[1]); pk[1] = pack_h2(hh[2], hh[3]);
+                pk[2] = pack_h2(hl[0], hl[1]); pk[3] = pack_h2(hl[2], hl[3]);
+                *reinterpret_cast<uint4*>(T.b2 + r * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+            fence_async_smem();
+            tc_fence_before();
+            team_sync(team);
+            // layer 2: four MMAs per warp (two K steps x two parts of W2)
+            if (l == 0 && !*aborted) {
+                tc_fence_after();
+                mma_f16_ts(acc_w, l2_a0, l2_b0, kIdesc, 0u);
+                umma_bf16(acc_w, l2_s0, l2_b0, kIdesc, 1u);
+                mma_f16_ts(acc_w, l2_a0 + 8u, l2_b1, kIdesc, 1u);
+                umma_bf16(acc_w, l2_s1, l2_b1, kIdesc, 1u);
+                umma_commit(bar);
+            }
+            __syncwarp();
+            wait_or_abort(&T.abort, &T.bar, parity, status); parity ^= 1u;
+            tc_fence_after();
+            {
+                float v[32];
+                tmem_ld32(tm_lane + kColAcc, v);
+                const int rs = r + (r >> 5) * 4;               // skewed column
+#pragma unroll
+                for (int ee = 0; ee < kEB; ++ee) {
+                    const float pre = bias2 + ((v[ee] + v[4 + ee]) + (v[8 + ee] + v[12 + ee])) +
+                                      ((v[16 + ee] + v[20 + ee]) + (v[24 + ee] + v[28 + ee]));
+                    T.h2[ee][rs] = tanh_sfu(pre);
+                }
+            }
+            tc_fence_before();
+            team_sync(team);
+            // action layer on the fp32 pipe: warp = episode e, lane = (o, q)
+            {
+                const float4* hp = reinterpret_cast<const float4*>(&T.h2[e][36 * q]);
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float4 hv = hp[j];
+                    s0 = fmaf(w3[4 * j], hv.x, s0); s1 = fmaf(w3[4 * j + 1], hv.y, s1);
+                    s2 = fmaf(w3[4 * j + 2], hv.z, s2); s3 = fmaf(w3[4 * j + 3], hv.w, s3);
+                }
+                float s = (s0 + s1) + (s2 + s3);
+                s += __shfl_xor_sync(0xffffffffu, s, 8);
+                s += __shfl_xor_sync(0xffffffffu, s, 16);
+                const float act = a.action_scale * tanh_sfu(s + bias3);
+                if (q == 0) { T.act[e][o] = act; ret = fmaf(-0.01f * act, act, ret); }
+            }
+            __syncwarp();
+            // task dynamics x' = tanh(A x + B a): warp = episode e, lane = output i
+            {
+                if (l < kNx) ret = fmaf(-xcur, xcur, ret);        // reward on (x_t, a_t)
+                const float4* dr = reinterpret_cast<const float4*>(&S.dyn[di][0]);
+                const float4* xp = reinterpret_cast<const float4*>(&T.x[e][0]);
+                const float4* ap = reinterpret_cast<const float4*>(&T.act[e][0]);
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int j = 0; j < kNx / 4; ++j) {
+                    const float4 c = dr[j], xv = xp[j];
+                    s0 = fmaf(c.x, xv.x, s0); s1 = fmaf(c.y, xv.y, s1); s2 = fmaf(c.z, xv.z, s2); s3 = fmaf(c.w, xv.w, s3);
+                }
+#pragma unroll
+                for (int j = 0; j < kNa / 4; ++j) {
+                    const float4 c = dr[kNx / 4 + j], av = ap[j];
+                    s0 = fmaf(c.x, av.x, s0); s1 = fmaf(c.y, av.y, s1); s2 = fmaf(c.z, av.z, s2); s3 = fmaf(c.w, av.w, s3);
+                }
+                const float xn = tanh_sfu((s0 + s1) + (s2 + s3));
+                __syncwarp();                                      // every lane has read x[e][.]
+                if (l < kNx) {
+                    __half hi, lo;
+                    split_f16(xn, hi, lo);
+                    T.x[e][l] = xn;
+                    reinterpret_cast<__half*>(T.b1 + l * 16)[e] = hi;
+                    reinterpret_cast<__half*>(T.b1 + l * 16)[4 + e] = lo;
+                    if (tracing && t < a.trace_T && e < nE)
+                        a.trace[((static_cast<size_t>(member) * a.E + e0 + e) * a.trace_T + t) * kNx + l] = xn;
+                }
+                xcur = xn;
+            }
+            fence_async_smem();
+            tc_fence_before();
+            team_sync(team);
+        }
+
+        // ---- the item's return: episodes summed in order (fixed tree inside a warp) ------------------
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) ret += __shfl_xor_sync(0xffffffffu, ret, off);
+        if (l == 0) T.ret[e] = ret;
+        team_sync(team);
+        if (r == 0) {
+            float v = 0.f;
+            for (int ee = 0; ee < nE; ++ee) v += T.ret[ee];
+            // after a time-out the numbers mean nothing: report NaN, which makes tell skip the update
+            a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = T.abort ? __int_as_float(0x7FC00000) : v;
+        }
+        team_sync(team);
+    }
+
+    // ---- leave: after a time-out MMAs may still be running (a commit covers the MMAs its own thread
+    // issued, so every issuing thread commits once more); the block gives them one bounded wait
+    __syncthreads();
+    bool any_abort = false;
+#pragma unroll
+    for (int i = 0; i < kTeams; ++i) any_abort |= S.team[i].abort != 0;
+    if (any_abort) {
+        if (l == 0) umma_commit(smem_u32(&S.drain_bar));
+        if (tid == 0) mbar_wait_bounded(smem_u32(&S.drain_bar), 0u, &status->wait_cycles_log2);
+        __syncthreads();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (tid < 32) tmem_dealloc(S.tmem_slot, 512);
+}
+
+}  // namespace tl
+
+bool rollout_tl_tc_supported(const RolloutMlpArgs& a)
+{
+    return a.task == EVO_TASK_TANH_LINEAR && a.n_layers == 3 && a.sizes[0] == tl::kNx && a.sizes[1] == tl::kH &&
+           a.sizes[2] == tl::kH && a.sizes[3] == tl::kNa && a.EB == tl::kEB;
+}
+
+int launch_rollout_tl_tc(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus* status)
+{
+    if (!rollout_tl_tc_supported(a)) return -2;
+    const size_t bytes = sizeof(tl::Smem);
+    if (!a.attr_done &&
+        cudaFuncSetAttribute(tl::k_rollout_tl_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) != cudaSuccess)
+        return -1;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+    const uint32_t items = a.P * a.n_eb;
+    const uint32_t blocks = min(static_cast<uint32_t>(sms), (items + tl::kTeams - 1u) / tl::kTeams);
+    tl::k_rollout_tl_tc<<<blocks, tl::kThreads, bytes, st>>>(a, status);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace evo

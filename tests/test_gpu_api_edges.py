@@ -63,12 +63,12 @@ def test_rollout_argument_errors():
                                W.CFG4.with_(pop_size=4, horizon=5)])
 def test_a_device_wait_that_runs_out_raises_timeout_and_leaves_the_solver_usable(w):
     """The failure path of the bounded waits, made to happen without disturbing the device: with
-    EVO_DEBUG_DROP_PARAM_COPY the roll-out blocks never start the copy they wait for, and with a
+    EVO_DEBUG_DROP_COMPLETION the roll-out blocks never start the copy they wait for, and with a
     limit of 2^16 clocks the wait gives up after ~30 us.  Every block must return by itself, raise
     EVO_ERR_TIMEOUT and report NaN; evo_sync_status must report the condition once and clear it; a
     tell on that fitness must skip the update (NaN fitness)."""
-    from paper_2202_05008_b200.binding import DEBUG_DROP_PARAM_COPY
-    s = Solver(w, wait_cycles_log2=16, debug_flags=DEBUG_DROP_PARAM_COPY)
+    from paper_2202_05008_b200.binding import DEBUG_DROP_COMPLETION
+    s = Solver(w, wait_cycles_log2=16, debug_flags=DEBUG_DROP_COMPLETION)
     s.ask()
     fit = s.rollout()
     assert s.sync_status() == 6                        # EVO_ERR_TIMEOUT, reported ...

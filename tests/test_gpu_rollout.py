@@ -64,12 +64,35 @@ def test_cfg2_T200_sampled_members(kernel):
     _rollout_check(W.CFG2, 200, [0, 1, 77, 128, 255], kernel)
 
 
-@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_AUTO])
+# AUTO = the tensor-core kernel (wide layers as split-fp16 tcgen05 MMAs), TILED = the fp32-pipe kernel
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_TILED, ROLLOUT_AUTO])
 def test_cfg4_T200_sampled_members(kernel):
-    _rollout_check(W.CFG4, 200, [0, 1, 2047, 4095], kernel)
+    _rollout_check(W.CFG4, 200, [0, 1, 591, 592, 2047, 4095], kernel)
 
 
-@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_AUTO])
+@pytest.mark.parametrize("pop,episodes", [(2, 4), (6, 3), (10, 6), (1186, 4), (6, 9)])
+def test_cfg4_tensor_core_kernel_ragged_members_and_episodes(pop, episodes):
+    """Populations that do not fill the four teams of a block, episode counts that leave a partial
+    episode block, and more items than resident teams (1186 > 2 * 592: teams loop three times)."""
+    w = W.CFG4.with_(pop_size=pop, episodes=episodes)
+    members = sorted({0, 1, pop // 2, pop - 1})
+    T = 40 if pop > 100 else 120
+    _rollout_check(w, T, members, ROLLOUT_AUTO, check_trace=pop <= 100)
+
+
+def test_cfg4_tensor_core_and_fp32_kernels_agree_and_repeat():
+    w = W.CFG4.with_(pop_size=600, horizon=100)
+    a = Solver(w, rollout_kernel=ROLLOUT_AUTO)
+    b = Solver(w, rollout_kernel=ROLLOUT_TILED)
+    a.ask(); b.ask()
+    fa = a.rollout().clone(); fa2 = a.rollout().clone(); fb = b.rollout().clone()
+    assert torch.equal(fa, fa2)                                    # run-to-run bitwise
+    assert rel_err(fa.cpu().numpy(), fb.cpu().numpy(), floor=1.0) < 1e-4
+    assert a.sync_status() == 0 and b.sync_status() == 0
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_TILED, ROLLOUT_AUTO])
 def test_cfg4_random_policies(kernel):
     w = W.CFG4.with_(pop_size=8)
     theta = W.random_parameters(2, 8, w.param_dim, scale=0.05)   # contracting closed loop
