@@ -432,13 +432,27 @@ def roofline_of(w, workload_key, noise, stages, work, peaks, sm_count, max_mhz, 
              "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"], "traffic": None}
     else:
         achieved = stages["rollout"]["TFLOP/s"]
-        r = {"kernel": "k_paint" if w.task_kind == W.TASK_PAINT else "k_rollout_mlp (tiled / warp-specialised)",
+        kernel = {W.TASK_PAINT: "k_paint", W.TASK_TANH_LINEAR: "k_rollout_tl_tc",
+                  W.TASK_CARTPOLE: "k_rollout_cartpole_ws / k_rollout_mlp_tiled"}[w.task_kind]
+        r = {"kernel": kernel,
              "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
              "frac": achieved / alu_peak,
              "peak_source": f"{sm_count} SMs x 128 fp32 lanes x 2 x {max_mhz} MHz", "traffic": None}
         if fma_measured:
             r.update({"peak_measured": fma_measured, "frac_of_measured": achieved / fma_measured,
                       "peak_measured_source": "bench_fma_probe (16 FMA chains per thread, best of 5 launches)"})
+        if w.task_kind == W.TASK_TANH_LINEAR and tuple(w.layer_sizes) == (28, 128, 128, 8):
+            # the two wide layers run on the tensor cores as split-fp16 MMAs (hi/lo parts of weights and
+            # activations: 4 tensor flops per algorithmic flop, in 128 x 8 x 16 tiles)
+            wide = 2.0 * (28 * 128 + 128 * 128) * w.env_steps_per_generation
+            t_s = stages["rollout"]["ms"] * 1e-3
+            r["tensor"] = {"algorithmic_TFLOP/s_of_the_wide_layers": wide / t_s / 1e12,
+                           "mma_TFLOP/s_issued": 4.0 * wide * (32.0 / 28.0 * 28 * 128 + 128 * 128) / (28 * 128 + 128 * 128) / t_s / 1e12,
+                           "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " (bf16 dense; fp16 runs at the same rate)"}
+            r["tensor"]["frac"] = r["tensor"]["mma_TFLOP/s_issued"] / peaks["bf16_tflops"]
+            r["note"] = ("fp32-accurate arithmetic reported against the fp32 pipe (the ceiling of any formulation on the "
+                         "CUDA cores); the wide layers run on the tensor cores, whose own figures are under 'tensor'; the "
+                         "kernel is bound by the latency of a step's serial chain, not by either pipe")
         if w.task_kind == W.TASK_PAINT:
             r["note"] = ("algorithmic flop = every pixel against every triangle; the kernel skips the pairs "
                          "outside a triangle's bounding box, so this is an equivalent rate, not pipe utilisation")

@@ -43,12 +43,13 @@ constexpr uint32_t kColW2hi = 0, kColW1hi = 64, kColW1lo = 80, kColAcc = 96, kCo
 constexpr int kOffW1 = 0, kOffB1 = kH * kNx, kOffW2 = kOffB1 + kH, kOffB2 = kOffW2 + kH * kH,
               kOffW3 = kOffB2 + kH, kOffB3 = kOffW3 + kNa * kH;
 static_assert(kOffB3 + kNa == 21256, "parameter layout of the 28-128-128-8 policy");
-constexpr int kH2Pitch = kH + 16;       // h2 rows in shared memory, 4 floats of skew per 32
+constexpr int kH2Pitch = kH + 32;       // h2 rows in shared memory, 4 floats of skew per 16
+constexpr int kB1Lbo = 144;             // layer-1 B operand: bytes between its 8-input groups (skewed: no bank conflicts)
 
 struct TeamSmem {
     alignas(128) unsigned char w2lo[kH * kH * 2];    // fp16, K-major 8x8 core matrices (A operand)
-    alignas(128) unsigned char b1[kK1 * 16];         // layer-1 B operand: [k][hi e0..3 | lo e0..3] fp16
-    alignas(128) unsigned char b2[kH * 16];          // layer-2 B operand
+    alignas(128) unsigned char b1[640];              // layer-1 B operand, K-major: (k, n) at (k/8) 144 + 16 n + 2 (k%8)
+    alignas(128) unsigned char b2[kH * 16];          // layer-2 B operand, N-major: [k][hi e0..3 | lo e0..3] fp16
     alignas(16) float h2[kEB][kH2Pitch];             // second hidden layer, fp32, [episode][unit]
     alignas(16) float x[kEB][32];                    // task state, fp32
     alignas(16) float act[kEB][kNa];                 // action, fp32
@@ -85,21 +86,19 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* u)
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// 32 lanes x 32 consecutive columns (the four accumulators of a team): thread = lane
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* r)
+// Pre-activations of this thread's row from the team's four accumulators (8 columns each: the
+// products with the hi parts of the four episodes' activations, then those with the lo parts):
+// pre[e] = bias + sum over the accumulators of (col e + col 4+e).  Two 16-column loads, so that only
+// 16 registers are live at a time.
+__device__ __forceinline__ void acc_sums(uint32_t taddr, float bias, float* pre)
 {
-    uint32_t u[32];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
-                   "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
-                   "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
-                   "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
-                 : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    float v[16];
+    tmem_ld16(taddr, v);
 #pragma unroll
-    for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
+    for (int e = 0; e < 4; ++e) pre[e] = bias + ((v[e] + v[4 + e]) + (v[8 + e] + v[12 + e]));
+    tmem_ld16(taddr + 16u, v);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) pre[e] += (v[e] + v[4 + e]) + (v[8 + e] + v[12 + e]);
 }
 
 // tanh(x) = 1 - 2/(exp(2x)+1) on the special-function unit; absolute error ~2e-7
@@ -143,7 +142,7 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
         const int row = i / 36, col = i % 36;
         S.dyn[row][col] = col < kNx ? a.task_const[row * kNx + col] : a.task_const[kNx * kNx + row * kNa + (col - kNx)];
     }
-    for (int i = r; i < kK1 * 16 / 4; i += kTeamThreads) reinterpret_cast<uint32_t*>(T.b1)[i] = 0u;   // rows 28..31 stay zero
+    for (int i = r; i < 640 / 4; i += kTeamThreads) reinterpret_cast<uint32_t*>(T.b1)[i] = 0u;   // inputs 28..31 stay zero
     if (r == 0) { mbar_init(smem_u32(&T.bar), 4); mbar_init_fence(); T.abort = 0; }
     if (tid == 0) { mbar_init(smem_u32(&S.drain_bar), kTeams * 4); mbar_init_fence(); }
     if (tid < 32) tmem_alloc(smem_u32(&S.tmem_slot), 512);
@@ -157,27 +156,34 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
     uint32_t parity = 0;
 
     // operand descriptors of this warp's MMAs (only lane 0 issues)
-    constexpr uint32_t kIdesc = idesc_f16(kH, 8, true);
+    constexpr uint32_t kIdescL1 = idesc_f16(kH, 8, false), kIdescL2 = idesc_f16(kH, 8, true);
     //   layer 1: warp w takes part (w & 1) of W1 and K step (w >> 1)
     const uint32_t l1_a = tm + ((w & 1) ? kColW1lo : kColW1hi) + 8u * static_cast<uint32_t>(w >> 1);
-    const uint64_t l1_b = umma_smem_desc(smem_u32(T.b1) + static_cast<uint32_t>(w >> 1) * 256u, 128u, 128u);
-    //   layer 2: warp w takes K steps 2w and 2w+1, both parts of W2
+    const uint64_t l1_b = umma_smem_desc(smem_u32(T.b1) + static_cast<uint32_t>(w >> 1) * 2u * kB1Lbo, kB1Lbo, 128u);
+    //   layer 2: warp w takes K steps 2w and 2w+1, both parts of W2 (the second step's operands lie 256
+    //   bytes = 16 descriptor units further on)
     const uint32_t l2_a0 = tm + kColW2hi + 8u * static_cast<uint32_t>(2 * w);
     const uint64_t l2_b0 = umma_smem_desc(smem_u32(T.b2) + static_cast<uint32_t>(2 * w) * 256u, 128u, 128u);
-    const uint64_t l2_b1 = umma_smem_desc(smem_u32(T.b2) + static_cast<uint32_t>(2 * w + 1) * 256u, 128u, 128u);
     const uint64_t l2_s0 = umma_smem_desc(smem_u32(T.w2lo) + static_cast<uint32_t>(2 * w) * 256u, 128u, 2048u);
-    const uint64_t l2_s1 = umma_smem_desc(smem_u32(T.w2lo) + static_cast<uint32_t>(2 * w + 1) * 256u, 128u, 2048u);
     const uint32_t acc_w = tm + kColAcc + 8u * static_cast<uint32_t>(w);
     const bool drop_first_commit = (status->debug_flags & EVO_DEBUG_DROP_COMPLETION) != 0u;
 
     // the narrow layers use another thread mapping: warp = episode, lane = (action o, input quarter q)
     // for the action layer and lane = output i for the task dynamics
-    const int e = w, o = l & 7, q = l >> 3, di = min(l, kNx - 1);
+    const int e = w, q8 = l & 7, op = l >> 3, di = min(l, kNx - 1);
+    float dynw[36];                                   // row di of [A | B]
+#pragma unroll
+    for (int j = 0; j < 36; ++j) dynw[j] = S.dyn[di][j];
     const bool tracing = a.trace != nullptr;
     volatile int* const aborted = &T.abort;
 
+    // the four teams run the same chain with the same period: started together they would all want
+    // the tensor pipe at the same moment and then all leave it idle, so team t starts t/4 step late
+    if (team > 0) __nanosleep(static_cast<uint32_t>(team) * 500u);
     const uint32_t items = a.P * a.n_eb;
-    for (uint32_t item = blockIdx.x * kTeams + team; item < items; item += gridDim.x * kTeams) {
+    // items go to the blocks round-robin first and to a block's teams second, so that a small
+    // population spreads over all SMs before any SM runs two members at a time
+    for (uint32_t item = blockIdx.x + gridDim.x * team; item < items; item += gridDim.x * kTeams) {
         const uint32_t member = item / a.n_eb, eb = item % a.n_eb;
         const uint32_t e0 = eb * kEB;
         const int nE = min(static_cast<uint32_t>(kEB), a.E - e0);
@@ -231,13 +237,15 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
         }
         tmem_st_wait();
         const float bias1 = __ldg(th + kOffB1 + r), bias2 = __ldg(th + kOffB2 + r);
-        float w3[32];                           // action layer: row o, inputs 32q .. 32q+31
+        float w3[2][16];                        // action layer: rows 2 op and 2 op + 1, inputs 16 q8 .. 16 q8 + 15
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float4 v = __ldg(reinterpret_cast<const float4*>(th + kOffW3 + o * kH + 32 * q) + j);
-            w3[4 * j] = v.x; w3[4 * j + 1] = v.y; w3[4 * j + 2] = v.z; w3[4 * j + 3] = v.w;
-        }
-        const float bias3 = __ldg(th + kOffB3 + o);
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(th + kOffW3 + (2 * op + i) * kH + 16 * q8) + j);
+                w3[i][4 * j] = v.x; w3[i][4 * j + 1] = v.y; w3[i][4 * j + 2] = v.z; w3[i][4 * j + 3] = v.w;
+            }
+        const float bias3a = __ldg(th + kOffB3 + 2 * op), bias3b = __ldg(th + kOffB3 + 2 * op + 1);
 
         // ---- reset: seeded start states, the same for every member ----------------------------------
         if (r < kEB * (kNx / 4)) {
@@ -248,9 +256,11 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
             for (int j = 0; j < 4; ++j) {
                 __half hi, lo;
                 split_f16(zs[j], hi, lo);
-                T.x[ee][4 * qq + j] = zs[j];
-                reinterpret_cast<__half*>(T.b1 + (4 * qq + j) * 16)[ee] = hi;
-                reinterpret_cast<__half*>(T.b1 + (4 * qq + j) * 16)[4 + ee] = lo;
+                const int k = 4 * qq + j;
+                T.x[ee][k] = zs[j];
+                unsigned char* bp = T.b1 + (k >> 3) * kB1Lbo + (k & 7) * 2;
+                *reinterpret_cast<__half*>(bp + ee * 16) = hi;
+                *reinterpret_cast<__half*>(bp + (4 + ee) * 16) = lo;
             }
         }
         fence_async_smem();
@@ -264,23 +274,19 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
             // layer 1: one MMA per warp
             if (l == 0 && !*aborted) {
                 tc_fence_after();
-                mma_f16_ts(acc_w, l1_a, l1_b, kIdesc, 0u);
+                mma_f16_ts(acc_w, l1_a, l1_b, kIdescL1, 0u);
                 if (!(drop_first_commit && t == 0u)) umma_commit(bar);
             }
             __syncwarp();
             wait_or_abort(&T.abort, &T.bar, parity, status); parity ^= 1u;
             tc_fence_after();
             {
-                float v[32];
-                tmem_ld32(tm_lane + kColAcc, v);
+                float pre[kEB];
+                acc_sums(tm_lane + kColAcc, bias1, pre);
                 uint32_t pk[4];
                 __half hh[kEB], hl[kEB];
 #pragma unroll
-                for (int ee = 0; ee < kEB; ++ee) {
-                    const float pre = bias1 + ((v[ee] + v[4 + ee]) + (v[8 + ee] + v[12 + ee])) +
-                                      ((v[16 + ee] + v[20 + ee]) + (v[24 + ee] + v[28 + ee]));
-                    split_f16(tanh_sfu(pre), hh[ee], hl[ee]);
-                }
+                for (int ee = 0; ee < kEB; ++ee) split_f16(tanh_sfu(pre[ee]), hh[ee], hl[ee]);
                 pk[0] = pack_h2(hh[0], hh[1]); pk[1] = pack_h2(hh[2], hh[3]);
                 pk[2] = pack_h2(hl[0], hl[1]); pk[3] = pack_h2(hl[2], hl[3]);
                 *reinterpret_cast<uint4*>(T.b2 + r * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
@@ -291,61 +297,67 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
             // layer 2: four MMAs per warp (two K steps x two parts of W2)
             if (l == 0 && !*aborted) {
                 tc_fence_after();
-                mma_f16_ts(acc_w, l2_a0, l2_b0, kIdesc, 0u);
-                umma_bf16(acc_w, l2_s0, l2_b0, kIdesc, 1u);
-                mma_f16_ts(acc_w, l2_a0 + 8u, l2_b1, kIdesc, 1u);
-                umma_bf16(acc_w, l2_s1, l2_b1, kIdesc, 1u);
+                mma_f16_ts(acc_w, l2_a0, l2_b0, kIdescL2, 0u);
+                umma_bf16(acc_w, l2_s0, l2_b0, kIdescL2, 1u);
+                mma_f16_ts(acc_w, l2_a0 + 8u, l2_b0 + 16u, kIdescL2, 1u);
+                umma_bf16(acc_w, l2_s0 + 16u, l2_b0 + 16u, kIdescL2, 1u);
                 umma_commit(bar);
             }
             __syncwarp();
             wait_or_abort(&T.abort, &T.bar, parity, status); parity ^= 1u;
             tc_fence_after();
             {
-                float v[32];
-                tmem_ld32(tm_lane + kColAcc, v);
-                const int rs = r + (r >> 5) * 4;               // skewed column
+                float pre[kEB];
+                acc_sums(tm_lane + kColAcc, bias2, pre);
+                const int rs = r + (r >> 4) * 4;               // skewed column
 #pragma unroll
-                for (int ee = 0; ee < kEB; ++ee) {
-                    const float pre = bias2 + ((v[ee] + v[4 + ee]) + (v[8 + ee] + v[12 + ee])) +
-                                      ((v[16 + ee] + v[20 + ee]) + (v[24 + ee] + v[28 + ee]));
-                    T.h2[ee][rs] = tanh_sfu(pre);
-                }
+                for (int ee = 0; ee < kEB; ++ee) T.h2[ee][rs] = tanh_sfu(pre[ee]);
             }
             tc_fence_before();
             team_sync(team);
-            // action layer on the fp32 pipe: warp = episode e, lane = (o, q)
+            // action layer on the fp32 pipe: warp = episode e, lane = (input eighth q8, output pair op)
             {
-                const float4* hp = reinterpret_cast<const float4*>(&T.h2[e][36 * q]);
-                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                const float4* hp = reinterpret_cast<const float4*>(&T.h2[e][20 * q8]);
+                float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
+                for (int j = 0; j < 4; ++j) {
                     const float4 hv = hp[j];
-                    s0 = fmaf(w3[4 * j], hv.x, s0); s1 = fmaf(w3[4 * j + 1], hv.y, s1);
-                    s2 = fmaf(w3[4 * j + 2], hv.z, s2); s3 = fmaf(w3[4 * j + 3], hv.w, s3);
+                    s0 = fmaf(w3[0][4 * j], hv.x, s0);     s1 = fmaf(w3[0][4 * j + 1], hv.y, s1);
+                    u0 = fmaf(w3[1][4 * j], hv.x, u0);     u1 = fmaf(w3[1][4 * j + 1], hv.y, u1);
+                    s0 = fmaf(w3[0][4 * j + 2], hv.z, s0); s1 = fmaf(w3[0][4 * j + 3], hv.w, s1);
+                    u0 = fmaf(w3[1][4 * j + 2], hv.z, u0); u1 = fmaf(w3[1][4 * j + 3], hv.w, u1);
                 }
-                float s = (s0 + s1) + (s2 + s3);
-                s += __shfl_xor_sync(0xffffffffu, s, 8);
-                s += __shfl_xor_sync(0xffffffffu, s, 16);
-                const float act = a.action_scale * tanh_sfu(s + bias3);
-                if (q == 0) { T.act[e][o] = act; ret = fmaf(-0.01f * act, act, ret); }
+                float sa = s0 + s1, sb = u0 + u1;
+#pragma unroll
+                for (int off = 1; off < 8; off <<= 1) {
+                    sa += __shfl_xor_sync(0xffffffffu, sa, off);
+                    sb += __shfl_xor_sync(0xffffffffu, sb, off);
+                }
+                const float aa = a.action_scale * tanh_sfu(sa + bias3a), ab = a.action_scale * tanh_sfu(sb + bias3b);
+                if (q8 == 0) {
+                    *reinterpret_cast<float2*>(&T.act[e][2 * op]) = make_float2(aa, ab);
+                    ret = fmaf(-0.01f * aa, aa, ret);
+                    ret = fmaf(-0.01f * ab, ab, ret);
+                }
             }
             __syncwarp();
             // task dynamics x' = tanh(A x + B a): warp = episode e, lane = output i
             {
                 if (l < kNx) ret = fmaf(-xcur, xcur, ret);        // reward on (x_t, a_t)
-                const float4* dr = reinterpret_cast<const float4*>(&S.dyn[di][0]);
                 const float4* xp = reinterpret_cast<const float4*>(&T.x[e][0]);
                 const float4* ap = reinterpret_cast<const float4*>(&T.act[e][0]);
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
                 for (int j = 0; j < kNx / 4; ++j) {
-                    const float4 c = dr[j], xv = xp[j];
-                    s0 = fmaf(c.x, xv.x, s0); s1 = fmaf(c.y, xv.y, s1); s2 = fmaf(c.z, xv.z, s2); s3 = fmaf(c.w, xv.w, s3);
+                    const float4 xv = xp[j];
+                    s0 = fmaf(dynw[4 * j], xv.x, s0); s1 = fmaf(dynw[4 * j + 1], xv.y, s1);
+                    s2 = fmaf(dynw[4 * j + 2], xv.z, s2); s3 = fmaf(dynw[4 * j + 3], xv.w, s3);
                 }
 #pragma unroll
                 for (int j = 0; j < kNa / 4; ++j) {
-                    const float4 c = dr[kNx / 4 + j], av = ap[j];
-                    s0 = fmaf(c.x, av.x, s0); s1 = fmaf(c.y, av.y, s1); s2 = fmaf(c.z, av.z, s2); s3 = fmaf(c.w, av.w, s3);
+                    const float4 av = ap[j];
+                    s0 = fmaf(dynw[kNx + 4 * j], av.x, s0); s1 = fmaf(dynw[kNx + 4 * j + 1], av.y, s1);
+                    s2 = fmaf(dynw[kNx + 4 * j + 2], av.z, s2); s3 = fmaf(dynw[kNx + 4 * j + 3], av.w, s3);
                 }
                 const float xn = tanh_sfu((s0 + s1) + (s2 + s3));
                 __syncwarp();                                      // every lane has read x[e][.]
@@ -353,8 +365,9 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
                     __half hi, lo;
                     split_f16(xn, hi, lo);
                     T.x[e][l] = xn;
-                    reinterpret_cast<__half*>(T.b1 + l * 16)[e] = hi;
-                    reinterpret_cast<__half*>(T.b1 + l * 16)[4 + e] = lo;
+                    unsigned char* bp = T.b1 + (l >> 3) * kB1Lbo + (l & 7) * 2;
+                    *reinterpret_cast<__half*>(bp + e * 16) = hi;
+                    *reinterpret_cast<__half*>(bp + (4 + e) * 16) = lo;
                     if (tracing && t < a.trace_T && e < nE)
                         a.trace[((static_cast<size_t>(member) * a.E + e0 + e) * a.trace_T + t) * kNx + l] = xn;
                 }
@@ -414,7 +427,7 @@ int launch_rollout_tl_tc(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus*
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
     const uint32_t items = a.P * a.n_eb;
-    const uint32_t blocks = min(static_cast<uint32_t>(sms), (items + tl::kTeams - 1u) / tl::kTeams);
+    const uint32_t blocks = min(static_cast<uint32_t>(sms), items);
     tl::k_rollout_tl_tc<<<blocks, tl::kThreads, bytes, st>>>(a, status);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
