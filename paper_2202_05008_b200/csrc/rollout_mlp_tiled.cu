@@ -125,8 +125,10 @@ struct Dense {
     int   row0, s;
     bool  active;
 
-    // weights from a row-major [NO][NI] matrix followed by bias[NO] (shared or global memory)
-    __device__ __forceinline__ void load(const float* W, const float* b, int tid)
+    // weights from a row-major [no][ni] matrix followed by bias[no] (shared or global memory).  The
+    // layer may be narrower than the compiled tile (no <= NO, ni <= NI): the missing rows and columns
+    // are zeros, so the padded units are tanh(0) = 0 and feed nothing into the next layer.
+    __device__ __forceinline__ void load(const float* W, const float* b, int tid, int ni = NI, int no = NO)
     {
         active = tid < ACTIVE;
         s = tid % S;
@@ -135,9 +137,9 @@ struct Dense {
 #pragma unroll
         for (int r = 0; r < TI; ++r) {
             const int row = row0 + (r ^ rm);                     // slot r holds this output row
-            const bool ok = active && (row < NO);
+            const bool ok = active && (row < no);
 #pragma unroll
-            for (int k = 0; k < KS; ++k) w[r][k] = ok ? W[row * NI + k * S + s] : 0.f;
+            for (int k = 0; k < KS; ++k) w[r][k] = (ok && k * S + s < ni) ? W[row * ni + k * S + s] : 0.f;
             bias[r] = (ok && s == 0 && b) ? b[row] : 0.f;
         }
     }
@@ -297,10 +299,11 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     Dense<H1, H2, TI2, S2, EB, THREADS> L2;
     Dense<H2, NOUT, TI3, S3, EB, THREADS> L3;
     {
+        const int n1 = static_cast<int>(a.sizes[1]), n2 = static_cast<int>(a.sizes[2]);   // real widths <= H1, H2
         const float* p = stage;
-        L1.load(p, p + H1 * NIN, tid); p += H1 * NIN + H1;
-        L2.load(p, p + H2 * H1, tid);  p += H2 * H1 + H2;
-        L3.load(p, p + NOUT * H2, tid);
+        L1.load(p, p + n1 * NIN, tid, NIN, n1); p += n1 * NIN + n1;
+        L2.load(p, p + n2 * n1, tid, n1, n2);   p += n2 * n1 + n2;
+        L3.load(p, p + NOUT * n2, tid, n2, NOUT);
     }
     // tanh-linear dynamics x' = tanh([A B][x ; a]) as a fourth layer with shared weights
     constexpr int SD = CART ? 1 : 4;
@@ -464,9 +467,10 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
     if (!copy_ok) return;
 
     const bool tracing = a.trace != nullptr;
+    const int n1 = static_cast<int>(a.sizes[1]), n2 = static_cast<int>(a.sizes[2]);       // real widths <= H1, H2
     const float* p1 = stage;
-    const float* p2 = p1 + H1 * NIN + H1;
-    const float* p3 = p2 + H2 * H1 + H2;
+    const float* p2 = p1 + n1 * NIN + n1;
+    const float* p3 = p2 + n2 * n1 + n2;
 
     if (tid >= 32) {
         // ---------------- policy warps: hidden layers of one group per half step ----------------
@@ -476,8 +480,8 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
         const int eoff = team * ET;
         Dense<NIN, H1, TI1, S1, ET, MT, EB> L1;
         Dense<H1, H2, TI2, S2, ET, MT, EB> L2;
-        L1.load(p1, p1 + H1 * NIN, mt);
-        L2.load(p2, p2 + H2 * H1, mt);
+        L1.load(p1, p1 + n1 * NIN, mt, NIN, n1);
+        L2.load(p2, p2 + n2 * n1, mt, n1, n2);
         auto hidden = [&](int g) {
             L1.template run<true>(obs + g * NIN * EB + eoff, h1 + eoff, 1.0f, NoHook{});
             asm volatile("bar.sync %0, %1;" :: "r"(1 + team), "n"(MT) : "memory");   // the team's own barrier
@@ -501,8 +505,8 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
         const int le = tid % EB, lq = tid / EB;
         float w3[KQ];
 #pragma unroll
-        for (int i = 0; i < KQ; ++i) w3[i] = p3[lq + Q * i];
-        const float b3 = p3[H2];
+        for (int i = 0; i < KQ; ++i) w3[i] = (lq + Q * i < n2) ? p3[lq + Q * i] : 0.f;
+        const float b3 = p3[n2];
         auto advance = [&](int g, uint32_t t) {
             const float* hin = h2 + g * H2 * EB;
             float acc0 = 0.f, acc1 = 0.f;
@@ -562,15 +566,19 @@ static const TiledShape kShapes[] = {
 };
 static bool has_two_group_kernel(int shape) { return shape == 1 || shape == 3 || shape == 4; }
 
+// The compiled shape that runs a policy with two hidden layers: the narrowest one whose hidden
+// widths cover the policy's (the kernels pad narrower layers with zeros); -1 if none does.
 int rollout_mlp_tiled_shape(uint32_t task, uint32_t n_layers, const uint32_t* sizes)
 {
     if (n_layers != 3) return -1;
+    int best = -1;
     for (int i = 0; i < static_cast<int>(sizeof(kShapes) / sizeof(kShapes[0])); ++i) {
         const TiledShape& s = kShapes[i];
-        if (s.task == task && s.nin == sizes[0] && s.h1 == sizes[1] && s.h2 == sizes[2] && s.nout == sizes[3])
-            return i;
+        if (s.task == task && s.nin == sizes[0] && s.nout == sizes[3] && s.h1 >= sizes[1] && s.h2 >= sizes[2] &&
+            (best < 0 || s.h1 < kShapes[best].h1))
+            best = i;
     }
-    return -1;
+    return best;
 }
 
 // episodes per block; the wider cart-pole shapes switch to the warp-specialised kernel

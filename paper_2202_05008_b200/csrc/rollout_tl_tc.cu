@@ -39,10 +39,6 @@ constexpr int kEB = 4;                  // episodes per team item
 constexpr int kTeams = 4, kTeamThreads = 128, kThreads = kTeams * kTeamThreads;
 // tensor-memory columns of a team
 constexpr uint32_t kColW2hi = 0, kColW1hi = 64, kColW1lo = 80, kColAcc = 96, kColsTeam = 128;
-// offsets in the flat parameter row
-constexpr int kOffW1 = 0, kOffB1 = kH * kNx, kOffW2 = kOffB1 + kH, kOffB2 = kOffW2 + kH * kH,
-              kOffW3 = kOffB2 + kH, kOffB3 = kOffW3 + kNa * kH;
-static_assert(kOffB3 + kNa == 21256, "parameter layout of the 28-128-128-8 policy");
 constexpr int kH2Pitch = kH + 32;       // h2 rows in shared memory, 4 floats of skew per 16
 constexpr int kB1Lbo = 144;             // layer-1 B operand: bytes between its 8-input groups (skewed: no bank conflicts)
 
@@ -186,15 +182,22 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
     for (uint32_t item = blockIdx.x + gridDim.x * team; item < items; item += gridDim.x * kTeams) {
         const uint32_t member = item / a.n_eb, eb = item % a.n_eb;
         const uint32_t e0 = eb * kEB;
+        const bool full_width = a.sizes[1] == kH && a.sizes[2] == kH;
         const int nE = min(static_cast<uint32_t>(kEB), a.E - e0);
         const float* th = a.theta + static_cast<size_t>(member) * a.ldD;
+        // offsets in the flat parameter row; hidden widths h1, h2 <= 128 (narrower layers are padded with
+        // zero rows and columns, so the padded units are tanh(0) = 0 and feed nothing onwards)
+        const int h1 = static_cast<int>(a.sizes[1]), h2 = static_cast<int>(a.sizes[2]);
+        const int kOffW1 = 0, kOffB1 = h1 * kNx, kOffW2 = kOffB1 + h1, kOffB2 = kOffW2 + h2 * h1,
+                  kOffW3 = kOffB2 + h2, kOffB3 = kOffW3 + kNa * h2;
 
         // ---- the member's weights: registers -> tensor memory / shared memory ---------------------
         {   // W1 row r (28 inputs, padded with zeros to 32): both parts into tensor memory
             float wrow[kK1];
 #pragma unroll
-            for (int c = 0; c < kNx / 4; ++c) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(th + kOffW1 + r * kNx) + c);
+            for (int c = 0; c < kNx / 4; ++c) {             // rows are 112 bytes: 16-byte aligned
+                const float4 v = r < h1 ? __ldg(reinterpret_cast<const float4*>(th + kOffW1 + r * kNx) + c)
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
                 wrow[4 * c] = v.x; wrow[4 * c + 1] = v.y; wrow[4 * c + 2] = v.z; wrow[4 * c + 3] = v.w;
             }
 #pragma unroll
@@ -216,10 +219,16 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
 #pragma unroll 1
         for (int c = 0; c < kH / 16; ++c) {   // W2 row r, 16 inputs at a time: hi -> tensor memory, lo -> shared memory
             float wv[16];
+            if (full_width) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(th + kOffW2 + r * kH + 16 * c) + j);
-                wv[4 * j] = v.x; wv[4 * j + 1] = v.y; wv[4 * j + 2] = v.z; wv[4 * j + 3] = v.w;
+                for (int j = 0; j < 4; ++j) {
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(th + kOffW2 + r * kH + 16 * c) + j);
+                    wv[4 * j] = v.x; wv[4 * j + 1] = v.y; wv[4 * j + 2] = v.z; wv[4 * j + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    wv[j] = (r < h2 && 16 * c + j < h1) ? __ldg(th + kOffW2 + r * h1 + 16 * c + j) : 0.f;
             }
             uint32_t hi[8], lo[8];
 #pragma unroll
@@ -236,15 +245,13 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
             *reinterpret_cast<uint4*>(dst + 128) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
         }
         tmem_st_wait();
-        const float bias1 = __ldg(th + kOffB1 + r), bias2 = __ldg(th + kOffB2 + r);
+        const float bias1 = r < h1 ? __ldg(th + kOffB1 + r) : 0.f, bias2 = r < h2 ? __ldg(th + kOffB2 + r) : 0.f;
         float w3[2][16];                        // action layer: rows 2 op and 2 op + 1, inputs 16 q8 .. 16 q8 + 15
 #pragma unroll
         for (int i = 0; i < 2; ++i)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(th + kOffW3 + (2 * op + i) * kH + 16 * q8) + j);
-                w3[i][4 * j] = v.x; w3[i][4 * j + 1] = v.y; w3[i][4 * j + 2] = v.z; w3[i][4 * j + 3] = v.w;
-            }
+            for (int j = 0; j < 16; ++j)
+                w3[i][j] = (16 * q8 + j < h2) ? __ldg(th + kOffW3 + (2 * op + i) * h2 + 16 * q8 + j) : 0.f;
         const float bias3a = __ldg(th + kOffB3 + 2 * op), bias3b = __ldg(th + kOffB3 + 2 * op + 1);
 
         // ---- reset: seeded start states, the same for every member ----------------------------------
@@ -412,8 +419,8 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
 
 bool rollout_tl_tc_supported(const RolloutMlpArgs& a)
 {
-    return a.task == EVO_TASK_TANH_LINEAR && a.n_layers == 3 && a.sizes[0] == tl::kNx && a.sizes[1] == tl::kH &&
-           a.sizes[2] == tl::kH && a.sizes[3] == tl::kNa && a.EB == tl::kEB;
+    return a.task == EVO_TASK_TANH_LINEAR && a.n_layers == 3 && a.sizes[0] == tl::kNx && a.sizes[1] <= tl::kH &&
+           a.sizes[2] <= tl::kH && a.sizes[3] == tl::kNa && a.EB == tl::kEB;
 }
 
 int launch_rollout_tl_tc(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus* status)

@@ -23,8 +23,9 @@ def test_create_rejects_small_workspace_and_unsupported_tiled_request():
     h = C.c_void_p()
     assert lib.evo_create(C.byref(cfg), ptr, n.value - 1, None, C.byref(h)) == 3      # workspace too small
     assert lib.evo_create(C.byref(cfg), ptr + 4, n.value, None, C.byref(h)) == 1      # misaligned
-    # a shape without a compiled fast kernel: AUTO falls back to the generic kernel, TILED is refused at rollout
-    sizes = (5, 7, 3, 1)
+    # a shape no compiled fast kernel covers (wider than all of them): AUTO falls back to the generic
+    # kernel, TILED is refused at rollout
+    sizes = (5, 200, 12, 1)
     w = W.CFG1.with_(layer_sizes=sizes, param_dim=W.mlp_param_count(sizes), horizon=10)
     s = Solver(w, rollout_kernel=ROLLOUT_TILED)
     s.ask()

@@ -135,6 +135,45 @@ def test_other_cartpole_widths_have_fast_kernels(hidden, episodes):
     _rollout_check(w, 60, list(range(6)), ROLLOUT_TILED, theta_np=theta)
 
 
+@pytest.mark.parametrize("sizes,kernel", [((5, 48, 48, 1), ROLLOUT_TILED), ((5, 20, 50, 1), ROLLOUT_TILED),
+                                          ((5, 100, 7, 1), ROLLOUT_AUTO), ((28, 96, 96, 8), ROLLOUT_AUTO),
+                                          ((28, 96, 96, 8), ROLLOUT_TILED), ((28, 40, 120, 8), ROLLOUT_AUTO)])
+def test_policies_narrower_than_a_compiled_shape_run_on_its_fast_kernel(sizes, kernel):
+    """Any two-hidden-layer policy whose hidden widths fit a compiled shape runs on that shape's kernel
+    with the missing rows and columns as zeros (TILED is refused when no fast kernel applies, so a
+    pass also shows that the fast path was taken)."""
+    base = W.CFG2 if sizes[0] == 5 else W.CFG4
+    w = base.with_(pop_size=6, episodes=16 if sizes[0] == 5 else 4, layer_sizes=sizes, param_dim=W.mlp_param_count(sizes))
+    theta = W.random_parameters(sum(sizes), 6, w.param_dim, scale=0.25 if sizes[0] == 5 else 0.05)
+    _rollout_check(w, 60, list(range(6)), kernel, theta_np=theta)
+
+
+def _rollout_ms(w, kernel, repeats=3):
+    s = Solver(w, rollout_kernel=kernel)
+    s.ask()
+    fit = torch.empty(w.pop_size, device="cuda")
+    s.rollout(fitness=fit)
+    best = 1e9
+    for _ in range(repeats):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); s.rollout(fitness=fit); e1.record(); e1.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    assert s.sync_status() == 0
+    s.close()
+    return best
+
+
+@pytest.mark.parametrize("base,narrow,wide", [(W.CFG2, (5, 48, 48, 1), (5, 64, 64, 1)),
+                                               (W.CFG4, (28, 96, 96, 8), (28, 128, 128, 8))])
+def test_narrower_policies_run_within_twice_the_time_of_the_compiled_shape(base, narrow, wide):
+    """A 5-48-48-1 and a 28-96-96-8 policy at the full population must not fall back to the slow
+    runtime-shape kernel: their roll-out takes at most twice as long as the compiled shape's."""
+    T = 200
+    t_narrow = _rollout_ms(base.with_(horizon=T, layer_sizes=narrow, param_dim=W.mlp_param_count(narrow)), ROLLOUT_AUTO)
+    t_wide = _rollout_ms(base.with_(horizon=T, layer_sizes=wide, param_dim=W.mlp_param_count(wide)), ROLLOUT_AUTO)
+    assert t_narrow < 2.0 * t_wide, (t_narrow, t_wide)
+
+
 def test_cfg1_shape_with_several_episodes():
     w = W.CFG1.with_(episodes=3)
     _rollout_check(w, 80, list(range(16)), ROLLOUT_TILED)
