@@ -236,6 +236,18 @@ evo_status evo_set_state(evo_solver* s, const float* d_center, const float* d_m,
  * EVO_ERR_NONFINITE, EVO_ERR_TIMEOUT) or EVO_ERR_CUDA if the stream reports a fault. */
 evo_status evo_sync_status(evo_solver* s);
 
+/*
+ * Checked build only (libevo_debug.so, compiled with -DEVO_DEBUG; the paper has no counterpart: this
+ * stands in for a memory checker where none can be run).  In that build every region of the
+ * workspace is followed by 256 guard bytes written at evo_create, and the kernels' global stores
+ * test their index against the array size, skip the store when it is outside and record the first
+ * such site.  evo_debug_check waits for the stream and reports *damaged_region = the index (in
+ * layout order) of the first region whose guard bytes changed, or -1; *bounds_site = the first
+ * store site that was skipped (0 = none) and *bounds_index = its index.  The normal build returns
+ * EVO_ERR_UNSUPPORTED.  Errors: INVALID_ARG (NULL), CUDA.
+ */
+evo_status evo_debug_check(evo_solver* s, int32_t* damaged_region, uint32_t* bounds_site, uint64_t* bounds_index);
+
 /* Number of kernels the library has launched for this solver so far. */
 evo_status evo_launch_count(evo_solver* s, uint64_t* launches);
 

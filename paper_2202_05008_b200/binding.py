@@ -16,6 +16,7 @@ from . import workloads as W
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libevo.so")
+LIB_DEBUG_PATH = os.path.join(_HERE, "libevo_debug.so")     # checked build (-DEVO_DEBUG)
 
 EVO_MAX_LAYERS = 8
 STATUS = {0: "EVO_OK", 1: "EVO_ERR_INVALID_ARG", 2: "EVO_ERR_BAD_ORDER", 3: "EVO_ERR_WORKSPACE",
@@ -49,17 +50,22 @@ class EvoError(RuntimeError):
 
 
 _lib = None
+_lib_debug = None
 
 
-def load_library():
-    """Loads libevo.so; raises if it has not been built (no CPU fallback exists)."""
-    global _lib
-    if _lib is not None:
+def load_library(debug: bool = False):
+    """Loads libevo.so (or the checked build libevo_debug.so); raises if it has not been built
+    (no CPU fallback exists)."""
+    global _lib, _lib_debug
+    if debug and _lib_debug is not None:
+        return _lib_debug
+    if not debug and _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
+    path = LIB_DEBUG_PATH if debug else LIB_PATH
+    if not os.path.exists(path):
         raise FileNotFoundError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2202_05008_b200.build`")
-    L = C.CDLL(LIB_PATH)
+            f"{path} is missing: build it with `python -m paper_2202_05008_b200.build`")
+    L = C.CDLL(path)
     vp, u32p, szp = C.c_void_p, C.POINTER(C.c_uint32), C.POINTER(C.c_size_t)
     cfgp = C.POINTER(EvoConfig)
     L.evo_workspace_bytes.argtypes = [cfgp, szp]
@@ -95,7 +101,12 @@ def load_library():
                  "evo_get_gradient", "evo_get_ranks", "evo_get_eps", "evo_get_sigma", "evo_set_sigma", "evo_get_counters",
                  "evo_set_state", "evo_sync_status", "evo_launch_count"):
         getattr(L, name).restype = C.c_int
-    _lib = L
+    L.evo_debug_check.argtypes = [vp, C.POINTER(C.c_int32), u32p, C.POINTER(C.c_uint64)]
+    L.evo_debug_check.restype = C.c_int
+    if debug:
+        _lib_debug = L
+    else:
+        _lib = L
     return L
 
 
@@ -132,8 +143,8 @@ class Solver:
     """One ES solver bound to a CUDA device, a stream and a caller-owned workspace tensor."""
 
     def __init__(self, workload: W.Workload, device="cuda:0", stream: Optional[torch.cuda.Stream] = None,
-                 **cfg_kw):
-        self.lib = load_library()
+                 debug: bool = False, **cfg_kw):
+        self.lib = load_library(debug)
         self.workload = workload
         self.cfg = make_config(workload, **cfg_kw)
         self.device = torch.device(device)
@@ -293,6 +304,12 @@ class Solver:
             return x.data_ptr()
         _check(self.lib.evo_set_state(self._h, ptr(center), ptr(m), ptr(v), generation, adam_step),
                "evo_set_state")
+
+    def debug_check(self):
+        """Checked build only: (damaged region or -1, skipped store site or 0, its index)."""
+        reg, site, idx = C.c_int32(), C.c_uint32(), C.c_uint64()
+        _check(self.lib.evo_debug_check(self._h, C.byref(reg), C.byref(site), C.byref(idx)), "evo_debug_check")
+        return reg.value, site.value, idx.value
 
     def sync_status(self) -> int:
         return self.lib.evo_sync_status(self._h)

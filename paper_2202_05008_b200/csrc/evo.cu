@@ -29,6 +29,7 @@ struct evo_solver {
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+constexpr int kCanaryByte = 0xA5;
 
 static evo_status check_config(const evo_config* c)
 {
@@ -104,7 +105,14 @@ static evo_status make_layout(const evo_config& c, Layout* L)
     if (c.task_kind == EVO_TASK_CARTPOLE || c.task_kind == EVO_TASK_TANH_LINEAR)
         rollout_mlp_plan(c, &L->EB, &L->n_eb);
     size_t off = 0;
-    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L->n_canaries = 0;
+    // every region starts 256-byte aligned; the checked build puts kCanaryBytes of guard words behind each
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off = align_up(off + bytes, 256);
+        if (kCanaryBytes && L->n_canaries < kMaxRegions) { L->canary[L->n_canaries++] = off; off += kCanaryBytes; }
+        return o;
+    };
     const size_t row = static_cast<size_t>(ldD) * sizeof(float);
     L->status = take(sizeof(DeviceStatus));
     L->center = take(row);
@@ -200,6 +208,11 @@ evo_status evo_create(const evo_config* cfg_in, void* d_workspace, size_t worksp
                               reinterpret_cast<float*>(s->ws + L.task_const));
     if (n < 0) { delete s; return EVO_ERR_CUDA; }
     s->launches += n;
+    for (int i = 0; i < L.n_canaries; ++i)          // checked build only (n_canaries is 0 otherwise)
+        if (cudaMemsetAsync(s->ws + L.canary[i], kCanaryByte, kCanaryBytes, s->stream) != cudaSuccess) {
+            delete s;
+            return EVO_ERR_CUDA;
+        }
     *out = s;
     return EVO_OK;
 }
@@ -522,6 +535,29 @@ evo_status evo_sync_status(evo_solver* s)
         return EVO_ERR_CUDA;
     }
     return EVO_OK;
+}
+
+evo_status evo_debug_check(evo_solver* s, int32_t* damaged_region, uint32_t* bounds_site, uint64_t* bounds_index)
+{
+    if (!s || !damaged_region || !bounds_site || !bounds_index) return EVO_ERR_INVALID_ARG;
+#ifdef EVO_DEBUG
+    *damaged_region = -1; *bounds_site = 0; *bounds_index = 0;
+    if (cudaStreamSynchronize(s->stream) != cudaSuccess) return EVO_ERR_CUDA;
+    unsigned char guard[kCanaryBytes];
+    for (int i = 0; i < s->lay.n_canaries && *damaged_region < 0; ++i) {
+        if (cudaMemcpy(guard, s->ws + s->lay.canary[i], kCanaryBytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+            return EVO_ERR_CUDA;
+        for (size_t b = 0; b < kCanaryBytes; ++b)
+            if (guard[b] != kCanaryByte) { *damaged_region = i; break; }
+    }
+    DeviceStatus h;
+    if (cudaMemcpy(&h, s->ws + s->lay.status, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return EVO_ERR_CUDA;
+    *bounds_site = h.bounds_site;
+    *bounds_index = (static_cast<uint64_t>(h.bounds_index_hi) << 32) | h.bounds_index_lo;
+    return EVO_OK;
+#else
+    return EVO_ERR_UNSUPPORTED;
+#endif
 }
 
 evo_status evo_launch_count(evo_solver* s, uint64_t* launches)

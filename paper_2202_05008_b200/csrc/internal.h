@@ -16,7 +16,36 @@ struct DeviceStatus {
     uint32_t generation;    // counter word of every random stream; advanced by the kernel that closes a tell
     uint32_t wait_cycles_log2;  // every bounded device-side wait gives up after 2^this SM clocks
     uint32_t debug_flags;   // EVO_DEBUG_* bits of the configuration
+    uint32_t bounds_site;   // checked build: first store site whose index left its array (0 = none)
+    uint32_t bounds_index_lo, bounds_index_hi;   // ... and that index
+    uint32_t reserved;
 };
+
+// Checked build (-DEVO_DEBUG, libevo_debug.so): a global store whose index lies outside its array is
+// not executed; the first such site and index are recorded in the status block and the sticky
+// EVO_ERR_CUDA bit is raised.  In the normal build the macro is the constant true.
+enum { EVO_SITE_ASK_THETA = 1, EVO_SITE_ASK_EPS = 2, EVO_SITE_RANK = 3, EVO_SITE_GRAD_PARTIAL = 4,
+       EVO_SITE_UPDATE = 5, EVO_SITE_FIT_PARTIAL = 6, EVO_SITE_TRACE = 7, EVO_SITE_FITNESS = 8 };
+#ifdef EVO_DEBUG
+__device__ __forceinline__ bool debug_in_bounds(const DeviceStatus* st, uint32_t site, unsigned long long idx,
+                                                unsigned long long limit)
+{
+    if (idx < limit) return true;
+    DeviceStatus* s = const_cast<DeviceStatus*>(st);
+    if (atomicCAS(&s->bounds_site, 0u, site) == 0u) {
+        s->bounds_index_lo = static_cast<uint32_t>(idx);
+        s->bounds_index_hi = static_cast<uint32_t>(idx >> 32);
+    }
+    atomicOr(&s->sticky, 1u << EVO_ERR_CUDA);
+    return false;
+}
+#define EVO_IN_BOUNDS(st, site, idx, limit) ::evo::debug_in_bounds(st, site, idx, limit)
+constexpr size_t kCanaryBytes = 256;      // guard words behind every workspace region
+#else
+#define EVO_IN_BOUNDS(st, site, idx, limit) true
+constexpr size_t kCanaryBytes = 0;
+#endif
+constexpr int kMaxRegions = 24;
 
 constexpr uint32_t kTlNx = 28;   // tanh-linear task: state width
 constexpr uint32_t kTlNa = 8;    // tanh-linear task: action width
@@ -47,6 +76,8 @@ struct Layout {                  // byte offsets into the workspace
            sigma_sum, norms,
            fit_partial, task_const, cnn_scratch, total;
     uint32_t ldD, grad_splits, n_eb, EB;
+    size_t canary[kMaxRegions];  // checked build: offset of the guard words behind each region, in layout order
+    int    n_canaries;
 };
 
 // ---- launchers (each returns the number of kernels it launched, or -1 on a launch error) ----

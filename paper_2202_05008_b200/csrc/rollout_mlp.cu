@@ -149,7 +149,8 @@ k_rollout_mlp_generic(const RolloutMlpArgs a, const DeviceStatus* __restrict__ s
     if (tid == 0) {
         float s = 0.f;
         for (uint32_t e = 0; e < nE; ++e) s += rets[e];
-        a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = s;
+        if (EVO_IN_BOUNDS(status, EVO_SITE_FIT_PARTIAL, static_cast<size_t>(member) * a.n_eb + eb, static_cast<size_t>(a.P) * a.n_eb))
+            a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = s;
     }
 }
 

@@ -398,7 +398,9 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
         else      v = (tid < SD) ? ret : 0.f;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-        if (tid == 0) a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = v;
+        if (tid == 0 && EVO_IN_BOUNDS(status, EVO_SITE_FIT_PARTIAL, static_cast<size_t>(member) * a.n_eb + eb,
+                                      static_cast<size_t>(a.P) * a.n_eb))
+            a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = v;
     }
 }
 
@@ -549,7 +551,9 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
         float v = ((tid < nA) ? ret[0] : 0.f) + ((tid < nB) ? ret[1] : 0.f);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-        if (tid == 0) a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = v;
+        if (tid == 0 && EVO_IN_BOUNDS(status, EVO_SITE_FIT_PARTIAL, static_cast<size_t>(member) * a.n_eb + eb,
+                                      static_cast<size_t>(a.P) * a.n_eb))
+            a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = v;
     }
 }
 

@@ -375,7 +375,9 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
                     unsigned char* bp = T.b1 + (l >> 3) * kB1Lbo + (l & 7) * 2;
                     *reinterpret_cast<__half*>(bp + e * 16) = hi;
                     *reinterpret_cast<__half*>(bp + (4 + e) * 16) = lo;
-                    if (tracing && t < a.trace_T && e < nE)
+                    if (tracing && t < a.trace_T && e < nE &&
+                        EVO_IN_BOUNDS(status, EVO_SITE_TRACE, ((static_cast<size_t>(member) * a.E + e0 + e) * a.trace_T + t) * kNx + l,
+                                      static_cast<size_t>(a.P) * a.E * a.trace_T * kNx))
                         a.trace[((static_cast<size_t>(member) * a.E + e0 + e) * a.trace_T + t) * kNx + l] = xn;
                 }
                 xcur = xn;
@@ -394,7 +396,9 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
             float v = 0.f;
             for (int ee = 0; ee < nE; ++ee) v += T.ret[ee];
             // after a time-out the numbers mean nothing: report NaN, which makes tell skip the update
-            a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = T.abort ? __int_as_float(0x7FC00000) : v;
+            if (EVO_IN_BOUNDS(status, EVO_SITE_FIT_PARTIAL, static_cast<size_t>(member) * a.n_eb + eb,
+                              static_cast<size_t>(a.P) * a.n_eb))
+                a.fit_partial[static_cast<size_t>(member) * a.n_eb + eb] = T.abort ? __int_as_float(0x7FC00000) : v;
         }
         team_sync(team);
     }

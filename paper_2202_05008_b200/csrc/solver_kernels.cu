@@ -18,6 +18,7 @@ __global__ void k_init(float* center, float* m, float* v, float* g, float* sigma
     if (i == 0) {
         status->sticky = 0; status->nonfinite = 0; status->adam_step = 0; status->generation = 0;
         status->wait_cycles_log2 = wait_cycles_log2; status->debug_flags = debug_flags;
+        status->bounds_site = 0; status->bounds_index_lo = 0; status->bounds_index_hi = 0; status->reserved = 0;
     }
 }
 
@@ -88,9 +89,14 @@ k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, Phi
             const float4 tm = make_float4(__fmaf_rn(-sg.x, z.x, c.x), __fmaf_rn(-sg.y, z.y, c.y),
                                           __fmaf_rn(-sg.z, z.z, c.z), __fmaf_rn(-sg.w, z.w, c.w));
             float* row = theta + static_cast<size_t>(2u * jj) * ldD + d0;
-            __stcs(reinterpret_cast<float4*>(row), tp);
-            __stcs(reinterpret_cast<float4*>(row + ldD), tm);
-            if (eps) __stcs(reinterpret_cast<float4*>(eps + static_cast<size_t>(jj) * ldD + d0), z);
+            if (EVO_IN_BOUNDS(status, EVO_SITE_ASK_THETA, static_cast<size_t>(2u * jj + 1u) * ldD + d0 + 3u,
+                              static_cast<size_t>(2u * H) * ldD)) {
+                __stcs(reinterpret_cast<float4*>(row), tp);
+                __stcs(reinterpret_cast<float4*>(row + ldD), tm);
+            }
+            if (eps && EVO_IN_BOUNDS(status, EVO_SITE_ASK_EPS, static_cast<size_t>(jj) * ldD + d0 + 3u,
+                                     static_cast<size_t>(H) * ldD))
+                __stcs(reinterpret_cast<float4*>(eps + static_cast<size_t>(jj) * ldD + d0), z);
         }
     }
 }
@@ -132,7 +138,7 @@ k_rank(const float* __restrict__ fitness, uint32_t P, int32_t* __restrict__ rank
             }
         }
     }
-    if (m < P) {
+    if (m < P && EVO_IN_BOUNDS(status, EVO_SITE_RANK, m, P)) {
         rank[m] = static_cast<int32_t>(below);
         u[m] = __fadd_rn(__fdiv_rn(__uint2float_rn(below), __uint2float_rn(P - 1u)), -0.5f);
     }
@@ -278,8 +284,11 @@ k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, Philo
             if (quad * 4u + i >= D) r[i] = 0.;
     }
     double2* out = reinterpret_cast<double2*>(partial + static_cast<size_t>(blockIdx.y) * ldD) + 2u * quad;
-    out[0] = make_double2(r[0], r[1]);
-    out[1] = make_double2(r[2], r[3]);
+    if (EVO_IN_BOUNDS(status, EVO_SITE_GRAD_PARTIAL, static_cast<size_t>(blockIdx.y) * ldD + 4u * quad + 3u,
+                      static_cast<size_t>((H + pairs_per_split - 1u) / pairs_per_split) * ldD)) {
+        out[0] = make_double2(r[0], r[1]);
+        out[1] = make_double2(r[2], r[3]);
+    }
     if (SIGMA) {
         float4 sr = make_float4(sacc[0].x + sacc[1].x, sacc[0].y + sacc[1].y, sacc[0].z + sacc[1].z, sacc[0].w + sacc[1].w);
         if (quad * 4u + 4u > D) {                  // padding columns carry no sigma signal
@@ -347,7 +356,8 @@ k_update(const double* __restrict__ partial, const float* __restrict__ sigma_par
             }
             reinterpret_cast<float4*>(m)[quad] = make_float4(mm[0], mm[1], mm[2], mm[3]);
             reinterpret_cast<float4*>(v)[quad] = make_float4(vv[0], vv[1], vv[2], vv[3]);
-            reinterpret_cast<float4*>(center)[quad] = make_float4(cc[0], cc[1], cc[2], cc[3]);
+            if (EVO_IN_BOUNDS(status, EVO_SITE_UPDATE, 4u * quad + 3u, ldD))
+                reinterpret_cast<float4*>(center)[quad] = make_float4(cc[0], cc[1], cc[2], cc[3]);
         }
         if (sigma_partial) {                            // PGPE sigma step with a relative-change limit
             float ss[4] = { 0.f, 0.f, 0.f, 0.f };
