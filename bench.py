@@ -88,8 +88,26 @@ def stage_work(w, stored):
 # that digest; once a kernel's source changes its entry reads null until it is captured again.
 CSRC = os.path.join(ROOT, "paper_2202_05008_b200", "csrc")
 NCU_TRAFFIC = {
-    # filled in from the captures summarised under profiles/
+    ("cfg4", "stored"): {"kernel": "k_rollout_tl_tc", "bytes": 3.489119e+08,
+                         "files": ["rollout_tl_tc.cu", "umma.cuh", "async.cuh", "noise.cuh", "internal.h"],
+                         "digest": "6e58c19ffb460ae2",
+                         "capture": "P = 592 capture scaled by members (the traffic is the parameter rows, proportional to P)"},
+    ("cfg2", "stored"): {"kernel": "k_rollout_cartpole_ws", "bytes": 4.787712e+06,
+                         "files": ["rollout_mlp_tiled.cu", "async.cuh", "tasks.cuh", "noise.cuh", "fp32x2.cuh", "internal.h"],
+                         "digest": "4a82517f4f499ba6", "capture": "full size"},
+    ("cfg3", "stored"): {"kernel": "k_cnn_conv2_tc", "bytes": 1.528125e+08,
+                         "files": ["rollout_cnn_tc.cu", "umma.cuh", "async.cuh", "internal.h"],
+                         "digest": "02b4c007675e3419", "capture": "full size"},
+    ("cfg5", "stored"): {"kernel": "k_ask", "bytes": 1.011388e+11,
+                         "files": ["solver_kernels.cu", "noise.cuh", "internal.h"],
+                         "digest": "87386e067f759f75",
+                         "capture": "D = 32,768 capture scaled by 32 (columns are independent)"},
+    ("cfg5", "regenerated"): {"kernel": "k_ask", "bytes": 6.677962e+10,
+                              "files": ["solver_kernels.cu", "noise.cuh", "internal.h"],
+                              "digest": "87386e067f759f75", "capture": "D = 32,768 capture scaled by 32"},
 }
+NCU_TRAFFIC[("cfg4", "regenerated")] = NCU_TRAFFIC[("cfg4", "stored")]
+NCU_TRAFFIC[("cfg2", "regenerated")] = NCU_TRAFFIC[("cfg2", "stored")]
 
 
 def source_digest(files):
@@ -460,6 +478,7 @@ def roofline_of(w, workload_key, noise, stages, work, peaks, sm_count, max_mhz, 
     if entry is not None and (w.task_kind != W.TASK_NONE or r["kernel"] == entry["kernel"]):
         r["traffic"] = entry["bytes"]
         r["traffic_kernel"] = entry["kernel"]
+        r["traffic_capture"] = entry["capture"]
     return r
 
 
@@ -746,9 +765,16 @@ def main():
                     help="N > 1: independent solvers (weak scaling) instead of one population in pair shards")
     ap.add_argument("--graph", action="store_true",
                     help="also time the generation replayed from a CUDA graph (extra key graph_replay)")
+    ap.add_argument("--traffic-digests", action="store_true",
+                    help="print the source digest each NCU_TRAFFIC entry would need now (after a new capture) and exit")
     ap.add_argument("--pop", type=int, default=0, help="override the population size (experiments)")
     ap.add_argument("--dim", type=int, default=0, help="override the parameter count (cfg5 only)")
     args = ap.parse_args()
+    if args.traffic_digests:
+        for key, entry in NCU_TRAFFIC.items():
+            now = source_digest(entry["files"])
+            print(key, entry["kernel"], "stored", entry["digest"], "current", now, "OK" if now == entry["digest"] else "STALE")
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2202_05008_b200 import workloads as W
     w = W.CONFIGS[args.workload]
