@@ -10,25 +10,37 @@
 
 namespace evo {
 
-struct PhiloxKey { uint32_t k0, k1; };
+// The key with its schedule: round r uses (k0 + r W0, k1 + r W1), W = the Weyl increments.  The ten
+// pairs are computed once where the key is made (on the host for the solver kernels, whose key is a
+// launch parameter: the round keys then come straight out of the constant bank and the generator
+// spends no instruction on the schedule).
+struct PhiloxKey { uint32_t r[20]; };
+
+__host__ __device__ __forceinline__ PhiloxKey philox_key(uint32_t k0, uint32_t k1)
+{
+    PhiloxKey k;
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+        k.r[2 * i] = k0 + static_cast<uint32_t>(i) * 0x9E3779B9u;
+        k.r[2 * i + 1] = k1 + static_cast<uint32_t>(i) * 0xBB67AE85u;
+    }
+    return k;
+}
 
 // counter = (item, row, generation, stream)
 __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                               PhiloxKey key)
+                                               const PhiloxKey& key)
 {
-    uint32_t k0 = key.k0, k1 = key.k1;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         const uint64_t p0 = static_cast<uint64_t>(0xD2511F53u) * c0;      // one wide multiply each
         const uint64_t p1 = static_cast<uint64_t>(0xCD9E8D57u) * c2;
         const uint32_t hi0 = static_cast<uint32_t>(p0 >> 32), lo0 = static_cast<uint32_t>(p0);
         const uint32_t hi1 = static_cast<uint32_t>(p1 >> 32), lo1 = static_cast<uint32_t>(p1);
-        c0 = hi1 ^ c1 ^ k0;
+        c0 = hi1 ^ c1 ^ key.r[2 * r];
         c1 = lo1;
-        c2 = hi0 ^ c3 ^ k1;
+        c2 = hi0 ^ c3 ^ key.r[2 * r + 1];
         c3 = lo0;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
     }
     return make_uint4(c0, c1, c2, c3);
 }
@@ -121,7 +133,7 @@ __device__ __forceinline__ float4 normal4(uint4 r)
     return z;
 }
 
-__device__ __forceinline__ float4 stream_normal4(PhiloxKey key, uint32_t stream, uint32_t generation,
+__device__ __forceinline__ float4 stream_normal4(const PhiloxKey& key, uint32_t stream, uint32_t generation,
                                                  uint32_t row, uint32_t item)
 {
     return normal4(philox4x32_10(item, row, generation, stream, key));

@@ -29,7 +29,7 @@ k_rollout_mlp_generic(const RolloutMlpArgs a, const DeviceStatus* __restrict__ s
     const uint32_t nE = min(a.EB, a.E - e0);          // episodes of this block
     const uint32_t EB = a.EB;
     const uint32_t tid = threadIdx.x;
-    const PhiloxKey key{ a.k0, a.k1 };
+    const PhiloxKey key = philox_key(a.k0, a.k1);
     const uint32_t generation = status->generation;
 
     uint32_t n_params = 0;

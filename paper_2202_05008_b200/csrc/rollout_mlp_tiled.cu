@@ -244,7 +244,7 @@ k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
     const uint32_t member = blockIdx.x, eb = blockIdx.y;
     const uint32_t e0 = eb * EB;
     const int nE = min(static_cast<uint32_t>(EB), a.E - e0);
-    const PhiloxKey key{ a.k0, a.k1 };
+    const PhiloxKey key = philox_key(a.k0, a.k1);
 
     // ---- parameter row: one bulk copy HBM -> shared memory ---------------------------------
     const uint32_t bar = smem_u32(&mbar);
@@ -430,7 +430,7 @@ k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
     const uint32_t e0 = eb * (2 * EB);
     const int nE = min(static_cast<uint32_t>(2 * EB), a.E - e0);      // episodes of this block
     const int nA = min(nE, EB), nB = nE - nA;                        // group sizes
-    const PhiloxKey key{ a.k0, a.k1 };
+    const PhiloxKey key = philox_key(a.k0, a.k1);
 
     const uint32_t bar = smem_u32(&mbar);
     if (tid == 0) { mbar_init(bar, 1); mbar_init_fence(); }

@@ -41,7 +41,7 @@ constexpr int kS2sMaxTe = 2 * kS2sMaxDigits + 1, kS2sMaxTd = kS2sMaxDigits + 1;
 __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
 // Query i of a generation: a, b uniform on [0, 10^nd) from the first two words of stream 6.
-__device__ __forceinline__ void s2s_query(PhiloxKey key, uint32_t generation, uint32_t i, uint32_t nd,
+__device__ __forceinline__ void s2s_query(const PhiloxKey& key, uint32_t generation, uint32_t i, uint32_t nd,
                                           uint8_t* enc, uint8_t* dec, uint8_t* tgt)
 {
     uint32_t range = 1;
@@ -99,7 +99,7 @@ k_s2s_simple(const S2sArgs a)
     const uint32_t h = a.h, r = threadIdx.x, member = blockIdx.x, q0 = blockIdx.y * kSimpleQ;
     const uint32_t nq = min(static_cast<uint32_t>(kSimpleQ), a.B - q0);
     const uint32_t Te = 2 * a.nd + 1, Td = a.nd + 1;
-    const PhiloxKey key{a.k0, a.k1};
+    const PhiloxKey key = philox_key(a.k0, a.k1);
     if (r < kSimpleQ) {
         s2s_query(key, a.status->generation, q0 + min(r, nq - 1u), a.nd, enc[r], dec[r], tgt[r]);
         loss_s[r] = 0.f;
@@ -340,7 +340,7 @@ k_s2s_tc(const S2sArgs a, DeviceStatus* status)
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31u;
     const uint32_t Te = 2 * a.nd + 1, Td = a.nd + 1, T = Te + Td;
     const uint32_t n_items = a.P * a.n_chunks;
-    const PhiloxKey key{a.k0, a.k1};
+    const PhiloxKey key = philox_key(a.k0, a.k1);
 
     if (tid == 0) {
         mbar_init(smem_u32(&S.full[0]), 1); mbar_init(smem_u32(&S.full[1]), 1);

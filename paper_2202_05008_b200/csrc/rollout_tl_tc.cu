@@ -131,7 +131,7 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
     const int team = tid / kTeamThreads, r = tid % kTeamThreads;     // r = hidden unit = tensor-memory lane
     const int w = r / 32, l = r % 32;                                // team-local warp and lane
     TeamSmem& T = S.team[team];
-    const PhiloxKey key{ a.k0, a.k1 };
+    const PhiloxKey key = philox_key(a.k0, a.k1);
 
     // ---- block set-up: task matrices, barriers, tensor memory ---------------------------------------
     for (int i = tid; i < kNx * 36; i += kThreads) {

@@ -53,7 +53,7 @@ __global__ void k_tanh_linear_constants(PhiloxKey key, float* out)
 int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t k1, float* task_const)
 {
     if (task != EVO_TASK_TANH_LINEAR) return 0;
-    k_tanh_linear_constants<<<1, 256, 0, st>>>(PhiloxKey{k0, k1}, task_const);
+    k_tanh_linear_constants<<<1, 256, 0, st>>>(philox_key(k0, k1), task_const);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
@@ -63,7 +63,7 @@ int launch_task_constants(cudaStream_t st, uint32_t task, uint32_t k0, uint32_t 
 // ------------------------------------------------------------------------------------------
 constexpr uint32_t kAskPairsPerThread = 8;
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 8)
 k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, PhiloxKey key,
       const DeviceStatus* __restrict__ status, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* __restrict__ theta, float* __restrict__ eps)
 {
@@ -108,7 +108,7 @@ int launch_ask(cudaStream_t st, const float* center, const float* sigma_vec, uin
     const uint32_t quads = ldD / 4u;
     dim3 grid((quads + 255u) / 256u, (H + kAskPairsPerThread - 1u) / kAskPairsPerThread);
     if (grid.y > 65535u) grid.y = 65535u;
-    k_ask<<<grid, 256, 0, st>>>(center, sigma_vec, PhiloxKey{k0, k1}, status, pair0, H, D, ldD, theta, eps);
+    k_ask<<<grid, 256, 0, st>>>(center, sigma_vec, philox_key(k0, k1), status, pair0, H, D, ldD, theta, eps);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
@@ -475,7 +475,7 @@ size_t clipup_norm_doubles(uint32_t ldD) { return 2u * ((ldD / 4u + 255u) / 256u
 template <bool REGEN, bool SIGMA>
 static void launch_grad(dim3 grid, cudaStream_t st, const TellArgs& a, uint32_t pps)
 {
-    k_grad_partial<REGEN, SIGMA><<<grid, kGradThreads, 0, st>>>(a.u, a.eps, PhiloxKey{a.k0, a.k1}, a.pair0,
+    k_grad_partial<REGEN, SIGMA><<<grid, kGradThreads, 0, st>>>(a.u, a.eps, philox_key(a.k0, a.k1), a.pair0,
                                                                 a.H, a.D, a.ldD, pps, a.partial, a.sigma_partial,
                                                                 a.status);
 }

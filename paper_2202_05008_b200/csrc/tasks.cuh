@@ -62,7 +62,7 @@ __device__ __forceinline__ CpState cartpole_step(const CartpoleConst& c, const C
 }
 
 // seeded start shared by all members: (0, 0, pi, 0) + Uniform(-a, a)^4, stream 1, row = episode
-__device__ __forceinline__ CpState cartpole_reset(PhiloxKey key, uint32_t generation, uint32_t episode,
+__device__ __forceinline__ CpState cartpole_reset(const PhiloxKey& key, uint32_t generation, uint32_t episode,
                                                   float a)
 {
     const uint4 r = philox4x32_10(0u, episode, generation, 1u, key);
