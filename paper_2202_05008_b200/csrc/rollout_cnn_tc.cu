@@ -355,14 +355,14 @@ __device__ __forceinline__ void c2_issue_mma(uint32_t a0, uint32_t b0, uint32_t 
 
 __global__ void __launch_bounds__(kC2Threads)
 k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const unsigned char* __restrict__ pooled1,
-               const int32_t* __restrict__ labels, uint32_t batch, uint32_t items_per_member,
-               float* __restrict__ partial, uint32_t* work_counter, DeviceStatus* status)
+               const int32_t* __restrict__ labels, uint32_t batch,
+               float* __restrict__ loss, uint32_t* work_counter, DeviceStatus* status)
 {
     extern __shared__ __align__(1024) unsigned char dyn[];
     C2Smem& S = *reinterpret_cast<C2Smem*>(dyn);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t n_pairs = (batch + 1u) / 2u;
-    const uint32_t n_items = P * items_per_member;
+    const uint64_t n_units = static_cast<uint64_t>(P) * n_pairs;      // (member, image pair), member-major
 
     if (tid == 0) {
         for (int i = 0; i < kC2Bufs; ++i) mbar_init(smem_u32(&S.full[i]), 1);
@@ -406,20 +406,24 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         // both accumulators start out free
         if (lane == 0) { mbar_arrive(smem_u32(&S.acc_free[0])); mbar_arrive(smem_u32(&S.acc_free[1])); }
         uint32_t gp = 0, done_par = 0;
-        // Items are equal in cost, so every block takes one contiguous range of them: consecutive
-        // items belong to the same member almost always, and a member's weights are staged only
-        // when the member changes.
-        const uint32_t item_end = static_cast<uint32_t>((static_cast<uint64_t>(blockIdx.x) + 1u) * n_items / gridDim.x);
+        // Image pairs are equal in cost, so every block takes one contiguous range of (member, pair)
+        // units, equal to within one pair, and walks it in items of up to 16 pairs of one member:
+        // consecutive items belong to the same member almost always, and a member's weights are
+        // staged only when the member changes.  The loss is written per image, so the result does
+        // not depend on where the ranges are cut.
+        const uint32_t unit_end = static_cast<uint32_t>((static_cast<uint64_t>(blockIdx.x) + 1u) * n_units / gridDim.x);
         uint32_t staged_member = 0xFFFFFFFFu;
-        for (uint32_t next = static_cast<uint32_t>(static_cast<uint64_t>(blockIdx.x) * n_items / gridDim.x);; ++next) {
+        uint32_t next = static_cast<uint32_t>(static_cast<uint64_t>(blockIdx.x) * n_units / gridDim.x);
+        for (;;) {
             if (tid == 0)                            // one thread decides, so the whole team takes one branch
-                S.item = (S.abort || next >= item_end) ? kNoItem : next;
+                S.item = (S.abort || next >= unit_end) ? kNoItem : next;
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
             const uint32_t item = S.item;
-            if (item >= n_items) break;
-            const uint32_t member = item / items_per_member;
-            const uint32_t pair0 = (item % items_per_member) * kPairsPerItem;
-            const int n = static_cast<int>(min(n_pairs, pair0 + kPairsPerItem) - pair0);
+            if (item == kNoItem) break;
+            const uint32_t member = item / n_pairs;
+            const uint32_t pair0 = item % n_pairs;
+            const int n = static_cast<int>(min(min(n_pairs - pair0, unit_end - item), static_cast<uint32_t>(kPairsPerItem)));
+            next = item + static_cast<uint32_t>(n);
             const int n_img = static_cast<int>(min(batch, 2u * (pair0 + n)) - 2u * pair0);
             const float* prm = theta + static_cast<size_t>(member) * ldD;
             const unsigned char* src = pooled1 + (static_cast<size_t>(member) * n_pairs + pair0) * kPairBytes;
@@ -569,9 +573,9 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     const int lab = min(max(labels[2u * pair0 + lane], 0), 9);
                     l = (mx + logf(se)) - lg[lab];
                 }
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);   // fixed order
-                if (lane == 0 && !S.abort) partial[item] = l;
+                // after a time-out the numbers mean nothing: NaN, which makes tell skip the update
+                if (lane < n_img)
+                    loss[static_cast<size_t>(member) * batch + 2u * pair0 + lane] = S.abort ? __int_as_float(0x7FC00000) : l;
             }
             fence_async_smem();        // the ring buffers held partial logits; bulk copies write them next
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
@@ -585,30 +589,32 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     if (warp == 0) tmem_dealloc(tmem, 32);
 }
 
-__global__ void k_cnn_tc_finalize(const float* __restrict__ partial, uint32_t P, uint32_t items_per_member,
-                                  uint32_t batch, float* __restrict__ fitness)
+// fitness[m] = -mean over the batch of the per-image losses: one block per member, fixed order
+// (thread t adds images t, t + 256, ...; then a tree over the threads)
+__global__ void __launch_bounds__(256)
+k_cnn_tc_finalize(const float* __restrict__ loss, uint32_t batch, float* __restrict__ fitness)
 {
-    const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
-    if (m >= P) return;
+    __shared__ float red[256];
+    const uint32_t m = blockIdx.x;
     float s = 0.f;
-    for (uint32_t t = 0; t < items_per_member; ++t) s += partial[static_cast<size_t>(m) * items_per_member + t];
-    fitness[m] = -s / static_cast<float>(batch);
+    for (uint32_t i = threadIdx.x; i < batch; i += 256u) s += loss[static_cast<size_t>(m) * batch + i];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (uint32_t off = 128u; off > 0u; off >>= 1) {
+        if (threadIdx.x < off) red[threadIdx.x] += red[threadIdx.x + off];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) fitness[m] = -red[0] / static_cast<float>(batch);
 }
 
 // ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
-static uint32_t items_per_member_of(uint32_t batch)
-{
-    const uint32_t n_pairs = (batch + 1u) / 2u;
-    return (n_pairs + kPairsPerItem - 1u) / kPairsPerItem;
-}
-
 size_t cnn_tc_scratch_bytes(uint32_t P, uint32_t batch)
 {
     const size_t n_pairs = (batch + 1u) / 2u;
     size_t b = 256;                                                        // work counter
-    b += (static_cast<size_t>(P) * items_per_member_of(batch) * sizeof(float) + 255) / 256 * 256;
+    b += (static_cast<size_t>(P) * batch * sizeof(float) + 255) / 256 * 256;      // per-image losses
     b += static_cast<size_t>(P) * n_pairs * kPairBytes;
     return b;
 }
@@ -625,9 +631,8 @@ int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uin
     }
     unsigned char* base = static_cast<unsigned char*>(scratch);
     uint32_t* counter = reinterpret_cast<uint32_t*>(base);
-    float* partial = reinterpret_cast<float*>(base + 256);
-    const uint32_t ipm = items_per_member_of(batch);
-    unsigned char* pooled1 = base + 256 + (static_cast<size_t>(P) * ipm * sizeof(float) + 255) / 256 * 256;
+    float* loss = reinterpret_cast<float*>(base + 256);
+    unsigned char* pooled1 = base + 256 + (static_cast<size_t>(P) * batch * sizeof(float) + 255) / 256 * 256;
 
     if (cudaFuncSetAttribute(k_cnn_conv1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kC1DynRequest) != cudaSuccess) return -1;
     const uint32_t n_tiles = (batch * 144u + 127u) / 128u;
@@ -638,11 +643,11 @@ int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uin
 
     const int c2_bytes = static_cast<int>(sizeof(C2Smem));
     if (cudaFuncSetAttribute(k_cnn_conv2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, c2_bytes) != cudaSuccess) return -1;
-    const uint32_t n_items = P * ipm;
-    const uint32_t g2 = min(n_items, static_cast<uint32_t>(sm_count) * 4u);      // 4 blocks of ~55 KB per SM
-    k_cnn_conv2_tc<<<g2, kC2Threads, c2_bytes, st>>>(theta, ldD, P, pooled1, labels, batch, ipm, partial, counter, status);
+    const uint64_t n_units = static_cast<uint64_t>(P) * ((batch + 1u) / 2u);
+    const uint32_t g2 = static_cast<uint32_t>(min(n_units, static_cast<uint64_t>(sm_count) * 4u));   // 4 blocks of ~55 KB per SM
+    k_cnn_conv2_tc<<<g2, kC2Threads, c2_bytes, st>>>(theta, ldD, P, pooled1, labels, batch, loss, counter, status);
     if (cudaGetLastError() != cudaSuccess) return -1;
-    k_cnn_tc_finalize<<<(P + 255u) / 256u, 256, 0, st>>>(partial, P, ipm, batch, fitness);
+    k_cnn_tc_finalize<<<P, 256, 0, st>>>(loss, batch, fitness);
     if (cudaGetLastError() != cudaSuccess) return -1;
     return 3;
 }

@@ -79,14 +79,32 @@ def test_cfg2_full_population_full_horizon_bounds_and_sampled_parity():
     s.close()
 
 
-def test_cfg4_full_population_full_horizon_bounds():
+def test_cfg4_full_population_full_horizon_bounds_and_sampled_parity():
+    # the bench configuration (P=4096, E=4, T=1000) in its launch shape: bounds, determinism, and the
+    # fitness of sampled members (first, last, the team/block boundaries of the persistent kernel)
+    # against the oracle at the full horizon
     w = W.CFG4
     s = Solver(w)
-    s.ask()
+    theta = s.ask()
     a = s.rollout().clone(); b = s.rollout().clone()
     assert torch.equal(a, b)
     a = a.cpu().numpy()
     assert np.isfinite(a).all() and a.max() <= 0.0 and a.min() >= -(28.08 * w.horizon + 400)
+    members = [0, 147, 148, 591, 592, 2047, 4095]
+    fit_o, _ = oracle_fitness(w, theta[members].cpu().numpy(), 0, w.horizon)
+    assert rel_err(a[members], fit_o, floor=1.0) < 1e-3
+    assert s.sync_status() == 0
+    s.close()
+
+
+def test_cfg2_full_horizon_sampled_parity():
+    w = W.CFG2
+    s = Solver(w)
+    theta = s.ask()
+    fit = s.rollout().cpu().numpy()
+    members = [0, 37, 100, 255]
+    fit_o, _ = oracle_fitness(w, theta[members].cpu().numpy(), 0, w.horizon)
+    assert rel_err(fit[members], fit_o, floor=1.0) < 1e-3
     s.close()
 
 
