@@ -391,7 +391,7 @@ def config_of(w, args, stored):
     task = {W.TASK_NONE: "none", W.TASK_CARTPOLE: "cartpole_swingup", W.TASK_TANH_LINEAR: "tanh_linear",
             W.TASK_SUPERVISED: "supervised_28x28", W.TASK_SEQ2SEQ_ADD: "seq2seq_addition",
             W.TASK_PAINT: f"triangle_painting_{int(w.task_param[0]) if w.task_param else 0}x{int(w.task_param[1]) if len(w.task_param) > 1 else 0}"}[w.task_kind]
-    sharded_run = args.gpus > 1 and not args.replicas
+    sharded_run = (args.gpus > 1 and not args.replicas) or getattr(args, "sharded", False)
     return {"workload": w.name, "pop_size": w.pop_size, "param_dim": w.param_dim, "task": task,
             "policy": "mlp " + "-".join(map(str, w.layer_sizes)) if w.policy_kind == W.POLICY_MLP else
                       {W.POLICY_CNN_28: "cnn_28",
@@ -450,8 +450,10 @@ def roofline_of(w, workload_key, noise, stages, work, peaks, sm_count, max_mhz, 
              "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"], "traffic": None}
     else:
         achieved = stages["rollout"]["TFLOP/s"]
-        kernel = {W.TASK_PAINT: "k_paint", W.TASK_TANH_LINEAR: "k_rollout_tl_tc",
-                  W.TASK_CARTPOLE: "k_rollout_cartpole_ws / k_rollout_mlp_tiled"}[w.task_kind]
+        # cart-pole: more than 8 episodes on a 32/64/128-wide shape run the warp-specialised two-group kernel
+        cart = "k_rollout_cartpole_ws" if (w.episodes > 8 and len(w.layer_sizes) == 4 and
+                                           16 < max(w.layer_sizes[1:3]) <= 128) else "k_rollout_mlp_tiled"
+        kernel = {W.TASK_PAINT: "k_paint", W.TASK_TANH_LINEAR: "k_rollout_tl_tc", W.TASK_CARTPOLE: cart}[w.task_kind]
         r = {"kernel": kernel,
              "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
              "frac": achieved / alu_peak,
@@ -705,7 +707,7 @@ def run_ours(args, w):
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    sharded_run = world > 1 and not args.replicas
+    sharded_run = (world > 1 and not args.replicas) or args.sharded
     overridden = bool(args.pop or args.dim)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     sampler = ClockSampler(local)
@@ -763,6 +765,8 @@ def main():
                     help="headline workload only: leave out the records of the other configurations")
     ap.add_argument("--replicas", action="store_true",
                     help="N > 1: independent solvers (weak scaling) instead of one population in pair shards")
+    ap.add_argument("--sharded", action="store_true",
+                    help="take the pair-sharded code path even at N = 1 (one shard owning every pair; checks the path)")
     ap.add_argument("--graph", action="store_true",
                     help="also time the generation replayed from a CUDA graph (extra key graph_replay)")
     ap.add_argument("--traffic-digests", action="store_true",

@@ -3,7 +3,8 @@
 // A member's two wide layers are the A operands of tcgen05.mma and stay on chip for all T steps:
 // W (128 x K) as two fp16 parts, w = hi + lo with hi = fp16(w) and lo = fp16(w - hi) (22 mantissa
 // bits together; every product of two fp16 numbers is exact and sums accumulate in fp32, so the
-// layer is as accurate as an fp32 FMA chain).  The hi part of W2 and both parts of W1 live in
+// layer is as accurate as an fp32 FMA chain; weights beyond +-65,504, the fp16 range, are clamped to
+// it).  The hi part of W2 and both parts of W1 live in
 // tensor memory, the lo part of W2 in shared memory.  The B operand of a layer is the activation
 // block of the member's four episodes, also as two fp16 parts set side by side, N = 8 columns
 // [hi(e0..e3) | lo(e0..e3)]: one MMA with A = W_part then yields W_part . a_hi and W_part . a_lo at once
@@ -112,6 +113,12 @@ __device__ __forceinline__ void split_f16(float x, __half& hi, __half& lo)
     hi = __float2half_rn(x);
     lo = __float2half_rn(x - __half2float(hi));
 }
+// weights of the wide layers: magnitudes above the largest fp16 number are taken as that number (the
+// tanh behind them is saturated long before; without the clamp they would turn into infinities)
+__device__ __forceinline__ void split_weight(float w, __half& hi, __half& lo)
+{
+    split_f16(fminf(fmaxf(w, -65504.0f), 65504.0f), hi, lo);
+}
 __device__ __forceinline__ uint32_t pack_h2(__half a, __half b)      // a in the low half
 {
     return static_cast<uint32_t>(__half_as_ushort(a)) | (static_cast<uint32_t>(__half_as_ushort(b)) << 16);
@@ -208,8 +215,8 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     __half h0, l0, h1, l1;
-                    split_f16(wrow[16 * c + 2 * i], h0, l0);
-                    split_f16(wrow[16 * c + 2 * i + 1], h1, l1);
+                    split_weight(wrow[16 * c + 2 * i], h0, l0);
+                    split_weight(wrow[16 * c + 2 * i + 1], h1, l1);
                     hi[i] = pack_h2(h0, h1); lo[i] = pack_h2(l0, l1);
                 }
                 tmem_st8(tm_lane + kColW1hi + 8u * c, hi);
@@ -234,8 +241,8 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 __half h0, l0, h1, l1;
-                split_f16(wv[2 * i], h0, l0);
-                split_f16(wv[2 * i + 1], h1, l1);
+                split_weight(wv[2 * i], h0, l0);
+                split_weight(wv[2 * i + 1], h1, l1);
                 hi[i] = pack_h2(h0, h1); lo[i] = pack_h2(l0, l1);
             }
             tmem_st8(tm_lane + kColW2hi + 8u * c, hi);

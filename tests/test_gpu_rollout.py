@@ -80,6 +80,24 @@ def test_cfg4_tensor_core_kernel_ragged_members_and_episodes(pop, episodes):
     _rollout_check(w, T, members, ROLLOUT_AUTO, check_trace=pop <= 100)
 
 
+def test_cfg4_tensor_core_kernel_with_weights_beyond_the_fp16_range():
+    """The tensor-core kernel holds the wide layers as fp16 pairs; a weight beyond +-65,504 is clamped
+    to that when staged.  The tanh behind it is saturated either way, so the fitness still agrees with
+    the oracle (which uses the weight as it is), and nothing turns into an infinity."""
+    w = W.CFG4.with_(pop_size=4, horizon=60)
+    theta = W.random_parameters(11, 4, w.param_dim, scale=0.05)
+    theta[0, 5] = 1.0e7                      # first layer, unit 0
+    theta[1, 28 * 128 + 128 + 300] = -3.0e6  # second layer
+    theta[2, 7] = 70000.0
+    s = Solver(w, rollout_kernel=ROLLOUT_AUTO)
+    arg = s.padded_rows(4); arg[:, :w.param_dim] = torch.tensor(theta, device="cuda")
+    fit = s.rollout(arg).cpu().numpy()
+    assert s.sync_status() == 0 and np.isfinite(fit).all()
+    fit_o, _ = oracle_fitness(w, theta, 0, 60)
+    assert rel_err(fit, fit_o, floor=1.0) < FIT_TOL
+    s.close()
+
+
 def test_cfg4_tensor_core_and_fp32_kernels_agree_and_repeat():
     w = W.CFG4.with_(pop_size=600, horizon=100)
     a = Solver(w, rollout_kernel=ROLLOUT_AUTO)
