@@ -27,6 +27,7 @@
 #include "internal.h"
 #include "umma.cuh"
 #include "noise.cuh"
+#include "fp32x2.cuh"
 
 #include <cuda_fp16.h>
 
@@ -332,16 +333,18 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
             // action layer on the fp32 pipe: warp = episode e, lane = (input eighth q8, output pair op)
             {
                 const float4* hp = reinterpret_cast<const float4*>(&T.h2[e][20 * q8]);
-                float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
+                // two inputs per paired FMA (fma.rn.f32x2): half the instructions of the scalar form
+                float2 s01 = make_float2(0.f, 0.f), s23 = s01, u01 = s01, u23 = s01;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float4 hv = hp[j];
-                    s0 = fmaf(w3[0][4 * j], hv.x, s0);     s1 = fmaf(w3[0][4 * j + 1], hv.y, s1);
-                    u0 = fmaf(w3[1][4 * j], hv.x, u0);     u1 = fmaf(w3[1][4 * j + 1], hv.y, u1);
-                    s0 = fmaf(w3[0][4 * j + 2], hv.z, s0); s1 = fmaf(w3[0][4 * j + 3], hv.w, s1);
-                    u0 = fmaf(w3[1][4 * j + 2], hv.z, u0); u1 = fmaf(w3[1][4 * j + 3], hv.w, u1);
+                    const float2 h01 = make_float2(hv.x, hv.y), h23 = make_float2(hv.z, hv.w);
+                    ffma2(s01, make_float2(w3[0][4 * j], w3[0][4 * j + 1]), h01);
+                    ffma2(u01, make_float2(w3[1][4 * j], w3[1][4 * j + 1]), h01);
+                    ffma2(s23, make_float2(w3[0][4 * j + 2], w3[0][4 * j + 3]), h23);
+                    ffma2(u23, make_float2(w3[1][4 * j + 2], w3[1][4 * j + 3]), h23);
                 }
-                float sa = s0 + s1, sb = u0 + u1;
+                float sa = (s01.x + s01.y) + (s23.x + s23.y), sb = (u01.x + u01.y) + (u23.x + u23.y);
 #pragma unroll
                 for (int off = 1; off < 8; off <<= 1) {
                     sa += __shfl_xor_sync(0xffffffffu, sa, off);
@@ -360,20 +363,20 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
                 if (l < kNx) ret = fmaf(-xcur, xcur, ret);        // reward on (x_t, a_t)
                 const float4* xp = reinterpret_cast<const float4*>(&T.x[e][0]);
                 const float4* ap = reinterpret_cast<const float4*>(&T.act[e][0]);
-                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                float2 s01 = make_float2(0.f, 0.f), s23 = s01;
 #pragma unroll
                 for (int j = 0; j < kNx / 4; ++j) {
                     const float4 xv = xp[j];
-                    s0 = fmaf(dynw[4 * j], xv.x, s0); s1 = fmaf(dynw[4 * j + 1], xv.y, s1);
-                    s2 = fmaf(dynw[4 * j + 2], xv.z, s2); s3 = fmaf(dynw[4 * j + 3], xv.w, s3);
+                    ffma2(s01, make_float2(dynw[4 * j], dynw[4 * j + 1]), make_float2(xv.x, xv.y));
+                    ffma2(s23, make_float2(dynw[4 * j + 2], dynw[4 * j + 3]), make_float2(xv.z, xv.w));
                 }
 #pragma unroll
                 for (int j = 0; j < kNa / 4; ++j) {
                     const float4 av = ap[j];
-                    s0 = fmaf(dynw[kNx + 4 * j], av.x, s0); s1 = fmaf(dynw[kNx + 4 * j + 1], av.y, s1);
-                    s2 = fmaf(dynw[kNx + 4 * j + 2], av.z, s2); s3 = fmaf(dynw[kNx + 4 * j + 3], av.w, s3);
+                    ffma2(s01, make_float2(dynw[kNx + 4 * j], dynw[kNx + 4 * j + 1]), make_float2(av.x, av.y));
+                    ffma2(s23, make_float2(dynw[kNx + 4 * j + 2], dynw[kNx + 4 * j + 3]), make_float2(av.z, av.w));
                 }
-                const float xn = tanh_sfu((s0 + s1) + (s2 + s3));
+                const float xn = tanh_sfu((s01.x + s01.y) + (s23.x + s23.y));
                 __syncwarp();                                      // every lane has read x[e][.]
                 if (l < kNx) {
                     __half hi, lo;
