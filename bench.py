@@ -88,23 +88,23 @@ def stage_work(w, stored):
 # that digest; once a kernel's source changes its entry reads null until it is captured again.
 CSRC = os.path.join(ROOT, "paper_2202_05008_b200", "csrc")
 NCU_TRAFFIC = {
-    ("cfg4", "stored"): {"kernel": "k_rollout_tl_tc", "bytes": 3.489119e+08,
-                         "files": ["rollout_tl_tc.cu", "umma.cuh", "async.cuh", "noise.cuh", "internal.h"],
-                         "digest": "6e58c19ffb460ae2",
+    ("cfg4", "stored"): {"kernel": "k_rollout_tl_tc", "bytes": 3.489491e+08,
+                         "files": ['rollout_tl_tc.cu', 'umma.cuh', 'async.cuh', 'noise.cuh', 'fp32x2.cuh', 'internal.h'],
+                         "digest": "f5b3bd1bbf199a6b",
                          "capture": "P = 592 capture scaled by members (the traffic is the parameter rows, proportional to P)"},
-    ("cfg2", "stored"): {"kernel": "k_rollout_cartpole_ws", "bytes": 4.787712e+06,
-                         "files": ["rollout_mlp_tiled.cu", "async.cuh", "tasks.cuh", "noise.cuh", "fp32x2.cuh", "internal.h"],
-                         "digest": "4a82517f4f499ba6", "capture": "full size"},
-    ("cfg3", "stored"): {"kernel": "k_cnn_conv2_tc", "bytes": 1.528125e+08,
-                         "files": ["rollout_cnn_tc.cu", "umma.cuh", "async.cuh", "internal.h"],
-                         "digest": "02b4c007675e3419", "capture": "full size"},
-    ("cfg5", "stored"): {"kernel": "k_ask", "bytes": 1.011388e+11,
-                         "files": ["solver_kernels.cu", "noise.cuh", "internal.h"],
-                         "digest": "87386e067f759f75",
+    ("cfg2", "stored"): {"kernel": "k_rollout_cartpole_ws", "bytes": 4.787968e+06,
+                         "files": ['rollout_mlp_tiled.cu', 'async.cuh', 'tasks.cuh', 'noise.cuh', 'fp32x2.cuh', 'internal.h'],
+                         "digest": "dd779dfecc56ca08", "capture": "full size"},
+    ("cfg3", "stored"): {"kernel": "k_cnn_conv2_tc", "bytes": 1.534646e+08,
+                         "files": ['rollout_cnn_tc.cu', 'umma.cuh', 'async.cuh', 'internal.h'],
+                         "digest": "dc67f31e2ffe836a", "capture": "full size"},
+    ("cfg5", "stored"): {"kernel": "k_ask", "bytes": 1.011768e+11,
+                         "files": ['solver_kernels.cu', 'noise.cuh', 'internal.h'],
+                         "digest": "3a3acbcf28e35af9",
                          "capture": "D = 32,768 capture scaled by 32 (columns are independent)"},
-    ("cfg5", "regenerated"): {"kernel": "k_ask", "bytes": 6.677962e+10,
-                              "files": ["solver_kernels.cu", "noise.cuh", "internal.h"],
-                              "digest": "87386e067f759f75", "capture": "D = 32,768 capture scaled by 32"},
+    ("cfg5", "regenerated"): {"kernel": "k_ask", "bytes": 6.679631e+10,
+                              "files": ['solver_kernels.cu', 'noise.cuh', 'internal.h'],
+                              "digest": "3a3acbcf28e35af9", "capture": "D = 32,768 capture scaled by 32"},
 }
 NCU_TRAFFIC[("cfg4", "regenerated")] = NCU_TRAFFIC[("cfg4", "stored")]
 NCU_TRAFFIC[("cfg2", "regenerated")] = NCU_TRAFFIC[("cfg2", "stored")]

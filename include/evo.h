@@ -51,6 +51,12 @@ enum { EVO_NOISE_STORED = 0, EVO_NOISE_REGENERATED = 1 };
 enum { EVO_POLICY_NONE = 0, EVO_POLICY_MLP = 1, EVO_POLICY_CNN_28 = 2, EVO_POLICY_LSTM_SEQ2SEQ = 3 };
 enum { EVO_TASK_NONE = 0, EVO_TASK_CARTPOLE = 1, EVO_TASK_TANH_LINEAR = 2, EVO_TASK_SUPERVISED = 3,
        EVO_TASK_SEQ2SEQ_ADD = 4, EVO_TASK_PAINT = 5 };
+/* Roll-out kernel of the control tasks.  GENERIC: runtime shapes, any MLP.  TILED: the fp32-pipe
+ * kernels with the weights in registers (two hidden layers, each at most as wide as a compiled shape:
+ * 16/32/64/128 for the cart-pole, 128 for the tanh-linear task); UNSUPPORTED at evo_rollout if none
+ * fits.  AUTO: for the tanh-linear task with hidden widths <= 128 the tensor-core kernel (wide layers
+ * as pairs of fp16 numbers on tcgen05, fp32-accurate; weights of those layers beyond +-65,504 are
+ * clamped), else TILED where it fits, else GENERIC. */
 enum { EVO_ROLLOUT_AUTO = 0, EVO_ROLLOUT_GENERIC = 1, EVO_ROLLOUT_TILED = 2 };
 enum { EVO_OPT_ADAM = 0, EVO_OPT_CLIPUP = 1 };
 enum { EVO_SIGMA_CONSTANT = 0, EVO_SIGMA_PGPE = 1 };
@@ -93,7 +99,7 @@ typedef struct evo_config {
     uint32_t horizon;              /* T >= 1 (control tasks)                                    */
     uint32_t batch;                /* images (supervised) or queries (seq2seq) per member       */
     uint32_t trace_steps;          /* leading steps recorded when evo_rollout gets d_trace, <= T */
-    uint32_t rollout_kernel;       /* EVO_ROLLOUT_*: AUTO picks the tiled kernel when one fits  */
+    uint32_t rollout_kernel;       /* EVO_ROLLOUT_*: AUTO picks the fastest kernel that fits    */
     float    task_param[16];       /* EVO_CP_* / EVO_S2S_* / EVO_PAINT_* by task; else unused   */
     uint32_t optimizer;            /* EVO_OPT_*: how the centre follows the ES gradient         */
     float    clipup_momentum;      /* ClipUp: 0 selects 0.9                                     */
