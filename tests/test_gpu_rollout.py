@@ -80,6 +80,22 @@ def test_cfg4_tensor_core_kernel_ragged_members_and_episodes(pop, episodes):
     _rollout_check(w, T, members, ROLLOUT_AUTO, check_trace=pop <= 100)
 
 
+@pytest.mark.parametrize("kernel", [ROLLOUT_GENERIC, ROLLOUT_TILED, ROLLOUT_AUTO])
+def test_cfg4_action_scale_and_later_generation(kernel):
+    """An action scale other than 1 and the initial states of a later generation (the roll-out seeds
+    depend on the generation counter) through all three kernels of the tanh-linear task."""
+    w = W.CFG4.with_(pop_size=6, action_scale=0.5, horizon=80)
+    s = Solver(w, rollout_kernel=kernel)
+    for gen in range(2):
+        theta = s.ask().cpu().numpy()
+        fit = s.rollout().cpu().numpy()
+        fit_o, _ = oracle_fitness(w, theta, gen, 80)
+        assert rel_err(fit, fit_o, floor=1.0) < FIT_TOL, gen
+        s.tell(torch.tensor(fit, device="cuda"))
+    assert s.sync_status() == 0
+    s.close()
+
+
 def test_cfg4_tensor_core_kernel_with_weights_beyond_the_fp16_range():
     """The tensor-core kernel holds the wide layers as fp16 pairs; a weight beyond +-65,504 is clamped
     to that when staged.  The tanh behind it is saturated either way, so the fitness still agrees with
