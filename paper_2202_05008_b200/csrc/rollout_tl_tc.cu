@@ -41,6 +41,10 @@ constexpr int kEB = 4;                  // episodes per team item
 constexpr int kTeams = 4, kTeamThreads = 128, kThreads = kTeams * kTeamThreads;
 // tensor-memory columns of a team
 constexpr uint32_t kColW2hi = 0, kColW1hi = 64, kColW1lo = 80, kColAcc = 96, kColsTeam = 128;
+// clocks the layer-2 MMA batch of one team keeps the tensor pipe busy (16 MMAs of ~25 clocks); measured
+// optimum of the spacing between two teams' batches (200..600 all help, 450 is best, 1000 throttles;
+// spacing the short layer-1 batches as well costs more than it gains)
+constexpr unsigned long long kL2Gap = 450;
 constexpr int kH2Pitch = kH + 32;       // h2 rows in shared memory, 4 floats of skew per 16
 constexpr int kB1Lbo = 144;             // layer-1 B operand: bytes between its 8-input groups (skewed: no bank conflicts)
 
@@ -59,6 +63,7 @@ struct Smem {
     TeamSmem team[kTeams];
     alignas(16) float dyn[kNx][36];                  // [A | B] of the task, row i = output i
     alignas(8) uint64_t drain_bar;
+    unsigned long long next_l2_slot;                 // clock at which the next team may start its layer-2 batch
     uint32_t tmem_slot;
 };
 
@@ -125,6 +130,25 @@ __device__ __forceinline__ uint32_t pack_h2(__half a, __half b)      // a in the
     return static_cast<uint32_t>(__half_as_ushort(a)) | (static_cast<uint32_t>(__half_as_ushort(b)) << 16);
 }
 
+// The teams share the tensor pipe and run the same chain with the same period.  Left alone, their
+// MMA batches interleave in the pipe (two batches issued together both finish late) and the teams
+// bunch up.  A team therefore books the pipe before it issues a batch: slots are handed out in
+// order of arrival, `clocks` apart (about the time the batch keeps the pipe busy), and a team that
+// is early sleeps until its slot (bounded: the loop ends after 64 short sleeps in any case).
+__device__ __forceinline__ void book_tensor_pipe(unsigned long long* next_slot, unsigned long long clocks)
+{
+    if (clocks == 0ull) return;
+    const unsigned long long now = static_cast<unsigned long long>(clock64());
+    unsigned long long old = *reinterpret_cast<volatile unsigned long long*>(next_slot), mine;
+    for (;;) {
+        mine = old > now ? old : now;
+        const unsigned long long seen = atomicCAS(next_slot, old, mine + clocks);
+        if (seen == old) break;
+        old = seen;
+    }
+    for (int i = 0; i < 64 && static_cast<unsigned long long>(clock64()) < mine; ++i) __nanosleep(40);
+}
+
 __device__ __forceinline__ void team_sync(int team)
 {
     asm volatile("bar.sync %0, %1;" :: "r"(1 + team), "n"(kTeamThreads) : "memory");
@@ -148,7 +172,7 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
     }
     for (int i = r; i < 640 / 4; i += kTeamThreads) reinterpret_cast<uint32_t*>(T.b1)[i] = 0u;   // inputs 28..31 stay zero
     if (r == 0) { mbar_init(smem_u32(&T.bar), 4); mbar_init_fence(); T.abort = 0; }
-    if (tid == 0) { mbar_init(smem_u32(&S.drain_bar), kTeams * 4); mbar_init_fence(); }
+    if (tid == 0) { mbar_init(smem_u32(&S.drain_bar), kTeams * 4); mbar_init_fence(); S.next_l2_slot = 0ull; }
     if (tid < 32) tmem_alloc(smem_u32(&S.tmem_slot), 512);
     fence_async_smem();
     tc_fence_before();
@@ -308,6 +332,7 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
             }
             fence_async_smem();
             tc_fence_before();
+            if (r == 0) book_tensor_pipe(&S.next_l2_slot, kL2Gap);
             team_sync(team);
             // layer 2: four MMAs per warp (two K steps x two parts of W2)
             if (l == 0 && !*aborted) {
