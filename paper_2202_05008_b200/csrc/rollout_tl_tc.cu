@@ -196,8 +196,8 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
     const uint32_t acc_w = tm + kColAcc + 8u * static_cast<uint32_t>(w);
     const bool drop_first_commit = (status->debug_flags & EVO_DEBUG_DROP_COMPLETION) != 0u;
 
-    // the narrow layers use another thread mapping: warp = episode, lane = (action o, input quarter q)
-    // for the action layer and lane = output i for the task dynamics
+    // the narrow layers use another thread mapping: warp = episode; for the action layer lane = (eighth
+    // q8 of the 128 inputs, pair op of the 8 outputs), for the task dynamics lane = output i
     const int e = w, q8 = l & 7, op = l >> 3, di = min(l, kNx - 1);
     float dynw[36];                                   // row di of [A | B]
 #pragma unroll
@@ -337,6 +337,8 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
             // layer 2: four MMAs per warp (two K steps x two parts of W2)
             if (l == 0 && !*aborted) {
                 tc_fence_after();
+                // (umma_bf16 is the kind::f16 MMA with A from shared memory; the operand type, fp16 here,
+                // comes from the instruction descriptor)
                 mma_f16_ts(acc_w, l2_a0, l2_b0, kIdescL2, 0u);
                 umma_bf16(acc_w, l2_s0, l2_b0, kIdescL2, 1u);
                 mma_f16_ts(acc_w, l2_a0 + 8u, l2_b0 + 16u, kIdescL2, 1u);
