@@ -103,8 +103,9 @@ __device__ __forceinline__ void c1_stage_rows(unsigned char* Abuf, int row, int 
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             const int k0 = 2 * k, k1 = 2 * k + 1;
-            const float v0 = (k0 < 25) ? patch[(dy + k0 / 5) * 6 + dx + k0 % 5] : 0.f;
-            const float v1 = (k1 < 25) ? patch[(dy + k1 / 5) * 6 + dx + k1 % 5] : 0.f;
+            // taps 25..27 of the padded K = 32 are the constant 1: their weights carry the bias (below)
+            const float v0 = (k0 < 25) ? patch[(dy + k0 / 5) * 6 + dx + k0 % 5] : (k0 < 28 ? 1.f : 0.f);
+            const float v1 = (k1 < 25) ? patch[(dy + k1 / 5) * 6 + dx + k1 % 5] : (k1 < 28 ? 1.f : 0.f);
             packed[k] = pack_bf16(v0, v1);
         }
 #pragma unroll
@@ -123,7 +124,6 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 
     unsigned char* Bsm = dyn;                                           // 32 KB
     unsigned char* Asm = dyn + kC1SmemB;                                // 2 x 32 KB
-    float* bias = reinterpret_cast<float*>(dyn + kC1SmemB + 2 * kC1SmemA);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t group0 = blockIdx.y * 64u;                           // first member of this block's group
@@ -142,16 +142,24 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         uint32_t w[4] = { 0, 0, 0, 0 };
         if (m < n_members) {
             const float* src = theta + static_cast<size_t>(group0 + m) * ldD + ch * 25u + kg * 8u;
+            // The bias rides in the contraction: against the three constant-1 taps stand three bf16 pieces of
+            // it, b = b0 + b1 + b2 to 24 bits, so the fp32 accumulator starts from the unrounded bias and
+            // the epilogue has nothing to add.
+            const float b = theta[static_cast<size_t>(group0 + m) * ldD + 200u + ch];
+            const float b0 = __bfloat162float(__float2bfloat16_rn(b));
+            const float b1 = __bfloat162float(__float2bfloat16_rn(b - b0));
+            const float b2 = (b - b0) - b1;
             float v[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) v[k] = (kg * 8u + k < 25u) ? src[k] : 0.f;
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t kk = kg * 8u + k;
+                v[k] = kk < 25u ? src[k] : (kk == 25u ? b0 : (kk == 26u ? b1 : (kk == 27u ? b2 : 0.f)));
+            }
 #pragma unroll
             for (int k = 0; k < 4; ++k) w[k] = pack_bf16(v[2 * k], v[2 * k + 1]);
         }
         *reinterpret_cast<uint4*>(Bsm + (kg * 64u + (f >> 3)) * 128u + (f & 7u) * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
     }
-    for (uint32_t f = tid; f < 512u; f += kC1Threads)
-        bias[f] = ((f >> 3) < n_members) ? theta[static_cast<size_t>(group0 + (f >> 3)) * ldD + 200u + (f & 7u)] : 0.f;
 
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
@@ -246,10 +254,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                         if (lane == 0) mbar_arrive(smem_u32(&ctl.acc_free[buf]));
                     }
                     const uint32_t m = gm * 8u + half * 4u + j;
-                    const float4 b0 = *reinterpret_cast<const float4*>(bias + m * 8u);
-                    const float4 b1 = *reinterpret_cast<const float4*>(bias + m * 8u + 4u);
-                    const float bb[8] = { b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w };
-                    // relu(max4 + b) = max(max4, -b) + b: two 3-input max and one add per value
+                    // the accumulators already contain the bias: relu(max4) = two 3-input max per value
                     uint32_t o[4];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -258,7 +263,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                         for (int h = 0; h < 2; ++h) {
                             const int k = 2 * c + h;
                             const float m3 = fmax3(__uint_as_float(cur[0][k]), __uint_as_float(cur[1][k]), __uint_as_float(cur[2][k]));
-                            v[h] = fmax3(m3, __uint_as_float(cur[3][k]), -bb[k]) + bb[k];
+                            v[h] = fmax3(m3, __uint_as_float(cur[3][k]), 0.f);
                         }
                         o[c] = pack_bf16(v[0], v[1]);
                     }
