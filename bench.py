@@ -95,9 +95,9 @@ NCU_TRAFFIC = {
     ("cfg2", "stored"): {"kernel": "k_rollout_cartpole_ws", "bytes": 4.787968e+06,
                          "files": ['rollout_mlp_tiled.cu', 'async.cuh', 'tasks.cuh', 'noise.cuh', 'fp32x2.cuh', 'internal.h'],
                          "digest": "dd779dfecc56ca08", "capture": "full size"},
-    ("cfg3", "stored"): {"kernel": "k_cnn_conv2_tc", "bytes": 1.534646e+08,
+    ("cfg3", "stored"): {"kernel": "k_cnn_conv2_tc", "bytes": 1.534469e+08,
                          "files": ['rollout_cnn_tc.cu', 'umma.cuh', 'async.cuh', 'internal.h'],
-                         "digest": "dc67f31e2ffe836a", "capture": "full size"},
+                         "digest": "5e888c2af8001fe0", "capture": "full size"},
     ("cfg5", "stored"): {"kernel": "k_ask", "bytes": 1.011768e+11,
                          "files": ['solver_kernels.cu', 'noise.cuh', 'internal.h'],
                          "digest": "3a3acbcf28e35af9",
