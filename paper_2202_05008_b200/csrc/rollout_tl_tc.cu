@@ -239,10 +239,10 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
                 uint32_t hi[8], lo[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    __half h0, l0, h1, l1;
-                    split_weight(wrow[16 * c + 2 * i], h0, l0);
-                    split_weight(wrow[16 * c + 2 * i + 1], h1, l1);
-                    hi[i] = pack_h2(h0, h1); lo[i] = pack_h2(l0, l1);
+                    __half ha, la, hb, lb;
+                    split_weight(wrow[16 * c + 2 * i], ha, la);
+                    split_weight(wrow[16 * c + 2 * i + 1], hb, lb);
+                    hi[i] = pack_h2(ha, hb); lo[i] = pack_h2(la, lb);
                 }
                 tmem_st8(tm_lane + kColW1hi + 8u * c, hi);
                 tmem_st8(tm_lane + kColW1lo + 8u * c, lo);
@@ -265,10 +265,10 @@ k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
             uint32_t hi[8], lo[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                __half h0, l0, h1, l1;
-                split_weight(wv[2 * i], h0, l0);
-                split_weight(wv[2 * i + 1], h1, l1);
-                hi[i] = pack_h2(h0, h1); lo[i] = pack_h2(l0, l1);
+                __half ha, la, hb, lb;
+                split_weight(wv[2 * i], ha, la);
+                split_weight(wv[2 * i + 1], hb, lb);
+                hi[i] = pack_h2(ha, hb); lo[i] = pack_h2(la, lb);
             }
             tmem_st8(tm_lane + kColW2hi + 8u * c, hi);
             // core matrix (row group r/8, K chunk): 8 rows x 16 bytes; K chunks 128 B apart, row groups 2048 B
