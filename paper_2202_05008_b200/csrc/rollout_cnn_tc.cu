@@ -34,12 +34,13 @@ namespace evo {
 // four separate A operands (the same 6x6 image patch shifted by (dy,dx)) accumulated into four
 // TMEM column blocks, so the max-pool is a max over four registers of one thread, with no
 // shuffles.  Unit of work = (tile, 8 members = 64 filters): 8 MMAs (4 windows x K = 2 x 16)
-// into one of two 256-column accumulators.  Warp 4 issues the MMAs and runs ahead; warps 0-3 read
-// the accumulators (pool, bias, ReLU, bf16) and store 16 bytes per (member, pixel), and stage the
-// next tile's A operands from a register-prefetched image patch.
+// into one of two 256-column accumulators.  Warp 8 issues the MMAs and runs ahead; warps 0-7 read
+// the accumulators (pool, ReLU, bf16; the bias rides in the contraction) and store 16 bytes per
+// (member, pixel); warps 9-12 build the next tile's A operands while the epilogues run.
 // ------------------------------------------------------------------------------------------
 constexpr int kC1EpiThreads = 256;                     // two warps per TMEM lane quarter
-constexpr int kC1Threads = kC1EpiThreads + 32;
+constexpr int kC1StageThreads = 128;                   // one thread per pooled pixel of a tile: builds the A operands
+constexpr int kC1Threads = kC1EpiThreads + 32 + kC1StageThreads;
 constexpr int kC1SmemB = 512 * 32 * 2;                  // all filters of the group, bf16, K = 32
 constexpr int kC1SmemAWin = 128 * 32 * 2;               // one window's im2col tile
 constexpr int kC1SmemA = 4 * kC1SmemAWin;               // four windows
@@ -49,6 +50,7 @@ constexpr int kC1DynRequest = 120 * 1024;
 
 struct C1Ctl {
     uint64_t a_full[2];          // the A operands of a tile are staged
+    uint64_t a_free[2];          // every MMA that read an A buffer has completed
     uint64_t mma_done[2];        // an accumulator is complete
     uint64_t acc_free[2];        // an accumulator has been read out
     uint32_t tmem_slot;
@@ -164,6 +166,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl.a_full[i]), 1);
+            mbar_init(smem_u32(&ctl.a_free[i]), 1);
             mbar_init(smem_u32(&ctl.mma_done[i]), 1);
             mbar_init(smem_u32(&ctl.acc_free[i]), kC1EpiThreads / 32);
         }
@@ -201,28 +204,37 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                         }
                     umma_commit(smem_u32(&ctl.mma_done[buf]));
                 }
+                umma_commit(smem_u32(&ctl.a_free[ti & 1u]));       // arrives once this tile's MMAs are done
             }
         }
-    } else {
-        // ================= epilogue warps (also stage the A operands) ==============================
-        if (lane == 0) { mbar_arrive(smem_u32(&ctl.acc_free[0])); mbar_arrive(smem_u32(&ctl.acc_free[1])); }
+    } else if (warp > kC1EpiThreads / 32) {
+        // ================= staging warps: im2col rows of the tiles, one tile ahead of the MMAs ============
+        // thread = pooled pixel of the tile; the 6x6 image patch under it gives the rows of all four
+        // pooling windows.  The buffer of tile ti is free once the MMAs of tile ti - 2 have completed.
+        const int row = tid - (kC1EpiThreads + 32);
         float patch[36];
-        // first tile
-        const int row = tid & 127, half = tid >> 7;       // my pooled pixel (= TMEM lane) and my half of the work
-        c1_load_patch(images, blockIdx.x * 128u + row, n_pooled, patch);
-        if (blockIdx.x < n_tiles) {
-            if (half) c1_stage_rows(Asm, row, 1, patch); else c1_stage_rows(Asm, row, 0, patch);
+        uint32_t ti = 0;
+        for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++ti) {
+            c1_load_patch(images, tile * 128u + row, n_pooled, patch);
+            if (ti >= 2u) wait_or_abort(&ctl.abort, &ctl.a_free[ti & 1u], ((ti >> 1) - 1u) & 1u, status);
+            unsigned char* Abuf = Asm + (ti & 1u) * kC1SmemA;
+            c1_stage_rows(Abuf, row, 0, patch);
+            c1_stage_rows(Abuf, row, 1, patch);
             fence_async_smem();
-            asm volatile("bar.sync 1, %0;" :: "n"(kC1EpiThreads) : "memory");
-            if (tid == 0) mbar_arrive(smem_u32(&ctl.a_full[0]));
+            asm volatile("bar.sync 2, %0;" :: "n"(kC1StageThreads) : "memory");
+            if (row == 0) mbar_arrive(smem_u32(&ctl.a_full[ti & 1u]));
         }
+        // the last arrivals on a_free land in this block's shared memory: see them in before the block ends
+        if (row < 2 && ti > static_cast<uint32_t>(row)) {
+            const uint32_t n_done = (ti - row + 1u) >> 1;              // completions of buffer `row`
+            wait_or_abort(&ctl.abort, &ctl.a_free[row], (n_done - 1u) & 1u, status);
+        }
+    } else {
+        // ================= epilogue warps ==========================================================
+        if (lane == 0) { mbar_arrive(smem_u32(&ctl.acc_free[0])); mbar_arrive(smem_u32(&ctl.acc_free[1])); }
+        const int row = tid & 127, half = tid >> 7;       // my pooled pixel (= TMEM lane) and my half of the members
         uint32_t u = 0, ti = 0;
         for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++ti) {
-            const uint32_t next = tile + gridDim.x;
-            const bool has_next = next < n_tiles;
-            if (has_next) c1_load_patch(images, next * 128u + row, n_pooled, patch);     // lands during the epilogues
-            const uint32_t stage_after = min(2u, n_gm - 1u);
-
             const uint32_t gp = tile * 128u + row;                     // my pooled pixel = my TMEM lane
             const bool pix_ok = gp < n_pooled;
             const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
@@ -269,20 +281,6 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     }
                     if (pix_ok && m < n_members)
                         pooled1[pix_off + static_cast<size_t>(group0 + m) * member_stride] = make_uint4(o[0], o[1], o[2], o[3]);
-                }
-                if (has_next && gm == stage_after) {
-                    // the other A buffer was last read by the previous tile, whose accumulators have all
-                    // been waited for: refill it for the next tile
-                    // keep the conversion of the patch here: hoisted to the loads at the top of the tile it
-                    // would make every warp wait there for the images instead of letting them land under
-                    // the epilogues
-#pragma unroll
-                    for (int i = 0; i < 36; ++i) asm volatile("" : "+f"(patch[i]));
-                    if (half) c1_stage_rows(Asm + ((ti + 1u) & 1u) * kC1SmemA, row, 1, patch);
-                    else      c1_stage_rows(Asm + ((ti + 1u) & 1u) * kC1SmemA, row, 0, patch);
-                    fence_async_smem();
-                    asm volatile("bar.sync 1, %0;" :: "n"(kC1EpiThreads) : "memory");
-                    if (tid == 0) mbar_arrive(smem_u32(&ctl.a_full[(ti + 1u) & 1u]));
                 }
             }
         }
