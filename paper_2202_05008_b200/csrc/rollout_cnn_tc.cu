@@ -4,19 +4,19 @@
 // 256->10) evaluated for every member on the same batch is two dense contractions:
 //
 //   k_cnn_conv1_tc   conv1 for ALL members at once.  The batch is shared, so the im2col rows
-//                    (K = 25 taps padded to 32) are the A operand for every member and the 8P
-//                    filters of the population sit side by side on N.  GEMM rows are pooled
-//                    pixels; the four conv outputs under a pooling window are four A operands
-//                    accumulated into four TMEM column blocks, so the 2x2 max-pool is a max over
-//                    registers.  The epilogue adds bias, applies ReLU and writes the pooled
-//                    activation as bf16, 8 channels = 16 bytes per pixel.
-//   k_cnn_conv2_tc   per member: conv2 as an implicit GEMM with NO im2col copy.  With channels
-//                    innermost, the 8 channels of a pixel are one 16-byte row of a UMMA core
-//                    matrix, 8 consecutive output columns are 8 consecutive pixels = one 128-byte
-//                    core matrix, and the (kh,kw) tap is just an address offset, so the shared
-//                    memory descriptors of the A operand point straight into the pooled image
-//                    pair that a single bulk copy brought in.  D[128 = 2 images x 8x8][16 filters]
-//                    in TMEM; pool, linear layer and cross-entropy on CUDA cores.
+//                    (K = 25 taps padded to 32, three of the pad taps carrying the bias) are the A
+//                    operand for every member and the 8P filters of the population sit side by side
+//                    on N.  GEMM rows are pooled pixels; the four conv outputs under a pooling window
+//                    are four A operands accumulated into four TMEM column blocks, so the 2x2
+//                    max-pool is a max over registers.  The epilogue applies ReLU and writes the
+//                    pooled activation as bf16, 8 channels = 16 bytes per pixel, in the operand
+//                    layout of conv2.
+//   k_cnn_conv2_tc   per member and group of 16 images: conv2 as a contraction over whole input
+//                    rows against a banded copy of the member's filter rows, with NO im2col copy:
+//                    the 8 channels of a pixel are one 16-byte row of a UMMA core matrix, 8 images
+//                    are its 8 rows, and filter row and column offsets are address offsets into
+//                    the group that a single bulk copy brought in.  D[128 = 8 rows x 16 images][4
+//                    columns x 16 filters] in TMEM; pool, linear layer and cross-entropy on CUDA cores.
 //
 // Operands are bf16 (round to nearest even), accumulation fp32 in TMEM.  Every wait is bounded:
 // on expiry the block records EVO_ERR_TIMEOUT, frees its TMEM and leaves.
@@ -24,6 +24,7 @@
 #include "internal.h"
 #include "async.cuh"
 #include "umma.cuh"
+#include "fp32x2.cuh"
 
 namespace evo {
 
@@ -57,11 +58,14 @@ struct C1Ctl {
     volatile int abort;
 };
 
-// pooled-1 layout: [member][image pair][y 12][image in pair 2][x 12][channel 8] bf16
-__device__ __forceinline__ size_t pooled1_offset(uint32_t member, uint32_t n_pairs, uint32_t image,
-                                                 uint32_t py, uint32_t px)
+// pooled-1 layout: [member][group of 16 images][y 12][image octet 2][x 12][image in octet 8][channel 8] bf16,
+// i.e. the operand layout of the second convolution.  A GEMM row of conv1 is one 16-byte element of
+// it, rows in storage order, so a tile of 128 rows is 2 KB of consecutive output.
+struct C1Row { uint32_t image, py, px; };
+__device__ __forceinline__ C1Row c1_row(uint32_t r)
 {
-    return (((static_cast<size_t>(member) * n_pairs + (image >> 1)) * 12 + py) * 2 + (image & 1u)) * 12 + px;
+    const uint32_t group = r / 2304u, e = r % 2304u, q = e / 96u;         // q = y * 2 + octet
+    return { group * 16u + (q & 1u) * 8u + (e & 7u), q >> 1, (e >> 3) % 12u };
 }
 
 // max of three values in one instruction (the 3-input form of max.f32)
@@ -72,13 +76,13 @@ __device__ __forceinline__ float fmax3(float a, float b, float c)
     return r;
 }
 
-// 6x6 image patch under one pooled pixel (zero for rows past the batch)
-__device__ __forceinline__ void c1_load_patch(const float* __restrict__ images, uint32_t gp, uint32_t n_pooled,
+// 6x6 image patch under the pooled pixel of GEMM row r (zero for images past the batch)
+__device__ __forceinline__ void c1_load_patch(const float* __restrict__ images, uint32_t r, uint32_t batch,
                                               float (&patch)[36])
 {
-    if (gp < n_pooled) {
-        const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
-        const float* src = images + static_cast<size_t>(img) * 784u + (2u * py) * 28u + 2u * px;
+    const C1Row at = c1_row(r);
+    if (at.image < batch) {
+        const float* src = images + static_cast<size_t>(at.image) * 784u + (2u * at.py) * 28u + 2u * at.px;
 #pragma unroll
         for (int r = 0; r < 6; ++r) {
             const float2* row = reinterpret_cast<const float2*>(src + r * 28);     // 2*px is even: 8-byte aligned
@@ -119,7 +123,7 @@ __device__ __forceinline__ void c1_stage_rows(unsigned char* Abuf, int row, int 
 
 __global__ void __launch_bounds__(kC1Threads, 1)
 k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const float* __restrict__ images,
-               uint32_t batch, uint4* __restrict__ pooled1, uint32_t* work_counter, DeviceStatus* status)
+               uint32_t batch, uint4* __restrict__ pooled1, DeviceStatus* status)
 {
     extern __shared__ __align__(1024) unsigned char dyn[];
     __shared__ __align__(8) C1Ctl ctl;
@@ -131,11 +135,8 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     const uint32_t group0 = blockIdx.y * 64u;                           // first member of this block's group
     const uint32_t n_members = min(64u, P - group0);
     const uint32_t n_gm = (n_members + 7u) / 8u;                        // units per tile
-    const uint32_t n_pairs = (batch + 1u) / 2u;
-    const uint32_t n_pooled = batch * 144u;
-    const uint32_t n_tiles = (n_pooled + 127u) / 128u;
-
-    if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *work_counter = 0;   // for the conv2 kernel
+    const uint32_t n_groups = (batch + 15u) / 16u;
+    const uint32_t n_tiles = n_groups * 18u;                            // 16 images x 144 pooled pixels = 18 tiles
 
     // ---- B operand: W1 of every member of the group, [filter][k] -> core matrices (k-group, member)
     for (uint32_t idx = tid; idx < 512u * 4u; idx += kC1Threads) {
@@ -215,7 +216,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         float patch[36];
         uint32_t ti = 0;
         for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++ti) {
-            c1_load_patch(images, tile * 128u + row, n_pooled, patch);
+            c1_load_patch(images, tile * 128u + row, batch, patch);
             if (ti >= 2u) wait_or_abort(&ctl.abort, &ctl.a_free[ti & 1u], ((ti >> 1) - 1u) & 1u, status);
             unsigned char* Abuf = Asm + (ti & 1u) * kC1SmemA;
             c1_stage_rows(Abuf, row, 0, patch);
@@ -235,11 +236,9 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         const int row = tid & 127, half = tid >> 7;       // my pooled pixel (= TMEM lane) and my half of the members
         uint32_t u = 0, ti = 0;
         for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++ti) {
-            const uint32_t gp = tile * 128u + row;                     // my pooled pixel = my TMEM lane
-            const bool pix_ok = gp < n_pooled;
-            const uint32_t img = gp / 144u, rem = gp % 144u, py = rem / 12u, px = rem % 12u;
-            const size_t pix_off = pooled1_offset(0u, n_pairs, img, py, px);     // + member * member_stride
-            const size_t member_stride = static_cast<size_t>(n_pairs) * (12u * 2u * 12u);
+            const uint32_t pix_off = tile * 128u + row;                // my GEMM row = my TMEM lane = my output element
+            const bool pix_ok = c1_row(pix_off).image < batch;
+            const size_t member_stride = static_cast<size_t>(n_groups) * 2304u;
 
             for (uint32_t gm = 0; gm < n_gm; ++gm, ++u) {
                 const uint32_t buf = u & 1u;
@@ -292,40 +291,56 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 }
 
 // ------------------------------------------------------------------------------------------
-// conv2 + pool + linear + cross-entropy, one work item = (member, 16 image pairs).
-// Warp-specialised: warp 4 only issues tensor-core work (13 MMAs per image pair, running ahead
-// of the epilogue through two 16-column TMEM accumulators); warps 0-3 take the accumulators out
-// of TMEM (pool, bias, ReLU), keep the pooled activations of the item's 32 images in shared
-// memory and run the linear layer and the cross-entropy once per item.  Pooled image pairs
-// arrive through a 4-deep ring of bulk copies.  The roles meet only on mbarriers; every wait is
-// bounded, and after a time-out all later waits fall through so that no role is left behind.
+// conv2 + pool + linear + cross-entropy.  Unit of work = (member, group of 16 images).
+//
+// The contraction runs over a whole input row at a time.  For one filter row dy, the 4 output
+// columns x 16 filters of half a row (N = 64) are a product of the 8 input columns x 8 channels under
+// them (K = 64) with a banded matrix that holds the member's 5 taps of that filter row at the
+// offsets column - output column (zero elsewhere; 5/8 dense).  The band does not depend on which
+// half of the row is computed, so one 40 KB operand serves both.  GEMM rows are (output row, image):
+// with the group stored as [y][image octet][x][image in octet][8 channels], the 8 images of an
+// octet are one core matrix, a step in y is a fixed byte offset, and filter row dy is the same
+// operand started dy rows lower.  Per unit: 2 halves x 5 filter rows x 4 K-steps = 40 MMAs of
+// M = 128, N = 64, K = 16, where the tap-by-tap implicit GEMM needed 104 (13 per image pair, N = 16):
+// an MMA reads its 4 KB A operand from shared memory whatever N is, and that read, not the
+// arithmetic, is what paces it.
+//
+// Roles: warps 0-3 read the accumulators (2x2 max over two columns of a thread and two lanes,
+// bias, ReLU, bf16) into a per-image activation buffer; warps 4-7 run the linear layer and the
+// cross-entropy from that buffer; warps 8-11 each issue the MMAs of one (accumulator, half);
+// warp 12 brings the groups in, one bulk copy each, two units ahead.  The roles meet only on
+// mbarriers; every wait is bounded, and after a time-out all later waits fall through so that no
+// role is left behind.
 // ------------------------------------------------------------------------------------------
 constexpr int kC2EpiThreads = 128;
-constexpr int kC2Threads = kC2EpiThreads + 32;
-constexpr int kPairsPerItem = 16;
-constexpr uint32_t kPairBytes = 12 * 2 * 12 * 16;        // 4608
-constexpr int kC2Bufs = 4;
-constexpr int kP2Stride = 258;                           // bf16 elements; 129 words: image rows fall in distinct banks
-constexpr uint32_t kNoItem = 0xFFFFFFFFu;
+constexpr int kC2LinThreads = 128;
+constexpr int kC2Issuers = 4;
+constexpr int kC2Threads = kC2EpiThreads + kC2LinThreads + 32 * kC2Issuers + 32;
+constexpr uint32_t kGroupRowBytes = 12 * 8 * 16;         // one (y, image octet): 12 pixels x 8 images x 16 bytes
+constexpr uint32_t kGroupBytes = 12 * 2 * kGroupRowBytes;   // 36,864
+constexpr uint32_t kC2SmemB = 5 * 8 * 8 * 128;           // (filter row, input column, 8-column group of N) core matrices
+constexpr int kP2Pitch = 264;                            // bf16 per image: 132 words, images fall in distinct banks
+constexpr int kRawPitch = 201;                           // floats per filter in the weight scratch (odd: no bank conflicts)
 
 struct __align__(128) C2Smem {
-    unsigned char a[kC2Bufs][kPairBytes];                // pooled image pairs (ring)
-    unsigned char b[26 * 2 * 128];                       // W2 as core matrices (tap, filter group)
+    unsigned char a[2][kGroupBytes];                     // pooled-1 groups (double buffer)
+    unsigned char b[kC2SmemB];                           // banded W2
+    float raw[16 * kRawPitch];                           // W2 as stored, one padded row per filter
     float wfT[256 * 12];                                 // linear layer transposed [k][class], bf16-rounded
-    __align__(16) __nv_bfloat16 p2[2 * kPairsPerItem][kP2Stride];   // pooled-2 activations of the item's images (they are
-                                                         // bf16 operands of the linear layer anyway; half the size lets
-                                                         // four blocks share an SM)
-    float logit[2 * kPairsPerItem][12];
+    __align__(16) __nv_bfloat16 p2[2][16][kP2Pitch];     // pooled-2 activations of a unit's images, k = pixel*16 + channel
+    float part[2][4][16][12];                            // partial logits of the four linear warps
     float b2[16];
     float bfc[12];
-    uint64_t full[kC2Bufs];                              // a ring slot has landed
+    uint64_t a_full[2];                                  // a group has landed
+    uint64_t a_free[2];                                  // every MMA that read a group has completed
     uint64_t mma_done[2];                                // an accumulator is complete
     uint64_t acc_free[2];                                // an accumulator has been read out
-    uint64_t item_ready;                                 // weights of the next item are staged
+    uint64_t p2_full[2];                                 // the activations of a unit are written
+    uint64_t p2_free[2];                                 // ... and have been consumed by the linear layer
+    uint64_t drain;                                      // all MMAs of the block have completed
+    uint32_t staged;                                     // members of the block's range whose band has been staged
     uint32_t tmem_slot;
     volatile int abort;
-    volatile uint32_t item;
-    volatile int n;
 };
 
 __device__ __forceinline__ void c2_wait(C2Smem& S, uint64_t* bar, uint32_t parity, DeviceStatus* status)
@@ -333,129 +348,199 @@ __device__ __forceinline__ void c2_wait(C2Smem& S, uint64_t* bar, uint32_t parit
     wait_or_abort(&S.abort, bar, parity, status);
 }
 
-__device__ __forceinline__ void c2_load_pair(C2Smem& S, int buf, const unsigned char* src)
+// The band is staged once per member, in order, and the count of staged members only grows: an
+// issuer that has no unit of some member (a group count of one) would lose track of an mbarrier's
+// phase parity, a counter cannot be misread.  Bounded like every other wait.
+__device__ __forceinline__ void c2_wait_staged(C2Smem& S, uint32_t need, DeviceStatus* status)
 {
-    bulk_copy_g2s(smem_u32(S.a[buf]), src, kPairBytes, smem_u32(&S.full[buf]));
-}
-
-// 13 MMAs (K = 16 each = two 5x5 taps x 8 channels) of one image pair into one accumulator.
-// Tap g = (kh, kw) of the A operand is the pooled pair shifted by kh rows (384 B) and kw pixels
-// (16 B); the loop is unrolled so that all offsets are immediates.
-__device__ __forceinline__ void c2_issue_mma(uint32_t a0, uint32_t b0, uint32_t d_tmem, uint32_t bar)
-{
-    constexpr uint32_t idesc = umma_idesc_bf16(128, 16);
-#pragma unroll
-    for (uint32_t j = 0; j < 13u; ++j) {
-        const uint32_t g0 = 2u * j, g1 = 2u * j + 1u;
-        const uint32_t off0 = (g0 / 5u) * 384u + (g0 % 5u) * 16u;
-        const uint32_t off1 = (g1 < 25u) ? (g1 / 5u) * 384u + (g1 % 5u) * 16u : off0;   // tap 25 = zero weights
-        const uint64_t ad = umma_smem_desc(a0 + off0, off1 - off0, 192u);
-        const uint64_t bd = umma_smem_desc(b0 + j * 512u, 256u, 128u);
-        umma_bf16(d_tmem, ad, bd, idesc, j);
+    const uint32_t addr = smem_u32(&S.staged);
+    uint32_t have;
+    long long t0 = 0;
+    for (;;) {
+        if (S.abort) return;
+        asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(have) : "r"(addr) : "memory");
+        if (have >= need) return;
+        if (t0 == 0) t0 = clock64();
+        if (clock64() - t0 > (1ll << status->wait_cycles_log2)) {
+            S.abort = 1;
+            atomicOr(&status->sticky, 1u << EVO_ERR_TIMEOUT);
+            return;
+        }
+        __nanosleep(64);
     }
-    umma_commit(bar);
 }
 
-__global__ void __launch_bounds__(kC2Threads)
+// The 20 MMAs of one half-row block of a unit.  a0 = the group, advanced to the half's first input
+// column; filter row dy starts the A operand dy rows lower and selects band dy; a K-step is two
+// input columns.
+__device__ __forceinline__ void c2_issue_mma(uint32_t a0, uint32_t b0, uint32_t d_tmem)
+{
+    constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
+#pragma unroll
+    for (uint32_t dy = 0; dy < 5u; ++dy)
+#pragma unroll
+        for (uint32_t ks = 0; ks < 4u; ++ks) {
+            const uint64_t ad = umma_smem_desc(a0 + dy * 2u * kGroupRowBytes + ks * 256u, 128u, kGroupRowBytes);
+            const uint64_t bd = umma_smem_desc(b0 + dy * 8192u + ks * 2048u, 1024u, 128u);
+            umma_bf16(d_tmem, ad, bd, idesc, dy | ks);
+        }
+}
+
+__global__ void __launch_bounds__(kC2Threads, 1)
 k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const unsigned char* __restrict__ pooled1,
                const int32_t* __restrict__ labels, uint32_t batch,
-               float* __restrict__ loss, uint32_t* work_counter, DeviceStatus* status)
+               float* __restrict__ loss, DeviceStatus* status)
 {
     extern __shared__ __align__(1024) unsigned char dyn[];
     C2Smem& S = *reinterpret_cast<C2Smem*>(dyn);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t n_pairs = (batch + 1u) / 2u;
-    const uint64_t n_units = static_cast<uint64_t>(P) * n_pairs;      // (member, image pair), member-major
+    const uint32_t n_groups = (batch + 15u) / 16u;
+    const uint64_t n_units = static_cast<uint64_t>(P) * n_groups;     // (member, group), member-major
+    // Units are equal in cost, so every block takes one contiguous range, equal to within one unit.
+    // The loss is written per image, so the result does not depend on where the ranges are cut.
+    const uint32_t u_begin = static_cast<uint32_t>(static_cast<uint64_t>(blockIdx.x) * n_units / gridDim.x);
+    const uint32_t u_end = static_cast<uint32_t>((static_cast<uint64_t>(blockIdx.x) + 1u) * n_units / gridDim.x);
+    const uint32_t n_mine = u_end - u_begin;
 
     if (tid == 0) {
-        for (int i = 0; i < kC2Bufs; ++i) mbar_init(smem_u32(&S.full[i]), 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&S.mma_done[i]), 1); mbar_init(smem_u32(&S.acc_free[i]), 4); }
-        mbar_init(smem_u32(&S.item_ready), 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&S.a_full[i]), 1);
+            mbar_init(smem_u32(&S.a_free[i]), 2);
+            mbar_init(smem_u32(&S.mma_done[i]), 2);
+            mbar_init(smem_u32(&S.acc_free[i]), kC2EpiThreads / 32);
+            mbar_init(smem_u32(&S.p2_full[i]), kC2EpiThreads / 32);
+            mbar_init(smem_u32(&S.p2_free[i]), kC2LinThreads / 32);
+        }
+        S.staged = 0;
+        mbar_init(smem_u32(&S.drain), kC2Issuers);
         S.abort = 0;
         mbar_init_fence();
     }
+    // the zeros of the band stay where they are for every member
+    for (uint32_t i = tid; i < kC2SmemB / 16u; i += kC2Threads) reinterpret_cast<uint4*>(S.b)[i] = make_uint4(0u, 0u, 0u, 0u);
     for (int k = tid; k < 256; k += kC2Threads) { S.wfT[k * 12 + 10] = 0.f; S.wfT[k * 12 + 11] = 0.f; }
     if (tid < 2) S.bfc[10 + tid] = 0.f;
     __syncwarp();
-    if (warp == 0) tmem_alloc(smem_u32(&S.tmem_slot), 32);
+    if (warp == 0) tmem_alloc(smem_u32(&S.tmem_slot), 256);
+    fence_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = S.tmem_slot;
 
-    if (warp == 4) {
-        // ================= MMA issuer: one thread, runs ahead of the epilogue =================
-        if (lane == 0) {
-            uint32_t gp = 0, item_par = 0, full_par = 0, free_par = 0;
-            const uint32_t b0 = smem_u32(S.b);
-            for (;;) {
-                c2_wait(S, &S.item_ready, item_par, status);
-                item_par ^= 1u;
-                if (S.item == kNoItem || S.abort) break;
-                const int n = S.n;
-                for (int i = 0; i < n; ++i, ++gp) {
-                    const uint32_t slot = gp % kC2Bufs, acc = gp & 1u;
-                    c2_wait(S, &S.full[slot], (full_par >> slot) & 1u, status);
-                    full_par ^= (1u << slot);
-                    c2_wait(S, &S.acc_free[acc], (free_par >> acc) & 1u, status);
-                    free_par ^= (1u << acc);
-                    tc_fence_after();
-                    c2_issue_mma(smem_u32(S.a[slot]), b0, tmem + 16u * acc, smem_u32(&S.mma_done[acc]));
-                }
-            }
-        }
-    } else {
-        // ================= epilogue warps ========================================================
+    if (warp < kC2EpiThreads / 32) {
+        // ================= accumulator warps: pool, bias, ReLU -> activations ====================
         // both accumulators start out free
         if (lane == 0) { mbar_arrive(smem_u32(&S.acc_free[0])); mbar_arrive(smem_u32(&S.acc_free[1])); }
-        uint32_t gp = 0, done_par = 0;
-        // Image pairs are equal in cost, so every block takes one contiguous range of (member, pair)
-        // units, equal to within one pair, and walks it in items of up to 16 pairs of one member:
-        // consecutive items belong to the same member almost always, and a member's weights are
-        // staged only when the member changes.  The loss is written per image, so the result does
-        // not depend on where the ranges are cut.
-        const uint32_t unit_end = static_cast<uint32_t>((static_cast<uint64_t>(blockIdx.x) + 1u) * n_units / gridDim.x);
+        // TMEM lane = output row y (2 per warp) x image: the warp owns pooled row py = warp; a thread
+        // holds the 4 x 16 (column, filter) outputs of a half row.  Column pairs are a max over two
+        // registers; the row pair is lane ^ 16, done as an exchange: the thread of the even row keeps
+        // the left pooled pixel of the half, the thread of the odd row the right one.
+        const int img = lane & 15, odd = lane >> 4, py = warp;
+        const uint32_t first_member = u_begin / n_groups;
+        float bias[16];
         uint32_t staged_member = 0xFFFFFFFFu;
-        uint32_t next = static_cast<uint32_t>(static_cast<uint64_t>(blockIdx.x) * n_units / gridDim.x);
-        for (;;) {
-            if (tid == 0)                            // one thread decides, so the whole team takes one branch
-                S.item = (S.abort || next >= unit_end) ? kNoItem : next;
-            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-            const uint32_t item = S.item;
-            if (item == kNoItem) break;
-            const uint32_t member = item / n_pairs;
-            const uint32_t pair0 = item % n_pairs;
-            const int n = static_cast<int>(min(min(n_pairs - pair0, unit_end - item), static_cast<uint32_t>(kPairsPerItem)));
-            next = item + static_cast<uint32_t>(n);
-            const int n_img = static_cast<int>(min(batch, 2u * (pair0 + n)) - 2u * pair0);
-            const float* prm = theta + static_cast<size_t>(member) * ldD;
-            const unsigned char* src = pooled1 + (static_cast<size_t>(member) * n_pairs + pair0) * kPairBytes;
-
-            // every earlier pair has been consumed (its accumulator was waited for), so the ring is free
-            if (tid == 0)
-                for (int i = 0; i < min(kC2Bufs, n); ++i)
-                    c2_load_pair(S, (gp + i) % kC2Bufs, src + static_cast<size_t>(i) * kPairBytes);
-
-            // ---- weights: coalesced reads, then the operand layouts are built from shared memory ----
-            float* raw = reinterpret_cast<float*>(&S.p2[0][0]);     // 3,200 floats of scratch
-            static_assert(sizeof(S.p2) >= 3200 * sizeof(float), "weight scratch fits in the activation buffer");
+        for (uint32_t j = 0; j < n_mine; ++j) {
+            const uint32_t member = (u_begin + j) / n_groups, ab = j & 1u, par = (j >> 1) & 1u;
             if (member != staged_member) {
-            staged_member = member;
-            {   // conv2 weights (offset 208) and linear weights (offset 3424) start 16-byte aligned
-                const float4* w2v = reinterpret_cast<const float4*>(prm + 208u);
-                const float4* wfv = reinterpret_cast<const float4*>(prm + 3424u);
-                float4 t2[7], tf[5];
-#pragma unroll
-                for (int k = 0; k < 7; ++k) t2[k] = (tid + k * kC2EpiThreads < 800) ? __ldg(w2v + tid + k * kC2EpiThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int k = 0; k < 5; ++k) tf[k] = __ldg(wfv + tid + k * kC2EpiThreads);
+                // Every MMA of the previous member has been waited for, so the band can be rewritten.
+                staged_member = member;
+                const float* prm = theta + static_cast<size_t>(member) * ldD;
+                const float4* w2v = reinterpret_cast<const float4*>(prm + 208u);      // 16-byte aligned
+                float4 t2[7];
 #pragma unroll
                 for (int k = 0; k < 7; ++k)
-                    if (tid + k * kC2EpiThreads < 800) reinterpret_cast<float4*>(raw)[tid + k * kC2EpiThreads] = t2[k];
+                    t2[k] = (tid + k * kC2EpiThreads < 800) ? __ldg(w2v + tid + k * kC2EpiThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int k = 0; k < 7; ++k) {
+                    const uint32_t i = 4u * (tid + k * kC2EpiThreads);               // flat (filter*8 + channel)*25 + tap
+                    if (i < 3200u) {
+                        float* d = S.raw + (i / 200u) * kRawPitch + i % 200u;       // 200 = 4 * 50: a float4 stays in its filter
+                        d[0] = t2[k].x; d[1] = t2[k].y; d[2] = t2[k].z; d[3] = t2[k].w;
+                    }
+                }
+                if (tid < 16) S.b2[tid] = prm[3408u + tid];
+                asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+                // band dy, K row (input column xi, channel), N column (output column xo, filter f) = W2[f][channel][dy][xi - xo]
+                for (uint32_t idx = tid; idx < 1600u; idx += kC2EpiThreads) {
+                    const uint32_t f = idx & 15u, q = idx >> 4, dx = q % 5u, xo = (q / 5u) & 3u, dy = q / 20u;
+                    const float* src = S.raw + f * kRawPitch + dy * 5u + dx;
+                    uint32_t w[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) w[k] = pack_bf16(src[(2 * k) * 25], src[(2 * k + 1) * 25]);
+                    const uint32_t n = xo * 16u + f;
+                    *reinterpret_cast<uint4*>(S.b + ((dy * 8u + xo + dx) * 8u + (n >> 3)) * 128u + (n & 7u) * 16u) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
+                }
+#pragma unroll
+                for (int f = 0; f < 16; ++f) bias[f] = S.b2[f];
+                fence_async_smem();
+                asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+                if (tid == 0)
+                    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;"
+                                 :: "r"(smem_u32(&S.staged)), "r"(member - first_member + 1u) : "memory");
+            }
+            c2_wait(S, &S.mma_done[ab], par, status);
+            tc_fence_after();
+            c2_wait(S, &S.p2_free[ab], par, status);
+            const uint32_t t0 = tmem + (static_cast<uint32_t>(warp * 32) << 16) + ab * 128u;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t r[4][16];                                     // [output column in the half][filter]
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld16_issue(t0 + h * 64u + c * 16u, r[c]);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld16_fence(r[c]);
+                if (h == 1) {                                          // the accumulator is in registers now
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&S.acc_free[ab]));
+                }
+                uint32_t o[8];
+#pragma unroll
+                for (int f = 0; f < 16; f += 2) {
+                    float v[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float left = fmaxf(__uint_as_float(r[0][f + e]), __uint_as_float(r[1][f + e]));
+                        const float right = fmaxf(__uint_as_float(r[2][f + e]), __uint_as_float(r[3][f + e]));
+                        const float keep = odd ? right : left;
+                        const float give = odd ? left : right;
+                        v[e] = fmaxf(fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 16)) + bias[f + e], 0.f);
+                    }
+                    o[f >> 1] = pack_bf16(v[0], v[1]);
+                }
+                const int px = 2 * h + odd;
+                uint4* dst = reinterpret_cast<uint4*>(&S.p2[ab][img][(py * 4 + px) * 16]);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&S.p2_full[ab]));
+        }
+    } else if (warp < (kC2EpiThreads + kC2LinThreads) / 32) {
+        // ================= linear layer 256 -> 10 and cross-entropy ==============================
+        // thread = (images ip and ip + 8, slice s of the inputs: the pairs k = 2(s + 16 i), +1); the 16
+        // slices meet by two shuffles inside a warp and through shared memory across the four warps.
+        if (lane == 0) { mbar_arrive(smem_u32(&S.p2_free[0])); mbar_arrive(smem_u32(&S.p2_free[1])); }
+        const int lt = tid - kC2EpiThreads, wl = lt >> 5;
+        const int ip = lane & 7, s = wl * 4 + (lane >> 3);
+        uint32_t staged_member = 0xFFFFFFFFu;
+        for (uint32_t j = 0; j < n_mine; ++j) {
+            const uint32_t unit = u_begin + j, member = unit / n_groups, group = unit % n_groups;
+            const uint32_t pb = j & 1u, par = (j >> 1) & 1u;
+            if (member != staged_member) {
+                // every linear warp is past the previous unit's products (the barrier below)
+                staged_member = member;
+                const float* prm = theta + static_cast<size_t>(member) * ldD;
+                const float4* wfv = reinterpret_cast<const float4*>(prm + 3424u);     // 16-byte aligned
+                float4 tf[5];
+#pragma unroll
+                for (int k = 0; k < 5; ++k) tf[k] = __ldg(wfv + lt + k * kC2LinThreads);
 #pragma unroll
                 for (int k = 0; k < 5; ++k) {
                     // flat index cls*256 + (c*16 + pos), 4 consecutive pos; stored at row pos*16 + c
-                    const uint32_t i = 4u * (tid + k * kC2EpiThreads);
+                    const uint32_t i = 4u * (lt + k * kC2LinThreads);
                     const uint32_t cls = i >> 8, c = (i >> 4) & 15u, pos = i & 15u;
                     float* d = S.wfT + (pos * 16u + c) * 12u + cls;
                     d[0 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].x));
@@ -463,133 +548,136 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     d[2 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].z));
                     d[3 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].w));
                 }
+                if (lt < 10) S.bfc[lt] = prm[5984u + lt];
+                asm volatile("bar.sync 2, %0;" :: "n"(kC2LinThreads) : "memory");
             }
-            if (tid < 16) S.b2[tid] = prm[3408u + tid];
-            if (tid < 10) S.bfc[tid] = prm[5984u + tid];
-            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-            // W2[oc][ic][kh][kw] -> k = (kh*5+kw)*8 + ic: core matrix (tap g, oc/8), row oc%8, 16 bytes = 8 ic
-            for (uint32_t idx = tid; idx < 26u * 16u; idx += kC2EpiThreads) {
-                const uint32_t g = idx >> 4, oc = idx & 15u;
-                uint32_t w[4] = { 0, 0, 0, 0 };
-                if (g < 25u) {
+            c2_wait(S, &S.p2_full[pb], par, status);
+            float2 acc[2][5];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        w[k] = pack_bf16(raw[(oc * 8u + 2 * k) * 25u + g], raw[(oc * 8u + 2 * k + 1) * 25u + g]);
-                }
-                *reinterpret_cast<uint4*>(S.b + (g * 2u + (oc >> 3)) * 128u + (oc & 7u) * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            fence_async_smem();
-            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-            }
-            if (tid == 0) { S.n = n; __threadfence_block(); mbar_arrive(smem_u32(&S.item_ready)); }
-
-            // After the 2x2 max (lanes ^1 = x parity, ^16 = y parity) done as a reduce-scatter, this
-            // lane owns channels c0..c0+3 of pooled pixel (image im, row py = warp, column px).
-            const int c0 = 8 * (lane & 1) + 4 * ((lane >> 4) & 1);
-            const int im = (lane >> 3) & 1, px = (lane & 7) >> 1, py = warp;
-            float bias4[4];
+            for (int e = 0; e < 2; ++e)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) bias4[j] = S.b2[c0 + j];
-
-            for (int i = 0; i < n; ++i, ++gp) {
-                const uint32_t slot = gp % kC2Bufs, acc = gp & 1u;
-                c2_wait(S, &S.mma_done[acc], (done_par >> acc) & 1u, status);
-                done_par ^= (1u << acc);
-                tc_fence_after();
-                // pair i has been consumed by the tensor core: its ring slot takes pair i + ring depth
-                if (tid == 0 && i + kC2Bufs < n) c2_load_pair(S, slot, src + static_cast<size_t>(i + kC2Bufs) * kPairBytes);
-                // lane = (y%2, image, x); 2x2 max = lanes ^1 and ^16; + bias, ReLU, bf16
-                float r[16];
-                tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + 16u * acc, r);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&S.acc_free[acc]));   // values are in registers now
-                {
-                    const bool up0 = lane & 1, up1 = lane & 16;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const float keep = up0 ? r[8 + c] : r[c];
-                        const float give = up0 ? r[c] : r[8 + c];
-                        r[c] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 1));
-                    }
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const float keep = up1 ? r[4 + c] : r[c];
-                        const float give = up1 ? r[c] : r[4 + c];
-                        r[c] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 16));
-                    }
-                    // activation index inside the item: (pixel, channel), channel innermost
-                    uint32_t* dst = reinterpret_cast<uint32_t*>(&S.p2[2 * i + im][(py * 4 + px) * 16 + c0]);
-                    dst[0] = pack_bf16(fmaxf(r[0] + bias4[0], 0.f), fmaxf(r[1] + bias4[1], 0.f));
-                    dst[1] = pack_bf16(fmaxf(r[2] + bias4[2], 0.f), fmaxf(r[3] + bias4[3], 0.f));
-                }
-            }
-            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-
-            // ---- linear 256 -> 10 for all images of the item: thread = (image, quarter of the inputs);
-            //      the partial logits meet in the ring buffers, which are idle now ----
-            float* part = reinterpret_cast<float*>(S.a[0]);            // [4][32][12]
-            {
-                float acc[12];
-#pragma unroll
-                for (int j = 0; j < 12; ++j) acc[j] = 0.f;
-                if (lane < 2 * n) {
-                    const uint32_t* x2 = reinterpret_cast<const uint32_t*>(&S.p2[lane][64 * warp]);   // two inputs per word
-                    const float* wr = S.wfT + 64 * warp * 12;
+                for (int c = 0; c < 5; ++c) acc[e][c] = make_float2(0.f, 0.f);
+            const uint32_t* x0 = reinterpret_cast<const uint32_t*>(&S.p2[pb][ip][0]) + s;        // two inputs per word
+            const uint32_t* x1 = reinterpret_cast<const uint32_t*>(&S.p2[pb][ip + 8][0]) + s;
+            const float* wr = S.wfT + s * 24;
 #pragma unroll 2
-                    for (int k2 = 0; k2 < 32; ++k2) {
-                        const uint32_t pair = x2[k2];
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t xa = x0[16 * i], xb = x1[16 * i];
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const float xv = __uint_as_float(h ? (pair & 0xFFFF0000u) : (pair << 16));
-                            const float* wk = wr + (2 * k2 + h) * 12;
-                            const float4 w0 = *reinterpret_cast<const float4*>(wk);
-                            const float4 w1 = *reinterpret_cast<const float4*>(wk + 4);
-                            const float4 w2 = *reinterpret_cast<const float4*>(wk + 8);
-                            acc[0] = fmaf(w0.x, xv, acc[0]); acc[1] = fmaf(w0.y, xv, acc[1]);
-                            acc[2] = fmaf(w0.z, xv, acc[2]); acc[3] = fmaf(w0.w, xv, acc[3]);
-                            acc[4] = fmaf(w1.x, xv, acc[4]); acc[5] = fmaf(w1.y, xv, acc[5]);
-                            acc[6] = fmaf(w1.z, xv, acc[6]); acc[7] = fmaf(w1.w, xv, acc[7]);
-                            acc[8] = fmaf(w2.x, xv, acc[8]); acc[9] = fmaf(w2.y, xv, acc[9]);
-                        }
-                    }
+                for (int hh = 0; hh < 2; ++hh) {
+                    const float fa = __uint_as_float(hh ? (xa & 0xFFFF0000u) : (xa << 16));
+                    const float fb = __uint_as_float(hh ? (xb & 0xFFFF0000u) : (xb << 16));
+                    const float2 va = make_float2(fa, fa), vb = make_float2(fb, fb);
+                    const float* wk = wr + (16 * i) * 24 + hh * 12;
+                    const float4 w0 = *reinterpret_cast<const float4*>(wk);
+                    const float4 w1 = *reinterpret_cast<const float4*>(wk + 4);
+                    const float2 w2 = *reinterpret_cast<const float2*>(wk + 8);
+                    ffma2(acc[0][0], make_float2(w0.x, w0.y), va); ffma2(acc[1][0], make_float2(w0.x, w0.y), vb);
+                    ffma2(acc[0][1], make_float2(w0.z, w0.w), va); ffma2(acc[1][1], make_float2(w0.z, w0.w), vb);
+                    ffma2(acc[0][2], make_float2(w1.x, w1.y), va); ffma2(acc[1][2], make_float2(w1.x, w1.y), vb);
+                    ffma2(acc[0][3], make_float2(w1.z, w1.w), va); ffma2(acc[1][3], make_float2(w1.z, w1.w), vb);
+                    ffma2(acc[0][4], w2, va);                      ffma2(acc[1][4], w2, vb);
                 }
-                float4* pw = reinterpret_cast<float4*>(part + (warp * 32 + lane) * 12);
-                pw[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-                pw[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
-                pw[2] = make_float4(acc[8], acc[9], 0.f, 0.f);
             }
-            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-            for (int o = tid; o < 32 * 12; o += kC2EpiThreads)          // quarters added in a fixed order
-                S.logit[o / 12][o % 12] = ((part[o] + part[384 + o]) + (part[768 + o] + part[1152 + o])) + S.bfc[o % 12];
-            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-            if (warp == 0) {
-                float l = 0.f;
-                if (lane < n_img) {
-                    const float* lg = S.logit[lane];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&S.p2_free[pb]));      // the activations have been read
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+#pragma unroll
+                for (int c = 0; c < 5; ++c) {
+                    float2 v = acc[e][c];
+                    v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
+                    v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
+                    acc[e][c] = v;
+                }
+            if (lane < 8) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    float* d = &S.part[pb][wl][ip + 8 * e][0];
+                    *reinterpret_cast<float4*>(d) = make_float4(acc[e][0].x, acc[e][0].y, acc[e][1].x, acc[e][1].y);
+                    *reinterpret_cast<float4*>(d + 4) = make_float4(acc[e][2].x, acc[e][2].y, acc[e][3].x, acc[e][3].y);
+                    *reinterpret_cast<float2*>(d + 8) = acc[e][4];
+                }
+            }
+            asm volatile("bar.sync 2, %0;" :: "n"(kC2LinThreads) : "memory");
+            if (wl == 0) {
+                const uint32_t image = group * 16u + lane;
+                if (lane < 16 && image < batch) {
+                    float lg[10];
+#pragma unroll
+                    for (int k = 0; k < 10; ++k)                            // warps added in a fixed order
+                        lg[k] = ((S.part[pb][0][lane][k] + S.part[pb][1][lane][k]) +
+                                 (S.part[pb][2][lane][k] + S.part[pb][3][lane][k])) + S.bfc[k];
                     float mx = lg[0];
 #pragma unroll
                     for (int k = 1; k < 10; ++k) mx = fmaxf(mx, lg[k]);
                     float se = 0.f;
 #pragma unroll
                     for (int k = 0; k < 10; ++k) se += expf(lg[k] - mx);
-                    const int lab = min(max(labels[2u * pair0 + lane], 0), 9);
-                    l = (mx + logf(se)) - lg[lab];
+                    const int lab = min(max(labels[image], 0), 9);
+                    float at_label = lg[0];
+#pragma unroll
+                    for (int k = 1; k < 10; ++k) at_label = (k == lab) ? lg[k] : at_label;
+                    const float l = (mx + logf(se)) - at_label;
+                    // after a time-out the numbers mean nothing: NaN, which makes tell skip the update
+                    loss[static_cast<size_t>(member) * batch + image] = S.abort ? __int_as_float(0x7FC00000) : l;
                 }
-                // after a time-out the numbers mean nothing: NaN, which makes tell skip the update
-                if (lane < n_img)
-                    loss[static_cast<size_t>(member) * batch + 2u * pair0 + lane] = S.abort ? __int_as_float(0x7FC00000) : l;
+                __syncwarp();
             }
-            fence_async_smem();        // the ring buffers held partial logits; bulk copies write them next
-            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
         }
-        // release the issuer
-        if (tid == 0) { S.item = kNoItem; __threadfence_block(); mbar_arrive(smem_u32(&S.item_ready)); }
+    } else if (warp < (kC2EpiThreads + kC2LinThreads) / 32 + kC2Issuers) {
+        // ================= MMA issuers: one thread per (accumulator, half row) ====================
+        if (lane == 0) {
+            const uint32_t wi = warp - (kC2EpiThreads + kC2LinThreads) / 32, ab = wi >> 1, h = wi & 1u;
+            const uint32_t a0 = smem_u32(S.a[ab]) + h * 4u * 128u, b0 = smem_u32(S.b);
+            const uint32_t first_member = u_begin / n_groups;
+            uint32_t seen_member = 0xFFFFFFFFu;
+            for (uint32_t j = ab; j < n_mine; j += 2u) {
+                const uint32_t member = (u_begin + j) / n_groups, par = (j >> 1) & 1u;
+                if (member != seen_member) {
+                    seen_member = member;
+                    c2_wait_staged(S, member - first_member + 1u, status);
+                }
+                c2_wait(S, &S.a_full[ab], par, status);
+                c2_wait(S, &S.acc_free[ab], par, status);
+                if (S.abort) break;
+                tc_fence_after();
+                c2_issue_mma(a0, b0, tmem + ab * 128u + h * 64u);
+                umma_commit(smem_u32(&S.mma_done[ab]));
+                umma_commit(smem_u32(&S.a_free[ab]));
+            }
+            umma_commit(smem_u32(&S.drain));                          // arrives when all my MMAs have completed
+        }
+    } else {
+        // ================= producer: one bulk copy per unit, two units ahead =======================
+        if (lane == 0) {
+            const unsigned char* src = pooled1 + static_cast<size_t>(u_begin) * kGroupBytes;
+            uint32_t issued = 0;
+            for (uint32_t j = 0; j < n_mine; ++j) {
+                const uint32_t ab = j & 1u;
+                if (j >= 2u) c2_wait(S, &S.a_free[ab], ((j >> 1) - 1u) & 1u, status);
+                if (S.abort) break;
+                bulk_copy_g2s(smem_u32(S.a[ab]), src + static_cast<size_t>(j) * kGroupBytes, kGroupBytes, smem_u32(&S.a_full[ab]));
+                issued = j + 1u;
+            }
+            // no copy may still be in flight when the block ends (only a time-out leaves any unconsumed)
+            for (uint32_t ab = 0; ab < 2u; ++ab)
+                if (issued > ab) {
+                    const uint32_t n_ab = (issued - ab + 1u) >> 1;
+                    mbar_wait_bounded(smem_u32(&S.a_full[ab]), (n_ab - 1u) & 1u, &status->wait_cycles_log2);
+                }
+        }
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 32);
+    if (warp == 0) {
+        // the accumulator warps have waited for every unit's MMAs; after a time-out some may still run
+        if (lane == 0) mbar_wait_bounded(smem_u32(&S.drain), 0u, &status->wait_cycles_log2);
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem, 256);
+    }
 }
 
 // fitness[m] = -mean over the batch of the per-image losses: one block per member, fixed order
@@ -615,10 +703,9 @@ k_cnn_tc_finalize(const float* __restrict__ loss, uint32_t batch, float* __restr
 // ------------------------------------------------------------------------------------------
 size_t cnn_tc_scratch_bytes(uint32_t P, uint32_t batch)
 {
-    const size_t n_pairs = (batch + 1u) / 2u;
-    size_t b = 256;                                                        // work counter
-    b += (static_cast<size_t>(P) * batch * sizeof(float) + 255) / 256 * 256;      // per-image losses
-    b += static_cast<size_t>(P) * n_pairs * kPairBytes;
+    const size_t n_groups = (batch + 15u) / 16u;
+    size_t b = (static_cast<size_t>(P) * batch * sizeof(float) + 255) / 256 * 256;      // per-image losses
+    b += static_cast<size_t>(P) * n_groups * kGroupBytes;                  // pooled-1 activations
     return b;
 }
 
@@ -633,22 +720,22 @@ int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uin
         if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
     }
     unsigned char* base = static_cast<unsigned char*>(scratch);
-    uint32_t* counter = reinterpret_cast<uint32_t*>(base);
-    float* loss = reinterpret_cast<float*>(base + 256);
-    unsigned char* pooled1 = base + 256 + (static_cast<size_t>(P) * batch * sizeof(float) + 255) / 256 * 256;
+    float* loss = reinterpret_cast<float*>(base);
+    unsigned char* pooled1 = base + (static_cast<size_t>(P) * batch * sizeof(float) + 255) / 256 * 256;
 
     if (cudaFuncSetAttribute(k_cnn_conv1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kC1DynRequest) != cudaSuccess) return -1;
-    const uint32_t n_tiles = (batch * 144u + 127u) / 128u;
+    const uint32_t n_groups = (batch + 15u) / 16u;
+    const uint32_t n_tiles = n_groups * 18u;
     dim3 g1(min(static_cast<uint32_t>(sm_count), n_tiles), (P + 63u) / 64u);
     k_cnn_conv1_tc<<<g1, kC1Threads, kC1DynRequest, st>>>(theta, ldD, P, images, batch,
-                                                          reinterpret_cast<uint4*>(pooled1), counter, status);
+                                                          reinterpret_cast<uint4*>(pooled1), status);
     if (cudaGetLastError() != cudaSuccess) return -1;
 
     const int c2_bytes = static_cast<int>(sizeof(C2Smem));
     if (cudaFuncSetAttribute(k_cnn_conv2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, c2_bytes) != cudaSuccess) return -1;
-    const uint64_t n_units = static_cast<uint64_t>(P) * ((batch + 1u) / 2u);
-    const uint32_t g2 = static_cast<uint32_t>(min(n_units, static_cast<uint64_t>(sm_count) * 4u));   // 4 blocks of ~55 KB per SM
-    k_cnn_conv2_tc<<<g2, kC2Threads, c2_bytes, st>>>(theta, ldD, P, pooled1, labels, batch, loss, counter, status);
+    const uint64_t n_units = static_cast<uint64_t>(P) * n_groups;
+    const uint32_t g2 = static_cast<uint32_t>(min(n_units, static_cast<uint64_t>(sm_count)));         // one block per SM
+    k_cnn_conv2_tc<<<g2, kC2Threads, c2_bytes, st>>>(theta, ldD, P, pooled1, labels, batch, loss, status);
     if (cudaGetLastError() != cudaSuccess) return -1;
     k_cnn_tc_finalize<<<P, 256, 0, st>>>(loss, batch, fitness);
     if (cudaGetLastError() != cudaSuccess) return -1;
