@@ -293,52 +293,53 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 // ------------------------------------------------------------------------------------------
 // conv2 + pool + linear + cross-entropy.  Unit of work = (member, group of 16 images).
 //
-// The contraction runs over a whole input row at a time.  For one filter row dy, the 4 output
-// columns x 16 filters of half a row (N = 64) are a product of the 8 input columns x 8 channels under
-// them (K = 64) with a banded matrix that holds the member's 5 taps of that filter row at the
-// offsets column - output column (zero elsewhere; 5/8 dense).  The band does not depend on which
-// half of the row is computed, so one 40 KB operand serves both.  GEMM rows are (output row, image):
-// with the group stored as [y][image octet][x][image in octet][8 channels], the 8 images of an
-// octet are one core matrix, a step in y is a fixed byte offset, and filter row dy is the same
-// operand started dy rows lower.  Per unit: 2 halves x 5 filter rows x 4 K-steps = 40 MMAs of
-// M = 128, N = 64, K = 16, where the tap-by-tap implicit GEMM needed 104 (13 per image pair, N = 16):
-// an MMA reads its 4 KB A operand from shared memory whatever N is, and that read, not the
-// arithmetic, is what paces it.
+// The contraction runs over a whole input row at a time, with the member's filters as the operand
+// that stays.  For filter row dy, the 8 output columns x 16 filters of an output row (M = 128) are a
+// product of a banded matrix, holding the 5 taps of that filter row at the offsets input column -
+// output column (zero elsewhere; 5/12 dense), with the 12 input columns x 8 channels (K = 96) of the
+// input row dy lower.  The five bands (240 columns) live in TENSOR MEMORY for as long as the member
+// lasts, so an MMA reads only its activation operand from shared memory: N = (output row, image), and
+// with the group stored as [y][image octet][x][image in octet][8 channels] the 8 images of an octet
+// are one core matrix, a step in y is a fixed byte offset, and filter row dy is the same operand
+// started dy rows lower.  Per unit: 5 filter rows x 6 K-steps on two halves of N = 60 MMAs of
+// M = 128, N = 64, K = 16 that each read 2 KB of shared memory, where a tap-by-tap implicit GEMM with the
+// pixels on M (13 MMAs of N = 16 per image pair, 104 per unit) read 4.5 KB each and was paced by that.
 //
 // Roles: warps 0-3 read the accumulators (2x2 max over two columns of a thread and two lanes,
-// bias, ReLU, bf16) into a per-image activation buffer; warps 4-7 run the linear layer and the
-// cross-entropy from that buffer; warps 8-11 each issue the MMAs of one (accumulator, half);
-// warp 12 brings the groups in, one bulk copy each, two units ahead.  The roles meet only on
-// mbarriers; every wait is bounded, and after a time-out all later waits fall through so that no
-// role is left behind.
+// bias, ReLU, bf16) into a per-image activation buffer; warps 4-11 run the linear layer and the
+// cross-entropy from that buffer; warps 12-15 each issue the MMAs of one (accumulator, half of N);
+// warp 16 brings the groups in, one bulk copy each, through a ring of three.  The roles meet only
+// on mbarriers; every wait is bounded, and after a time-out all later waits fall through so that
+// no role is left behind.
 // ------------------------------------------------------------------------------------------
 constexpr int kC2EpiThreads = 128;
-constexpr int kC2LinThreads = 128;
+constexpr int kC2LinThreads = 256;
 constexpr int kC2Issuers = 4;
 constexpr int kC2Threads = kC2EpiThreads + kC2LinThreads + 32 * kC2Issuers + 32;
 constexpr uint32_t kGroupRowBytes = 12 * 8 * 16;         // one (y, image octet): 12 pixels x 8 images x 16 bytes
 constexpr uint32_t kGroupBytes = 12 * 2 * kGroupRowBytes;   // 36,864
-constexpr uint32_t kC2SmemB = 5 * 8 * 8 * 128;           // (filter row, input column, 8-column group of N) core matrices
+constexpr uint32_t kC2Ring = 3;                          // groups in flight
+constexpr uint32_t kC2BandCols = 48;                     // tensor-memory columns of one band: K = 96 bf16
+constexpr uint32_t kC2AccCol = 256;                      // first accumulator column (the bands take 240)
 constexpr int kP2Pitch = 264;                            // bf16 per image: 132 words, images fall in distinct banks
 constexpr int kRawPitch = 201;                           // floats per filter in the weight scratch (odd: no bank conflicts)
 
 struct __align__(128) C2Smem {
-    unsigned char a[2][kGroupBytes];                     // pooled-1 groups (double buffer)
-    unsigned char b[kC2SmemB];                           // banded W2
+    unsigned char a[kC2Ring][kGroupBytes];               // pooled-1 groups (ring)
     float raw[16 * kRawPitch];                           // W2 as stored, one padded row per filter
     float wfT[256 * 12];                                 // linear layer transposed [k][class], bf16-rounded
     __align__(16) __nv_bfloat16 p2[2][16][kP2Pitch];     // pooled-2 activations of a unit's images, k = pixel*16 + channel
-    float part[2][4][16][12];                            // partial logits of the four linear warps
+    float part[2][8][16][12];                            // partial logits of the eight linear warps
     float b2[16];
     float bfc[12];
-    uint64_t a_full[2];                                  // a group has landed
-    uint64_t a_free[2];                                  // every MMA that read a group has completed
+    uint64_t a_full[kC2Ring];                            // a group has landed
+    uint64_t a_free[kC2Ring];                            // every MMA that read a group has completed
     uint64_t mma_done[2];                                // an accumulator is complete
     uint64_t acc_free[2];                                // an accumulator has been read out
     uint64_t p2_full[2];                                 // the activations of a unit are written
     uint64_t p2_free[2];                                 // ... and have been consumed by the linear layer
     uint64_t drain;                                      // all MMAs of the block have completed
-    uint32_t staged;                                     // members of the block's range whose band has been staged
+    uint32_t staged;                                     // members of the block's range whose bands have been staged
     uint32_t tmem_slot;
     volatile int abort;
 };
@@ -348,7 +349,7 @@ __device__ __forceinline__ void c2_wait(C2Smem& S, uint64_t* bar, uint32_t parit
     wait_or_abort(&S.abort, bar, parity, status);
 }
 
-// The band is staged once per member, in order, and the count of staged members only grows: an
+// The bands are staged once per member, in order, and the count of staged members only grows: an
 // issuer that has no unit of some member (a group count of one) would lose track of an mbarrier's
 // phase parity, a counter cannot be misread.  Bounded like every other wait.
 __device__ __forceinline__ void c2_wait_staged(C2Smem& S, uint32_t need, DeviceStatus* status)
@@ -370,19 +371,18 @@ __device__ __forceinline__ void c2_wait_staged(C2Smem& S, uint32_t need, DeviceS
     }
 }
 
-// The 20 MMAs of one half-row block of a unit.  a0 = the group, advanced to the half's first input
-// column; filter row dy starts the A operand dy rows lower and selects band dy; a K-step is two
-// input columns.
-__device__ __forceinline__ void c2_issue_mma(uint32_t a0, uint32_t b0, uint32_t d_tmem)
+// The 30 MMAs of one half (4 output rows x 16 images) of a unit.  b0 = the group, advanced to the
+// half's first row; filter row dy takes band dy and starts the activation operand dy rows lower;
+// a K-step is two input columns.
+__device__ __forceinline__ void c2_issue_mma(uint32_t bands, uint32_t b0, uint32_t d_tmem)
 {
     constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
 #pragma unroll
     for (uint32_t dy = 0; dy < 5u; ++dy)
 #pragma unroll
-        for (uint32_t ks = 0; ks < 4u; ++ks) {
-            const uint64_t ad = umma_smem_desc(a0 + dy * 2u * kGroupRowBytes + ks * 256u, 128u, kGroupRowBytes);
-            const uint64_t bd = umma_smem_desc(b0 + dy * 8192u + ks * 2048u, 1024u, 128u);
-            umma_bf16(d_tmem, ad, bd, idesc, dy | ks);
+        for (uint32_t ks = 0; ks < 6u; ++ks) {
+            const uint64_t bd = umma_smem_desc(b0 + dy * 2u * kGroupRowBytes + ks * 256u, 128u, kGroupRowBytes);
+            umma_bf16_ts(d_tmem, bands + dy * kC2BandCols + ks * 8u, bd, idesc, dy | ks);
         }
 }
 
@@ -403,47 +403,47 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     const uint32_t n_mine = u_end - u_begin;
 
     if (tid == 0) {
-        for (int i = 0; i < 2; ++i) {
+        for (uint32_t i = 0; i < kC2Ring; ++i) {
             mbar_init(smem_u32(&S.a_full[i]), 1);
             mbar_init(smem_u32(&S.a_free[i]), 2);
+        }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&S.mma_done[i]), 2);
             mbar_init(smem_u32(&S.acc_free[i]), kC2EpiThreads / 32);
             mbar_init(smem_u32(&S.p2_full[i]), kC2EpiThreads / 32);
             mbar_init(smem_u32(&S.p2_free[i]), kC2LinThreads / 32);
         }
-        S.staged = 0;
         mbar_init(smem_u32(&S.drain), kC2Issuers);
+        S.staged = 0;
         S.abort = 0;
         mbar_init_fence();
     }
-    // the zeros of the band stay where they are for every member
-    for (uint32_t i = tid; i < kC2SmemB / 16u; i += kC2Threads) reinterpret_cast<uint4*>(S.b)[i] = make_uint4(0u, 0u, 0u, 0u);
     for (int k = tid; k < 256; k += kC2Threads) { S.wfT[k * 12 + 10] = 0.f; S.wfT[k * 12 + 11] = 0.f; }
     if (tid < 2) S.bfc[10 + tid] = 0.f;
     __syncwarp();
-    if (warp == 0) tmem_alloc(smem_u32(&S.tmem_slot), 256);
-    fence_async_smem();
+    if (warp == 0) tmem_alloc(smem_u32(&S.tmem_slot), 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = S.tmem_slot;
 
     if (warp < kC2EpiThreads / 32) {
-        // ================= accumulator warps: pool, bias, ReLU -> activations ====================
+        // ================= accumulator warps: bands -> tensor memory; pool, bias, ReLU -> activations ===
         // both accumulators start out free
         if (lane == 0) { mbar_arrive(smem_u32(&S.acc_free[0])); mbar_arrive(smem_u32(&S.acc_free[1])); }
-        // TMEM lane = output row y (2 per warp) x image: the warp owns pooled row py = warp; a thread
-        // holds the 4 x 16 (column, filter) outputs of a half row.  Column pairs are a max over two
-        // registers; the row pair is lane ^ 16, done as an exchange: the thread of the even row keeps
-        // the left pooled pixel of the half, the thread of the odd row the right one.
-        const int img = lane & 15, odd = lane >> 4, py = warp;
+        // TMEM lane = output column x (2 per warp) x filter: the warp owns pooled column px = warp; a
+        // thread holds the 8 x 16 (output row, image) outputs of its (column, filter).  Row pairs are
+        // a max over two registers; the column pair is lane ^ 16, done as an exchange: of a pair of
+        // pooled rows (a, a + 2) the thread of the even column keeps row a, that of the odd column a + 2.
+        const int f = lane & 15, odd = lane >> 4, xo = 2 * warp + odd, px = warp;
+        const uint32_t tm_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
         const uint32_t first_member = u_begin / n_groups;
-        float bias[16];
+        float bias = 0.f;
         uint32_t staged_member = 0xFFFFFFFFu;
         for (uint32_t j = 0; j < n_mine; ++j) {
             const uint32_t member = (u_begin + j) / n_groups, ab = j & 1u, par = (j >> 1) & 1u;
             if (member != staged_member) {
-                // Every MMA of the previous member has been waited for, so the band can be rewritten.
+                // Every MMA of the previous member has been waited for, so the bands can be rewritten.
                 staged_member = member;
                 const float* prm = theta + static_cast<size_t>(member) * ldD;
                 const float4* w2v = reinterpret_cast<const float4*>(prm + 208u);      // 16-byte aligned
@@ -461,20 +461,25 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 }
                 if (tid < 16) S.b2[tid] = prm[3408u + tid];
                 asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-                // band dy, K row (input column xi, channel), N column (output column xo, filter f) = W2[f][channel][dy][xi - xo]
-                for (uint32_t idx = tid; idx < 1600u; idx += kC2EpiThreads) {
-                    const uint32_t f = idx & 15u, q = idx >> 4, dx = q % 5u, xo = (q / 5u) & 3u, dy = q / 20u;
-                    const float* src = S.raw + f * kRawPitch + dy * 5u + dx;
-                    uint32_t w[4];
+                // band dy, row (output column xo, filter f), K = (input column xi, channel): W2[f][channel][dy][xi - xo];
+                // a tensor-memory column holds two consecutive K, 8 columns = two input columns = one K-step
+                const float* mine = S.raw + f * kRawPitch;
+#pragma unroll 1
+                for (uint32_t dy = 0; dy < 5u; ++dy)
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) w[k] = pack_bf16(src[(2 * k) * 25], src[(2 * k + 1) * 25]);
-                    const uint32_t n = xo * 16u + f;
-                    *reinterpret_cast<uint4*>(S.b + ((dy * 8u + xo + dx) * 8u + (n >> 3)) * 128u + (n & 7u) * 16u) =
-                        make_uint4(w[0], w[1], w[2], w[3]);
-                }
+                    for (int ks = 0; ks < 6; ++ks) {
+                        uint32_t u[8];
 #pragma unroll
-                for (int f = 0; f < 16; ++f) bias[f] = S.b2[f];
-                fence_async_smem();
+                        for (int e = 0; e < 8; ++e) {
+                            const int dx = 2 * ks + (e >> 2) - xo, ch = 2 * (e & 3);
+                            u[e] = 0u;
+                            if (dx >= 0 && dx <= 4) u[e] = pack_bf16(mine[ch * 25 + dy * 5 + dx], mine[(ch + 1) * 25 + dy * 5 + dx]);
+                        }
+                        tmem_st8(tm_lane + dy * kC2BandCols + ks * 8u, u);
+                    }
+                tmem_st_wait();
+                tc_fence_before();
+                bias = S.b2[f];
                 asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
                 if (tid == 0)
                     asm volatile("st.release.cta.shared::cta.u32 [%0], %1;"
@@ -483,45 +488,38 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             c2_wait(S, &S.mma_done[ab], par, status);
             tc_fence_after();
             c2_wait(S, &S.p2_free[ab], par, status);
-            const uint32_t t0 = tmem + (static_cast<uint32_t>(warp * 32) << 16) + ab * 128u;
+            const uint32_t t0 = tm_lane + kC2AccCol + ab * 128u;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t r[4][16];                                     // [output column in the half][filter]
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld16_issue(t0 + h * 64u + c * 16u, r[c]);
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld16_fence(r[c]);
-                if (h == 1) {                                          // the accumulator is in registers now
+            for (int a = 0; a < 2; ++a) {
+                // accumulator column = output row * 16 + image: pooled rows a and a + 2 are output rows 2a, 2a+1 and 2a+4, 2a+5
+                uint32_t lo[2][16], hi[2][16];
+                tmem_ld16_issue(t0 + (2 * a) * 16u, lo[0]);     tmem_ld16_issue(t0 + (2 * a + 1) * 16u, lo[1]);
+                tmem_ld16_issue(t0 + (2 * a + 4) * 16u, hi[0]); tmem_ld16_issue(t0 + (2 * a + 5) * 16u, hi[1]);
+                tmem_ld16_fence(lo[0]); tmem_ld16_fence(lo[1]); tmem_ld16_fence(hi[0]); tmem_ld16_fence(hi[1]);
+                if (a == 1) {                                          // the accumulator is in registers now
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&S.acc_free[ab]));
                 }
-                uint32_t o[8];
+                const int py = a + 2 * odd;
+                __nv_bfloat16* dst = &S.p2[ab][0][(py * 4 + px) * 16 + f];
 #pragma unroll
-                for (int f = 0; f < 16; f += 2) {
-                    float v[2];
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const float left = fmaxf(__uint_as_float(r[0][f + e]), __uint_as_float(r[1][f + e]));
-                        const float right = fmaxf(__uint_as_float(r[2][f + e]), __uint_as_float(r[3][f + e]));
-                        const float keep = odd ? right : left;
-                        const float give = odd ? left : right;
-                        v[e] = fmaxf(fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 16)) + bias[f + e], 0.f);
-                    }
-                    o[f >> 1] = pack_bf16(v[0], v[1]);
+                for (int img = 0; img < 16; ++img) {
+                    const float va = fmaxf(__uint_as_float(lo[0][img]), __uint_as_float(lo[1][img]));
+                    const float vb = fmaxf(__uint_as_float(hi[0][img]), __uint_as_float(hi[1][img]));
+                    const float keep = odd ? vb : va;
+                    const float give = odd ? va : vb;
+                    const float v = fmaxf(fmaxf(keep, __shfl_xor_sync(0xffffffffu, give, 16)) + bias, 0.f);
+                    dst[img * kP2Pitch] = __float2bfloat16_rn(v);
                 }
-                const int px = 2 * h + odd;
-                uint4* dst = reinterpret_cast<uint4*>(&S.p2[ab][img][(py * 4 + px) * 16]);
-                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&S.p2_full[ab]));
         }
     } else if (warp < (kC2EpiThreads + kC2LinThreads) / 32) {
         // ================= linear layer 256 -> 10 and cross-entropy ==============================
-        // thread = (images ip and ip + 8, slice s of the inputs: the pairs k = 2(s + 16 i), +1); the 16
-        // slices meet by two shuffles inside a warp and through shared memory across the four warps.
+        // thread = (images ip and ip + 8, slice s of the inputs: the pairs k = 2(s + 32 i), +1); the 32
+        // slices meet by two shuffles inside a warp and through shared memory across the eight warps.
         if (lane == 0) { mbar_arrive(smem_u32(&S.p2_free[0])); mbar_arrive(smem_u32(&S.p2_free[1])); }
         const int lt = tid - kC2EpiThreads, wl = lt >> 5;
         const int ip = lane & 7, s = wl * 4 + (lane >> 3);
@@ -534,19 +532,22 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 staged_member = member;
                 const float* prm = theta + static_cast<size_t>(member) * ldD;
                 const float4* wfv = reinterpret_cast<const float4*>(prm + 3424u);     // 16-byte aligned
-                float4 tf[5];
+                float4 tf[3];
 #pragma unroll
-                for (int k = 0; k < 5; ++k) tf[k] = __ldg(wfv + lt + k * kC2LinThreads);
+                for (int k = 0; k < 3; ++k)
+                    tf[k] = (lt + k * kC2LinThreads < 640) ? __ldg(wfv + lt + k * kC2LinThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int k = 0; k < 5; ++k) {
+                for (int k = 0; k < 3; ++k) {
                     // flat index cls*256 + (c*16 + pos), 4 consecutive pos; stored at row pos*16 + c
                     const uint32_t i = 4u * (lt + k * kC2LinThreads);
-                    const uint32_t cls = i >> 8, c = (i >> 4) & 15u, pos = i & 15u;
-                    float* d = S.wfT + (pos * 16u + c) * 12u + cls;
-                    d[0 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].x));
-                    d[1 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].y));
-                    d[2 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].z));
-                    d[3 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].w));
+                    if (i < 2560u) {
+                        const uint32_t cls = i >> 8, c = (i >> 4) & 15u, pos = i & 15u;
+                        float* d = S.wfT + (pos * 16u + c) * 12u + cls;
+                        d[0 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].x));
+                        d[1 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].y));
+                        d[2 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].z));
+                        d[3 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].w));
+                    }
                 }
                 if (lt < 10) S.bfc[lt] = prm[5984u + lt];
                 asm volatile("bar.sync 2, %0;" :: "n"(kC2LinThreads) : "memory");
@@ -560,15 +561,15 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             const uint32_t* x0 = reinterpret_cast<const uint32_t*>(&S.p2[pb][ip][0]) + s;        // two inputs per word
             const uint32_t* x1 = reinterpret_cast<const uint32_t*>(&S.p2[pb][ip + 8][0]) + s;
             const float* wr = S.wfT + s * 24;
-#pragma unroll 2
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t xa = x0[16 * i], xb = x1[16 * i];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t xa = x0[32 * i], xb = x1[32 * i];
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     const float fa = __uint_as_float(hh ? (xa & 0xFFFF0000u) : (xa << 16));
                     const float fb = __uint_as_float(hh ? (xb & 0xFFFF0000u) : (xb << 16));
                     const float2 va = make_float2(fa, fa), vb = make_float2(fb, fb);
-                    const float* wk = wr + (16 * i) * 24 + hh * 12;
+                    const float* wk = wr + (32 * i) * 24 + hh * 12;
                     const float4 w0 = *reinterpret_cast<const float4*>(wk);
                     const float4 w1 = *reinterpret_cast<const float4*>(wk + 4);
                     const float2 w2 = *reinterpret_cast<const float2*>(wk + 8);
@@ -591,6 +592,12 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     acc[e][c] = v;
                 }
             if (lane < 8) {
+                if (wl == 0) {                          // the bias joins the first warp's part: nothing reads it after the barrier
+#pragma unroll
+                    for (int e = 0; e < 2; ++e)
+#pragma unroll
+                        for (int c = 0; c < 5; ++c) { acc[e][c].x += S.bfc[2 * c]; acc[e][c].y += S.bfc[2 * c + 1]; }
+                }
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     float* d = &S.part[pb][wl][ip + 8 * e][0];
@@ -600,71 +607,67 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 }
             }
             asm volatile("bar.sync 2, %0;" :: "n"(kC2LinThreads) : "memory");
-            if (wl == 0) {
-                const uint32_t image = group * 16u + lane;
-                if (lane < 16 && image < batch) {
-                    float lg[10];
-#pragma unroll
-                    for (int k = 0; k < 10; ++k)                            // warps added in a fixed order
-                        lg[k] = ((S.part[pb][0][lane][k] + S.part[pb][1][lane][k]) +
-                                 (S.part[pb][2][lane][k] + S.part[pb][3][lane][k])) + S.bfc[k];
-                    float mx = lg[0];
-#pragma unroll
-                    for (int k = 1; k < 10; ++k) mx = fmaxf(mx, lg[k]);
-                    float se = 0.f;
-#pragma unroll
-                    for (int k = 0; k < 10; ++k) se += expf(lg[k] - mx);
-                    const int lab = min(max(labels[image], 0), 9);
-                    float at_label = lg[0];
-#pragma unroll
-                    for (int k = 1; k < 10; ++k) at_label = (k == lab) ? lg[k] : at_label;
-                    const float l = (mx + logf(se)) - at_label;
-                    // after a time-out the numbers mean nothing: NaN, which makes tell skip the update
-                    loss[static_cast<size_t>(member) * batch + image] = S.abort ? __int_as_float(0x7FC00000) : l;
+            // cross-entropy: warp = two images, 16 lanes each, lane = class (10 of the 16 in use)
+            {
+                const int cls = lane & 15, il = 2 * wl + (lane >> 4);
+                const uint32_t image = group * 16u + il;
+                float lg = -INFINITY;
+                if (cls < 10) {
+                    const float* q = &S.part[pb][0][il][cls];                // warps added in a fixed order
+                    lg = ((q[0] + q[192]) + (q[384] + q[576])) + ((q[768] + q[960]) + (q[1152] + q[1344]));
                 }
-                __syncwarp();
+                float mx = lg;
+#pragma unroll
+                for (int d = 8; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+                float se = cls < 10 ? expf(lg - mx) : 0.f;
+#pragma unroll
+                for (int d = 8; d > 0; d >>= 1) se += __shfl_xor_sync(0xffffffffu, se, d);
+                const int lab = image < batch ? min(max(labels[image], 0), 9) : 0;
+                const float at_label = __shfl_sync(0xffffffffu, lg, (lane & 16) + lab);
+                // after a time-out the numbers mean nothing: NaN, which makes tell skip the update
+                if (cls == 0 && image < batch)
+                    loss[static_cast<size_t>(member) * batch + image] = S.abort ? __int_as_float(0x7FC00000) : (mx + logf(se)) - at_label;
             }
         }
     } else if (warp < (kC2EpiThreads + kC2LinThreads) / 32 + kC2Issuers) {
-        // ================= MMA issuers: one thread per (accumulator, half row) ====================
+        // ================= MMA issuers: one thread per (accumulator, half of the output rows) =====
         if (lane == 0) {
             const uint32_t wi = warp - (kC2EpiThreads + kC2LinThreads) / 32, ab = wi >> 1, h = wi & 1u;
-            const uint32_t a0 = smem_u32(S.a[ab]) + h * 4u * 128u, b0 = smem_u32(S.b);
             const uint32_t first_member = u_begin / n_groups;
             uint32_t seen_member = 0xFFFFFFFFu;
             for (uint32_t j = ab; j < n_mine; j += 2u) {
-                const uint32_t member = (u_begin + j) / n_groups, par = (j >> 1) & 1u;
+                const uint32_t member = (u_begin + j) / n_groups, slot = j % kC2Ring;
                 if (member != seen_member) {
                     seen_member = member;
                     c2_wait_staged(S, member - first_member + 1u, status);
                 }
-                c2_wait(S, &S.a_full[ab], par, status);
-                c2_wait(S, &S.acc_free[ab], par, status);
+                c2_wait(S, &S.a_full[slot], (j / kC2Ring) & 1u, status);
+                c2_wait(S, &S.acc_free[ab], (j >> 1) & 1u, status);
                 if (S.abort) break;
                 tc_fence_after();
-                c2_issue_mma(a0, b0, tmem + ab * 128u + h * 64u);
+                c2_issue_mma(tmem, smem_u32(S.a[slot]) + h * 8u * kGroupRowBytes, tmem + kC2AccCol + ab * 128u + h * 64u);
                 umma_commit(smem_u32(&S.mma_done[ab]));
-                umma_commit(smem_u32(&S.a_free[ab]));
+                umma_commit(smem_u32(&S.a_free[slot]));
             }
             umma_commit(smem_u32(&S.drain));                          // arrives when all my MMAs have completed
         }
     } else {
-        // ================= producer: one bulk copy per unit, two units ahead =======================
+        // ================= producer: one bulk copy per unit, up to three units ahead ===============
         if (lane == 0) {
             const unsigned char* src = pooled1 + static_cast<size_t>(u_begin) * kGroupBytes;
             uint32_t issued = 0;
             for (uint32_t j = 0; j < n_mine; ++j) {
-                const uint32_t ab = j & 1u;
-                if (j >= 2u) c2_wait(S, &S.a_free[ab], ((j >> 1) - 1u) & 1u, status);
+                const uint32_t slot = j % kC2Ring;
+                if (j >= kC2Ring) c2_wait(S, &S.a_free[slot], (j / kC2Ring - 1u) & 1u, status);
                 if (S.abort) break;
-                bulk_copy_g2s(smem_u32(S.a[ab]), src + static_cast<size_t>(j) * kGroupBytes, kGroupBytes, smem_u32(&S.a_full[ab]));
+                bulk_copy_g2s(smem_u32(S.a[slot]), src + static_cast<size_t>(j) * kGroupBytes, kGroupBytes, smem_u32(&S.a_full[slot]));
                 issued = j + 1u;
             }
             // no copy may still be in flight when the block ends (only a time-out leaves any unconsumed)
-            for (uint32_t ab = 0; ab < 2u; ++ab)
-                if (issued > ab) {
-                    const uint32_t n_ab = (issued - ab + 1u) >> 1;
-                    mbar_wait_bounded(smem_u32(&S.a_full[ab]), (n_ab - 1u) & 1u, &status->wait_cycles_log2);
+            for (uint32_t slot = 0; slot < kC2Ring; ++slot)
+                if (issued > slot) {
+                    const uint32_t n_slot = (issued - slot + kC2Ring - 1u) / kC2Ring;     // copies into this slot
+                    mbar_wait_bounded(smem_u32(&S.a_full[slot]), (n_slot - 1u) & 1u, &status->wait_cycles_log2);
                 }
         }
     }
@@ -676,7 +679,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         if (lane == 0) mbar_wait_bounded(smem_u32(&S.drain), 0u, &status->wait_cycles_log2);
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem, 256);
+        tmem_dealloc(tmem, 512);
     }
 }
 
