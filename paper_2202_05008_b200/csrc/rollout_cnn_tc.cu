@@ -314,7 +314,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 // ------------------------------------------------------------------------------------------
 constexpr int kC2EpiThreads = 128;
 constexpr int kC2LinThreads = 256;
-constexpr int kC2Issuers = 4;
+constexpr int kC2Issuers = 2;
 constexpr int kC2Threads = kC2EpiThreads + kC2LinThreads + 32 * kC2Issuers + 32;
 constexpr uint32_t kGroupRowBytes = 12 * 8 * 16;         // one (y, image octet): 12 pixels x 8 images x 16 bytes
 constexpr uint32_t kGroupBytes = 12 * 2 * kGroupRowBytes;   // 36,864
@@ -327,11 +327,11 @@ constexpr int kRawPitch = 201;                           // floats per filter in
 struct __align__(128) C2Smem {
     unsigned char a[kC2Ring][kGroupBytes];               // pooled-1 groups (ring)
     float raw[16 * kRawPitch];                           // W2 as stored, one padded row per filter
-    float wfT[256 * 12];                                 // linear layer transposed [k][class], bf16-rounded
+    float wfT[2][256 * 12];                              // linear layer transposed [k][class], bf16-rounded, one copy per linear team
     __align__(16) __nv_bfloat16 p2[2][16][kP2Pitch];     // pooled-2 activations of a unit's images, k = pixel*16 + channel
-    float part[2][8][16][12];                            // partial logits of the eight linear warps
+    float part[2][2][4][16][12];                         // [team][unit parity in the team] partial logits of the four warps
     float b2[16];
-    float bfc[12];
+    float bfc[2][12];
     uint64_t a_full[kC2Ring];                            // a group has landed
     uint64_t a_free[kC2Ring];                            // every MMA that read a group has completed
     uint64_t mma_done[2];                                // an accumulator is complete
@@ -376,7 +376,7 @@ __device__ __forceinline__ void c2_wait_staged(C2Smem& S, uint32_t need, DeviceS
 // a K-step is two input columns.
 __device__ __forceinline__ void c2_issue_mma(uint32_t bands, uint32_t b0, uint32_t d_tmem)
 {
-    constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
+    constexpr uint32_t idesc = umma_idesc_bf16(128, 128);
 #pragma unroll
     for (uint32_t dy = 0; dy < 5u; ++dy)
 #pragma unroll
@@ -405,21 +405,21 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     if (tid == 0) {
         for (uint32_t i = 0; i < kC2Ring; ++i) {
             mbar_init(smem_u32(&S.a_full[i]), 1);
-            mbar_init(smem_u32(&S.a_free[i]), 2);
+            mbar_init(smem_u32(&S.a_free[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&S.mma_done[i]), 2);
+            mbar_init(smem_u32(&S.mma_done[i]), 1);
             mbar_init(smem_u32(&S.acc_free[i]), kC2EpiThreads / 32);
             mbar_init(smem_u32(&S.p2_full[i]), kC2EpiThreads / 32);
-            mbar_init(smem_u32(&S.p2_free[i]), kC2LinThreads / 32);
+            mbar_init(smem_u32(&S.p2_free[i]), kC2LinThreads / 64);
         }
         mbar_init(smem_u32(&S.drain), kC2Issuers);
         S.staged = 0;
         S.abort = 0;
         mbar_init_fence();
     }
-    for (int k = tid; k < 256; k += kC2Threads) { S.wfT[k * 12 + 10] = 0.f; S.wfT[k * 12 + 11] = 0.f; }
-    if (tid < 2) S.bfc[10 + tid] = 0.f;
+    for (int k = tid; k < 512; k += kC2Threads) { S.wfT[k >> 8][(k & 255) * 12 + 10] = 0.f; S.wfT[k >> 8][(k & 255) * 12 + 11] = 0.f; }
+    if (tid < 4) S.bfc[tid >> 1][10 + (tid & 1)] = 0.f;
     __syncwarp();
     if (warp == 0) tmem_alloc(smem_u32(&S.tmem_slot), 512);
     tc_fence_before();
@@ -440,6 +440,12 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         const uint32_t first_member = u_begin / n_groups;
         float bias = 0.f;
         uint32_t staged_member = 0xFFFFFFFFu;
+        {   // the zeros of the bands, once
+            const uint32_t z[8] = { 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u };
+#pragma unroll
+            for (uint32_t c = 0; c < 5u * kC2BandCols; c += 8u) tmem_st8(tm_lane + c, z);
+            tmem_st_wait();
+        }
         for (uint32_t j = 0; j < n_mine; ++j) {
             const uint32_t member = (u_begin + j) / n_groups, ab = j & 1u, par = (j >> 1) & 1u;
             if (member != staged_member) {
@@ -461,21 +467,23 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 }
                 if (tid < 16) S.b2[tid] = prm[3408u + tid];
                 asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-                // band dy, row (output column xo, filter f), K = (input column xi, channel): W2[f][channel][dy][xi - xo];
-                // a tensor-memory column holds two consecutive K, 8 columns = two input columns = one K-step
+                // band dy, row (output column xo, filter f), K = (input column xi, channel): W2[f][channel][dy][xi - xo].
+                // A tensor-memory column holds two consecutive K, 8 columns = two input columns = one K-step.
+                // Only the input columns xo .. xo + 4 of a row are not zero, the same for every member: they
+                // lie in the three K-steps from xo / 2 on.
                 const float* mine = S.raw + f * kRawPitch;
-#pragma unroll 1
+#pragma unroll
                 for (uint32_t dy = 0; dy < 5u; ++dy)
 #pragma unroll
-                    for (int ks = 0; ks < 6; ++ks) {
+                    for (int t = 0; t < 3; ++t) {
                         uint32_t u[8];
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
-                            const int dx = 2 * ks + (e >> 2) - xo, ch = 2 * (e & 3);
+                            const int dx = 2 * t + (e >> 2) - odd, ch = 2 * (e & 3);       // xo is 2 * warp + odd
                             u[e] = 0u;
                             if (dx >= 0 && dx <= 4) u[e] = pack_bf16(mine[ch * 25 + dy * 5 + dx], mine[(ch + 1) * 25 + dy * 5 + dx]);
                         }
-                        tmem_st8(tm_lane + dy * kC2BandCols + ks * 8u, u);
+                        tmem_st8(tm_lane + dy * kC2BandCols + static_cast<uint32_t>(warp + t) * 8u, u);
                     }
                 tmem_st_wait();
                 tc_fence_before();
@@ -518,58 +526,63 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         }
     } else if (warp < (kC2EpiThreads + kC2LinThreads) / 32) {
         // ================= linear layer 256 -> 10 and cross-entropy ==============================
-        // thread = (images ip and ip + 8, slice s of the inputs: the pairs k = 2(s + 32 i), +1); the 32
-        // slices meet by two shuffles inside a warp and through shared memory across the eight warps.
-        if (lane == 0) { mbar_arrive(smem_u32(&S.p2_free[0])); mbar_arrive(smem_u32(&S.p2_free[1])); }
-        const int lt = tid - kC2EpiThreads, wl = lt >> 5;
+        // Two teams of four warps take the units in turn (team = unit parity = activation buffer), so a
+        // team has two unit times for the chain products -> sums -> barrier -> softmax of its unit.
+        // thread = (images ip and ip + 8, slice s of the inputs: the pairs k = 2(s + 16 i), +1); the 16
+        // slices meet by two shuffles inside a warp and through shared memory across the four warps.
+        const int lt = (tid - kC2EpiThreads) & 127, wl = lt >> 5;
+        const uint32_t team = static_cast<uint32_t>(tid - kC2EpiThreads) >> 7;
+        if (lane == 0) mbar_arrive(smem_u32(&S.p2_free[team]));
         const int ip = lane & 7, s = wl * 4 + (lane >> 3);
         uint32_t staged_member = 0xFFFFFFFFu;
-        for (uint32_t j = 0; j < n_mine; ++j) {
+        for (uint32_t j = team; j < n_mine; j += 2u) {
             const uint32_t unit = u_begin + j, member = unit / n_groups, group = unit % n_groups;
-            const uint32_t pb = j & 1u, par = (j >> 1) & 1u;
+            const uint32_t par = (j >> 1) & 1u;
+            // softmax: warp = four images, 8 lanes each, lane = classes c and c + 8; the label comes early
+            const int cls = lane & 7, il = 4 * wl + (lane >> 3);
+            const uint32_t image = group * 16u + il;
+            const int lab = image < batch ? min(max(__ldg(labels + image), 0), 9) : 0;
             if (member != staged_member) {
-                // every linear warp is past the previous unit's products (the barrier below)
+                // The teams keep their own copy of the layer (theirs to rewrite once they are past the
+                // previous unit's products: the barrier below).
                 staged_member = member;
                 const float* prm = theta + static_cast<size_t>(member) * ldD;
                 const float4* wfv = reinterpret_cast<const float4*>(prm + 3424u);     // 16-byte aligned
-                float4 tf[3];
+                float4 tf[5];
 #pragma unroll
-                for (int k = 0; k < 3; ++k)
-                    tf[k] = (lt + k * kC2LinThreads < 640) ? __ldg(wfv + lt + k * kC2LinThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k = 0; k < 5; ++k) tf[k] = __ldg(wfv + lt + k * 128);
 #pragma unroll
-                for (int k = 0; k < 3; ++k) {
+                for (int k = 0; k < 5; ++k) {
                     // flat index cls*256 + (c*16 + pos), 4 consecutive pos; stored at row pos*16 + c
-                    const uint32_t i = 4u * (lt + k * kC2LinThreads);
-                    if (i < 2560u) {
-                        const uint32_t cls = i >> 8, c = (i >> 4) & 15u, pos = i & 15u;
-                        float* d = S.wfT + (pos * 16u + c) * 12u + cls;
-                        d[0 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].x));
-                        d[1 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].y));
-                        d[2 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].z));
-                        d[3 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].w));
-                    }
+                    const uint32_t i = 4u * (lt + k * 128);
+                    const uint32_t oc = i >> 8, c = (i >> 4) & 15u, pos = i & 15u;
+                    float* d = S.wfT[team] + (pos * 16u + c) * 12u + oc;
+                    d[0 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].x));
+                    d[1 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].y));
+                    d[2 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].z));
+                    d[3 * 192]  = __bfloat162float(__float2bfloat16_rn(tf[k].w));
                 }
-                if (lt < 10) S.bfc[lt] = prm[5984u + lt];
-                asm volatile("bar.sync 2, %0;" :: "n"(kC2LinThreads) : "memory");
+                if (lt < 10) S.bfc[team][lt] = prm[5984u + lt];
+                asm volatile("bar.sync %0, 128;" :: "r"(2u + team) : "memory");
             }
-            c2_wait(S, &S.p2_full[pb], par, status);
+            c2_wait(S, &S.p2_full[team], par, status);
             float2 acc[2][5];
 #pragma unroll
             for (int e = 0; e < 2; ++e)
 #pragma unroll
                 for (int c = 0; c < 5; ++c) acc[e][c] = make_float2(0.f, 0.f);
-            const uint32_t* x0 = reinterpret_cast<const uint32_t*>(&S.p2[pb][ip][0]) + s;        // two inputs per word
-            const uint32_t* x1 = reinterpret_cast<const uint32_t*>(&S.p2[pb][ip + 8][0]) + s;
-            const float* wr = S.wfT + s * 24;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t xa = x0[32 * i], xb = x1[32 * i];
+            const uint32_t* x0 = reinterpret_cast<const uint32_t*>(&S.p2[team][ip][0]) + s;        // two inputs per word
+            const uint32_t* x1 = reinterpret_cast<const uint32_t*>(&S.p2[team][ip + 8][0]) + s;
+            const float* wr = S.wfT[team] + s * 24;
+#pragma unroll 4
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t xa = x0[16 * i], xb = x1[16 * i];
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     const float fa = __uint_as_float(hh ? (xa & 0xFFFF0000u) : (xa << 16));
                     const float fb = __uint_as_float(hh ? (xb & 0xFFFF0000u) : (xb << 16));
                     const float2 va = make_float2(fa, fa), vb = make_float2(fb, fb);
-                    const float* wk = wr + (32 * i) * 24 + hh * 12;
+                    const float* wk = wr + (16 * i) * 24 + hh * 12;
                     const float4 w0 = *reinterpret_cast<const float4*>(wk);
                     const float4 w1 = *reinterpret_cast<const float4*>(wk + 4);
                     const float2 w2 = *reinterpret_cast<const float2*>(wk + 8);
@@ -581,7 +594,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&S.p2_free[pb]));      // the activations have been read
+            if (lane == 0) mbar_arrive(smem_u32(&S.p2_free[team]));    // the activations have been read
 #pragma unroll
             for (int e = 0; e < 2; ++e)
 #pragma unroll
@@ -596,34 +609,30 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 #pragma unroll
                     for (int e = 0; e < 2; ++e)
 #pragma unroll
-                        for (int c = 0; c < 5; ++c) { acc[e][c].x += S.bfc[2 * c]; acc[e][c].y += S.bfc[2 * c + 1]; }
+                        for (int c = 0; c < 5; ++c) { acc[e][c].x += S.bfc[team][2 * c]; acc[e][c].y += S.bfc[team][2 * c + 1]; }
                 }
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    float* d = &S.part[pb][wl][ip + 8 * e][0];
+                    float* d = &S.part[team][par][wl][ip + 8 * e][0];
                     *reinterpret_cast<float4*>(d) = make_float4(acc[e][0].x, acc[e][0].y, acc[e][1].x, acc[e][1].y);
                     *reinterpret_cast<float4*>(d + 4) = make_float4(acc[e][2].x, acc[e][2].y, acc[e][3].x, acc[e][3].y);
                     *reinterpret_cast<float2*>(d + 8) = acc[e][4];
                 }
             }
-            asm volatile("bar.sync 2, %0;" :: "n"(kC2LinThreads) : "memory");
-            // cross-entropy: warp = two images, 16 lanes each, lane = class (10 of the 16 in use)
+            asm volatile("bar.sync %0, 128;" :: "r"(2u + team) : "memory");
             {
-                const int cls = lane & 15, il = 2 * wl + (lane >> 4);
-                const uint32_t image = group * 16u + il;
-                float lg = -INFINITY;
-                if (cls < 10) {
-                    const float* q = &S.part[pb][0][il][cls];                // warps added in a fixed order
-                    lg = ((q[0] + q[192]) + (q[384] + q[576])) + ((q[768] + q[960]) + (q[1152] + q[1344]));
-                }
-                float mx = lg;
+                const float* q = &S.part[team][par][0][il][cls];             // warps added in a fixed order
+                const float lg0 = (q[0] + q[192]) + (q[384] + q[576]);
+                const float lg1 = cls < 2 ? (q[8] + q[200]) + (q[392] + q[584]) : -INFINITY;
+                float mx = fmaxf(lg0, lg1);
 #pragma unroll
-                for (int d = 8; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
-                float se = cls < 10 ? expf(lg - mx) : 0.f;
+                for (int d = 4; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+                float se = expf(lg0 - mx) + (cls < 2 ? expf(lg1 - mx) : 0.f);
 #pragma unroll
-                for (int d = 8; d > 0; d >>= 1) se += __shfl_xor_sync(0xffffffffu, se, d);
-                const int lab = image < batch ? min(max(labels[image], 0), 9) : 0;
-                const float at_label = __shfl_sync(0xffffffffu, lg, (lane & 16) + lab);
+                for (int d = 4; d > 0; d >>= 1) se += __shfl_xor_sync(0xffffffffu, se, d);
+                const float a0 = __shfl_sync(0xffffffffu, lg0, (lane & 24) + (lab & 7));
+                const float a1 = __shfl_sync(0xffffffffu, lg1, (lane & 24) + (lab & 7));
+                const float at_label = lab < 8 ? a0 : a1;
                 // after a time-out the numbers mean nothing: NaN, which makes tell skip the update
                 if (cls == 0 && image < batch)
                     loss[static_cast<size_t>(member) * batch + image] = S.abort ? __int_as_float(0x7FC00000) : (mx + logf(se)) - at_label;
@@ -632,7 +641,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     } else if (warp < (kC2EpiThreads + kC2LinThreads) / 32 + kC2Issuers) {
         // ================= MMA issuers: one thread per (accumulator, half of the output rows) =====
         if (lane == 0) {
-            const uint32_t wi = warp - (kC2EpiThreads + kC2LinThreads) / 32, ab = wi >> 1, h = wi & 1u;
+            const uint32_t ab = warp - (kC2EpiThreads + kC2LinThreads) / 32;
             const uint32_t first_member = u_begin / n_groups;
             uint32_t seen_member = 0xFFFFFFFFu;
             for (uint32_t j = ab; j < n_mine; j += 2u) {
@@ -645,7 +654,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 c2_wait(S, &S.acc_free[ab], (j >> 1) & 1u, status);
                 if (S.abort) break;
                 tc_fence_after();
-                c2_issue_mma(tmem, smem_u32(S.a[slot]) + h * 8u * kGroupRowBytes, tmem + kC2AccCol + ab * 128u + h * 64u);
+                c2_issue_mma(tmem, smem_u32(S.a[slot]), tmem + kC2AccCol + ab * 128u);
                 umma_commit(smem_u32(&S.mma_done[ab]));
                 umma_commit(smem_u32(&S.a_free[slot]));
             }
