@@ -29,28 +29,35 @@
 namespace evo {
 
 // ------------------------------------------------------------------------------------------
-// conv1 for a group of up to 64 members.
+// conv1 for a group of up to 32 members.
 //
-// GEMM rows are POOLED pixels (128 per tile); the four conv outputs of a 2x2 pooling window are
-// four separate A operands (the same 6x6 image patch shifted by (dy,dx)) accumulated into four
-// TMEM column blocks, so the max-pool is a max over four registers of one thread, with no
-// shuffles.  Unit of work = (tile, 8 members = 64 filters): 8 MMAs (4 windows x K = 2 x 16)
-// into one of two 256-column accumulators.  Warp 8 issues the MMAs and runs ahead; warps 0-7 read
-// the accumulators (pool, ReLU, bf16; the bias rides in the contraction) and store 16 bytes per
-// (member, pixel); warps 9-12 build the next tile's A operands while the epilogues run.
+// GEMM rows are POOLED pixels (128 per tile).  The A operand of a row is the 6x6 image patch under
+// its pooling window (K = 36, padded to 48 with three constant-1 entries that carry the bias), the
+// same for every member.  A member's B operand has 32 columns: the 8 filters at each of the four
+// positions of the pooling window, i.e. the 5x5 filter placed at offset (dy, dx) in the 6x6 patch
+// (25/36 dense).  The four conv outputs of a window so land in four columns of one thread, and the
+// max-pool is a max over registers, with no shuffles.  Unit of work = (tile, 8 members): 3 MMAs
+// (K = 3 x 16) of N = 256 into one of two 256-column accumulators: an MMA of N = 64 holds the tensor
+// pipe about as long as one of N = 128, so few wide MMAs beat the 8 narrow ones that separate
+// per-position A operands needed.  One warp issues the MMAs and runs ahead; sixteen read the
+// accumulators (pool, ReLU, bf16) and store 16 bytes per (member, pixel); four build the next
+// tile's A operand while the epilogues run.
 // ------------------------------------------------------------------------------------------
-constexpr int kC1EpiThreads = 256;                     // two warps per TMEM lane quarter
-constexpr int kC1StageThreads = 128;                   // one thread per pooled pixel of a tile: builds the A operands
+constexpr int kC1EpiThreads = 512;                     // four warps per TMEM lane quarter
+constexpr int kC1PerThread = 8 * 128 / kC1EpiThreads;  // members of a unit per epilogue thread
+constexpr int kC1StageThreads = 128;                   // one thread per pooled pixel of a tile: builds the A operand
 constexpr int kC1Threads = kC1EpiThreads + 32 + kC1StageThreads;
-constexpr int kC1SmemB = 512 * 32 * 2;                  // all filters of the group, bf16, K = 32
-constexpr int kC1SmemAWin = 128 * 32 * 2;               // one window's im2col tile
-constexpr int kC1SmemA = 4 * kC1SmemAWin;               // four windows
-// the block owns all 512 TMEM columns, so it must be alone on its SM: ask for more than half
-// of the SM's shared memory (it uses ~100 KB of it)
-constexpr int kC1DynRequest = 120 * 1024;
+constexpr uint32_t kC1Group = 32;                      // members per block
+constexpr uint32_t kC1KGroups = 6;                     // K = 48 in groups of 8
+constexpr uint32_t kC1NGroups = kC1Group * 32 / 8;     // N = 32 columns per member, in groups of 8
+constexpr int kC1SmemB = kC1KGroups * kC1NGroups * 128;   // 96 KB: all members of the group, bf16
+constexpr int kC1SmemA = kC1KGroups * 16 * 128;        // 12 KB: one tile
+// the block owns all 512 TMEM columns, so it must be alone on its SM: it uses more than half of
+// the SM's shared memory
+constexpr int kC1DynRequest = kC1SmemB + 2 * kC1SmemA;
 
 struct C1Ctl {
-    uint64_t a_full[2];          // the A operands of a tile are staged
+    uint64_t a_full[2];          // the A operand of a tile is staged
     uint64_t a_free[2];          // every MMA that read an A buffer has completed
     uint64_t mma_done[2];        // an accumulator is complete
     uint64_t acc_free[2];        // an accumulator has been read out
@@ -98,27 +105,21 @@ __device__ __forceinline__ void c1_load_patch(const float* __restrict__ images, 
     }
 }
 
-// im2col rows of the four windows of pooled pixel `row` into the A buffers (core matrices: 8 rows
-// x 16 bytes, k-group kg at +kg*2048, row group at +128)
-__device__ __forceinline__ void c1_stage_rows(unsigned char* Abuf, int row, int dy, const float (&patch)[36])
+// the patch of pooled pixel `row` as its row of the A operand (core matrices: 8 rows x 16 bytes,
+// k-group kg at +kg*2048, row group at +128); k = 6 * patch row + patch column, then three times 1
+__device__ __forceinline__ void c1_stage_row(unsigned char* Abuf, int row, const float (&patch)[36])
 {
+    uint32_t packed[24];
 #pragma unroll
-    for (int dx = 0; dx < 2; ++dx) {                     // the two windows of conv row parity dy
-        const int w = 2 * dy + dx;
-        uint32_t packed[16];
+    for (int k = 0; k < 18; ++k) packed[k] = pack_bf16(patch[2 * k], patch[2 * k + 1]);
+    packed[18] = pack_bf16(1.f, 1.f);
+    packed[19] = pack_bf16(1.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-            const int k0 = 2 * k, k1 = 2 * k + 1;
-            // taps 25..27 of the padded K = 32 are the constant 1: their weights carry the bias (below)
-            const float v0 = (k0 < 25) ? patch[(dy + k0 / 5) * 6 + dx + k0 % 5] : (k0 < 28 ? 1.f : 0.f);
-            const float v1 = (k1 < 25) ? patch[(dy + k1 / 5) * 6 + dx + k1 % 5] : (k1 < 28 ? 1.f : 0.f);
-            packed[k] = pack_bf16(v0, v1);
-        }
+    for (int k = 20; k < 24; ++k) packed[k] = 0u;
 #pragma unroll
-        for (int kg = 0; kg < 4; ++kg)
-            *reinterpret_cast<uint4*>(Abuf + w * kC1SmemAWin + (kg * 16 + (row >> 3)) * 128 + (row & 7) * 16) =
-                make_uint4(packed[4 * kg], packed[4 * kg + 1], packed[4 * kg + 2], packed[4 * kg + 3]);
-    }
+    for (int kg = 0; kg < 6; ++kg)
+        *reinterpret_cast<uint4*>(Abuf + (kg * 16 + (row >> 3)) * 128 + (row & 7) * 16) =
+            make_uint4(packed[4 * kg], packed[4 * kg + 1], packed[4 * kg + 2], packed[4 * kg + 3]);
 }
 
 __global__ void __launch_bounds__(kC1Threads, 1)
@@ -128,40 +129,54 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     extern __shared__ __align__(1024) unsigned char dyn[];
     __shared__ __align__(8) C1Ctl ctl;
 
-    unsigned char* Bsm = dyn;                                           // 32 KB
-    unsigned char* Asm = dyn + kC1SmemB;                                // 2 x 32 KB
+    unsigned char* Bsm = dyn;                                           // 96 KB
+    unsigned char* Asm = dyn + kC1SmemB;                                // 2 x 12 KB
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t group0 = blockIdx.y * 64u;                           // first member of this block's group
-    const uint32_t n_members = min(64u, P - group0);
+    const uint32_t group0 = blockIdx.y * kC1Group;                      // first member of this block's group
+    const uint32_t n_members = min(kC1Group, P - group0);
     const uint32_t n_gm = (n_members + 7u) / 8u;                        // units per tile
     const uint32_t n_groups = (batch + 15u) / 16u;
     const uint32_t n_tiles = n_groups * 18u;                            // 16 images x 144 pooled pixels = 18 tiles
 
-    // ---- B operand: W1 of every member of the group, [filter][k] -> core matrices (k-group, member)
-    for (uint32_t idx = tid; idx < 512u * 4u; idx += kC1Threads) {
-        const uint32_t f = idx >> 2, kg = idx & 3u;                     // filter, 8-tap group
-        const uint32_t m = f >> 3, ch = f & 7u;
-        uint32_t w[4] = { 0, 0, 0, 0 };
+    // ---- B operand: column n = member * 32 + position (dy, dx) * 8 + filter, K = patch element (r, c):
+    //      W1[filter][r - dy][c - dx] where that is a tap, else 0; core matrices (k-group, n / 8).
+    //      thread = (member, filter): its 25 taps in registers give its four columns.
+    for (uint32_t pair = tid; pair < kC1Group * 8u; pair += kC1Threads) {
+        const uint32_t m = pair >> 3, ch = pair & 7u;
+        float wv[25], bp[3] = { 0.f, 0.f, 0.f };
+#pragma unroll
+        for (int i = 0; i < 25; ++i) wv[i] = 0.f;
         if (m < n_members) {
-            const float* src = theta + static_cast<size_t>(group0 + m) * ldD + ch * 25u + kg * 8u;
-            // The bias rides in the contraction: against the three constant-1 taps stand three bf16 pieces of
-            // it, b = b0 + b1 + b2 to 24 bits, so the fp32 accumulator starts from the unrounded bias and
+            const float* src = theta + static_cast<size_t>(group0 + m) * ldD;
+#pragma unroll
+            for (int i = 0; i < 25; ++i) wv[i] = __ldg(src + ch * 25u + i);
+            // The bias rides in the contraction: against the three constant-1 entries stand three bf16 pieces
+            // of it, b = b0 + b1 + b2 to 24 bits, so the fp32 accumulator starts from the unrounded bias and
             // the epilogue has nothing to add.
-            const float b = theta[static_cast<size_t>(group0 + m) * ldD + 200u + ch];
-            const float b0 = __bfloat162float(__float2bfloat16_rn(b));
-            const float b1 = __bfloat162float(__float2bfloat16_rn(b - b0));
-            const float b2 = (b - b0) - b1;
-            float v[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint32_t kk = kg * 8u + k;
-                v[k] = kk < 25u ? src[k] : (kk == 25u ? b0 : (kk == 26u ? b1 : (kk == 27u ? b2 : 0.f)));
-            }
-#pragma unroll
-            for (int k = 0; k < 4; ++k) w[k] = pack_bf16(v[2 * k], v[2 * k + 1]);
+            const float b = __ldg(src + 200u + ch);
+            bp[0] = __bfloat162float(__float2bfloat16_rn(b));
+            bp[1] = __bfloat162float(__float2bfloat16_rn(b - bp[0]));
+            bp[2] = (b - bp[0]) - bp[1];
         }
-        *reinterpret_cast<uint4*>(Bsm + (kg * 64u + (f >> 3)) * 128u + (f & 7u) * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+#pragma unroll
+        for (int pos = 0; pos < 4; ++pos) {
+            const int dy = pos >> 1, dx = pos & 1;
+            const uint32_t n = m * 32u + pos * 8u + ch;
+#pragma unroll
+            for (int kg = 0; kg < 6; ++kg) {
+                float v[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int k = kg * 8 + i, r = k / 6, c = k % 6;
+                    v[i] = 0.f;
+                    if (k < 36) { if (r >= dy && r < dy + 5 && c >= dx && c < dx + 5) v[i] = wv[(r - dy) * 5 + (c - dx)]; }
+                    else if (k < 39) v[i] = bp[k - 36];
+                }
+                *reinterpret_cast<uint4*>(Bsm + (kg * kC1NGroups + (n >> 3)) * 128u + (n & 7u) * 16u) =
+                    make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+            }
+        }
     }
 
     if (tid == 0) {
@@ -185,7 +200,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     if (warp == kC1EpiThreads / 32) {
         // ================= MMA issuer =============================================================
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(128, 64);
+            constexpr uint32_t idesc = umma_idesc_bf16(128, 256);
             const uint32_t a_base = smem_u32(Asm), b_base = smem_u32(Bsm);
             uint32_t u = 0, ti = 0;
             for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++ti) {
@@ -196,13 +211,11 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     wait_or_abort(&ctl.abort, &ctl.acc_free[buf], (u >> 1) & 1u, status);
                     tc_fence_after();
 #pragma unroll
-                    for (uint32_t w = 0; w < 4u; ++w)
-#pragma unroll
-                        for (uint32_t ks = 0; ks < 2u; ++ks) {
-                            const uint64_t ad = umma_smem_desc(a0 + w * kC1SmemAWin + ks * 2u * 2048u, 2048u, 128u);
-                            const uint64_t bd = umma_smem_desc(b_base + ks * 2u * 8192u + gm * 8u * 128u, 8192u, 128u);
-                            umma_bf16(tmem + buf * 256u + w * 64u, ad, bd, idesc, ks);
-                        }
+                    for (uint32_t ks = 0; ks < 3u; ++ks) {
+                        const uint64_t ad = umma_smem_desc(a0 + ks * 2u * 2048u, 2048u, 128u);
+                        const uint64_t bd = umma_smem_desc(b_base + ks * 2u * (kC1NGroups * 128u) + gm * 32u * 128u, kC1NGroups * 128u, 128u);
+                        umma_bf16(tmem + buf * 256u, ad, bd, idesc, ks);
+                    }
                     umma_commit(smem_u32(&ctl.mma_done[buf]));
                 }
                 umma_commit(smem_u32(&ctl.a_free[ti & 1u]));       // arrives once this tile's MMAs are done
@@ -210,8 +223,8 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         }
     } else if (warp > kC1EpiThreads / 32) {
         // ================= staging warps: im2col rows of the tiles, one tile ahead of the MMAs ============
-        // thread = pooled pixel of the tile; the 6x6 image patch under it gives the rows of all four
-        // pooling windows.  The buffer of tile ti is free once the MMAs of tile ti - 2 have completed.
+        // thread = pooled pixel of the tile; the 6x6 image patch under it is its row of the operand.
+        // The buffer of tile ti is free once the MMAs of tile ti - 2 have completed.
         const int row = tid - (kC1EpiThreads + 32);
         float patch[36];
         uint32_t ti = 0;
@@ -219,8 +232,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             c1_load_patch(images, tile * 128u + row, batch, patch);
             if (ti >= 2u) wait_or_abort(&ctl.abort, &ctl.a_free[ti & 1u], ((ti >> 1) - 1u) & 1u, status);
             unsigned char* Abuf = Asm + (ti & 1u) * kC1SmemA;
-            c1_stage_rows(Abuf, row, 0, patch);
-            c1_stage_rows(Abuf, row, 1, patch);
+            c1_stage_row(Abuf, row, patch);
             fence_async_smem();
             asm volatile("bar.sync 2, %0;" :: "n"(kC1StageThreads) : "memory");
             if (row == 0) mbar_arrive(smem_u32(&ctl.a_full[ti & 1u]));
@@ -233,7 +245,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     } else {
         // ================= epilogue warps ==========================================================
         if (lane == 0) { mbar_arrive(smem_u32(&ctl.acc_free[0])); mbar_arrive(smem_u32(&ctl.acc_free[1])); }
-        const int row = tid & 127, half = tid >> 7;       // my pooled pixel (= TMEM lane) and my half of the members
+        const int row = tid & 127, part = tid >> 7;       // my pooled pixel (= TMEM lane) and my share of the members
         uint32_t u = 0, ti = 0;
         for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++ti) {
             const uint32_t pix_off = tile * 128u + row;                // my GEMM row = my TMEM lane = my output element
@@ -244,27 +256,27 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 const uint32_t buf = u & 1u;
                 wait_or_abort(&ctl.abort, &ctl.mma_done[buf], (u >> 1) & 1u, status);
                 tc_fence_after();
-                const uint32_t t0 = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + buf * 256u + half * 32u;
-                // My four members of the unit, one at a time: the 8 filters of a member under the four
-                // pooling windows are 4 x 8 columns.  The loads of the next member are in flight while
-                // this one is pooled and stored (two register buffers).
+                const uint32_t t0 = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + buf * 256u + part * (32u * kC1PerThread);
+                // My members of the unit, one at a time: a member's 8 filters at the four positions of
+                // the pooling window are 32 consecutive columns.  The loads of the next member are in flight
+                // while this one is pooled and stored (two register buffers).
                 uint32_t ra[4][8], rb[4][8];
 #pragma unroll
-                for (int w = 0; w < 4; ++w) tmem_ld8_issue(t0 + w * 64u, ra[w]);
+                for (int w = 0; w < 4; ++w) tmem_ld8_issue(t0 + w * 8u, ra[w]);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < kC1PerThread; ++j) {
                     uint32_t (&cur)[4][8] = (j & 1) ? rb : ra;
                     uint32_t (&nxt)[4][8] = (j & 1) ? ra : rb;
                     tmem_ld8x4_fence(cur[0], cur[1], cur[2], cur[3]);
-                    if (j < 3) {
+                    if (j < kC1PerThread - 1) {
 #pragma unroll
-                        for (int w = 0; w < 4; ++w) tmem_ld8_issue(t0 + w * 64u + (j + 1) * 8u, nxt[w]);
+                        for (int w = 0; w < 4; ++w) tmem_ld8_issue(t0 + (j + 1) * 32u + w * 8u, nxt[w]);
                     } else {                                             // my part of the accumulator is in registers
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&ctl.acc_free[buf]));
                     }
-                    const uint32_t m = gm * 8u + half * 4u + j;
+                    const uint32_t m = gm * 8u + part * kC1PerThread + j;
                     // the accumulators already contain the bias: relu(max4) = two 3-input max per value
                     uint32_t o[4];
 #pragma unroll
@@ -435,7 +447,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         // thread holds the 8 x 16 (output row, image) outputs of its (column, filter).  Row pairs are
         // a max over two registers; the column pair is lane ^ 16, done as an exchange: of a pair of
         // pooled rows (a, a + 2) the thread of the even column keeps row a, that of the odd column a + 2.
-        const int f = lane & 15, odd = lane >> 4, xo = 2 * warp + odd, px = warp;
+        const int f = lane & 15, odd = lane >> 4, px = warp;     // output column 2 * warp + odd
         const uint32_t tm_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
         const uint32_t first_member = u_begin / n_groups;
         float bias = 0.f;
@@ -738,7 +750,8 @@ int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uin
     if (cudaFuncSetAttribute(k_cnn_conv1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kC1DynRequest) != cudaSuccess) return -1;
     const uint32_t n_groups = (batch + 15u) / 16u;
     const uint32_t n_tiles = n_groups * 18u;
-    dim3 g1(min(static_cast<uint32_t>(sm_count), n_tiles), (P + 63u) / 64u);
+    const uint32_t n_member_groups = (P + kC1Group - 1u) / kC1Group;
+    dim3 g1(min(max(static_cast<uint32_t>(sm_count) / n_member_groups, 1u), n_tiles), n_member_groups);
     k_cnn_conv1_tc<<<g1, kC1Threads, kC1DynRequest, st>>>(theta, ldD, P, images, batch,
                                                           reinterpret_cast<uint4*>(pooled1), status);
     if (cudaGetLastError() != cudaSuccess) return -1;
