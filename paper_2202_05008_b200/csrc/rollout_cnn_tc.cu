@@ -339,6 +339,7 @@ constexpr int kRawPitch = 201;                           // floats per filter in
 struct __align__(128) C2Smem {
     unsigned char a[kC2Ring][kGroupBytes];               // pooled-1 groups (ring)
     float raw[16 * kRawPitch];                           // W2 as stored, one padded row per filter
+    uint4 taps[16][25];                                  // W2 as bf16: the 8 channels of (filter, tap) = the 4 columns of an input column
     float wfT[2][256 * 12];                              // linear layer transposed [k][class], bf16-rounded, one copy per linear team
     __align__(16) __nv_bfloat16 p2[2][16][kP2Pitch];     // pooled-2 activations of a unit's images, k = pixel*16 + channel
     float part[2][2][4][16][12];                         // [team][unit parity in the team] partial logits of the four warps
@@ -450,63 +451,83 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         const int f = lane & 15, odd = lane >> 4, px = warp;     // output column 2 * warp + odd
         const uint32_t tm_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
         const uint32_t first_member = u_begin / n_groups;
-        float bias = 0.f;
-        uint32_t staged_member = 0xFFFFFFFFu;
+        // A member's filters on their way to tensor memory, in two steps.  The first needs no tensor memory and
+        // runs ahead, while the MMAs of the previous member's last unit are still busy: W2 as stored ->
+        // shared memory (coalesced) -> bf16, the 8 channels of a (filter, tap) as one 16-byte entry.
+        auto load_taps = [&](uint32_t member) {
+            const float* prm = theta + static_cast<size_t>(member) * ldD;
+            const float4* w2v = reinterpret_cast<const float4*>(prm + 208u);          // 16-byte aligned
+            float4 t2[7];
+#pragma unroll
+            for (int k = 0; k < 7; ++k)
+                t2[k] = (tid + k * kC2EpiThreads < 800) ? __ldg(w2v + tid + k * kC2EpiThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int k = 0; k < 7; ++k) {
+                const uint32_t i = 4u * (tid + k * kC2EpiThreads);                   // flat (filter*8 + channel)*25 + tap
+                if (i < 3200u) {
+                    float* d = S.raw + (i / 200u) * kRawPitch + i % 200u;           // 200 = 4 * 50: a float4 stays in its filter
+                    d[0] = t2[k].x; d[1] = t2[k].y; d[2] = t2[k].z; d[3] = t2[k].w;
+                }
+            }
+            if (tid < 16) S.b2[tid] = prm[3408u + tid];
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+            for (uint32_t i = tid; i < 400u; i += kC2EpiThreads) {
+                const float* src = S.raw + (i / 25u) * kRawPitch + i % 25u;           // (filter, tap), channels 25 apart
+                S.taps[i / 25u][i % 25u] = make_uint4(pack_bf16(src[0], src[25]), pack_bf16(src[50], src[75]),
+                                                      pack_bf16(src[100], src[125]), pack_bf16(src[150], src[175]));
+            }
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+        };
+        // The second step, once every MMA of the previous member has completed: band dy, row (output column
+        // xo, filter f), K = (input column xi, channel) is W2[f][channel][dy][xi - xo].  A tensor-memory column
+        // holds two consecutive K, 8 columns = two input columns = one K-step.  Only the input columns
+        // xo .. xo + 4 of a row are not zero, the same for every member: they lie in the three K-steps from
+        // xo / 2 on.  Then the issuers are told.
+        auto write_bands = [&](uint32_t member) {
+#pragma unroll
+            for (uint32_t dy = 0; dy < 5u; ++dy)
+#pragma unroll
+                for (int t = 0; t < 3; ++t) {
+                    uint4 q[2];
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        const int dx = 2 * t + c - odd;                                // xo is 2 * warp + odd
+                        q[c] = make_uint4(0u, 0u, 0u, 0u);
+                        if (dx >= 0 && dx <= 4) q[c] = S.taps[f][dy * 5 + dx];
+                    }
+                    const uint32_t u[8] = { q[0].x, q[0].y, q[0].z, q[0].w, q[1].x, q[1].y, q[1].z, q[1].w };
+                    tmem_st8(tm_lane + dy * kC2BandCols + static_cast<uint32_t>(warp + t) * 8u, u);
+                }
+            tmem_st_wait();
+            tc_fence_before();
+            asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
+            if (tid == 0)
+                asm volatile("st.release.cta.shared::cta.u32 [%0], %1;"
+                             :: "r"(smem_u32(&S.staged)), "r"(member - first_member + 1u) : "memory");
+        };
         {   // the zeros of the bands, once
             const uint32_t z[8] = { 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u };
 #pragma unroll
             for (uint32_t c = 0; c < 5u * kC2BandCols; c += 8u) tmem_st8(tm_lane + c, z);
             tmem_st_wait();
         }
+        load_taps(first_member);
+        write_bands(first_member);
+        float bias = S.b2[f];
         for (uint32_t j = 0; j < n_mine; ++j) {
             const uint32_t member = (u_begin + j) / n_groups, ab = j & 1u, par = (j >> 1) & 1u;
-            if (member != staged_member) {
-                // Every MMA of the previous member has been waited for, so the bands can be rewritten.
-                staged_member = member;
-                const float* prm = theta + static_cast<size_t>(member) * ldD;
-                const float4* w2v = reinterpret_cast<const float4*>(prm + 208u);      // 16-byte aligned
-                float4 t2[7];
-#pragma unroll
-                for (int k = 0; k < 7; ++k)
-                    t2[k] = (tid + k * kC2EpiThreads < 800) ? __ldg(w2v + tid + k * kC2EpiThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int k = 0; k < 7; ++k) {
-                    const uint32_t i = 4u * (tid + k * kC2EpiThreads);               // flat (filter*8 + channel)*25 + tap
-                    if (i < 3200u) {
-                        float* d = S.raw + (i / 200u) * kRawPitch + i % 200u;       // 200 = 4 * 50: a float4 stays in its filter
-                        d[0] = t2[k].x; d[1] = t2[k].y; d[2] = t2[k].z; d[3] = t2[k].w;
-                    }
-                }
-                if (tid < 16) S.b2[tid] = prm[3408u + tid];
-                asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-                // band dy, row (output column xo, filter f), K = (input column xi, channel): W2[f][channel][dy][xi - xo].
-                // A tensor-memory column holds two consecutive K, 8 columns = two input columns = one K-step.
-                // Only the input columns xo .. xo + 4 of a row are not zero, the same for every member: they
-                // lie in the three K-steps from xo / 2 on.
-                const float* mine = S.raw + f * kRawPitch;
-#pragma unroll
-                for (uint32_t dy = 0; dy < 5u; ++dy)
-#pragma unroll
-                    for (int t = 0; t < 3; ++t) {
-                        uint32_t u[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const int dx = 2 * t + (e >> 2) - odd, ch = 2 * (e & 3);       // xo is 2 * warp + odd
-                            u[e] = 0u;
-                            if (dx >= 0 && dx <= 4) u[e] = pack_bf16(mine[ch * 25 + dy * 5 + dx], mine[(ch + 1) * 25 + dy * 5 + dx]);
-                        }
-                        tmem_st8(tm_lane + dy * kC2BandCols + static_cast<uint32_t>(warp + t) * 8u, u);
-                    }
-                tmem_st_wait();
-                tc_fence_before();
-                bias = S.b2[f];
-                asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-                if (tid == 0)
-                    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;"
-                                 :: "r"(smem_u32(&S.staged)), "r"(member - first_member + 1u) : "memory");
-            }
+            // the unit after this one belongs to the next member: its filters are fetched while this unit's MMAs run
+            const bool last_of_member = j + 1u < n_mine && (u_begin + j + 1u) / n_groups != member;
+            if (last_of_member) load_taps(member + 1u);
             c2_wait(S, &S.mma_done[ab], par, status);
             tc_fence_after();
+            float next_bias = bias;
+            if (last_of_member) {
+                // This was the member's last MMA, so the bands can be rewritten, and the next member's MMAs
+                // run while this unit's accumulator is read out.
+                write_bands(member + 1u);
+                next_bias = S.b2[f];
+            }
             c2_wait(S, &S.p2_free[ab], par, status);
             const uint32_t t0 = tm_lane + kC2AccCol + ab * 128u;
 #pragma unroll
@@ -535,6 +556,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&S.p2_full[ab]));
+            bias = next_bias;
         }
     } else if (warp < (kC2EpiThreads + kC2LinThreads) / 32) {
         // ================= linear layer 256 -> 10 and cross-entropy ==============================
@@ -680,6 +702,9 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             for (uint32_t j = 0; j < n_mine; ++j) {
                 const uint32_t slot = j % kC2Ring;
                 if (j >= kC2Ring) c2_wait(S, &S.a_free[slot], (j / kC2Ring - 1u) & 1u, status);
+                // the first groups one after the other, so that memory serves every block's first group
+                // (and its weights) before anyone's second
+                else if (j >= 1u) c2_wait(S, &S.a_full[j - 1u], 0u, status);
                 if (S.abort) break;
                 bulk_copy_g2s(smem_u32(S.a[slot]), src + static_cast<size_t>(j) * kGroupBytes, kGroupBytes, smem_u32(&S.a_full[slot]));
                 issued = j + 1u;
