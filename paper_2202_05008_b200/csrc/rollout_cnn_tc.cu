@@ -431,6 +431,13 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         S.abort = 0;
         mbar_init_fence();
     }
+    // A block whose range runs into a second member will want that member's parameters in the middle of its
+    // work, from memory that is busy streaming activations by then: ask for them now, into L2.
+    if ((u_end - 1u) / n_groups != u_begin / n_groups) {
+        const float* nxt = theta + static_cast<size_t>(u_begin / n_groups + 1u) * ldD + 208u;     // conv2 and linear layers
+        for (uint32_t i = tid; i < (kCnnParams - 208u + 31u) / 32u; i += kC2Threads)
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(nxt + 32u * i));
+    }
     for (int k = tid; k < 512; k += kC2Threads) { S.wfT[k >> 8][(k & 255) * 12 + 10] = 0.f; S.wfT[k >> 8][(k & 255) * 12 + 11] = 0.f; }
     if (tid < 4) S.bfc[tid >> 1][10 + (tid & 1)] = 0.f;
     __syncwarp();
