@@ -69,9 +69,23 @@ def test_cnn_tensor_core_path_against_the_unrounded_oracle():
 
 
 def test_cnn_more_than_one_member_group_and_tiny_batch():
-    # 70 members = two conv1 groups (64 + 6); batch 3 = one full pair and one half pair
+    # 70 members = three conv1 groups (32 + 32 + 6); batch 3 = a fifth of one image group
     w = W.CFG3.with_(pop_size=70, batch=3)
-    _run(w, theta_np=W.random_parameters(6, 70, W.CNN_PARAMS, scale=0.1), members=[0, 5, 63, 64, 69])
+    _run(w, theta_np=W.random_parameters(6, 70, W.CNN_PARAMS, scale=0.1), members=[0, 5, 31, 32, 63, 64, 69])
+
+
+@pytest.mark.parametrize("pop,batch,members", [
+    (300, 24, [0, 1, 2, 3, 147, 148, 149, 298, 299]),   # 600 units on 148 blocks: every block runs through 2-3 members
+    (296, 16, [0, 1, 2, 3, 100, 295]),                  # one image group per member: every unit is a new member
+    (34, 16, [0, 31, 32, 33]),                          # a conv1 group of two members
+    (6, 1, [0, 5]),                                     # a single image
+    (4, 200, [0, 1, 2, 3]),                             # 13 image groups per member, the last half full
+])
+def test_cnn_block_ranges_across_members(pop, batch, members):
+    """conv2 blocks take contiguous ranges of (member, image group) units: cases where a range runs through
+    several members (filter bands restaged in flight), where each unit is a new member, and ragged ends."""
+    w = W.CFG3.with_(pop_size=pop, batch=batch)
+    _run(w, theta_np=W.random_parameters(11, pop, W.CNN_PARAMS, scale=0.1), members=members)
 
 
 def test_cnn_tensor_core_path_is_deterministic():
