@@ -319,15 +319,15 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 //
 // Roles: warps 0-3 read the accumulators (2x2 max over two columns of a thread and two lanes,
 // bias, ReLU, bf16) into a per-image activation buffer; warps 4-11 run the linear layer and the
-// cross-entropy from that buffer; warps 12-15 each issue the MMAs of one (accumulator, half of N);
-// warp 16 brings the groups in, one bulk copy each, through a ring of three.  The roles meet only
+// cross-entropy from that buffer; two warps each issue the MMAs of one accumulator; one warp fetches
+// the filters of the members to come; one brings the groups in, one bulk copy each, through a ring of three.  The roles meet only
 // on mbarriers; every wait is bounded, and after a time-out all later waits fall through so that
 // no role is left behind.
 // ------------------------------------------------------------------------------------------
 constexpr int kC2EpiThreads = 128;
 constexpr int kC2LinThreads = 256;
 constexpr int kC2Issuers = 2;
-constexpr int kC2Threads = kC2EpiThreads + kC2LinThreads + 32 * kC2Issuers + 32;
+constexpr int kC2Threads = kC2EpiThreads + kC2LinThreads + 32 * kC2Issuers + 32 + 32;
 constexpr uint32_t kGroupRowBytes = 12 * 8 * 16;         // one (y, image octet): 12 pixels x 8 images x 16 bytes
 constexpr uint32_t kGroupBytes = 12 * 2 * kGroupRowBytes;   // 36,864
 constexpr uint32_t kC2Ring = 3;                          // groups in flight
@@ -339,11 +339,12 @@ constexpr int kRawPitch = 201;                           // floats per filter in
 struct __align__(128) C2Smem {
     unsigned char a[kC2Ring][kGroupBytes];               // pooled-1 groups (ring)
     float raw[16 * kRawPitch];                           // W2 as stored, one padded row per filter
-    uint4 taps[16][25];                                  // W2 as bf16: the 8 channels of (filter, tap) = the 4 columns of an input column
+    uint4 taps[2][16][25];                               // W2 as bf16: the 8 channels of (filter, tap) = the 4 columns of an input column;
+                                                         // [member of the block's range & 1]: the next member's are fetched ahead
     float wfT[2][256 * 12];                              // linear layer transposed [k][class], bf16-rounded, one copy per linear team
     __align__(16) __nv_bfloat16 p2[2][16][kP2Pitch];     // pooled-2 activations of a unit's images, k = pixel*16 + channel
     float part[2][2][4][16][12];                         // [team][unit parity in the team] partial logits of the four warps
-    float b2[16];
+    float b2[2][16];
     float bfc[2][12];
     uint64_t a_full[kC2Ring];                            // a group has landed
     uint64_t a_free[kC2Ring];                            // every MMA that read a group has completed
@@ -353,6 +354,8 @@ struct __align__(128) C2Smem {
     uint64_t p2_free[2];                                 // ... and have been consumed by the linear layer
     uint64_t drain;                                      // all MMAs of the block have completed
     uint32_t staged;                                     // members of the block's range whose bands have been staged
+    uint32_t taps_loaded;                                // ... whose filters are in `taps`
+    uint32_t issued;                                     // units whose MMAs have been issued
     uint32_t tmem_slot;
     volatile int abort;
 };
@@ -362,12 +365,13 @@ __device__ __forceinline__ void c2_wait(C2Smem& S, uint64_t* bar, uint32_t parit
     wait_or_abort(&S.abort, bar, parity, status);
 }
 
-// The bands are staged once per member, in order, and the count of staged members only grows: an
-// issuer that has no unit of some member (a group count of one) would lose track of an mbarrier's
-// phase parity, a counter cannot be misread.  Bounded like every other wait.
-__device__ __forceinline__ void c2_wait_staged(C2Smem& S, uint32_t need, DeviceStatus* status)
+// Progress that is counted, not signalled: the members whose bands are staged, the members whose
+// filters are in shared memory, the units whose MMAs are issued.  Counts only grow, so a role that
+// skips some (an issuer with no unit of some member when a group count is one) cannot misread them
+// as it could an mbarrier's phase parity.  The wait is bounded like every other.
+__device__ __forceinline__ void c2_wait_count(C2Smem& S, const uint32_t* counter, uint32_t need, DeviceStatus* status)
 {
-    const uint32_t addr = smem_u32(&S.staged);
+    const uint32_t addr = smem_u32(counter);
     uint32_t have;
     long long t0 = 0;
     for (;;) {
@@ -382,6 +386,10 @@ __device__ __forceinline__ void c2_wait_staged(C2Smem& S, uint32_t need, DeviceS
         }
         __nanosleep(64);
     }
+}
+__device__ __forceinline__ void c2_set_count(uint32_t* counter, uint32_t value)
+{
+    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" :: "r"(smem_u32(counter)), "r"(value) : "memory");
 }
 
 // The 30 MMAs of one half (4 output rows x 16 images) of a unit.  b0 = the group, advanced to the
@@ -428,6 +436,8 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         }
         mbar_init(smem_u32(&S.drain), kC2Issuers);
         S.staged = 0;
+        S.taps_loaded = 0;
+        S.issued = 0;
         S.abort = 0;
         mbar_init_fence();
     }
@@ -458,9 +468,9 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         const int f = lane & 15, odd = lane >> 4, px = warp;     // output column 2 * warp + odd
         const uint32_t tm_lane = tmem + (static_cast<uint32_t>(warp * 32) << 16);
         const uint32_t first_member = u_begin / n_groups;
-        // A member's filters on their way to tensor memory, in two steps.  The first needs no tensor memory and
-        // runs ahead, while the MMAs of the previous member's last unit are still busy: W2 as stored ->
-        // shared memory (coalesced) -> bf16, the 8 channels of a (filter, tap) as one 16-byte entry.
+        // A member's filters on their way to tensor memory, in two steps.  The first needs no tensor memory: W2
+        // as stored -> shared memory (coalesced) -> bf16, the 8 channels of a (filter, tap) as one 16-byte
+        // entry.  Here for the block's first member; the weights warp does it for the later ones, ahead of time.
         auto load_taps = [&](uint32_t member) {
             const float* prm = theta + static_cast<size_t>(member) * ldD;
             const float4* w2v = reinterpret_cast<const float4*>(prm + 208u);          // 16-byte aligned
@@ -476,11 +486,11 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     d[0] = t2[k].x; d[1] = t2[k].y; d[2] = t2[k].z; d[3] = t2[k].w;
                 }
             }
-            if (tid < 16) S.b2[tid] = prm[3408u + tid];
+            if (tid < 16) S.b2[0][tid] = prm[3408u + tid];
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
             for (uint32_t i = tid; i < 400u; i += kC2EpiThreads) {
                 const float* src = S.raw + (i / 25u) * kRawPitch + i % 25u;           // (filter, tap), channels 25 apart
-                S.taps[i / 25u][i % 25u] = make_uint4(pack_bf16(src[0], src[25]), pack_bf16(src[50], src[75]),
+                S.taps[0][i / 25u][i % 25u] = make_uint4(pack_bf16(src[0], src[25]), pack_bf16(src[50], src[75]),
                                                       pack_bf16(src[100], src[125]), pack_bf16(src[150], src[175]));
             }
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
@@ -490,7 +500,8 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         // holds two consecutive K, 8 columns = two input columns = one K-step.  Only the input columns
         // xo .. xo + 4 of a row are not zero, the same for every member: they lie in the three K-steps from
         // xo / 2 on.  Then the issuers are told.
-        auto write_bands = [&](uint32_t member) {
+        auto write_bands = [&](uint32_t member) -> float {
+            const uint4 (&taps)[16][25] = S.taps[(member - first_member) & 1u];
 #pragma unroll
             for (uint32_t dy = 0; dy < 5u; ++dy)
 #pragma unroll
@@ -500,17 +511,17 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     for (int c = 0; c < 2; ++c) {
                         const int dx = 2 * t + c - odd;                                // xo is 2 * warp + odd
                         q[c] = make_uint4(0u, 0u, 0u, 0u);
-                        if (dx >= 0 && dx <= 4) q[c] = S.taps[f][dy * 5 + dx];
+                        if (dx >= 0 && dx <= 4) q[c] = taps[f][dy * 5 + dx];
                     }
                     const uint32_t u[8] = { q[0].x, q[0].y, q[0].z, q[0].w, q[1].x, q[1].y, q[1].z, q[1].w };
                     tmem_st8(tm_lane + dy * kC2BandCols + static_cast<uint32_t>(warp + t) * 8u, u);
                 }
             tmem_st_wait();
             tc_fence_before();
+            const float b = S.b2[(member - first_member) & 1u][f];      // read before the buffer is given back
             asm volatile("bar.sync 1, %0;" :: "n"(kC2EpiThreads) : "memory");
-            if (tid == 0)
-                asm volatile("st.release.cta.shared::cta.u32 [%0], %1;"
-                             :: "r"(smem_u32(&S.staged)), "r"(member - first_member + 1u) : "memory");
+            if (tid == 0) c2_set_count(&S.staged, member - first_member + 1u);
+            return b;                                                    // the member's bias for this thread's filter
         };
         {   // the zeros of the bands, once
             const uint32_t z[8] = { 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u };
@@ -519,21 +530,18 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
             tmem_st_wait();
         }
         load_taps(first_member);
-        write_bands(first_member);
-        float bias = S.b2[f];
+        float bias = write_bands(first_member);
         for (uint32_t j = 0; j < n_mine; ++j) {
             const uint32_t member = (u_begin + j) / n_groups, ab = j & 1u, par = (j >> 1) & 1u;
-            // the unit after this one belongs to the next member: its filters are fetched while this unit's MMAs run
             const bool last_of_member = j + 1u < n_mine && (u_begin + j + 1u) / n_groups != member;
-            if (last_of_member) load_taps(member + 1u);
             c2_wait(S, &S.mma_done[ab], par, status);
             tc_fence_after();
             float next_bias = bias;
             if (last_of_member) {
                 // This was the member's last MMA, so the bands can be rewritten, and the next member's MMAs
                 // run while this unit's accumulator is read out.
-                write_bands(member + 1u);
-                next_bias = S.b2[f];
+                c2_wait_count(S, &S.taps_loaded, member + 1u - first_member + 1u, status);
+                next_bias = write_bands(member + 1u);
             }
             c2_wait(S, &S.p2_free[ab], par, status);
             const uint32_t t0 = tm_lane + kC2AccCol + ab * 128u;
@@ -689,7 +697,10 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 const uint32_t member = (u_begin + j) / n_groups, slot = j % kC2Ring;
                 if (member != seen_member) {
                     seen_member = member;
-                    c2_wait_staged(S, member - first_member + 1u, status);
+                    c2_wait_count(S, &S.staged, member - first_member + 1u, status);
+                    // When a member's bands are staged both issuers are let go at once, and the MMAs of two
+                    // units taking turns in the pipe would finish the first unit late: in unit order here.
+                    c2_wait_count(S, &S.issued, j, status);
                 }
                 c2_wait(S, &S.a_full[slot], (j / kC2Ring) & 1u, status);
                 c2_wait(S, &S.acc_free[ab], (j >> 1) & 1u, status);
@@ -698,8 +709,31 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 c2_issue_mma(tmem, smem_u32(S.a[slot]), tmem + kC2AccCol + ab * 128u);
                 umma_commit(smem_u32(&S.mma_done[ab]));
                 umma_commit(smem_u32(&S.a_free[slot]));
+                c2_set_count(&S.issued, j + 1u);
             }
             umma_commit(smem_u32(&S.drain));                          // arrives when all my MMAs have completed
+        }
+    } else if (warp == (kC2EpiThreads + kC2LinThreads) / 32 + kC2Issuers) {
+        // ================= weights warp: the later members' filters, fetched ahead =================
+        // For the members after the block's first: W2 -> bf16 entries in the buffer that the member
+        // before the previous one has left (its bands are staged), straight from global memory (L2: they
+        // were asked for at the start); slow, but a member's worth of units ahead of when it is needed.
+        const uint32_t first_member = u_begin / n_groups, n_ord = (u_end - 1u) / n_groups - first_member + 1u;
+        for (uint32_t ord = 1; ord < n_ord; ++ord) {
+            c2_wait_count(S, &S.staged, ord - 1u, status);
+            if (S.abort) break;
+            const float* prm = theta + static_cast<size_t>(first_member + ord) * ldD;
+            for (uint32_t i = lane; i < 400u; i += 32u) {
+                const float* src = prm + 208u + (i / 25u) * 200u + i % 25u;             // (filter, tap), channels 25 apart
+                float v[8];
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch) v[ch] = __ldg(src + ch * 25);
+                S.taps[ord & 1u][i / 25u][i % 25u] = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]),
+                                                                pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+            }
+            if (lane < 16) S.b2[ord & 1u][lane] = __ldg(prm + 3408u + lane);
+            __syncwarp();
+            if (lane == 0) c2_set_count(&S.taps_loaded, ord + 1u);
         }
     } else {
         // ================= producer: one bulk copy per unit, up to three units ahead ===============
