@@ -355,7 +355,7 @@ struct __align__(128) C2Smem {
     uint64_t drain;                                      // all MMAs of the block have completed
     uint32_t staged;                                     // members of the block's range whose bands have been staged
     uint32_t taps_loaded;                                // ... whose filters are in `taps`
-    uint32_t issued;                                     // units whose MMAs have been issued
+    uint32_t issued[2];                                  // per issuer: one past the last unit whose MMAs it has issued
     uint32_t tmem_slot;
     volatile int abort;
 };
@@ -366,9 +366,10 @@ __device__ __forceinline__ void c2_wait(C2Smem& S, uint64_t* bar, uint32_t parit
 }
 
 // Progress that is counted, not signalled: the members whose bands are staged, the members whose
-// filters are in shared memory, the units whose MMAs are issued.  Counts only grow, so a role that
-// skips some (an issuer with no unit of some member when a group count is one) cannot misread them
-// as it could an mbarrier's phase parity.  The wait is bounded like every other.
+// filters are in shared memory, the units whose MMAs an issuer has issued.  Every counter has one
+// writer and only grows, so a role that skips some values (an issuer with no unit of some member
+// when a group count is one) cannot misread it as it could an mbarrier's phase parity.  The wait is
+// bounded like every other.
 __device__ __forceinline__ void c2_wait_count(C2Smem& S, const uint32_t* counter, uint32_t need, DeviceStatus* status)
 {
     const uint32_t addr = smem_u32(counter);
@@ -437,7 +438,8 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         mbar_init(smem_u32(&S.drain), kC2Issuers);
         S.staged = 0;
         S.taps_loaded = 0;
-        S.issued = 0;
+        S.issued[0] = 0;
+        S.issued[1] = 0;
         S.abort = 0;
         mbar_init_fence();
     }
@@ -700,7 +702,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                     c2_wait_count(S, &S.staged, member - first_member + 1u, status);
                     // When a member's bands are staged both issuers are let go at once, and the MMAs of two
                     // units taking turns in the pipe would finish the first unit late: in unit order here.
-                    c2_wait_count(S, &S.issued, j, status);
+                    c2_wait_count(S, &S.issued[ab ^ 1u], j, status);      // unit j - 1 is the other issuer's
                 }
                 c2_wait(S, &S.a_full[slot], (j / kC2Ring) & 1u, status);
                 c2_wait(S, &S.acc_free[ab], (j >> 1) & 1u, status);
@@ -709,7 +711,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 c2_issue_mma(tmem, smem_u32(S.a[slot]), tmem + kC2AccCol + ab * 128u);
                 umma_commit(smem_u32(&S.mma_done[ab]));
                 umma_commit(smem_u32(&S.a_free[slot]));
-                c2_set_count(&S.issued, j + 1u);
+                c2_set_count(&S.issued[ab], j + 1u);
             }
             umma_commit(smem_u32(&S.drain));                          // arrives when all my MMAs have completed
         }
