@@ -3,20 +3,24 @@
 // The convolutional policy (conv 1->8 5x5, ReLU, pool; conv 8->16 5x5, ReLU, pool; linear
 // 256->10) evaluated for every member on the same batch is two dense contractions:
 //
-//   k_cnn_conv1_tc   conv1 for ALL members at once.  The batch is shared, so the im2col rows
-//                    (K = 25 taps padded to 32, three of the pad taps carrying the bias) are the A
-//                    operand for every member and the 8P filters of the population sit side by side
-//                    on N.  GEMM rows are pooled pixels; the four conv outputs under a pooling window
-//                    are four A operands accumulated into four TMEM column blocks, so the 2x2
+//   k_cnn_conv1_tc   conv1 for a group of members at once.  The batch is shared, so a GEMM row (a pooled
+//                    pixel) has one A operand for every member: the 6x6 image patch under its pooling
+//                    window (K = 36, + 3 entries that carry the bias, padded to 48).  A member's B operand
+//                    places its 8 filters at the four positions of the window (N = 32 per member), so
+//                    the four conv outputs of a window are four columns of one thread and the 2x2
 //                    max-pool is a max over registers.  The epilogue applies ReLU and writes the
 //                    pooled activation as bf16, 8 channels = 16 bytes per pixel, in the operand
 //                    layout of conv2.
 //   k_cnn_conv2_tc   per member and group of 16 images: conv2 as a contraction over whole input
-//                    rows against a banded copy of the member's filter rows, with NO im2col copy:
-//                    the 8 channels of a pixel are one 16-byte row of a UMMA core matrix, 8 images
-//                    are its 8 rows, and filter row and column offsets are address offsets into
-//                    the group that a single bulk copy brought in.  D[128 = 8 rows x 16 images][4
-//                    columns x 16 filters] in TMEM; pool, linear layer and cross-entropy on CUDA cores.
+//                    rows.  The member's filter rows, as banded matrices, stay in TENSOR MEMORY as the A
+//                    operand (M = 8 output columns x 16 filters, K = 12 input columns x 8 channels);
+//                    the activations are the B operand with NO im2col copy: the 8 channels of a pixel
+//                    are one 16-byte row of a UMMA core matrix, 8 images are its 8 rows, and filter
+//                    row and K-step are address offsets into the group that a single bulk copy
+//                    brought in.  D[8 columns x 16 filters][8 rows x 16 images] in TMEM; pool, linear
+//                    layer and cross-entropy on CUDA cores.
+//
+// Few wide MMAs: an MMA of N = 16 or 64 holds the tensor pipe about as long as one of N = 128.
 //
 // Operands are bf16 (round to nearest even), accumulation fp32 in TMEM.  Every wait is bounded:
 // on expiry the block records EVO_ERR_TIMEOUT, frees its TMEM and leaves.
