@@ -107,3 +107,25 @@ def test_cnn_rollout_needs_a_batch():
         s.rollout()
     assert e.value.code == 2
     s.close()
+
+
+@pytest.mark.parametrize("pop,batch", [(64, 256), (70, 48), (296, 16), (128, 100)])
+def test_cnn_many_generations_stay_ok_and_deterministic(pop, batch):
+    """The roles of the tensor-core kernels meet on mbarriers and progress counters; a rare ordering that made
+    one of them wait for ever would show up as EVO_ERR_TIMEOUT (a bounded wait giving up) only after many
+    launches.  150 generations per shape, the roll-out repeated now and then: same bits, status ok."""
+    w = W.CFG3.with_(pop_size=pop, batch=batch)
+    s = Solver(w)
+    images, labels = W.image_batch(w.seed, 0, w.batch)
+    s.set_batch(torch.tensor(images, device="cuda"), torch.tensor(labels, device="cuda"))
+    fit = torch.empty(pop, dtype=torch.float32, device="cuda")
+    for g in range(150):
+        s.ask()
+        s.rollout(fitness=fit)
+        if g % 25 == 0:
+            first = fit.clone()
+            s.rollout(fitness=fit)
+            assert torch.equal(first, fit)
+        s.tell(fit)
+    assert s.sync_status() == 0
+    s.close()
