@@ -142,4 +142,31 @@ int launch_rollout_paint(cudaStream_t st, const float* theta, uint32_t ldD, uint
                          uint32_t W, uint32_t H, float background, const float* target, void* scratch,
                          float* fitness, float* canvas);
 
+// ------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  The small kernels of a generation follow one another in one
+// stream, and between two of them the launch of the second costs about as much as the kernel itself
+// runs.  A kernel launched with launch_dependent may be set up while its predecessor is still
+// running; it MUST call dep_wait() before it reads or writes anything (every thread, before any
+// return): that waits for the predecessor to have completed, and so, one after the other, for
+// everything before it.  A kernel lets its successor be set up with dep_trigger().  After a kernel that
+// never triggers, or after a copy, the launch is an ordinary one.
+// ------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 }  // namespace evo

@@ -200,6 +200,9 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = ctl.tmem_slot;
+    // conv2 is launched as a programmatic dependent: its blocks may become resident (and fetch their filters)
+    // as soon as blocks of this kernel leave; it waits for this whole grid before it reads an activation
+    if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kC1EpiThreads / 32) {
         // ================= MMA issuer =============================================================
@@ -462,6 +465,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = S.tmem_slot;
+    if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the finalize kernel may be set up
 
     if (warp < kC2EpiThreads / 32) {
         // ================= accumulator warps: bands -> tensor memory; pool, bias, ReLU -> activations ===
@@ -746,6 +750,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         if (lane == 0) {
             const unsigned char* src = pooled1 + static_cast<size_t>(u_begin) * kGroupBytes;
             uint32_t issued = 0;
+            asm volatile("griddepcontrol.wait;" ::: "memory");          // the activations are complete and visible
             for (uint32_t j = 0; j < n_mine; ++j) {
                 const uint32_t slot = j % kC2Ring;
                 if (j >= kC2Ring) c2_wait(S, &S.a_free[slot], (j / kC2Ring - 1u) & 1u, status);
@@ -782,6 +787,8 @@ __global__ void __launch_bounds__(256)
 k_cnn_tc_finalize(const float* __restrict__ loss, uint32_t batch, float* __restrict__ fitness)
 {
     __shared__ float red[256];
+    dep_wait();                                                         // the losses are complete and visible
+    dep_trigger();                                                      // the ranking that follows may be set up
     const uint32_t m = blockIdx.x;
     float s = 0.f;
     for (uint32_t i = threadIdx.x; i < batch; i += 256u) s += loss[static_cast<size_t>(m) * batch + i];
@@ -832,10 +839,28 @@ int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uin
     if (cudaFuncSetAttribute(k_cnn_conv2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, c2_bytes) != cudaSuccess) return -1;
     const uint64_t n_units = static_cast<uint64_t>(P) * n_groups;
     const uint32_t g2 = static_cast<uint32_t>(min(n_units, static_cast<uint64_t>(sm_count)));         // one block per SM
-    k_cnn_conv2_tc<<<g2, kC2Threads, c2_bytes, st>>>(theta, ldD, P, pooled1, labels, batch, loss, status);
-    if (cudaGetLastError() != cudaSuccess) return -1;
-    k_cnn_tc_finalize<<<P, 256, 0, st>>>(loss, batch, fitness);
-    if (cudaGetLastError() != cudaSuccess) return -1;
+    {
+        // conv2 may start (its blocks become resident, fetch their filters and build their bands) while the tail
+        // of conv1 is still running; it reads no activation before conv1 has completed (griddepcontrol.wait)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(g2); cfg.blockDim = dim3(kC2Threads); cfg.dynamicSmemBytes = static_cast<size_t>(c2_bytes); cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        const unsigned char* p1 = pooled1;
+        if (cudaLaunchKernelEx(&cfg, k_cnn_conv2_tc, theta, ldD, P, p1, labels, batch, loss, status) != cudaSuccess) return -1;
+    }
+    {   // likewise a programmatic dependent (of conv2): its launch latency goes under conv2's tail
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(P); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        const float* lp = loss;
+        if (cudaLaunchKernelEx(&cfg, k_cnn_tc_finalize, lp, batch, fitness) != cudaSuccess) return -1;
+    }
     return 3;
 }
 

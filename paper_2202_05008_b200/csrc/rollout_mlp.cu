@@ -158,6 +158,7 @@ k_rollout_mlp_generic(const RolloutMlpArgs a, const DeviceStatus* __restrict__ s
 __global__ void k_fitness_finalize(const float* __restrict__ partial, uint32_t P, uint32_t n_eb,
                                    uint32_t E, float* __restrict__ fitness)
 {
+    dep_trigger();                       // the ranking that follows may be set up
     const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
     if (m >= P) return;
     float s = 0.f;

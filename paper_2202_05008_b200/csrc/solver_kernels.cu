@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(256, 8)
 k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, PhiloxKey key,
       const DeviceStatus* __restrict__ status, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* __restrict__ theta, float* __restrict__ eps)
 {
+    dep_wait();
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
     const uint32_t generation = status->generation;
@@ -108,8 +109,8 @@ int launch_ask(cudaStream_t st, const float* center, const float* sigma_vec, uin
     const uint32_t quads = ldD / 4u;
     dim3 grid((quads + 255u) / 256u, (H + kAskPairsPerThread - 1u) / kAskPairsPerThread);
     if (grid.y > 65535u) grid.y = 65535u;
-    k_ask<<<grid, 256, 0, st>>>(center, sigma_vec, philox_key(k0, k1), status, pair0, H, D, ldD, theta, eps);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    return launch_dependent(k_ask, grid, dim3(256), 0, st, center, sigma_vec, philox_key(k0, k1), status, pair0, H, D, ldD,
+                            theta, eps) == cudaSuccess ? 1 : -1;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -122,6 +123,8 @@ k_rank(const float* __restrict__ fitness, uint32_t P, int32_t* __restrict__ rank
        float* __restrict__ u, DeviceStatus* status)
 {
     __shared__ float tile[kRankTile];
+    dep_wait();
+    dep_trigger();
     const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
     const float fm = (m < P) ? fitness[m] : 0.f;
     if (m < P && fm != fm) atomicOr(&status->nonfinite, 1u);
@@ -186,8 +189,7 @@ int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank
 {
     const uint32_t bx = (P + 255u) / 256u;
     if (P <= 2u * kRankTile) {
-        k_rank<<<bx, 256, 0, st>>>(fitness, P, rank, u, status);
-        return cudaGetLastError() == cudaSuccess ? 1 : -1;
+        return launch_dependent(k_rank, dim3(bx), dim3(256), 0, st, fitness, P, rank, u, status) == cudaSuccess ? 1 : -1;
     }
     k_rank_zero<<<bx, 256, 0, st>>>(rank, P);
     if (cudaGetLastError() != cudaSuccess) return -1;
@@ -238,6 +240,8 @@ k_grad_partial(const float* __restrict__ u, const float* __restrict__ eps, Philo
                uint32_t pairs_per_split, double* __restrict__ partial, float* __restrict__ sigma_partial,
                const DeviceStatus* status)
 {
+    dep_wait();
+    dep_trigger();
     if (status->nonfinite) return;
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
@@ -312,6 +316,8 @@ k_update(const double* __restrict__ partial, const float* __restrict__ sigma_par
          float* __restrict__ center, float* __restrict__ m, float* __restrict__ v, float* __restrict__ g,
          double* __restrict__ norm_partial, const DeviceStatus* status)
 {
+    dep_wait();
+    dep_trigger();
     if (status->nonfinite) return;
     __shared__ float corr[2];
     __shared__ double red[256];
@@ -449,6 +455,8 @@ k_clipup_apply(float* __restrict__ vel, float* __restrict__ center, uint32_t ldD
 // counter (the random streams of the next ask and roll-out) always does.
 __global__ void k_tell_finish(DeviceStatus* status)
 {
+    dep_wait();
+    dep_trigger();
     if (status->nonfinite) {
         status->sticky |= (1u << EVO_ERR_NONFINITE);
         status->nonfinite = 0;
@@ -475,9 +483,8 @@ size_t clipup_norm_doubles(uint32_t ldD) { return 2u * ((ldD / 4u + 255u) / 256u
 template <bool REGEN, bool SIGMA>
 static void launch_grad(dim3 grid, cudaStream_t st, const TellArgs& a, uint32_t pps)
 {
-    k_grad_partial<REGEN, SIGMA><<<grid, kGradThreads, 0, st>>>(a.u, a.eps, philox_key(a.k0, a.k1), a.pair0,
-                                                                a.H, a.D, a.ldD, pps, a.partial, a.sigma_partial,
-                                                                a.status);
+    launch_dependent(k_grad_partial<REGEN, SIGMA>, grid, dim3(kGradThreads), 0, st, a.u, a.eps, philox_key(a.k0, a.k1),
+                     a.pair0, a.H, a.D, a.ldD, pps, a.partial, a.sigma_partial, a.status);
 }
 
 static int launch_partials(cudaStream_t st, const TellArgs& a, uint32_t* used_out)
@@ -503,24 +510,21 @@ static int launch_step(cudaStream_t st, const TellArgs& a, const double* partial
     const uint32_t nb = (quads + 255u) / 256u;
     int launches = 0;
     if (a.optimizer == EVO_OPT_ADAM) {
-        k_update<true><<<nb, 256, 0, st>>>(partial, sigma_partial, splits, a.ldD, inv_pop, a.lr, a.beta1, a.beta2,
-                                           a.adam_eps, a.sigma_lr, a.sigma_max_change, inv_pairs, a.sigma_vec,
-                                           a.center, a.m, a.v, a.g, a.norms, a.status);
-        if (cudaGetLastError() != cudaSuccess) return -1;
+        if (launch_dependent(k_update<true>, dim3(nb), dim3(256), 0, st, partial, sigma_partial, splits, a.ldD, inv_pop, a.lr,
+                             a.beta1, a.beta2, a.adam_eps, a.sigma_lr, a.sigma_max_change, inv_pairs, a.sigma_vec,
+                             a.center, a.m, a.v, a.g, a.norms, a.status) != cudaSuccess) return -1;
         launches += 1;
     } else {
-        k_update<false><<<nb, 256, 0, st>>>(partial, sigma_partial, splits, a.ldD, inv_pop, a.lr, a.beta1, a.beta2,
-                                            a.adam_eps, a.sigma_lr, a.sigma_max_change, inv_pairs, a.sigma_vec,
-                                            a.center, a.m, a.v, a.g, a.norms, a.status);
-        if (cudaGetLastError() != cudaSuccess) return -1;
+        if (launch_dependent(k_update<false>, dim3(nb), dim3(256), 0, st, partial, sigma_partial, splits, a.ldD, inv_pop, a.lr,
+                             a.beta1, a.beta2, a.adam_eps, a.sigma_lr, a.sigma_max_change, inv_pairs, a.sigma_vec,
+                             a.center, a.m, a.v, a.g, a.norms, a.status) != cudaSuccess) return -1;
         k_clipup_velocity<<<nb, 256, 0, st>>>(a.g, a.m, a.ldD, a.lr, a.clipup_momentum, a.norms, nb, a.status);
         if (cudaGetLastError() != cudaSuccess) return -1;
         k_clipup_apply<<<nb, 256, 0, st>>>(a.m, a.center, a.ldD, a.clipup_max_speed, a.norms, nb, a.status);
         if (cudaGetLastError() != cudaSuccess) return -1;
         launches += 3;
     }
-    k_tell_finish<<<1, 1, 0, st>>>(a.status);
-    if (cudaGetLastError() != cudaSuccess) return -1;
+    if (launch_dependent(k_tell_finish, dim3(1), dim3(1), 0, st, a.status) != cudaSuccess) return -1;
     return launches + 1;
 }
 
