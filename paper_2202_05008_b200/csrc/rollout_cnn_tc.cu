@@ -132,6 +132,7 @@ k_cnn_conv1_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
 {
     extern __shared__ __align__(1024) unsigned char dyn[];
     __shared__ __align__(8) C1Ctl ctl;
+    dep_wait();
 
     unsigned char* Bsm = dyn;                                           // 96 KB
     unsigned char* Asm = dyn + kC1SmemB;                                // 2 x 12 KB
@@ -831,9 +832,8 @@ int launch_rollout_cnn_tc(cudaStream_t st, const float* theta, uint32_t ldD, uin
     const uint32_t n_tiles = n_groups * 18u;
     const uint32_t n_member_groups = (P + kC1Group - 1u) / kC1Group;
     dim3 g1(min(max(static_cast<uint32_t>(sm_count) / n_member_groups, 1u), n_tiles), n_member_groups);
-    k_cnn_conv1_tc<<<g1, kC1Threads, kC1DynRequest, st>>>(theta, ldD, P, images, batch,
-                                                          reinterpret_cast<uint4*>(pooled1), status);
-    if (cudaGetLastError() != cudaSuccess) return -1;
+    if (launch_dependent(k_cnn_conv1_tc, g1, dim3(kC1Threads), kC1DynRequest, st, theta, ldD, P, images, batch,
+                         reinterpret_cast<uint4*>(pooled1), status) != cudaSuccess) return -1;
 
     const int c2_bytes = static_cast<int>(sizeof(C2Smem));
     if (cudaFuncSetAttribute(k_cnn_conv2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, c2_bytes) != cudaSuccess) return -1;

@@ -158,6 +158,7 @@ k_rollout_mlp_generic(const RolloutMlpArgs a, const DeviceStatus* __restrict__ s
 __global__ void k_fitness_finalize(const float* __restrict__ partial, uint32_t P, uint32_t n_eb,
                                    uint32_t E, float* __restrict__ fitness)
 {
+    dep_wait();
     dep_trigger();                       // the ranking that follows may be set up
     const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
     if (m >= P) return;
@@ -256,8 +257,8 @@ int launch_rollout_mlp(cudaStream_t st, const RolloutMlpArgs& a_in, uint32_t ker
         if (cudaGetLastError() != cudaSuccess) return -1;
         launches += 1;
     }
-    k_fitness_finalize<<<(a.P + 255u) / 256u, 256, 0, st>>>(a.fit_partial, a.P, a.n_eb, a.E, fitness);
-    if (cudaGetLastError() != cudaSuccess) return -1;
+    if (launch_dependent(k_fitness_finalize, dim3((a.P + 255u) / 256u), dim3(256), 0, st, a.fit_partial, a.P, a.n_eb, a.E,
+                         fitness) != cudaSuccess) return -1;
     return launches + 1;
 }
 

@@ -226,6 +226,7 @@ template <int NIN, int H1, int H2, int NOUT, int EB, int THREADS, int TASK,
 __global__ void __launch_bounds__(THREADS)
 k_rollout_mlp_tiled(const RolloutMlpArgs a, DeviceStatus* status)
 {
+    dep_wait();
     constexpr bool CART = (TASK == EVO_TASK_CARTPOLE);
     constexpr int NOBS = CART ? 5 : (kTlNx + kTlNa);        // tanh-linear: [x ; a] feeds the dynamics
     static_assert(!CART || S3 * ((NOUT + TI3 - 1) / TI3) <= 32, "cart-pole action layer runs in warp 0");
@@ -416,6 +417,7 @@ template <int H1, int H2, int EB, int MT, int NT, int TI1, int S1, int TI2, int 
 __global__ void __launch_bounds__(32 + MT * NT)
 k_rollout_cartpole_ws(const RolloutMlpArgs a, DeviceStatus* status)
 {
+    dep_wait();
     constexpr int NIN = 5;
     extern __shared__ __align__(128) float smem[];
     __shared__ __align__(8) uint64_t mbar;
@@ -603,8 +605,7 @@ static int launch_one(K kernel, int threads, size_t act_floats, cudaStream_t st,
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) != cudaSuccess)
         return -1;
     dim3 grid(a.P, a.n_eb);
-    kernel<<<grid, threads, bytes, st>>>(a, status);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    return launch_dependent(kernel, grid, dim3(threads), bytes, st, a, status) == cudaSuccess ? 1 : -1;
 }
 
 int launch_rollout_mlp_tiled(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus* status)

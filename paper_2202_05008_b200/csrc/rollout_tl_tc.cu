@@ -157,6 +157,7 @@ __device__ __forceinline__ void team_sync(int team)
 __global__ void __launch_bounds__(kThreads, 1)
 k_rollout_tl_tc(const RolloutMlpArgs a, DeviceStatus* status)
 {
+    dep_wait();
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Smem& S = *reinterpret_cast<Smem*>(smem_raw);
     const int tid = threadIdx.x;
@@ -476,7 +477,7 @@ int launch_rollout_tl_tc(cudaStream_t st, const RolloutMlpArgs& a, DeviceStatus*
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
     const uint32_t items = a.P * a.n_eb;
     const uint32_t blocks = min(static_cast<uint32_t>(sms), items);
-    tl::k_rollout_tl_tc<<<blocks, tl::kThreads, bytes, st>>>(a, status);
+    launch_dependent(tl::k_rollout_tl_tc, dim3(blocks), dim3(tl::kThreads), bytes, st, a, status);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

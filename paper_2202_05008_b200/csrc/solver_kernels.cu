@@ -68,6 +68,7 @@ k_ask(const float* __restrict__ center, const float* __restrict__ sigma_vec, Phi
       const DeviceStatus* __restrict__ status, uint32_t pair0, uint32_t H, uint32_t D, uint32_t ldD, float* __restrict__ theta, float* __restrict__ eps)
 {
     dep_wait();
+    dep_trigger();                       // the roll-out that follows may be set up
     const uint32_t quad = blockIdx.x * blockDim.x + threadIdx.x;
     if (quad * 4u >= ldD) return;
     const uint32_t generation = status->generation;
