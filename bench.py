@@ -88,23 +88,23 @@ def stage_work(w, stored):
 # that digest; once a kernel's source changes its entry reads null until it is captured again.
 CSRC = os.path.join(ROOT, "paper_2202_05008_b200", "csrc")
 NCU_TRAFFIC = {
-    ("cfg4", "stored"): {"kernel": "k_rollout_tl_tc", "bytes": 3.489774e+08,
+    ("cfg4", "stored"): {"kernel": "k_rollout_tl_tc", "bytes": 3.490288e+08,
                          "files": ['rollout_tl_tc.cu', 'umma.cuh', 'async.cuh', 'noise.cuh', 'fp32x2.cuh', 'internal.h'],
-                         "digest": "d36dd8c98d87d12f",
+                         "digest": "6dc95ec37104ccff",
                          "capture": "P = 592 capture scaled by members (the traffic is the parameter rows, proportional to P)"},
-    ("cfg2", "stored"): {"kernel": "k_rollout_cartpole_ws", "bytes": 4.787968e+06,
+    ("cfg2", "stored"): {"kernel": "k_rollout_cartpole_ws", "bytes": 4.788480e+06,
                          "files": ['rollout_mlp_tiled.cu', 'async.cuh', 'tasks.cuh', 'noise.cuh', 'fp32x2.cuh', 'internal.h'],
-                         "digest": "dd779dfecc56ca08", "capture": "full size"},
-    ("cfg3", "stored"): {"kernel": "k_cnn_conv2_tc", "bytes": 1.530872e+08,
+                         "digest": "43ceffc3a9b4ab42", "capture": "full size"},
+    ("cfg3", "stored"): {"kernel": "k_cnn_conv2_tc", "bytes": 1.533949e+08,
                          "files": ['rollout_cnn_tc.cu', 'umma.cuh', 'async.cuh', 'fp32x2.cuh', 'internal.h'],
-                         "digest": "9fc1e24c9838d01f", "capture": "full size"},
-    ("cfg5", "stored"): {"kernel": "k_ask", "bytes": 1.011768e+11,
+                         "digest": "9bf648a0a51baa53", "capture": "full size"},
+    ("cfg5", "stored"): {"kernel": "k_ask", "bytes": 1.011610e+11,
                          "files": ['solver_kernels.cu', 'noise.cuh', 'internal.h'],
-                         "digest": "3a3acbcf28e35af9",
+                         "digest": "08fdd2bb750833bc",
                          "capture": "D = 32,768 capture scaled by 32 (columns are independent)"},
-    ("cfg5", "regenerated"): {"kernel": "k_ask", "bytes": 6.679631e+10,
+    ("cfg5", "regenerated"): {"kernel": "k_ask", "bytes": 6.677521e+10,
                               "files": ['solver_kernels.cu', 'noise.cuh', 'internal.h'],
-                              "digest": "3a3acbcf28e35af9", "capture": "D = 32,768 capture scaled by 32"},
+                              "digest": "08fdd2bb750833bc", "capture": "D = 32,768 capture scaled by 32"},
 }
 NCU_TRAFFIC[("cfg4", "regenerated")] = NCU_TRAFFIC[("cfg4", "stored")]
 NCU_TRAFFIC[("cfg2", "regenerated")] = NCU_TRAFFIC[("cfg2", "stored")]
