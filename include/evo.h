@@ -60,11 +60,11 @@ enum { EVO_TASK_NONE = 0, EVO_TASK_CARTPOLE = 1, EVO_TASK_TANH_LINEAR = 2, EVO_T
 enum { EVO_ROLLOUT_AUTO = 0, EVO_ROLLOUT_GENERIC = 1, EVO_ROLLOUT_TILED = 2 };
 enum { EVO_OPT_ADAM = 0, EVO_OPT_CLIPUP = 1 };
 enum { EVO_SIGMA_CONSTANT = 0, EVO_SIGMA_PGPE = 1 };
-/* evo_config.debug_flags.  DROP_COMPLETION: the control-task roll-out kernels leave out the
- * asynchronous completion their first bounded wait depends on (the copy of a member's parameter
- * row; in the tensor-core kernel the commit of the first batch of MMAs), so that wait must run
- * out: every block raises EVO_ERR_TIMEOUT, reports NaN as its return and leaves by itself, with
- * nothing left in flight.  It exists so that the time-out path can be tested without disturbing
+/* evo_config.debug_flags.  DROP_COMPLETION: the roll-out kernels leave out the asynchronous
+ * completion their first bounded wait depends on (the copy of a member's parameter row; in the
+ * tensor-core control kernel the commit of the first batch of MMAs; in the tensor-core CNN the
+ * copy of a block's first group of activations), so that wait must run out: every block raises
+ * EVO_ERR_TIMEOUT, reports NaN as its return and leaves by itself, with nothing left in flight.  It exists so that the time-out path can be tested without disturbing
  * the device. */
 enum { EVO_DEBUG_DROP_COMPLETION = 1 };
 

@@ -751,6 +751,8 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
         if (lane == 0) {
             const unsigned char* src = pooled1 + static_cast<size_t>(u_begin) * kGroupBytes;
             uint32_t issued = 0;
+            // a test of the failure path: the first group is never fetched, so the waits for it run out
+            const bool drop_first = (status->debug_flags & EVO_DEBUG_DROP_COMPLETION) != 0u;
             asm volatile("griddepcontrol.wait;" ::: "memory");          // the activations are complete and visible
             for (uint32_t j = 0; j < n_mine; ++j) {
                 const uint32_t slot = j % kC2Ring;
@@ -759,6 +761,7 @@ k_cnn_conv2_tc(const float* __restrict__ theta, uint32_t ldD, uint32_t P, const 
                 // (and its weights) before anyone's second
                 else if (j >= 1u) c2_wait(S, &S.a_full[j - 1u], 0u, status);
                 if (S.abort) break;
+                if (drop_first && j == 0u) continue;
                 bulk_copy_g2s(smem_u32(S.a[slot]), src + static_cast<size_t>(j) * kGroupBytes, kGroupBytes, smem_u32(&S.a_full[slot]));
                 issued = j + 1u;
             }

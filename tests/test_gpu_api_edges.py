@@ -60,8 +60,15 @@ def test_rollout_argument_errors():
     s.close()
 
 
+def _with_batch(s, w):
+    if w.task_kind == W.TASK_SUPERVISED:
+        images, labels = W.image_batch(w.seed, 0, w.batch)
+        s.set_batch(torch.tensor(images, device="cuda"), torch.tensor(labels, device="cuda"))
+    return s
+
+
 @pytest.mark.parametrize("w", [W.CFG1.with_(horizon=5), W.CFG2.with_(pop_size=4, horizon=5),
-                               W.CFG4.with_(pop_size=4, horizon=5)])
+                               W.CFG4.with_(pop_size=4, horizon=5), W.CFG3.with_(pop_size=6, batch=40)])
 def test_a_device_wait_that_runs_out_raises_timeout_and_leaves_the_solver_usable(w):
     """The failure path of the bounded waits, made to happen without disturbing the device: with
     EVO_DEBUG_DROP_COMPLETION the roll-out blocks never start the copy they wait for, and with a
@@ -69,7 +76,7 @@ def test_a_device_wait_that_runs_out_raises_timeout_and_leaves_the_solver_usable
     EVO_ERR_TIMEOUT and report NaN; evo_sync_status must report the condition once and clear it; a
     tell on that fitness must skip the update (NaN fitness)."""
     from paper_2202_05008_b200.binding import DEBUG_DROP_COMPLETION
-    s = Solver(w, wait_cycles_log2=16, debug_flags=DEBUG_DROP_COMPLETION)
+    s = _with_batch(Solver(w, wait_cycles_log2=16, debug_flags=DEBUG_DROP_COMPLETION), w)
     s.ask()
     fit = s.rollout()
     assert s.sync_status() == 6                        # EVO_ERR_TIMEOUT, reported ...
@@ -81,7 +88,7 @@ def test_a_device_wait_that_runs_out_raises_timeout_and_leaves_the_solver_usable
     assert torch.equal(s.center(), c0) and s.counters() == (1, 0)
     s.close()
     # the same configuration without the flag runs normally afterwards on the same device
-    s = Solver(w, wait_cycles_log2=22)
+    s = _with_batch(Solver(w, wait_cycles_log2=22), w)
     s.ask()
     fit = s.rollout()
     assert s.sync_status() == 0 and bool(torch.isfinite(fit).all())
