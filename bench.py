@@ -95,9 +95,9 @@ NCU_TRAFFIC = {
     ("cfg2", "stored"): {"kernel": "k_rollout_cartpole_ws", "bytes": 4.788480e+06,
                          "files": ['rollout_mlp_tiled.cu', 'async.cuh', 'tasks.cuh', 'noise.cuh', 'fp32x2.cuh', 'internal.h'],
                          "digest": "43ceffc3a9b4ab42", "capture": "full size"},
-    ("cfg3", "stored"): {"kernel": "k_cnn_conv2_tc", "bytes": 1.533949e+08,
+    ("cfg3", "stored"): {"kernel": "k_cnn_conv2_tc", "bytes": 1.530819e+08,
                          "files": ['rollout_cnn_tc.cu', 'umma.cuh', 'async.cuh', 'fp32x2.cuh', 'internal.h'],
-                         "digest": "9bf648a0a51baa53", "capture": "full size"},
+                         "digest": "9d6c703703822230", "capture": "full size"},
     ("cfg5", "stored"): {"kernel": "k_ask", "bytes": 1.011610e+11,
                          "files": ['solver_kernels.cu', 'noise.cuh', 'internal.h'],
                          "digest": "08fdd2bb750833bc",
