@@ -148,16 +148,19 @@ k_rank(const float* __restrict__ fitness, uint32_t P, int32_t* __restrict__ rank
     }
 }
 
-// Large populations: the comparisons of a member are split over blockIdx.y (one fitness tile each)
-// and summed with integer atomics (exact, order-independent); a second kernel turns counts into
-// centred ranks.
+// Larger populations: the comparisons of a member are split over blockIdx.y (one fitness tile of
+// `tile_n` <= kRankTile entries each) and summed with integer atomics (exact, order-independent); a
+// second kernel turns counts into centred ranks.
 __global__ void __launch_bounds__(256)
-k_rank_count(const float* __restrict__ fitness, uint32_t P, int32_t* __restrict__ rank, DeviceStatus* status)
+k_rank_count(const float* __restrict__ fitness, uint32_t P, uint32_t tile_n, int32_t* __restrict__ rank,
+             DeviceStatus* status)
 {
     __shared__ float tile[kRankTile];
+    dep_wait();
+    dep_trigger();
     const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t base = blockIdx.y * kRankTile;
-    const uint32_t n = min(kRankTile, P - base);
+    const uint32_t base = blockIdx.y * tile_n;
+    const uint32_t n = min(tile_n, P - base);
     for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) tile[i] = fitness[base + i];
     __syncthreads();
     if (m >= P) return;
@@ -174,12 +177,16 @@ k_rank_count(const float* __restrict__ fitness, uint32_t P, int32_t* __restrict_
 
 __global__ void k_rank_zero(int32_t* __restrict__ rank, uint32_t P)
 {
+    dep_wait();
+    dep_trigger();
     const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
     if (m < P) rank[m] = 0;
 }
 
 __global__ void k_rank_finish(const int32_t* __restrict__ rank, uint32_t P, float* __restrict__ u)
 {
+    dep_wait();
+    dep_trigger();
     const uint32_t m = blockIdx.x * blockDim.x + threadIdx.x;
     if (m < P)
         u[m] = __fadd_rn(__fdiv_rn(__uint2float_rn(static_cast<uint32_t>(rank[m])), __uint2float_rn(P - 1u)), -0.5f);
@@ -189,16 +196,16 @@ int launch_rank(cudaStream_t st, const float* fitness, uint32_t P, int32_t* rank
                 DeviceStatus* status)
 {
     const uint32_t bx = (P + 255u) / 256u;
-    if (P <= 2u * kRankTile) {
+    if (P <= 1024u) {      // a handful of blocks, each thread against the whole population: a few microseconds
         return launch_dependent(k_rank, dim3(bx), dim3(256), 0, st, fitness, P, rank, u, status) == cudaSuccess ? 1 : -1;
     }
-    k_rank_zero<<<bx, 256, 0, st>>>(rank, P);
-    if (cudaGetLastError() != cudaSuccess) return -1;
-    dim3 grid(bx, (P + kRankTile - 1u) / kRankTile);
-    k_rank_count<<<grid, 256, 0, st>>>(fitness, P, rank, status);
-    if (cudaGetLastError() != cudaSuccess) return -1;
-    k_rank_finish<<<bx, 256, 0, st>>>(rank, P, u);
-    return cudaGetLastError() == cudaSuccess ? 3 : -1;
+    // From there on one kernel of P / 256 blocks leaves most of the GPU idle (P = 4,096: 16 blocks, 63 us):
+    // tiles of 256 comparisons up to P = 8,192 (P = 4,096: 256 blocks), of 2,048 beyond.
+    const uint32_t tile_n = P <= 8192u ? 256u : kRankTile;
+    if (launch_dependent(k_rank_zero, dim3(bx), dim3(256), 0, st, rank, P) != cudaSuccess) return -1;
+    dim3 grid(bx, (P + tile_n - 1u) / tile_n);
+    if (launch_dependent(k_rank_count, grid, dim3(256), 0, st, fitness, P, tile_n, rank, status) != cudaSuccess) return -1;
+    return launch_dependent(k_rank_finish, dim3(bx), dim3(256), 0, st, rank, P, u) == cudaSuccess ? 3 : -1;
 }
 
 // ------------------------------------------------------------------------------------------
