@@ -151,17 +151,19 @@ def test_fma_probe_reports_a_plausible_fp32_rate_and_rejects_bad_shapes():
     assert flops.value == 2 * 16 * 8 * 1024
 
 
-def test_graph_replay_of_a_generation_matches_plain_calls():
+@pytest.mark.parametrize("w", [W.CFG1.with_(pop_size=32), W.CFG3.with_(pop_size=70, batch=48),
+                               W.CFG4.with_(pop_size=8, horizon=20)])
+def test_graph_replay_of_a_generation_matches_plain_calls(w):
     """ask -> rollout -> tell captured once and replayed must walk through the same generations
-    (same noise, same episode seeds, same centre) as the three calls made one by one."""
-    w = W.CFG1.with_(pop_size=32)
-    plain = Solver(w)
+    (same noise, same episode seeds, same centre) as the three calls made one by one.  The kernels of a
+    generation are programmatic dependents of one another; the capture must keep those edges."""
+    plain = _with_batch(Solver(w), w)
     for _ in range(4):
         plain.ask()
         plain.tell(plain.rollout())
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
-        g = Solver(w, stream=side)
+        g = _with_batch(Solver(w, stream=side), w)
         fit = torch.empty(w.pop_size, device="cuda")
         g.ask(); g.tell(g.rollout(fitness=fit))                  # generation 0 by hand (also warms up)
         graph = g.capture_generation(fit)                         # capturing does not run anything
